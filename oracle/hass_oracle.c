@@ -1,0 +1,274 @@
+/*
+ * fp64 CPU oracle for the fused LM-head + Top-K distillation loss of HASS
+ * (Harmonized Objective Distillation, Section 3.1, Eq. 1) and its gradient with
+ * respect to the draft features.
+ *
+ * THIS IS TEST INFRASTRUCTURE. It is slow on purpose, shares no code with the
+ * CUDA library and must never be called from the product path. Only the tests,
+ * the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Per row i (rows are independent), in the paper's notation (q: target LLM's
+ * next-token distribution, p: draft model's, Omega: vocabulary, Omega_hat: the K
+ * tokens with the highest target probability):
+ *
+ *   step 1  z_t[v] = sum_k H_t[i,k] W[v,k],  z_d[v] = sum_k H_d[i,k] W[v,k]
+ *           (the shared LM head applied to target and draft features; training
+ *            listing in Section 3.2: lm_head(hidden_states_target), lm_head(predict))
+ *   step 2  q = softmax(z_t), p = softmax(z_d) over the whole vocabulary (Eq. 1: q and p
+ *           are next-token probability distributions; they are NOT renormalised over
+ *           Omega_hat - that is the separate "Normed Top-K" variant of Section 4.3)
+ *   step 3  Omega_hat = K largest q (Section 3.1), by a full sort on (-z_t, index):
+ *           ties go to the lower index
+ *   step 4  L = - sum_{x in Omega_hat} q(x) log p(x)                        (Eq. 1)
+ *   step 5  dL/dz_d[v] = g (S_q p[v] - q[v] [v in Omega_hat]),  S_q = sum_{x in Omega_hat} q(x)
+ *           dH_d[i,:] = sum_v dL/dz_d[v] W[v,:]
+ *           (derivative of Eq. 1 with q and Omega_hat constant: the target side needs no
+ *            gradient, Appendix "Training Overhead"; g is the upstream weight of row i)
+ *
+ * Inputs of the feature-level entry are bf16 bit patterns widened exactly to fp64.
+ * The only liberty taken with summation order is SIMD reassociation of the inner
+ * dot-product loop (omp simd reduction), i.e. rounding order.
+ *
+ * Pins (tests/test_oracle_pins.py): K = V reduces to soft-target cross-entropy
+ * (library log_softmax), one-hot target gives NLL, shift invariances, brute-force
+ * subset enumeration with a literal unshifted Eq. 1, finite differences, and an
+ * autograd restatement. Every function here is pinned by at least one of them.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#if defined(__x86_64__) && defined(__GNUC__) && !defined(__clang__)
+#define HASS_CLONES __attribute__((target_clones("avx512f", "avx2,fma", "default")))
+#else
+#define HASS_CLONES
+#endif
+
+static inline double bf16_to_f64(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int hass_oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---- step 1 helpers ------------------------------------------------------- */
+
+HASS_CLONES
+static void dot2(const double* a, const double* b, const double* w, int64_t d, double* out_a,
+                 double* out_b) {
+    double sa = 0.0, sb = 0.0;
+#pragma omp simd reduction(+ : sa, sb)
+    for (int64_t k = 0; k < d; ++k) {
+        sa += a[k] * w[k];
+        sb += b[k] * w[k];
+    }
+    *out_a = sa;
+    *out_b = sb;
+}
+
+HASS_CLONES
+static void axpy(double alpha, const double* w, double* y, int64_t d) {
+    for (int64_t k = 0; k < d; ++k) y[k] += alpha * w[k];
+}
+
+HASS_CLONES
+static void widen_bf16(const uint16_t* src, double* dst, int64_t d) {
+    for (int64_t k = 0; k < d; ++k) dst[k] = bf16_to_f64(src[k]);
+}
+
+/* ---- steps 2-5 on given logits ------------------------------------------------ */
+
+typedef struct {
+    double z;
+    int32_t v;
+} zi_t;
+
+static int cmp_desc(const void* pa, const void* pb) {
+    const zi_t* a = (const zi_t*)pa;
+    const zi_t* b = (const zi_t*)pb;
+    if (a->z > b->z) return -1;
+    if (a->z < b->z) return 1;
+    return (a->v > b->v) - (a->v < b->v);
+}
+
+static double log_sum_exp(const double* z, int64_t V) {
+    double m = z[0];
+    for (int64_t v = 1; v < V; ++v)
+        if (z[v] > m) m = z[v];
+    double s = 0.0;
+    for (int64_t v = 0; v < V; ++v) s += exp(z[v] - m);
+    return m + log(s);
+}
+
+/*
+ * Steps 2-5 for one row from its logits.
+ *   forced_idx  NULL: Omega_hat is the top-K of z_t (step 3). Otherwise K indices that are
+ *               taken as Omega_hat as given (used to score a row whose K-th and (K+1)-th
+ *               target logits are a near-tie on a set the caller supplies).
+ *   idx, q_k    [K] out: Omega_hat in descending q (ties: lower index first) and q there.
+ *   dz_d        [V] out or NULL.
+ * Returns 0, or -1 on bad arguments.
+ */
+int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V, int32_t K, double g,
+                                const int32_t* forced_idx, double* loss, int32_t* idx, double* q_k,
+                                double* lse_t_out, double* lse_d_out, double* dz_d) {
+    if (V < 1 || K < 1 || K > V) return -1;
+    const double lse_t = log_sum_exp(z_t, V);
+    const double lse_d = log_sum_exp(z_d, V);
+
+    zi_t* order = NULL;
+    if (forced_idx) {
+        order = (zi_t*)malloc(sizeof(zi_t) * (size_t)K);
+        for (int32_t j = 0; j < K; ++j) {
+            if (forced_idx[j] < 0 || forced_idx[j] >= V) {
+                free(order);
+                return -1;
+            }
+            order[j].z = z_t[forced_idx[j]];
+            order[j].v = forced_idx[j];
+        }
+        qsort(order, (size_t)K, sizeof(zi_t), cmp_desc);
+    } else {
+        order = (zi_t*)malloc(sizeof(zi_t) * (size_t)V);
+        for (int64_t v = 0; v < V; ++v) {
+            order[v].z = z_t[v];
+            order[v].v = (int32_t)v;
+        }
+        qsort(order, (size_t)V, sizeof(zi_t), cmp_desc);
+    }
+
+    double S_q = 0.0, L = 0.0;
+    for (int32_t j = 0; j < K; ++j) {
+        const int32_t x = order[j].v;
+        const double q = exp(z_t[x] - lse_t);
+        const double logp = z_d[x] - lse_d;
+        idx[j] = x;
+        q_k[j] = q;
+        S_q += q;
+        L -= q * logp;
+    }
+    *loss = L;
+    if (lse_t_out) *lse_t_out = lse_t;
+    if (lse_d_out) *lse_d_out = lse_d;
+
+    if (dz_d) {
+        for (int64_t v = 0; v < V; ++v) dz_d[v] = g * S_q * exp(z_d[v] - lse_d);
+        for (int32_t j = 0; j < K; ++j) dz_d[idx[j]] -= g * q_k[j];
+    }
+    free(order);
+    return 0;
+}
+
+/* ---- feature-level entries -------------------------------------------------------- */
+
+/*
+ * Steps 1-5 for a set of rows.
+ *   elem_bytes  2: H_t, H_d, W hold bf16 bit patterns; 8: they hold doubles.
+ *   rows        NULL (all N rows, n_rows == N) or n_rows row numbers into H_t / H_d.
+ *   grad_loss   NULL (g = 1) or [N] upstream weights, indexed by the original row number.
+ *   forced_idx  NULL or [n_rows, K].
+ * Outputs are indexed by position in `rows`: loss, lse_t, lse_d [n_rows]; idx, q_k [n_rows, K];
+ * dH_d [n_rows, d] (may be NULL to skip step 5's back-projection).
+ */
+int hass_oracle_features(const void* H_t, const void* H_d, const void* W, int elem_bytes, int64_t N,
+                         int64_t d, int64_t V, int32_t K, const double* grad_loss, const int64_t* rows,
+                         int64_t n_rows, const int32_t* forced_idx, double* loss, int32_t* idx,
+                         double* q_k, double* lse_t, double* lse_d, double* dH_d) {
+    if (N < 1 || d < 1 || V < 1 || K < 1 || K > V || n_rows < 0) return -1;
+    if (elem_bytes != 2 && elem_bytes != 8) return -1;
+    if (!rows && n_rows != N) return -1;
+    for (int64_t r = 0; r < n_rows; ++r)
+        if (rows && (rows[r] < 0 || rows[r] >= N)) return -1;
+    int status = 0;
+
+#pragma omp parallel
+    {
+        double* ht = (double*)malloc(sizeof(double) * (size_t)d);
+        double* hd = (double*)malloc(sizeof(double) * (size_t)d);
+        double* wr = (double*)malloc(sizeof(double) * (size_t)d);
+        double* zt = (double*)malloc(sizeof(double) * (size_t)V);
+        double* zd = (double*)malloc(sizeof(double) * (size_t)V);
+        double* dz = (double*)malloc(sizeof(double) * (size_t)V);
+
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            const int64_t i = rows ? rows[r] : r;
+            const double g = grad_loss ? grad_loss[i] : 1.0;
+            if (elem_bytes == 2) {
+                widen_bf16((const uint16_t*)H_t + i * d, ht, d);
+                widen_bf16((const uint16_t*)H_d + i * d, hd, d);
+            } else {
+                memcpy(ht, (const double*)H_t + i * d, sizeof(double) * (size_t)d);
+                memcpy(hd, (const double*)H_d + i * d, sizeof(double) * (size_t)d);
+            }
+            /* step 1 */
+            for (int64_t v = 0; v < V; ++v) {
+                const double* w;
+                if (elem_bytes == 2) {
+                    widen_bf16((const uint16_t*)W + v * d, wr, d);
+                    w = wr;
+                } else {
+                    w = (const double*)W + v * d;
+                }
+                dot2(ht, hd, w, d, &zt[v], &zd[v]);
+            }
+            /* steps 2-5 on the logits */
+            int rc = hass_oracle_row_from_logits(zt, zd, V, K, g, forced_idx ? forced_idx + r * K : NULL,
+                                                 &loss[r], idx + r * K, q_k + r * K, &lse_t[r], &lse_d[r],
+                                                 dH_d ? dz : NULL);
+            if (rc != 0) {
+#pragma omp atomic write
+                status = -1;
+                continue;
+            }
+            /* step 5: back-projection through the LM head */
+            if (dH_d) {
+                double* out = dH_d + r * d;
+                for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+                for (int64_t v = 0; v < V; ++v) {
+                    const double* w;
+                    if (elem_bytes == 2) {
+                        widen_bf16((const uint16_t*)W + v * d, wr, d);
+                        w = wr;
+                    } else {
+                        w = (const double*)W + v * d;
+                    }
+                    axpy(dz[v], w, out, d);
+                }
+            }
+        }
+        free(ht);
+        free(hd);
+        free(wr);
+        free(zt);
+        free(zd);
+        free(dz);
+    }
+    return status;
+}
+
+/* Step 1 for selected (row, token) pairs: z[j] = sum_k H[row_j, k] W[tok_j, k], bf16 inputs.
+ * The parity comparator uses it to look up target logits of tokens the GPU selected. */
+int hass_oracle_logits_at(const uint16_t* H, const uint16_t* W, int64_t N, int64_t d, int64_t V,
+                          const int64_t* row, const int32_t* tok, int64_t n, double* z) {
+    for (int64_t j = 0; j < n; ++j) {
+        if (row[j] < 0 || row[j] >= N || tok[j] < 0 || tok[j] >= V) return -1;
+        double s = 0.0;
+        for (int64_t k = 0; k < d; ++k)
+            s += bf16_to_f64(H[row[j] * d + k]) * bf16_to_f64(W[(int64_t)tok[j] * d + k]);
+        z[j] = s;
+    }
+    return 0;
+}
