@@ -1,0 +1,172 @@
+/*
+ * hass.h - C ABI of the B200 (sm_100a) fused LM-head + Top-K distillation library.
+ *
+ * The library computes, for N rows of target features H_t and draft features H_d and the
+ * frozen LM head W that both share, the Top-K distillation loss of HASS and its gradient
+ * with respect to H_d, without ever holding an N x V logit matrix in memory.
+ *
+ * Notation follows the paper (Section 3.1): q = softmax(H_t W^T) is the target LLM's
+ * next-token distribution, p = softmax(H_d W^T) the draft model's, Omega the vocabulary
+ * (size V), Omega_hat the K tokens with the highest q.
+ *
+ * Common conventions
+ *   - Every pointer is DEVICE memory owned by the caller unless a parameter says "host".
+ *     The library allocates nothing, frees nothing and (except hass_check and the *_host
+ *     entry) never synchronises: work is enqueued on `cuda_stream` (a cudaStream_t passed as
+ *     void*; NULL = the default stream) and outputs are valid once the stream reaches that point.
+ *   - Matrices are dense row-major: H_t, H_d [N, d], W [V, d], bf16 (raw 16-bit patterns).
+ *     All pointers must be 16-byte aligned; d must be a multiple of 8 (a row is then a whole
+ *     number of 16-byte units, which the TMA engine requires).
+ *   - 1 <= K <= min(V, HASS_K_MAX). N >= 1 and V >= 1 are otherwise arbitrary; ragged row and
+ *     vocabulary tiles are handled inside.
+ *   - The return value is a hass_status. Argument errors are found on the host before anything
+ *     is launched. A device-side problem (a bounded wait that gave up) is recorded in a status
+ *     word at the start of the workspace and reported by hass_check. Nothing traps or aborts.
+ *   - The device must be compute capability 10.x; anything else returns HASS_ERR_ARCH. There is
+ *     no fallback path.
+ *   - `workspace` is scratch the caller provides (hass_topk_distill_workspace_bytes gives the
+ *     size; 256-byte aligned). The same workspace may be reused by successive calls on one
+ *     stream; calls that may overlap on the GPU need separate workspaces.
+ */
+#ifndef HASS_H_
+#define HASS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HASS_K_MAX 128
+
+typedef enum {
+    HASS_OK = 0,
+    HASS_ERR_INVALID_ARG = -1, /* null / misaligned pointer, size out of range */
+    HASS_ERR_UNSUPPORTED = -2, /* legal but not implemented (e.g. N too large for one call) */
+    HASS_ERR_WORKSPACE = -3,   /* workspace missing or too small */
+    HASS_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed, or no CUDA device */
+    HASS_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (see hass_check) */
+    HASS_ERR_ARCH = -6         /* device is not sm_100 */
+} hass_status;
+
+typedef enum { HASS_BF16 = 0, HASS_FP32 = 1 } hass_dtype; /* element type of dH_d */
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* hass_status_string(int status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int hass_version(void);
+
+/*
+ * Bytes of workspace that every entry point below accepts for this problem size.
+ * The figure covers: a status block, per-CTA partial softmax statistics and Top-K candidates of
+ * the forward sweep, the index-sorted Top-K lists of the backward, and a bounded scratch for one
+ * chunk of rows of the gradient with respect to the draft logits (bf16, chunk_rows x V; the
+ * chunk is a fixed number of 128-row tiles that does not grow with N).
+ * Needs no GPU (assumes 148 SMs if none is present).
+ */
+int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes);
+
+/*
+ * Forward: Eq. 1 of the paper, L_i = - sum_{x in Omega_hat_i} q_i(x) log p_i(x), per row.
+ *
+ * Steps (Section 3.1 and the training listing of Section 3.2: lm_head(hidden_states_target),
+ * lm_head(predict), logit loss): target logits z_t = H_t W^T and draft logits z_d = H_d W^T over
+ * the whole vocabulary (computed tile by tile, never stored), their log-sum-exp, the K largest
+ * target logits per row (= K most probable tokens under q), and the loss.
+ * q and p are full-vocabulary softmaxes; they are not renormalised over Omega_hat.
+ *
+ *   loss      [N]    out  per-row loss, unweighted
+ *   topk_idx  [N,K]  out  Omega_hat, in descending q; equal logits: lower token id first
+ *   topk_q    [N,K]  out  q(x) for those tokens
+ *   lse_t     [N]    out  log sum_v exp z_t[v]
+ *   lse_d     [N]    out  log sum_v exp z_d[v]
+ */
+int hass_topk_distill_fwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
+                          int64_t V, int32_t K, float* loss, int32_t* topk_idx, float* topk_q,
+                          float* lse_t, float* lse_d, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream);
+
+/*
+ * Forward for aligning steps j >= 2 of harmonized context alignment (Section 3.2): the target
+ * side (q, Omega_hat) does not change between steps - the paper counts it in the "constant
+ * part" of the cost (Appendix, Training Overhead) - so topk_idx / topk_q from an earlier
+ * hass_topk_distill_fwd are INPUTS here and only the draft projection is computed.
+ *
+ *   topk_idx [N,K] in, topk_q [N,K] in;  loss [N] out, lse_d [N] out.
+ */
+int hass_topk_distill_fwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                                int32_t K, const int32_t* topk_idx, const float* topk_q, float* loss,
+                                float* lse_d, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream);
+
+/*
+ * Backward: gradient of sum_i grad_loss[i] * L_i with respect to H_d (the loss.backward() of the
+ * training listing; the target side and the LM head receive no gradient - Section 2 says the
+ * head is the target LLM's, and the Appendix says the constant part needs no gradient).
+ *
+ *   dz_d[i,v] = grad_loss[i] * ( S_q,i * p_i(v) - q_i(v) * [v in Omega_hat_i] ),  S_q = sum of topk_q
+ *   dH_d      = dz_d W
+ *
+ * dz_d is formed one bounded chunk of rows at a time (recomputing z_d tile by tile from H_d, W
+ * and lse_d) in bf16 inside the workspace and contracted with W on the tensor cores.
+ *
+ *   topk_idx, topk_q, lse_d   in   as written by the forward
+ *   grad_loss [N]             in   upstream weight per row (loss weight w, step re-weighting
+ *                                  beta^(j-1), masks, 1/N ...), or NULL for all ones
+ *   dH_d      [N,d]           out  bf16 or fp32 according to dH_dtype (a hass_dtype)
+ */
+int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
+                          const int32_t* topk_idx, const float* topk_q, const float* lse_d,
+                          const float* grad_loss, void* dH_d, int dH_dtype, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Forward and backward in one call (the whole hot path of one aligning step): same outputs as
+ * hass_topk_distill_fwd followed by hass_topk_distill_bwd with the same arguments.
+ */
+int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
+                              int64_t V, int32_t K, const float* grad_loss, float* loss,
+                              int32_t* topk_idx, float* topk_q, float* lse_t, float* lse_d,
+                              void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream);
+
+/*
+ * The same forward + backward for callers whose features live in HOST memory (the training
+ * listing reads precomputed target hidden states per batch): H_t_host, H_d_host [N,d] bf16 are
+ * copied to the device, the path runs, and loss_host [N] (fp32) and dH_d_host [N,d] (dH_dtype)
+ * are copied back; topk_idx_host / topk_q_host may be NULL to skip their copy. W stays a DEVICE
+ * pointer: the LM head is frozen and shared, so it is uploaded once, not per step.
+ * grad_loss_host is a host pointer or NULL. Host buffers should be page-locked for the copies
+ * to be asynchronous. The call returns after the stream has been synchronised (the host results
+ * are then valid) and reports device-side errors like hass_check.
+ * `workspace` must hold hass_topk_distill_host_workspace_bytes(...) bytes: the normal workspace
+ * plus device staging for the inputs and outputs.
+ */
+int hass_topk_distill_host_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, int dH_dtype,
+                                           size_t* bytes);
+int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, const void* W,
+                                   int64_t N, int64_t d, int64_t V, int32_t K,
+                                   const float* grad_loss_host, float* loss_host,
+                                   int32_t* topk_idx_host, float* topk_q_host, void* dH_d_host,
+                                   int dH_dtype, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and returns the status word of `workspace`: HASS_OK, or
+ * HASS_ERR_TIMEOUT if a kernel gave up on a bounded wait (its outputs are then undefined), or
+ * HASS_ERR_CUDA if the stream reports an error. Clears the status word.
+ */
+int hass_check(void* workspace, void* cuda_stream);
+
+/*
+ * Number of kernels of this library launched by the calling process so far (all entry points).
+ * Lets a benchmark report how many of the library's own kernels ran in a timed region.
+ */
+int64_t hass_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HASS_H_ */

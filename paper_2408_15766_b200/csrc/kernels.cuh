@@ -1,0 +1,601 @@
+// Device code of the fused LM-head + Top-K distillation path (sm_100a).
+//
+// One warp-specialised, persistent GEMM kernel (TMA -> shared memory -> tcgen05.mma -> TMEM ->
+// epilogue warps) is instantiated with three epilogues:
+//   MODE_STATS  logits tile -> running max / sum-exp per row (+ Top-K candidates for target rows)
+//   MODE_PROBS  draft logits tile -> dz_d tile = g (S_q p - q [v in Omega_hat]) in bf16 -> scratch
+//   MODE_OUT    plain store of the accumulator (dH_d = dz_d W)
+// plus two small kernels: finalize (merge partial statistics, pick Omega_hat, Eq. 1) and
+// bwd_prep (index-sorted Top-K lists and per-row coefficients for MODE_PROBS).
+#pragma once
+#include <cuda_bf16.h>
+#include <float.h>
+#include <limits.h>
+
+#include "ptx.cuh"
+
+namespace hass {
+
+constexpr int BM = 128;        // rows per tile (TMEM lanes)
+constexpr int BN = 256;        // columns per tile (one UMMA N)
+constexpr int BK = 64;         // contraction elements per pipeline stage (128 B of bf16: one swizzle row)
+constexpr int UMMA_K = 16;     // contraction elements per tcgen05.mma (bf16)
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int NUM_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
+constexpr int MAX_PHASES = 48;
+constexpr int K_CAP = 128;         // == HASS_K_MAX
+constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr float LOG2E = 1.4426950408889634f;
+
+enum { MODE_STATS = 0, MODE_PROBS = 1, MODE_OUT = 2 };
+
+// A phase gives G consecutive row tiles S "lanes" each; lane l of a row tile sweeps the column
+// tiles l, l + S, l + 2S, ... CTA b < G * S works on row tile row_tile_begin + b / S, lane b % S, and
+// owns partial-result slot slot_base + b. All CTAs of a phase walk the column tiles in lockstep,
+// so a column tile of B is fetched from HBM once and then served from L2 to the G row tiles.
+struct Phase {
+    int row_tile_begin, G, S, slot_base;
+};
+struct Schedule {
+    int n_phases;
+    int total_slots;
+    int max_ctas;          // largest G * S over the phases = grid size
+    int pad;
+    Phase ph[MAX_PHASES];
+};
+
+struct GemmParams {
+    CUtensorMap tmA0, tmA1, tmB;
+    Schedule sched;
+    int row_tiles0;        // row tiles [0, row_tiles0) read A0, the others A1 (tile index - row_tiles0)
+    int topk_row_tiles;    // leading row tiles whose rows collect Top-K candidates (MODE_STATS)
+    int a_row_offset;      // added to A0's row coordinate (chunked backward)
+    int row_global_offset; // global row number of local row 0 (per-row inputs / outputs)
+    int rows_valid;        // global rows >= rows_valid are padding
+    int n_cols;            // extent of the tile-column dimension (V, or d for MODE_OUT)
+    int col_tiles;
+    int k_blocks;          // ceil(contraction extent / BK)
+    int K;                 // Top-K
+    // MODE_STATS outputs (per slot)
+    float* part_m;
+    float* part_s;
+    float* cand_v;
+    int* cand_i;
+    // MODE_PROBS
+    const float* lse2;     // [N] lse_d * log2(e)
+    const float* coef;     // [N] g * S_q
+    const int* sidx;       // [N, K] Omega_hat sorted by token id
+    const float* sgq;      // [N, K] g * q in the same order
+    __nv_bfloat16* P;      // [chunk rows, p_pitch]
+    long long p_pitch;
+    // MODE_OUT
+    void* out;
+    int out_fp32;
+    long long out_pitch;   // elements
+    unsigned int* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Replace-the-minimum insertion into an unsorted K-list kept in local memory. Returns the new
+// admission threshold: -inf while the list is not full, else its smallest value. Among equal
+// smallest values the one with the highest token id is the next to be evicted, and admission is
+// strict (x > threshold) with token ids visited in increasing order, so equal logits resolve to
+// the lower token id.
+__device__ __noinline__ float topk_insert(float* lv, int* li, int* cnt_minpos, int K, float x, int idx) {
+    int cnt = cnt_minpos[0];
+    if (cnt < K) {
+        lv[cnt] = x;
+        li[cnt] = idx;
+        cnt_minpos[0] = ++cnt;
+        if (cnt < K) return -INFINITY;
+    } else {
+        const int mp = cnt_minpos[1];
+        lv[mp] = x;
+        li[mp] = idx;
+    }
+    float mn = lv[0];
+    int mi = li[0], mp = 0;
+    for (int j = 1; j < K; ++j) {
+        const float a = lv[j];
+        const int b = li[j];
+        if (a < mn || (a == mn && b > mi)) {
+            mn = a;
+            mi = b;
+            mp = j;
+        }
+    }
+    cnt_minpos[1] = mp;
+    return mn;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+    constexpr bool B_MN_MAJOR = (MODE == MODE_OUT);
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smemA = smem_base;
+    const uint32_t smemB = smem_base + STAGES * A_STAGE_BYTES;
+    const uint32_t bar_base = smemB + STAGES * B_STAGE_BYTES;
+    // barriers: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem pointer, abort flag
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint32_t* tmem_ptr_smem =
+        reinterpret_cast<uint32_t*>(smem_gen + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 8 * (2 * STAGES + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&p.tmA0);
+        prefetch_tensormap(&p.tmB);
+        if (MODE == MODE_STATS) prefetch_tensormap(&p.tmA1);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_ptr_smem), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    // Calls f(row_tile, lane, S, slot) for every item of this CTA; f returns false to stop.
+    auto for_each_item = [&](auto&& f) {
+        for (int ph = 0; ph < p.sched.n_phases; ++ph) {
+            const Phase P = p.sched.ph[ph];
+            if (cta < P.G * P.S) {
+                const int gi = cta / P.S;
+                if (!f(P.row_tile_begin + gi, cta - gi * P.S, P.S, P.slot_base + cta)) return;
+            }
+        }
+    };
+
+    if (warp == 0) {
+        // ===================== TMA producer =====================
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for_each_item([&](int rt, int ln, int S, int) {
+                const bool second = (MODE == MODE_STATS) && rt >= p.row_tiles0;
+                const CUtensorMap* tmA = second ? &p.tmA1 : &p.tmA0;
+                const int row0 = second ? (rt - p.row_tiles0) * BM : p.a_row_offset + rt * BM;
+                for (int ct = ln; ct < p.col_tiles; ct += S) {
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!wait_barrier(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) return false;
+                        mbar_arrive_expect_tx(full_bar(stage), A_STAGE_BYTES + B_STAGE_BYTES);
+                        tma_load_2d(smemA + stage * A_STAGE_BYTES, tmA, full_bar(stage), kb * BK, row0);
+                        if (!B_MN_MAJOR) {
+                            tma_load_2d(smemB + stage * B_STAGE_BYTES, &p.tmB, full_bar(stage), kb * BK, ct * BN);
+                        } else {
+                            // B tile = BK contraction rows x BN contiguous columns, fetched as BN/64 boxes
+                            // of 64 columns (one 128-byte swizzle row) x BK rows
+#pragma unroll
+                            for (int j = 0; j < BN / 64; ++j)
+                                tma_load_2d(smemB + stage * B_STAGE_BYTES + j * (BK * 128), &p.tmB, full_bar(stage),
+                                            ct * BN + j * 64, kb * BK);
+                        }
+                        if (++stage == STAGES) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                }
+                return true;
+            });
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer =====================
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN, 0, B_MN_MAJOR ? 1 : 0);
+            int stage = 0;
+            uint32_t phase = 0;
+            int ab = 0;
+            uint32_t aphase = 0;
+            for_each_item([&](int, int ln, int S, int) {
+                for (int ct = ln; ct < p.col_tiles; ct += S) {
+                    if (!wait_barrier(tempty_bar(ab), aphase ^ 1u, abort_flag, p.status, 2)) return false;
+                    tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + ab * BN;
+                    for (int kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!wait_barrier(full_bar(stage), phase, abort_flag, p.status, 3)) return false;
+                        tc_fence_after_sync();
+                        // A: K-major, 8-row groups 1024 B apart. B: K-major likewise, or MN-major with
+                        // 64-column groups BK*128 B apart (LBO) and 8-row contraction groups 1024 B apart (SBO).
+                        const uint64_t a_desc = make_smem_desc_sw128(smemA + stage * A_STAGE_BYTES, 0, 1024);
+                        const uint64_t b_desc =
+                            B_MN_MAJOR ? make_smem_desc_sw128(smemB + stage * B_STAGE_BYTES, BK * 128, 1024)
+                                       : make_smem_desc_sw128(smemB + stage * B_STAGE_BYTES, 0, 1024);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            // advance the start address (>>4) along the contraction
+                            const uint64_t a_adv = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);
+                            const uint64_t b_adv = B_MN_MAJOR ? static_cast<uint64_t>((k * UMMA_K * 128) >> 4)
+                                                              : static_cast<uint64_t>((k * UMMA_K * 2) >> 4);
+                            umma_bf16(d_tmem, a_desc + a_adv, b_desc + b_adv, idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                        if (++stage == STAGES) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                    umma_commit(tfull_bar(ab));          // accumulator complete
+                    ab ^= 1;
+                    if (ab == 0) aphase ^= 1u;
+                }
+                return true;
+            });
+        }
+    } else {
+        // ===================== epilogue warps =====================
+        const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int r_local = quad * 32 + lane;      // row inside the tile
+        int ab = 0;
+        uint32_t aphase = 0;
+        // Top-K list of this thread's row (MODE_STATS); lives in local memory, touched only on admission
+        float lv[MODE == MODE_STATS ? K_CAP : 1];
+        int li[MODE == MODE_STATS ? K_CAP : 1];
+        int cnt_minpos[2];
+
+        for_each_item([&](int rt, int ln, int S, int slot) {
+            const int g_row = p.row_global_offset + rt * BM + r_local;
+            const bool row_ok = g_row < p.rows_valid;
+            // ---- per-item state ----
+            float m = -INFINITY, s = 0.f, thr = -INFINITY;        // MODE_STATS
+            bool want_topk = false;
+            float lse2 = 0.f, coef = 0.f;                         // MODE_PROBS
+            const int* si = nullptr;
+            const float* sg = nullptr;
+            int cur = 0, nxt = INT_MAX;
+            if (MODE == MODE_STATS) {
+                want_topk = rt < p.topk_row_tiles;
+                cnt_minpos[0] = 0;
+                cnt_minpos[1] = 0;
+            }
+            if (MODE == MODE_PROBS && row_ok) {
+                lse2 = p.lse2[g_row];
+                coef = p.coef[g_row];
+                si = p.sidx + static_cast<long long>(g_row) * p.K;
+                sg = p.sgq + static_cast<long long>(g_row) * p.K;
+                nxt = si[0];
+            }
+            for (int ct = ln; ct < p.col_tiles; ct += S) {
+                // the whole warp must agree before the warp-collective TMEM loads below
+                const bool ready = wait_barrier(tfull_bar(ab), aphase, abort_flag, p.status, 4);
+                if (!__all_sync(0xffffffffu, ready)) return false;
+                tc_fence_after_sync();
+                const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + ab * BN;
+                const int col_base = ct * BN;
+#pragma unroll 1
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t r[32];
+                    tmem_ld32(t_row + ch * 32, r);
+                    tmem_ld_wait(r);
+                    const int col0 = col_base + ch * 32;
+                    if (MODE == MODE_STATS) {
+                        if (col0 + 32 > p.n_cols) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j >= p.n_cols) r[j] = __float_as_uint(-INFINITY);
+                        }
+                        float cm = __uint_as_float(r[0]);
+#pragma unroll
+                        for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
+                        if (cm > m) {
+                            s *= ex2((m - cm) * LOG2E);
+                            m = cm;
+                        }
+                        const float mneg = -m * LOG2E;
+                        float acc = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), LOG2E, mneg));
+                        s += acc;
+                        if (want_topk && cm > thr) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float x = __uint_as_float(r[j]);
+                                if (x > thr) thr = topk_insert(lv, li, cnt_minpos, p.K, x, col0 + j);
+                            }
+                        }
+                    } else if (MODE == MODE_PROBS) {
+                        while (nxt < col0) {
+                            ++cur;
+                            nxt = cur < p.K ? si[cur] : INT_MAX;
+                        }
+                        float e[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) e[j] = coef * ex2(fmaf(__uint_as_float(r[j]), LOG2E, -lse2));
+                        while (nxt < col0 + 32) {
+                            const int off = nxt - col0;
+                            const float gq = sg[cur];
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j == off) e[j] -= gq;
+                            ++cur;
+                            nxt = cur < p.K ? si[cur] : INT_MAX;
+                        }
+                        if (col0 + 32 > p.n_cols) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j >= p.n_cols) e[j] = 0.f;
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(p.P + static_cast<long long>(rt * BM + r_local) * p.p_pitch + col0);
+#pragma unroll
+                        for (int g8 = 0; g8 < 4; ++g8) {
+                            uint4 w;
+                            w.x = pack_bf16x2(e[8 * g8 + 0], e[8 * g8 + 1]);
+                            w.y = pack_bf16x2(e[8 * g8 + 2], e[8 * g8 + 3]);
+                            w.z = pack_bf16x2(e[8 * g8 + 4], e[8 * g8 + 5]);
+                            w.w = pack_bf16x2(e[8 * g8 + 6], e[8 * g8 + 7]);
+                            dst[g8] = w;
+                        }
+                    } else {
+                        if (row_ok) {
+                            if (p.out_fp32) {
+                                float* dst = reinterpret_cast<float*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+#pragma unroll
+                                for (int g4 = 0; g4 < 8; ++g4) {
+                                    if (col0 + 4 * g4 < p.n_cols) {
+                                        *reinterpret_cast<float4*>(dst + 4 * g4) =
+                                            make_float4(__uint_as_float(r[4 * g4]), __uint_as_float(r[4 * g4 + 1]),
+                                                        __uint_as_float(r[4 * g4 + 2]), __uint_as_float(r[4 * g4 + 3]));
+                                    }
+                                }
+                            } else {
+                                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+#pragma unroll
+                                for (int g8 = 0; g8 < 4; ++g8) {
+                                    if (col0 + 8 * g8 < p.n_cols) {
+                                        uint4 w;
+                                        w.x = pack_bf16x2(__uint_as_float(r[8 * g8 + 0]), __uint_as_float(r[8 * g8 + 1]));
+                                        w.y = pack_bf16x2(__uint_as_float(r[8 * g8 + 2]), __uint_as_float(r[8 * g8 + 3]));
+                                        w.z = pack_bf16x2(__uint_as_float(r[8 * g8 + 4]), __uint_as_float(r[8 * g8 + 5]));
+                                        w.w = pack_bf16x2(__uint_as_float(r[8 * g8 + 6]), __uint_as_float(r[8 * g8 + 7]));
+                                        *reinterpret_cast<uint4*>(dst + 8 * g8) = w;
+                                    }
+                                }
+                            }
+                        }
+                    }
+                }
+                // accumulator drained: hand the buffer back to the MMA warp
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(ab));
+                ab ^= 1;
+                if (ab == 0) aphase ^= 1u;
+            }
+            if (MODE == MODE_STATS) {
+                const long long so = static_cast<long long>(slot) * BM + r_local;
+                p.part_m[so] = m;
+                p.part_s[so] = s;
+                if (want_topk) {
+                    const int cnt = cnt_minpos[0];
+                    for (int k = 0; k < p.K; ++k) {
+                        const long long co = (static_cast<long long>(slot) * p.K + k) * BM + r_local;
+                        p.cand_v[co] = k < cnt ? lv[k] : -INFINITY;
+                        p.cand_i[co] = k < cnt ? li[k] : -1;
+                    }
+                }
+            }
+            return true;
+        });
+    }
+
+    // ---- teardown ----
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait gave up: let copies that may still be in flight land before the CTA's memory is released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// finalize: one warp per row. Merges the per-slot (max, sum-exp) pairs into lse_t / lse_d, selects
+// Omega_hat from the slots' candidates (or takes it as an input), gathers the draft logits at
+// Omega_hat with K dot products, and evaluates Eq. 1.
+struct FinalizeParams {
+    Schedule sched;
+    int N, d, K;
+    int row_tiles_t;       // row tiles of the target matrix in the schedule (0: Omega_hat is an input)
+    const float* part_m;
+    const float* part_s;
+    const float* cand_v;
+    const int* cand_i;
+    const __nv_bfloat16* H_d;
+    const __nv_bfloat16* W;
+    const int* idx_in;     // [N,K] when row_tiles_t == 0
+    const float* q_in;
+    float* loss;
+    int* idx_out;
+    float* q_out;
+    float* lse_t;
+    float* lse_d;
+};
+
+__device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
+    slot0 = 0;
+    S = 0;
+    for (int ph = 0; ph < sc.n_phases; ++ph) {
+        const Phase P = sc.ph[ph];
+        if (row_tile >= P.row_tile_begin && row_tile < P.row_tile_begin + P.G) {
+            slot0 = P.slot_base + (row_tile - P.row_tile_begin) * P.S;
+            S = P.S;
+            return;
+        }
+    }
+}
+
+__device__ __forceinline__ float warp_lse(const float* pm, const float* ps, int slot0, int S, int r, int lane) {
+    float m = -INFINITY;
+    for (int j = lane; j < S; j += 32) m = fmaxf(m, pm[static_cast<long long>(slot0 + j) * BM + r]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float s = 0.f;
+    for (int j = lane; j < S; j += 32) {
+        const long long so = static_cast<long long>(slot0 + j) * BM + r;
+        s += ps[so] * exp2f((pm[so] - m) * LOG2E);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return m + logf(s);
+}
+
+__global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ FinalizeParams p) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= p.N) return;
+    const int rt = row / BM, r = row % BM;
+    const int K = p.K;
+    int slot0, S;
+
+    // draft statistics
+    find_slots(p.sched, p.row_tiles_t + rt, slot0, S);
+    const float lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
+    if (lane == 0) p.lse_d[row] = lse_d;
+
+    float lse_t = 0.f;
+    if (p.row_tiles_t > 0) {
+        find_slots(p.sched, rt, slot0, S);
+        lse_t = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
+        if (lane == 0) p.lse_t[row] = lse_t;
+    }
+
+    const __nv_bfloat16* hrow = p.H_d + static_cast<long long>(row) * p.d;
+    float loss = 0.f;
+    float prev_v = INFINITY;
+    int prev_i = -1;
+    const int C = S * K;   // candidates of this row (target path)
+    for (int j = 0; j < K; ++j) {
+        int tok;
+        float qv;
+        if (p.row_tiles_t > 0) {
+            // next candidate after (prev_v, prev_i) in the order: logit descending, then token id ascending
+            float bv = -INFINITY;
+            int bi = INT_MAX;
+            for (int c = lane; c < C; c += 32) {
+                const long long co = (static_cast<long long>(slot0 + c / K) * K + (c % K)) * BM + r;
+                const float v = p.cand_v[co];
+                const int i = p.cand_i[co];
+                if (i < 0) continue;
+                const bool after_prev = (v < prev_v) || (v == prev_v && i > prev_i);
+                const bool better = (v > bv) || (v == bv && i < bi);
+                if (after_prev && better) {
+                    bv = v;
+                    bi = i;
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > bv || (ov == bv && oi < bi)) {
+                    bv = ov;
+                    bi = oi;
+                }
+            }
+            prev_v = bv;
+            prev_i = bi;
+            tok = bi == INT_MAX ? 0 : bi;     // cannot happen for K <= V; keeps the gather in range
+            qv = expf(bv - lse_t);
+            if (lane == 0) {
+                p.idx_out[static_cast<long long>(row) * K + j] = tok;
+                p.q_out[static_cast<long long>(row) * K + j] = qv;
+            }
+        } else {
+            tok = p.idx_in[static_cast<long long>(row) * K + j];
+            qv = p.q_in[static_cast<long long>(row) * K + j];
+        }
+        // draft logit of this token: <H_d[row], W[tok]>
+        const __nv_bfloat16* wrow = p.W + static_cast<long long>(tok) * p.d;
+        float acc = 0.f;
+        for (int k = lane * 8; k < p.d; k += 256) {
+            const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k);
+            const uint4 wv = *reinterpret_cast<const uint4*>(wrow + k);
+            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+            const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const float2 a = __bfloat1622float2(hp[t]);
+                const float2 b = __bfloat1622float2(wp[t]);
+                acc = fmaf(a.x, b.x, acc);
+                acc = fmaf(a.y, b.y, acc);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
+    }
+    if (lane == 0) p.loss[row] = loss;
+}
+
+// ---------------------------------------------------------------------------------------------
+// bwd_prep: one thread per row. Sorts Omega_hat by token id (the MODE_PROBS epilogue walks the
+// vocabulary in increasing order) and precomputes g * q, g * S_q and lse_d * log2(e).
+__global__ void bwd_prep_kernel(int N, int K, const int* __restrict__ idx, const float* __restrict__ q,
+                                const float* __restrict__ lse_d, const float* __restrict__ grad_loss,
+                                int* __restrict__ sidx, float* __restrict__ sgq, float* __restrict__ coef,
+                                float* __restrict__ lse2) {
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= N) return;
+    const float g = grad_loss ? grad_loss[row] : 1.f;
+    int li[K_CAP];
+    float lq[K_CAP];
+    float S_q = 0.f;
+    for (int j = 0; j < K; ++j) {
+        const int x = idx[static_cast<long long>(row) * K + j];
+        const float qq = q[static_cast<long long>(row) * K + j];
+        S_q += qq;
+        int t = j;
+        while (t > 0 && li[t - 1] > x) {
+            li[t] = li[t - 1];
+            lq[t] = lq[t - 1];
+            --t;
+        }
+        li[t] = x;
+        lq[t] = qq;
+    }
+    for (int j = 0; j < K; ++j) {
+        sidx[static_cast<long long>(row) * K + j] = li[j];
+        sgq[static_cast<long long>(row) * K + j] = g * lq[j];
+    }
+    coef[row] = g * S_q;
+    lse2[row] = lse_d[row] * LOG2E;
+}
+
+}  // namespace hass
