@@ -1,0 +1,198 @@
+"""ctypes binding of libhass_b200.so. See include/hass.h for the contract of every call."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhass_b200.so")
+
+HASS_BF16, HASS_FP32 = 0, 1
+K_MAX = 128
+
+
+class HassError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2408_15766_b200.build` "
+            "(needs nvcc with sm_100a support). There is no fallback path.")
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+    L.hass_status_string.restype = ctypes.c_char_p
+    L.hass_status_string.argtypes = [ctypes.c_int]
+    L.hass_version.restype = ctypes.c_int
+    L.hass_kernel_launch_count.restype = ctypes.c_int64
+    L.hass_topk_distill_workspace_bytes.argtypes = [i64, i64, i64, i32, ctypes.POINTER(sz)]
+    L.hass_topk_distill_host_workspace_bytes.argtypes = [i64, i64, i64, i32, ctypes.c_int, ctypes.POINTER(sz)]
+    L.hass_topk_distill_fwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.hass_topk_distill_fwd_draft.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, sz, vp]
+    L.hass_topk_distill_bwd.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+    L.hass_topk_distill_fwd_bwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp,
+                                            ctypes.c_int, vp, sz, vp]
+    L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
+                                                 ctypes.c_int, vp, sz, vp]
+    L.hass_check.argtypes = [vp, vp]
+    for name in ("hass_topk_distill_workspace_bytes", "hass_topk_distill_host_workspace_bytes",
+                 "hass_topk_distill_fwd", "hass_topk_distill_fwd_draft", "hass_topk_distill_bwd",
+                 "hass_topk_distill_fwd_bwd", "hass_topk_distill_fwd_bwd_host", "hass_check"):
+        getattr(L, name).restype = ctypes.c_int
+    return L
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.hass_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib.hass_version())
+
+
+def kernel_launch_count() -> int:
+    return int(lib.hass_kernel_launch_count())
+
+
+def _ok(status: int, where: str) -> None:
+    if status != 0:
+        raise HassError(status, where)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dims(H: torch.Tensor, W: torch.Tensor):
+    assert H.dtype == torch.bfloat16 and W.dtype == torch.bfloat16, "H and W must be bf16"
+    assert H.is_contiguous() and W.is_contiguous() and H.dim() == 2 and W.dim() == 2
+    assert H.shape[1] == W.shape[1], "H and W disagree on d"
+    return H.shape[0], H.shape[1], W.shape[0]
+
+
+def topk_distill_workspace_bytes(N: int, d: int, V: int, K: int) -> int:
+    out = ctypes.c_size_t(0)
+    _ok(lib.hass_topk_distill_workspace_bytes(N, d, V, K, ctypes.byref(out)), "hass_topk_distill_workspace_bytes")
+    return int(out.value)
+
+
+def topk_distill_host_workspace_bytes(N: int, d: int, V: int, K: int, dH_dtype: int = HASS_BF16) -> int:
+    out = ctypes.c_size_t(0)
+    _ok(lib.hass_topk_distill_host_workspace_bytes(N, d, V, K, dH_dtype, ctypes.byref(out)),
+        "hass_topk_distill_host_workspace_bytes")
+    return int(out.value)
+
+
+def _workspace(ws: Optional[torch.Tensor], nbytes: int, device) -> torch.Tensor:
+    if ws is None:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    assert ws.dtype == torch.uint8 and ws.is_cuda and ws.is_contiguous()
+    return ws
+
+
+def _dh_dtype(code: int):
+    return torch.float32 if code == HASS_FP32 else torch.bfloat16
+
+
+def topk_distill_fwd(H_t, H_d, W, K: int, workspace=None, stream=None) -> dict:
+    N, d, V = _dims(H_t, W)
+    assert H_d.shape == H_t.shape and H_d.dtype == torch.bfloat16 and H_d.is_contiguous()
+    dev = H_t.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+               topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+               topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+               lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+               lse_d=torch.empty(N, dtype=torch.float32, device=dev), workspace=ws)
+    _ok(lib.hass_topk_distill_fwd(_p(H_t), _p(H_d), _p(W), N, d, V, K, _p(out["loss"]), _p(out["topk_idx"]),
+                                  _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]), _p(ws), ws.numel(),
+                                  _stream(stream)), "hass_topk_distill_fwd")
+    return out
+
+
+def topk_distill_fwd_draft(H_d, W, topk_idx, topk_q, workspace=None, stream=None) -> dict:
+    N, d, V = _dims(H_d, W)
+    K = topk_idx.shape[1]
+    assert topk_idx.dtype == torch.int32 and topk_q.dtype == torch.float32
+    assert topk_idx.is_contiguous() and topk_q.is_contiguous() and topk_idx.shape == topk_q.shape == (N, K)
+    dev = H_d.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+               lse_d=torch.empty(N, dtype=torch.float32, device=dev), workspace=ws)
+    _ok(lib.hass_topk_distill_fwd_draft(_p(H_d), _p(W), N, d, V, K, _p(topk_idx), _p(topk_q), _p(out["loss"]),
+                                        _p(out["lse_d"]), _p(ws), ws.numel(), _stream(stream)),
+        "hass_topk_distill_fwd_draft")
+    return out
+
+
+def topk_distill_bwd(H_d, W, topk_idx, topk_q, lse_d, grad_loss=None, dH_dtype: int = HASS_BF16, workspace=None,
+                     stream=None, out=None) -> torch.Tensor:
+    N, d, V = _dims(H_d, W)
+    K = topk_idx.shape[1]
+    assert topk_idx.dtype == torch.int32 and topk_q.dtype == torch.float32 and lse_d.dtype == torch.float32
+    assert topk_idx.is_contiguous() and topk_q.is_contiguous() and lse_d.is_contiguous()
+    assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
+    dev = H_d.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    dH = torch.empty(N, d, dtype=_dh_dtype(dH_dtype), device=dev) if out is None else out
+    _ok(lib.hass_topk_distill_bwd(_p(H_d), _p(W), N, d, V, K, _p(topk_idx), _p(topk_q), _p(lse_d), _p(grad_loss),
+                                  _p(dH), dH_dtype, _p(ws), ws.numel(), _stream(stream)), "hass_topk_distill_bwd")
+    return dH
+
+
+def topk_distill_fwd_bwd(H_t, H_d, W, K: int, grad_loss=None, dH_dtype: int = HASS_BF16, workspace=None,
+                         stream=None, out: Optional[dict] = None) -> dict:
+    N, d, V = _dims(H_t, W)
+    assert H_d.shape == H_t.shape and H_d.dtype == torch.bfloat16 and H_d.is_contiguous()
+    assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
+    dev = H_t.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    if out is None:
+        out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+                   topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+                   topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+                   lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+                   lse_d=torch.empty(N, dtype=torch.float32, device=dev),
+                   dH_d=torch.empty(N, d, dtype=_dh_dtype(dH_dtype), device=dev))
+    out["workspace"] = ws
+    _ok(lib.hass_topk_distill_fwd_bwd(_p(H_t), _p(H_d), _p(W), N, d, V, K, _p(grad_loss), _p(out["loss"]),
+                                      _p(out["topk_idx"]), _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]),
+                                      _p(out["dH_d"]), dH_dtype, _p(ws), ws.numel(), _stream(stream)),
+        "hass_topk_distill_fwd_bwd")
+    return out
+
+
+def topk_distill_fwd_bwd_host(H_t_host, H_d_host, W, K: int, loss_host, dH_d_host, grad_loss_host=None,
+                              topk_idx_host=None, topk_q_host=None, dH_dtype: int = HASS_BF16, workspace=None,
+                              stream=None) -> None:
+    """H_t_host, H_d_host and the *_host outputs are CPU tensors (pinned for asynchronous copies);
+    W and the workspace are CUDA tensors. Returns once the host outputs are valid."""
+    assert not H_t_host.is_cuda and not H_d_host.is_cuda and W.is_cuda
+    N, d, V = _dims(H_t_host, W)
+    assert H_d_host.shape == H_t_host.shape and H_d_host.dtype == torch.bfloat16 and H_d_host.is_contiguous()
+    assert loss_host.dtype == torch.float32 and loss_host.shape == (N,) and not loss_host.is_cuda
+    assert dH_d_host.dtype == _dh_dtype(dH_dtype) and dH_d_host.shape == (N, d) and dH_d_host.is_contiguous()
+    ws = _workspace(workspace, topk_distill_host_workspace_bytes(N, d, V, K, dH_dtype), W.device)
+    _ok(lib.hass_topk_distill_fwd_bwd_host(_p(H_t_host), _p(H_d_host), _p(W), N, d, V, K, _p(grad_loss_host),
+                                           _p(loss_host), _p(topk_idx_host), _p(topk_q_host), _p(dH_d_host),
+                                           dH_dtype, _p(ws), ws.numel(), _stream(stream)),
+        "hass_topk_distill_fwd_bwd_host")
+
+
+def check(workspace: torch.Tensor, stream=None) -> None:
+    """Synchronises the stream and raises HassError if a kernel recorded a device-side problem."""
+    _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")

@@ -1,0 +1,603 @@
+// Host side of the C ABI declared in include/hass.h: argument checks, tile schedules, TMA
+// descriptors, workspace layout and kernel launches. No allocation, no synchronisation except in
+// hass_check and the *_host entry.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "../../include/hass.h"
+#include "kernels.cuh"
+
+namespace hass {
+
+static std::atomic<long long> g_launches{0};
+
+// ---- device info ------------------------------------------------------------------------------
+struct DeviceInfo {
+    int ok = 0;   // 0 unknown, 1 usable, <0 hass_status
+    int sms = 148;
+};
+static DeviceInfo g_dev[64];
+
+static int device_info(DeviceInfo* out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    DeviceInfo& di = g_dev[dev];
+    if (di.ok == 0) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        if (major != 10) {
+            di.ok = HASS_ERR_ARCH;
+        } else {
+            di.sms = sms;
+            cudaError_t e0 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<MODE_PROBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) {
+                cudaGetLastError();
+                return HASS_ERR_CUDA;
+            }
+            di.ok = 1;
+        }
+    }
+    if (di.ok < 0) return di.ok;
+    *out = di;
+    return HASS_OK;
+}
+
+static int sm_count_or_default() {
+    DeviceInfo di;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return 148;
+    }
+    return device_info(&di) == HASS_OK ? di.sms : 148;
+}
+
+// ---- tile schedule ----------------------------------------------------------------------------
+// Splits RT row tiles into phases (G row tiles x S lanes, G * S <= sms) minimising the summed phase
+// durations ceil(CT / S), by dynamic programming over the number of row tiles already covered.
+static int plan_schedule(int RT, int CT, int sms, Schedule* out) {
+    if (RT < 1 || CT < 1 || sms < 1) return HASS_ERR_INVALID_ARG;
+    const int INF = 1 << 30;
+    std::vector<int> best(RT + 1, INF), nph(RT + 1, INF), choice(RT + 1, 0);
+    best[0] = 0;
+    nph[0] = 0;
+    for (int n = 1; n <= RT; ++n) {
+        for (int G = 1; G <= n && G <= sms; ++G) {
+            int S = sms / G;
+            if (S > CT) S = CT;
+            const int cost = best[n - G] + (CT + S - 1) / S;
+            const int ph = nph[n - G] + 1;
+            if (cost < best[n] || (cost == best[n] && ph < nph[n])) {
+                best[n] = cost;
+                nph[n] = ph;
+                choice[n] = G;
+            }
+        }
+    }
+    if (nph[RT] > MAX_PHASES) return HASS_ERR_UNSUPPORTED;
+    std::vector<int> groups;
+    for (int n = RT; n > 0; n -= choice[n]) groups.push_back(choice[n]);
+    std::memset(out, 0, sizeof(*out));
+    int rt = 0, slot = 0, maxc = 0;
+    // largest groups first: the widest phases start together
+    for (size_t i = 0; i < groups.size(); ++i)
+        for (size_t j = i + 1; j < groups.size(); ++j)
+            if (groups[j] > groups[i]) std::swap(groups[i], groups[j]);
+    for (size_t i = 0; i < groups.size(); ++i) {
+        const int G = groups[i];
+        int S = sms / G;
+        if (S > CT) S = CT;
+        out->ph[i] = Phase{rt, G, S, slot};
+        rt += G;
+        slot += G * S;
+        if (G * S > maxc) maxc = G * S;
+    }
+    out->n_phases = static_cast<int>(groups.size());
+    out->total_slots = slot;
+    out->max_ctas = maxc;
+    return HASS_OK;
+}
+
+// ---- TMA descriptors --------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+static int get_encode() {
+    if (g_encode) return HASS_OK;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return HASS_OK;
+}
+
+// bf16 row-major matrix [rows, cols] with `pitch` elements between rows; box = box_cols x box_rows,
+// 128-byte swizzle (box_cols must be 64), out-of-range elements read as zero.
+static int make_tmap(CUtensorMap* tm, const void* base, long long rows, long long cols, long long pitch,
+                     int box_cols, int box_rows) {
+    cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    cuuint64_t gstride[1] = {static_cast<cuuint64_t>(pitch) * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HASS_OK : HASS_ERR_CUDA;
+}
+
+// ---- workspace layout -------------------------------------------------------------------------
+static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+struct Layout {
+    size_t status, part_m, part_s, cand_v, cand_i, sidx, sgq, coef, lse2, scratch, fixed_end;
+    size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
+    long long p_pitch;
+    int pref_chunk_tiles;
+    size_t total_pref;
+};
+
+static int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
+
+// The forward schedule covers 2 * RT row tiles (target then draft).
+static int make_layout(long long N, long long d, long long V, int K, int sms, Layout* L, Schedule* fwd_sched) {
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
+    Schedule s;
+    int rc = plan_schedule(2 * RT, CT, sms, &s);
+    if (rc != HASS_OK) return rc;
+    if (fwd_sched) *fwd_sched = s;
+    size_t off = 0;
+    L->status = off;
+    off += 256;
+    const size_t slots = static_cast<size_t>(s.total_slots);
+    L->part_m = off;
+    off = align256(off + slots * BM * 4);
+    L->part_s = off;
+    off = align256(off + slots * BM * 4);
+    L->cand_v = off;
+    off = align256(off + slots * BM * 4 * K);
+    L->cand_i = off;
+    off = align256(off + slots * BM * 4 * K);
+    L->sidx = off;
+    off = align256(off + static_cast<size_t>(N) * K * 4);
+    L->sgq = off;
+    off = align256(off + static_cast<size_t>(N) * K * 4);
+    L->coef = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    L->lse2 = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    L->scratch = off;
+    L->fixed_end = off;
+    L->p_pitch = static_cast<long long>(CT) * BN;
+    L->scratch_row_tile_bytes = static_cast<size_t>(BM) * L->p_pitch * 2;
+    int pref = sms / 4;
+    if (pref < 1) pref = 1;
+    if (pref > RT) pref = RT;
+    L->pref_chunk_tiles = pref;
+    L->total_pref = off + L->scratch_row_tile_bytes * pref;
+    return HASS_OK;
+}
+
+// ---- argument checks --------------------------------------------------------------------------
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_sizes(long long N, long long d, long long V, int K) {
+    if (N < 1 || d < 8 || V < 1 || K < 1) return HASS_ERR_INVALID_ARG;
+    if (d % 8 != 0) return HASS_ERR_INVALID_ARG;
+    if (K > V || K > HASS_K_MAX) return HASS_ERR_INVALID_ARG;
+    if (N > (1ll << 30) || V > (1ll << 30) || d > (1ll << 20)) return HASS_ERR_UNSUPPORTED;
+    return HASS_OK;
+}
+
+static const bool kLog = [] {
+    const char* e = std::getenv("HASS_LOG");
+    return e && e[0] == '1';
+}();
+
+static void log_schedule(const char* what, const Schedule& s) {
+    if (!kLog) return;
+    std::fprintf(stderr, "[hass] %s: %d phases, %d slots, grid %d:", what, s.n_phases, s.total_slots, s.max_ctas);
+    for (int i = 0; i < s.n_phases; ++i)
+        std::fprintf(stderr, " (rt0=%d G=%d S=%d)", s.ph[i].row_tile_begin, s.ph[i].G, s.ph[i].S);
+    std::fprintf(stderr, "\n");
+}
+
+template <int MODE>
+static int launch_gemm(const GemmParams& p, cudaStream_t st) {
+    gemm_kernel<MODE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
+}
+
+// ---- forward ----------------------------------------------------------------------------------
+// with_target: both projections + Omega_hat selection; otherwise draft only with Omega_hat given.
+static int forward_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
+                        long long V, int K, const int* idx_in, const float* q_in, float* loss, int* idx_out,
+                        float* q_out, float* lse_t, float* lse_d, void* workspace, size_t workspace_bytes,
+                        cudaStream_t st) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_d || !W || !loss || !lse_d || !aligned16(H_d) || !aligned16(W)) return HASS_ERR_INVALID_ARG;
+    if (with_target && (!H_t || !idx_out || !q_out || !lse_t || !aligned16(H_t))) return HASS_ERR_INVALID_ARG;
+    if (!with_target && (!idx_in || !q_in)) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+
+    Layout L;
+    Schedule full;
+    rc = make_layout(N, d, V, K, di.sms, &L, &full);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.fixed_end) return HASS_ERR_WORKSPACE;
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    // every public call starts with a clean status word
+    if (cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    if (with_target) {
+        p.sched = full;
+        p.row_tiles0 = RT;
+        p.topk_row_tiles = RT;
+        rc = make_tmap(&p.tmA0, H_t, N, d, d, BK, BM);
+        if (rc == HASS_OK) rc = make_tmap(&p.tmA1, H_d, N, d, d, BK, BM);
+    } else {
+        rc = plan_schedule(RT, CT, di.sms, &p.sched);   // never needs more slots than the full schedule
+        if (rc != HASS_OK) return rc;
+        if (p.sched.total_slots > full.total_slots) return HASS_ERR_WORKSPACE;
+        p.row_tiles0 = RT;
+        p.topk_row_tiles = 0;
+        rc = make_tmap(&p.tmA0, H_d, N, d, d, BK, BM);
+        if (rc == HASS_OK) rc = make_tmap(&p.tmA1, H_d, N, d, d, BK, BM);
+    }
+    if (rc == HASS_OK) rc = make_tmap(&p.tmB, W, V, d, d, BK, BN);
+    if (rc != HASS_OK) return rc;
+    log_schedule(with_target ? "fwd stats" : "fwd stats (draft)", p.sched);
+    p.a_row_offset = 0;
+    p.row_global_offset = 0;
+    p.rows_valid = static_cast<int>(N);
+    p.n_cols = static_cast<int>(V);
+    p.col_tiles = CT;
+    p.k_blocks = ceil_div(d, BK);
+    p.K = K;
+    p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+    p.part_s = reinterpret_cast<float*>(ws + L.part_s);
+    p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
+    p.cand_i = reinterpret_cast<int*>(ws + L.cand_i);
+    p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    rc = launch_gemm<MODE_STATS>(p, st);
+    if (rc != HASS_OK) return rc;
+
+    FinalizeParams f;
+    std::memset(&f, 0, sizeof(f));
+    f.sched = p.sched;
+    f.N = static_cast<int>(N);
+    f.d = static_cast<int>(d);
+    f.K = K;
+    f.row_tiles_t = with_target ? RT : 0;
+    f.part_m = p.part_m;
+    f.part_s = p.part_s;
+    f.cand_v = p.cand_v;
+    f.cand_i = p.cand_i;
+    f.H_d = static_cast<const __nv_bfloat16*>(H_d);
+    f.W = static_cast<const __nv_bfloat16*>(W);
+    f.idx_in = idx_in;
+    f.q_in = q_in;
+    f.loss = loss;
+    f.idx_out = idx_out;
+    f.q_out = q_out;
+    f.lse_t = lse_t;
+    f.lse_d = lse_d;
+    const int warps_per_block = 8;
+    finalize_kernel<<<ceil_div(N, warps_per_block), warps_per_block * 32, 0, st>>>(f);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
+}
+
+// ---- backward ---------------------------------------------------------------------------------
+static int backward_impl(const void* H_d, const void* W, long long N, long long d, long long V, int K,
+                         const int* topk_idx, const float* topk_q, const float* lse_d, const float* grad_loss,
+                         void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                         bool clear_status) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_d || !W || !topk_idx || !topk_q || !lse_d || !dH_d) return HASS_ERR_INVALID_ARG;
+    if (!aligned16(H_d) || !aligned16(W) || !aligned16(dH_d)) return HASS_ERR_INVALID_ARG;
+    if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.fixed_end + L.scratch_row_tile_bytes) return HASS_ERR_WORKSPACE;
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN), DT = ceil_div(d, BN);
+    long long fit = static_cast<long long>((workspace_bytes - L.fixed_end) / L.scratch_row_tile_bytes);
+    int chunk_tiles = L.pref_chunk_tiles;
+    if (fit < chunk_tiles) chunk_tiles = static_cast<int>(fit);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* sidx = reinterpret_cast<int*>(ws + L.sidx);
+    float* sgq = reinterpret_cast<float*>(ws + L.sgq);
+    float* coef = reinterpret_cast<float*>(ws + L.coef);
+    float* lse2 = reinterpret_cast<float*>(ws + L.lse2);
+    __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(ws + L.scratch);
+    if (clear_status && cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+
+    bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss, sidx,
+                                                       sgq, coef, lse2);
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+
+    CUtensorMap tmHd, tmWk, tmWn, tmP;
+    rc = make_tmap(&tmHd, H_d, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = make_tmap(&tmWk, W, V, d, d, BK, BN);      // B of z_d = H_d W^T: K-major
+    if (rc == HASS_OK) rc = make_tmap(&tmWn, W, V, d, d, 64, BK);      // B of dH_d = dz_d W: MN-major boxes
+    if (rc == HASS_OK) rc = make_tmap(&tmP, P, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
+    if (rc != HASS_OK) return rc;
+
+    for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
+        const int tiles = (RT - t0 < chunk_tiles) ? RT - t0 : chunk_tiles;
+        // (1) dz_d tiles of this chunk of rows -> scratch
+        GemmParams p;
+        std::memset(&p, 0, sizeof(p));
+        rc = plan_schedule(tiles, CT, di.sms, &p.sched);
+        if (rc != HASS_OK) return rc;
+        log_schedule("bwd dz_d", p.sched);
+        p.tmA0 = tmHd;
+        p.tmA1 = tmHd;
+        p.tmB = tmWk;
+        p.row_tiles0 = tiles;
+        p.a_row_offset = t0 * BM;
+        p.row_global_offset = t0 * BM;
+        p.rows_valid = static_cast<int>(N);
+        p.n_cols = static_cast<int>(V);
+        p.col_tiles = CT;
+        p.k_blocks = ceil_div(d, BK);
+        p.K = K;
+        p.lse2 = lse2;
+        p.coef = coef;
+        p.sidx = sidx;
+        p.sgq = sgq;
+        p.P = P;
+        p.p_pitch = L.p_pitch;
+        p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+        rc = launch_gemm<MODE_PROBS>(p, st);
+        if (rc != HASS_OK) return rc;
+        // (2) dH_d rows of this chunk = dz_d chunk x W
+        GemmParams o;
+        std::memset(&o, 0, sizeof(o));
+        rc = plan_schedule(tiles, DT, di.sms, &o.sched);
+        if (rc != HASS_OK) return rc;
+        log_schedule("bwd dH_d", o.sched);
+        o.tmA0 = tmP;
+        o.tmA1 = tmP;
+        o.tmB = tmWn;
+        o.row_tiles0 = tiles;
+        o.a_row_offset = 0;
+        o.row_global_offset = t0 * BM;
+        o.rows_valid = static_cast<int>(N);
+        o.n_cols = static_cast<int>(d);
+        o.col_tiles = DT;
+        o.k_blocks = ceil_div(V, BK);
+        o.K = K;
+        o.out = dH_d;
+        o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+        o.out_pitch = d;
+        o.status = p.status;
+        rc = launch_gemm<MODE_OUT>(o, st);
+        if (rc != HASS_OK) return rc;
+    }
+    return HASS_OK;
+}
+
+}  // namespace hass
+
+using namespace hass;
+
+extern "C" {
+
+const char* hass_status_string(int status) {
+    switch (status) {
+        case HASS_OK: return "HASS_OK";
+        case HASS_ERR_INVALID_ARG: return "HASS_ERR_INVALID_ARG";
+        case HASS_ERR_UNSUPPORTED: return "HASS_ERR_UNSUPPORTED";
+        case HASS_ERR_WORKSPACE: return "HASS_ERR_WORKSPACE";
+        case HASS_ERR_CUDA: return "HASS_ERR_CUDA";
+        case HASS_ERR_TIMEOUT: return "HASS_ERR_TIMEOUT";
+        case HASS_ERR_ARCH: return "HASS_ERR_ARCH";
+        default: return "HASS_ERR_UNKNOWN";
+    }
+}
+
+int hass_version(void) { return 100; }
+
+int64_t hass_kernel_launch_count(void) { return g_launches.load(); }
+
+int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes) {
+    if (!bytes) return HASS_ERR_INVALID_ARG;
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    Layout L;
+    rc = make_layout(N, d, V, K, sm_count_or_default(), &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    *bytes = L.total_pref;
+    return HASS_OK;
+}
+
+int hass_topk_distill_fwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
+                          float* loss, int32_t* topk_idx, float* topk_q, float* lse_t, float* lse_d, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
+    return forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
+                        workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int hass_topk_distill_fwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
+                                const int32_t* topk_idx, const float* topk_q, float* loss, float* lse_d,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return forward_impl(false, nullptr, H_d, W, N, d, V, K, topk_idx, topk_q, loss, nullptr, nullptr, nullptr, lse_d,
+                        workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
+                          const int32_t* topk_idx, const float* topk_q, const float* lse_d, const float* grad_loss,
+                          void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return backward_impl(H_d, W, N, d, V, K, topk_idx, topk_q, lse_d, grad_loss, dH_d, dH_dtype, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream), true);
+}
+
+int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                              int32_t K, const float* grad_loss, float* loss, int32_t* topk_idx, float* topk_q,
+                              float* lse_t, float* lse_d, void* dH_d, int dH_dtype, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+    // validate the backward's own arguments before anything is launched
+    if (!dH_d || !aligned16(dH_d) || (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32)) return HASS_ERR_INVALID_ARG;
+    int rc = forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
+                          workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+    if (rc != HASS_OK) return rc;
+    return backward_impl(H_d, W, N, d, V, K, topk_idx, topk_q, lse_d, grad_loss, dH_d, dH_dtype, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream), false);
+}
+
+// Device staging appended to the normal workspace by the *_host entry.
+struct HostStage {
+    size_t H_t, H_d, grad, loss, idx, q, lse_t, lse_d, dH, total;
+};
+static int host_stage(int64_t N, int64_t d, int64_t V, int32_t K, int dH_dtype, size_t base, HostStage* s) {
+    size_t off = align256(base);
+    s->H_t = off;
+    off = align256(off + static_cast<size_t>(N) * d * 2);
+    s->H_d = off;
+    off = align256(off + static_cast<size_t>(N) * d * 2);
+    s->grad = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    s->loss = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    s->idx = off;
+    off = align256(off + static_cast<size_t>(N) * K * 4);
+    s->q = off;
+    off = align256(off + static_cast<size_t>(N) * K * 4);
+    s->lse_t = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    s->lse_d = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    s->dH = off;
+    off = align256(off + static_cast<size_t>(N) * d * (dH_dtype == HASS_FP32 ? 4 : 2));
+    s->total = off;
+    (void)V;
+    return HASS_OK;
+}
+
+int hass_topk_distill_host_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, int dH_dtype, size_t* bytes) {
+    if (!bytes || (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32)) return HASS_ERR_INVALID_ARG;
+    size_t base = 0;
+    int rc = hass_topk_distill_workspace_bytes(N, d, V, K, &base);
+    if (rc != HASS_OK) return rc;
+    HostStage s;
+    host_stage(N, d, V, K, dH_dtype, base, &s);
+    *bytes = s.total;
+    return HASS_OK;
+}
+
+int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, const void* W, int64_t N, int64_t d,
+                                   int64_t V, int32_t K, const float* grad_loss_host, float* loss_host,
+                                   int32_t* topk_idx_host, float* topk_q_host, void* dH_d_host, int dH_dtype,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_t_host || !H_d_host || !W || !loss_host || !dH_d_host) return HASS_ERR_INVALID_ARG;
+    if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    size_t base = 0;
+    rc = hass_topk_distill_workspace_bytes(N, d, V, K, &base);
+    if (rc != HASS_OK) return rc;
+    HostStage s;
+    host_stage(N, d, V, K, dH_dtype, base, &s);
+    if (workspace_bytes < s.total) return HASS_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const size_t hbytes = static_cast<size_t>(N) * d * 2;
+    if (cudaMemcpyAsync(ws + s.H_t, H_t_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ws + s.H_d, H_d_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    const float* grad_dev = nullptr;
+    if (grad_loss_host) {
+        if (cudaMemcpyAsync(ws + s.grad, grad_loss_host, static_cast<size_t>(N) * 4, cudaMemcpyHostToDevice, st) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        grad_dev = reinterpret_cast<const float*>(ws + s.grad);
+    }
+    rc = hass_topk_distill_fwd_bwd(ws + s.H_t, ws + s.H_d, W, N, d, V, K, grad_dev, reinterpret_cast<float*>(ws + s.loss),
+                                   reinterpret_cast<int32_t*>(ws + s.idx), reinterpret_cast<float*>(ws + s.q),
+                                   reinterpret_cast<float*>(ws + s.lse_t), reinterpret_cast<float*>(ws + s.lse_d),
+                                   ws + s.dH, dH_dtype, workspace, base, st);
+    if (rc != HASS_OK) return rc;
+    bool ok = cudaMemcpyAsync(loss_host, ws + s.loss, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dH_d_host, ws + s.dH, static_cast<size_t>(N) * d * (dH_dtype == HASS_FP32 ? 4 : 2),
+                               cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (topk_idx_host)
+        ok = ok && cudaMemcpyAsync(topk_idx_host, ws + s.idx, static_cast<size_t>(N) * K * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (topk_q_host)
+        ok = ok && cudaMemcpyAsync(topk_q_host, ws + s.q, static_cast<size_t>(N) * K * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    return hass_check(workspace, cuda_stream);
+}
+
+int hass_check(void* workspace, void* cuda_stream) {
+    if (!workspace) return HASS_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    unsigned int word = 0;
+    if (cudaMemcpy(&word, workspace, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    if (word != 0) {
+        cudaMemset(workspace, 0, 4);
+        if (kLog) std::fprintf(stderr, "[hass] device status word 0x%x\n", word);
+        return HASS_ERR_TIMEOUT;
+    }
+    return HASS_OK;
+}
+
+}  // extern "C"

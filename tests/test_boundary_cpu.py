@@ -1,0 +1,77 @@
+"""Host-side checks that need no GPU: the library loads, exports what include/hass.h declares,
+rejects bad arguments before touching the device, and sizes its workspace sensibly."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def hass():
+    from paper_2408_15766_b200 import build
+    build.build_library()
+    import paper_2408_15766_b200 as h
+    return h
+
+
+def test_every_declared_symbol_is_exported(hass):
+    header = open(os.path.join(ROOT, "include", "hass.h")).read()
+    names = set(re.findall(r"\b(hass_[a-z_0-9]+)\s*\(", header))
+    assert {"hass_topk_distill_fwd", "hass_topk_distill_bwd", "hass_topk_distill_fwd_bwd"} <= names
+    for n in names:
+        assert hasattr(hass.lib, n), n
+
+
+def test_status_strings_and_version(hass):
+    assert hass.status_string(0) == "HASS_OK"
+    assert hass.status_string(-5) == "HASS_ERR_TIMEOUT"
+    assert hass.version() >= 100
+
+
+def test_workspace_bytes_is_bounded_in_N(hass):
+    a = hass.topk_distill_workspace_bytes(8192, 4096, 128256, 10)
+    b = hass.topk_distill_workspace_bytes(65536, 4096, 128256, 10)
+    scratch = 37 * 128 * 128256 * 2          # one chunk of dz_d rows, independent of N
+    assert scratch <= a < scratch + (64 << 20)
+    assert b - a < (256 << 20)               # grows only by O(N K) lists and partial statistics
+    assert a < 8192 * 128256 * 2             # less than one N x V bf16 matrix
+
+
+@pytest.mark.parametrize("N,d,V,K", [(0, 64, 64, 1), (4, 12, 64, 1), (4, 64, 64, 65), (4, 64, 64, 0),
+                                     (4, 64, 1000, 129), (4, 0, 64, 1)])
+def test_bad_sizes_rejected_without_a_device(hass, N, d, V, K):
+    out = ctypes.c_size_t(0)
+    rc = hass.lib.hass_topk_distill_workspace_bytes(N, d, V, K, ctypes.byref(out))
+    assert rc == -1
+    buf = ctypes.create_string_buffer(64)
+    p = ctypes.cast(buf, ctypes.c_void_p)
+    rc = hass.lib.hass_topk_distill_fwd(p, p, p, N, d, V, K, p, p, p, p, p, p, 1 << 20, None)
+    assert rc == -1
+
+
+def test_null_and_misaligned_pointers_rejected(hass):
+    buf = ctypes.create_string_buffer(4096)
+    base = ctypes.addressof(buf)
+    al = ctypes.c_void_p((base + 255) & ~255)
+    mis = ctypes.c_void_p(al.value + 2)
+    f = hass.lib.hass_topk_distill_fwd
+    assert f(None, al, al, 4, 64, 64, 2, al, al, al, al, al, al, 1 << 20, None) == -1
+    assert f(mis, al, al, 4, 64, 64, 2, al, al, al, al, al, al, 1 << 20, None) == -1
+    assert f(al, al, al, 4, 64, 64, 2, al, al, al, al, al, None, 1 << 20, None) == -3
+    assert f(al, al, al, 4, 64, 64, 2, al, al, al, al, al, mis, 1 << 20, None) == -3
+    b = hass.lib.hass_topk_distill_bwd
+    assert b(al, al, 4, 64, 64, 2, al, al, al, None, al, 7, al, 1 << 20, None) == -1
+    assert b(al, al, 4, 64, 64, 2, None, al, al, None, al, 0, al, 1 << 20, None) == -1
+
+
+def test_no_device_is_an_error_not_a_fallback(hass):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    buf = ctypes.create_string_buffer(1 << 16)
+    al = ctypes.c_void_p((ctypes.addressof(buf) + 255) & ~255)
+    rc = hass.lib.hass_topk_distill_fwd(al, al, al, 4, 64, 64, 2, al, al, al, al, al, al, 1 << 15, None)
+    assert rc in (-4, -6)

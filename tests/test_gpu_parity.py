@@ -1,0 +1,157 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import hass_inputs as hi
+from parity import compare
+
+pytestmark = pytest.mark.gpu
+
+FULL_ROWS = int(os.environ.get("HASS_ORACLE_ROWS", "192"))
+
+
+def _hass():
+    import paper_2408_15766_b200 as hass
+    return hass
+
+
+def _to_cpu(out):
+    return {k: v.cpu() for k, v in out.items() if k != "workspace"}
+
+
+def _run_and_compare(inp, K, step=0, dH_dtype=None, grad_loss=None, rows=None):
+    hass = _hass()
+    dH_dtype = hass.HASS_BF16 if dH_dtype is None else dH_dtype
+    dev = torch.device("cuda:0")
+    H_t, H_d, W = inp.H_t.to(dev), inp.H_d[step].to(dev), inp.W.to(dev)
+    gl = None if grad_loss is None else torch.tensor(grad_loss, dtype=torch.float32, device=dev)
+    out = hass.topk_distill_fwd_bwd(H_t, H_d, W, K, grad_loss=gl, dH_dtype=dH_dtype)
+    hass.check(out["workspace"])
+    return compare(inp.H_t, inp.H_d[step], inp.W, K, _to_cpu(out), rows=rows, grad_loss=grad_loss), out
+
+
+def test_tiny_config_all_rows():
+    wl = hi.WORKLOADS["tiny"]
+    stats, _ = _run_and_compare(hi.make_inputs(wl), wl.K, dH_dtype=_hass().HASS_FP32)
+    print(stats)
+
+
+@pytest.mark.parametrize("N,d,V,K", [
+    (1, 64, 64, 1), (64, 256, 1000, 2), (127, 264, 1024, 10), (129, 64, 32003, 10),
+    (300, 256, 5000, 64), (200, 128, 777, 100), (130, 512, 300, 128), (5, 8, 9, 9),
+])
+def test_awkward_shapes(N, d, V, K):
+    inp = hi.make_custom(N, d, V, K, seed=N + V, sigma_w=0.5 / np.sqrt(d) * 4)
+    rng = np.random.default_rng(0)
+    grad = rng.normal(size=N)
+    grad[0] = 0.0
+    stats, _ = _run_and_compare(inp, K, dH_dtype=_hass().HASS_FP32, grad_loss=grad)
+    print(stats)
+
+
+def test_split_calls_match_fused_call_and_draft_only_forward():
+    hass = _hass()
+    wl = hi.Workload("mid", N=384, d=512, V=4096, K=10, steps=2)
+    inp = hi.make_inputs(wl)
+    dev = torch.device("cuda:0")
+    H_t, W = inp.H_t.to(dev), inp.W.to(dev)
+    H_d0, H_d1 = inp.H_d[0].to(dev), inp.H_d[1].to(dev)
+    fused = hass.topk_distill_fwd_bwd(H_t, H_d0, W, wl.K)
+    f = hass.topk_distill_fwd(H_t, H_d0, W, wl.K)
+    dH = hass.topk_distill_bwd(H_d0, W, f["topk_idx"], f["topk_q"], f["lse_d"], workspace=f["workspace"])
+    hass.check(f["workspace"])
+    for k in ("loss", "topk_idx", "topk_q", "lse_t", "lse_d"):
+        assert torch.equal(fused[k], f[k])
+    assert torch.equal(fused["dH_d"], dH)
+    # aligning step 2: target statistics reused, only the draft side recomputed
+    s2 = hass.topk_distill_fwd_draft(H_d1, W, f["topk_idx"], f["topk_q"], workspace=f["workspace"])
+    dH2 = hass.topk_distill_bwd(H_d1, W, f["topk_idx"], f["topk_q"], s2["lse_d"], workspace=f["workspace"])
+    hass.check(f["workspace"])
+    gpu = dict(loss=s2["loss"].cpu(), lse_d=s2["lse_d"].cpu(), lse_t=f["lse_t"].cpu(), topk_idx=f["topk_idx"].cpu(),
+               topk_q=f["topk_q"].cpu(), dH_d=dH2.cpu())
+    print(compare(inp.H_t, inp.H_d[1], inp.W, wl.K, gpu))
+
+
+def test_host_buffer_entry_matches_device_entry():
+    hass = _hass()
+    wl = hi.Workload("mid", N=200, d=256, V=3000, K=10)
+    inp = hi.make_inputs(wl)
+    dev = torch.device("cuda:0")
+    W = inp.W.to(dev)
+    ref = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), W, wl.K)
+    loss_h = torch.empty(wl.N, dtype=torch.float32).pin_memory()
+    dH_h = torch.empty(wl.N, wl.d, dtype=torch.bfloat16).pin_memory()
+    idx_h = torch.empty(wl.N, wl.K, dtype=torch.int32).pin_memory()
+    hass.topk_distill_fwd_bwd_host(inp.H_t.pin_memory(), inp.H_d[0].pin_memory(), W, wl.K, loss_h, dH_h,
+                                   topk_idx_host=idx_h)
+    assert torch.equal(loss_h, ref["loss"].cpu())
+    assert torch.equal(dH_h, ref["dH_d"].cpu())
+    assert torch.equal(idx_h, ref["topk_idx"].cpu())
+
+
+def test_results_are_deterministic_run_to_run():
+    hass = _hass()
+    inp = hi.make_custom(500, 256, 9000, 10, seed=5, sigma_w=0.1)
+    dev = torch.device("cuda:0")
+    a = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), 10)
+    b = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), 10)
+    for k in ("loss", "topk_idx", "topk_q", "lse_t", "lse_d", "dH_d"):
+        assert torch.equal(a[k], b[k]), k
+
+
+def test_exact_ties_resolve_to_lower_token_id():
+    hass = _hass()
+    inp = hi.make_custom(70, 64, 600, 4, seed=9, sigma_w=0.2)
+    W = inp.W.clone()
+    W[300:600] = W[0:300]            # every logit appears twice: tokens v and v + 300
+    dev = torch.device("cuda:0")
+    out = hass.topk_distill_fwd(inp.H_t.to(dev), inp.H_d[0].to(dev), W.to(dev), 4)
+    hass.check(out["workspace"])
+    idx = out["topk_idx"].cpu().numpy()
+    assert np.all(idx[:, 1] == idx[:, 0] + 300) and np.all(idx[:, 3] == idx[:, 2] + 300)
+    assert np.all(idx[:, 0] < 300) and np.all(idx[:, 2] < 300)
+    print(compare(inp.H_t, inp.H_d[0], W, 4, _to_cpu(out) | {"dH_d": None}, check_dH=False))
+
+
+@pytest.mark.parametrize("name", ["l2-7b", "l3-8b"])
+def test_full_size_config_sampled_rows(name):
+    wl = hi.WORKLOADS[name]
+    inp = hi.make_inputs(wl)
+    rows = hi.sample_rows(wl.N, FULL_ROWS, seed=wl.seed)
+    stats, _ = _run_and_compare(inp, wl.K, rows=rows)
+    print(name, stats)
+
+
+def test_l2_13b_three_aligning_steps_sampled_rows():
+    hass = _hass()
+    wl = hi.WORKLOADS["l2-13b"]
+    inp = hi.make_inputs(wl)
+    rows = hi.sample_rows(wl.N, max(FULL_ROWS // 3, 32), seed=wl.seed)
+    dev = torch.device("cuda:0")
+    H_t, W = inp.H_t.to(dev), inp.W.to(dev)
+    first = None
+    for step in range(wl.steps):
+        H_d = inp.H_d[step].to(dev)
+        if step == 0:
+            out = hass.topk_distill_fwd_bwd(H_t, H_d, W, wl.K)
+            first = out
+        else:
+            s = hass.topk_distill_fwd_draft(H_d, W, first["topk_idx"], first["topk_q"], workspace=first["workspace"])
+            dH = hass.topk_distill_bwd(H_d, W, first["topk_idx"], first["topk_q"], s["lse_d"],
+                                       workspace=first["workspace"])
+            out = dict(loss=s["loss"], lse_d=s["lse_d"], lse_t=first["lse_t"], topk_idx=first["topk_idx"],
+                       topk_q=first["topk_q"], dH_d=dH)
+        hass.check(first["workspace"])
+        print("step", step, compare(inp.H_t, inp.H_d[step], inp.W, wl.K, _to_cpu(out), rows=rows))
+
+
+@pytest.mark.parametrize("K", [1, 10, 64])
+def test_l3_70b_k_sweep_sampled_rows(K):
+    wl = hi.WORKLOADS["l3-70b"]
+    inp = hi.make_inputs(wl)
+    rows = hi.sample_rows(wl.N, max(FULL_ROWS // 3, 32), seed=wl.seed)
+    stats, _ = _run_and_compare(inp, K, rows=rows)
+    print("l3-70b K", K, stats)
