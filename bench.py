@@ -1,0 +1,334 @@
+#!/usr/bin/env python
+"""Benchmark of the fused LM-head + Top-K distillation forward+backward (one aligning step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload l3-8b] [--impl reference]
+
+One "step" is one pass of the whole hot path (target and draft projections, softmax statistics,
+Top-K selection, Eq. 1 loss, dz_d and the back-projection to dH_d) over one batch of synthetic
+bf16 inputs of the named shape. Rows are independent, so with N > 1 GPUs every rank processes
+its own batch (weak scaling, no collective on the data path); `value` is the total tokens/s.
+
+Prints ONE JSON line (rank 0). Timing: CUDA events on the launching stream around exactly
+`steps` steps after `warmup` untimed ones, barrier + synchronize on both sides, max over ranks.
+The inputs (W alone is larger than L2) make every step start cold in L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import hass_inputs as hi  # noqa: E402
+
+METRIC = "tokens/sec fused top-K distill fwd+bwd"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---- clock sampling --------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()          # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(pw)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---- multi-rank plumbing ----------------------------------------------------------------------------
+def dist_setup(n_gpus: int):
+    """Returns (rank, world, local_rank). One process per GPU when launched by torch.distributed.run."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world == 1:
+        return 0, 1, 0
+    import torch.distributed as dist
+    rank = int(os.environ["RANK"])
+    local = int(os.environ.get("LOCAL_RANK", rank))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    backend = "nccl" if torch.cuda.is_available() else "gloo"
+    if backend == "nccl":
+        torch.cuda.set_device(local)
+    dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world, local
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """Whole-job time = the slowest rank's device time."""
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate(tokens_per_rank: int, world: int, ms_per_step_max: float) -> float:
+    """tokens/s of the whole job: all ranks' tokens over the slowest rank's time."""
+    return tokens_per_rank * world / (ms_per_step_max * 1e-3)
+
+
+# ---- CPU baseline (the oracle as it stands) ---------------------------------------------------------
+def time_oracle(inp, K: int, n_rows: int, seed: int = 0):
+    import oracle
+    rows = hi.sample_rows(inp.wl.N, n_rows, seed=seed)
+    Hb_t, Hb_d, Wb = hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W)
+    t0 = time.perf_counter()
+    oracle.from_features(Hb_t, Hb_d, Wb, K, rows=rows, want_dH=True)
+    dt = time.perf_counter() - t0
+    return rows.shape[0] / dt, dt, int(rows.shape[0]), oracle.threads()
+
+
+def run_reference(args, rank: int, world: int):
+    """--impl reference: the fp64 CPU oracle, untuned, on the host cores; each step is a bounded
+    sample of rows of the same workload. Rank 0 only."""
+    if rank != 0:
+        return
+    wl = hi.WORKLOADS[args.workload]
+    inp = hi.make_inputs(wl)
+    import oracle
+    oracle.build()
+    rows_per_step = args.oracle_rows
+    vals = []
+    for i in range(args.warmup + args.steps):
+        tps, dt, n, cores = time_oracle(inp, wl.K, rows_per_step, seed=i)
+        if i >= args.warmup:
+            vals.append((tps, dt))
+    tps = float(np.mean([v[0] for v in vals]))
+    ms = float(np.mean([v[1] for v in vals]) * 1e3)
+    sample = f"{rows_per_step} of {wl.N} rows per step (head, tail and seeded random rows), all {wl.V} tokens"
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "V": wl.V, "K": wl.K,
+                       "note": "fp64 CPU oracle on a row sample; rows are independent"},
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---- main --------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--K", type=int, default=None)
+    ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank, world, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        if args.oracle_rows is None:
+            args.oracle_rows = 64
+        run_reference(args, rank, world)
+        return
+
+    import paper_2408_15766_b200 as hass   # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    wl = hi.WORKLOADS[args.workload]
+    K = args.K or wl.K
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = load_peaks()
+
+    inp = hi.make_inputs(wl)
+    N, d, V = wl.N, wl.d, wl.V
+    H_t, H_d, W = inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev)
+    ws = torch.empty(hass.topk_distill_host_workspace_bytes(N, d, V, K), dtype=torch.uint8, device=dev)
+    out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+               topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+               topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+               lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+               lse_d=torch.empty(N, dtype=torch.float32, device=dev),
+               dH_d=torch.empty(N, d, dtype=torch.bfloat16, device=dev))
+    stream = torch.cuda.current_stream()
+
+    def step():
+        hass.topk_distill_fwd_bwd(H_t, H_d, W, K, workspace=ws, out=out, stream=stream)
+
+    # ---- device-resident timing ----
+    for _ in range(args.warmup):
+        step()
+    hass.check(ws)
+    barrier(world)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    hass.profile_enable(True)
+    launches0 = hass.kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    launches = hass.kernel_launch_count() - launches0
+    prof = hass.profile_summary()
+    hass.profile_enable(False)
+    clocks = sampler.stop()
+    hass.check(ws)
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
+    value = aggregate(N, world, ms_step)
+
+    # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        Ht_h, Hd_h = inp.H_t.pin_memory(), inp.H_d[0].pin_memory()
+        loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
+        dH_h = torch.empty(N, d, dtype=torch.bfloat16).pin_memory()
+        for _ in range(3):
+            hass.topk_distill_fwd_bwd_host(Ht_h, Hd_h, W, K, loss_h, dH_h, workspace=ws, stream=stream)
+        barrier(world)
+        torch.cuda.synchronize()
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            hass.topk_distill_fwd_bwd_host(Ht_h, Hd_h, W, K, loss_h, dH_h, workspace=ws, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1) / n_e2e, world, dev)
+        e2e = {"value": aggregate(N, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": 2 * N * d * 2, "d2h_bytes_per_step": N * 4 + N * d * 2,
+               "note": "H_t, H_d from pinned host memory; loss and dH_d back to host; frozen LM head W resident"}
+
+    if rank != 0:
+        return
+
+    # ---- roofline of the dominant kernel (tensor-core bound) ----
+    flops_credit = 6.0 * N * d * V                 # three d x V products per token
+    kinds = {"stats_gemm": 4.0 * N * d * V, "dz_gemm": 2.0 * N * d * V, "dH_gemm": 2.0 * N * d * V}
+    total_ms = sum(v[0] for v in prof.values())
+    kernel_rows = {}
+    for k, (ms, cnt) in prof.items():
+        if cnt:
+            kernel_rows[k] = {"ms_per_step": ms / args.steps, "launches_per_step": cnt / args.steps,
+                              "share": ms / total_ms if total_ms else None}
+            if k in kinds:
+                kernel_rows[k]["tflops"] = kinds[k] / (ms / args.steps * 1e-3) / 1e12
+    dom = max(kinds, key=lambda k: prof[k][0])
+    dom_ms, dom_cnt = prof[dom]
+    flops_per_launch = kinds[dom] * args.steps / dom_cnt
+    achieved = flops_per_launch / (dom_ms / dom_cnt * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops_sustained"])
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_kind": f"bf16_tflops_sustained, of {peak_kind} (kernel timed inside a long step)",
+                "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
+                "flops_per_launch": flops_per_launch, "avg_launch_ms": dom_ms / dom_cnt}
+    step_tflops = flops_credit / (ms_step * 1e-3) / 1e12
+    executed = sum(kinds.values())
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "N": N, "d": d, "V": V, "K": K, "rows_per_gpu": N,
+                       "l2": "inputs larger than L2 (W alone is %.0f MB)" % (V * d * 2 / 1e6),
+                       "dH_dtype": "bf16", "target_stats": "recomputed every step"},
+            "clocks": clocks, "gpu_launches": launches,
+            "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
+                       "executed_tflops": executed / (ms_step * 1e-3) / 1e12, "executed_flops_per_step": executed,
+                       "frac_of_burst_credited": step_tflops / float(peaks["bf16_tflops"]),
+                       "frac_of_sustained_credited": step_tflops / float(peaks["bf16_tflops_sustained"]),
+                       "frac_of_nominal_2250_credited": step_tflops / 2250.0, "peaks": peak_kind},
+            "kernels": kernel_rows, "roofline": roofline}
+    if e2e:
+        line["e2e"] = e2e
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload ----
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        oracle.build()
+        cores = oracle.threads()
+        n_rows = args.oracle_rows or max(16, min(N, int(16 * cores * (4096 * 128256) / (d * V))))
+        tps, dt, n, cores = time_oracle(inp, K, n_rows)
+        line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{n} of {N} rows (head, tail and seeded random rows), all {V} tokens, "
+                                          f"{dt:.1f} s"}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        import torch.distributed as dist
+        if dist.is_initialized():
+            dist.destroy_process_group()

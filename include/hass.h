@@ -166,6 +166,19 @@ int hass_check(void* workspace, void* cuda_stream);
  */
 int64_t hass_kernel_launch_count(void);
 
+/*
+ * Optional per-kernel timing for benchmarks (no counterpart in the paper). While enabled, each
+ * kernel launch of the library is bracketed by CUDA events on its stream (the events are created
+ * on the first enable). hass_profile_summary waits for the recorded events, adds the elapsed
+ * milliseconds and launch counts per kernel kind into arrays of at least HASS_PROFILE_KINDS
+ * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
+ * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation.
+ * At most 8192 launches are recorded between summaries. Not thread-safe.
+ */
+#define HASS_PROFILE_KINDS 5
+int hass_profile_enable(int on);
+int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
+
 #ifdef __cplusplus
 }
 #endif

@@ -13,6 +13,9 @@ from .binding import (  # noqa: F401
     check,
     kernel_launch_count,
     lib,
+    PROFILE_KINDS,
+    profile_enable,
+    profile_summary,
     status_string,
     topk_distill_bwd,
     topk_distill_fwd,

@@ -23,7 +23,7 @@ class HassError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(_LIB_PATH):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2408_15766_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python paper_2408_15766_b200/build.py` "
             "(needs nvcc with sm_100a support). There is no fallback path.")
     L = ctypes.CDLL(_LIB_PATH)
     vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
@@ -41,6 +41,10 @@ def _load() -> ctypes.CDLL:
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
     L.hass_check.argtypes = [vp, vp]
+    L.hass_profile_enable.argtypes = [ctypes.c_int]
+    L.hass_profile_enable.restype = ctypes.c_int
+    L.hass_profile_summary.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64), ctypes.c_int]
+    L.hass_profile_summary.restype = ctypes.c_int
     for name in ("hass_topk_distill_workspace_bytes", "hass_topk_distill_host_workspace_bytes",
                  "hass_topk_distill_fwd", "hass_topk_distill_fwd_draft", "hass_topk_distill_bwd",
                  "hass_topk_distill_fwd_bwd", "hass_topk_distill_fwd_bwd_host", "hass_check"):
@@ -196,3 +200,19 @@ def topk_distill_fwd_bwd_host(H_t_host, H_d_host, W, K: int, loss_host, dH_d_hos
 def check(workspace: torch.Tensor, stream=None) -> None:
     """Synchronises the stream and raises HassError if a kernel recorded a device-side problem."""
     _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")
+
+
+PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep")
+
+
+def profile_enable(on: bool) -> None:
+    _ok(lib.hass_profile_enable(1 if on else 0), "hass_profile_enable")
+
+
+def profile_summary() -> dict:
+    """{kind: (milliseconds, launches)} since the last summary / enable."""
+    n = len(PROFILE_KINDS)
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_int64 * n)()
+    _ok(lib.hass_profile_summary(ms, cnt, n), "hass_profile_summary")
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(PROFILE_KINDS)}

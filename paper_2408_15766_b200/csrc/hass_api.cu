@@ -14,6 +14,34 @@ namespace hass {
 
 static std::atomic<long long> g_launches{0};
 
+// ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
+// When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
+// summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, NUM_KINDS = 5 };
+constexpr int kMaxRecords = 8192;
+struct Profiler {
+    bool on = false;
+    int n = 0;
+    std::vector<cudaEvent_t> ev;     // 2 per record
+    std::vector<int> kind;
+};
+static Profiler g_prof;
+
+struct KernelTimer {
+    int rec = -1;
+    cudaStream_t st;
+    KernelTimer(int kind, cudaStream_t s) : st(s) {
+        if (g_prof.on && g_prof.n < kMaxRecords) {
+            rec = g_prof.n++;
+            g_prof.kind[rec] = kind;
+            cudaEventRecord(g_prof.ev[2 * rec], st);
+        }
+    }
+    ~KernelTimer() {
+        if (rec >= 0) cudaEventRecord(g_prof.ev[2 * rec + 1], st);
+    }
+};
+
 // ---- device info ------------------------------------------------------------------------------
 struct DeviceInfo {
     int ok = 0;   // 0 unknown, 1 usable, <0 hass_status
@@ -221,6 +249,7 @@ static void log_schedule(const char* what, const Schedule& s) {
 
 template <int MODE>
 static int launch_gemm(const GemmParams& p, cudaStream_t st) {
+    KernelTimer timer(MODE, st);
     gemm_kernel<MODE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
@@ -313,7 +342,10 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.lse_t = lse_t;
     f.lse_d = lse_d;
     const int warps_per_block = 8;
-    finalize_kernel<<<ceil_div(N, warps_per_block), warps_per_block * 32, 0, st>>>(f);
+    {
+        KernelTimer timer(KIND_FINALIZE, st);
+        finalize_kernel<<<ceil_div(N, warps_per_block), warps_per_block * 32, 0, st>>>(f);
+    }
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
 }
@@ -354,8 +386,11 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
         return HASS_ERR_CUDA;
     }
 
-    bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss, sidx,
-                                                       sgq, coef, lse2);
+    {
+        KernelTimer timer(KIND_PREP, st);
+        bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss,
+                                                           sidx, sgq, coef, lse2);
+    }
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
 
@@ -443,6 +478,45 @@ const char* hass_status_string(int status) {
 int hass_version(void) { return 100; }
 
 int64_t hass_kernel_launch_count(void) { return g_launches.load(); }
+
+int hass_profile_enable(int on) {
+    if (on && g_prof.ev.empty()) {
+        g_prof.ev.resize(2 * kMaxRecords);
+        g_prof.kind.resize(kMaxRecords);
+        for (auto& e : g_prof.ev)
+            if (cudaEventCreate(&e) != cudaSuccess) {
+                cudaGetLastError();
+                g_prof.ev.clear();
+                return HASS_ERR_CUDA;
+            }
+    }
+    g_prof.on = on != 0;
+    g_prof.n = 0;
+    return HASS_OK;
+}
+
+int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds) {
+    if (!ms_by_kind || !launches_by_kind || n_kinds < NUM_KINDS) return HASS_ERR_INVALID_ARG;
+    for (int k = 0; k < n_kinds; ++k) {
+        ms_by_kind[k] = 0.0;
+        launches_by_kind[k] = 0;
+    }
+    for (int r = 0; r < g_prof.n; ++r) {
+        if (cudaEventSynchronize(g_prof.ev[2 * r + 1]) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_prof.ev[2 * r], g_prof.ev[2 * r + 1]) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        ms_by_kind[g_prof.kind[r]] += ms;
+        launches_by_kind[g_prof.kind[r]] += 1;
+    }
+    g_prof.n = 0;
+    return HASS_OK;
+}
 
 int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes) {
     if (!bytes) return HASS_ERR_INVALID_ARG;

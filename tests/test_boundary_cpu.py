@@ -11,8 +11,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def hass():
-    from paper_2408_15766_b200 import build
-    build.build_library()
+    import sys
+    sys.path.insert(0, ROOT)
+    import __graft_entry__ as entry
+    entry.build()
     import paper_2408_15766_b200 as h
     return h
 
