@@ -167,6 +167,36 @@ int hass_check(void* workspace, void* cuda_stream);
 int64_t hass_kernel_launch_count(void);
 
 /*
+ * hass_topk_distill_fwd with no workspace argument. The paper has no counterpart to this entry:
+ * it exists for callers that cannot obtain device memory at the time of the call. Typical cases:
+ * a process whose framework reserved the whole GPU at start-up, so any later cudaMalloc fails; a
+ * plug-in interface that hands the callee its input and output buffers and nothing else; a
+ * latency-critical loop that must not run into the device-wide synchronisation cudaMalloc and
+ * cudaFree imply. For them the partial softmax statistics and Top-K candidates of the forward
+ * sweep live in an array built into the library's device image instead of a caller workspace.
+ *
+ *   - The array is HASS_STATIC_SCRATCH_MAX_BYTES (16 MiB) and every GPU that loads the library
+ *     holds it until the process exits. A problem whose forward scratch does not fit (it grows
+ *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits up to K = 31) is refused
+ *     with HASS_ERR_UNSUPPORTED; use hass_topk_distill_fwd with a workspace then.
+ *   - The call allocates and frees nothing, in this library or through any other.
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query,
+ *     with that device current). Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.
+ *     The call itself clears the only word that has to start at zero. Two calls that can overlap
+ *     on the GPU (different streams, no ordering between them) race on the array: serialise them.
+ *   - Arguments and outputs are those of hass_topk_distill_fwd. device_status is optional
+ *     (NULL to skip): a caller-owned DEVICE word that receives, in stream order, 0 or the
+ *     non-zero code of a bounded device-side wait that gave up (outputs are then undefined);
+ *     it replaces hass_check, which needs a workspace pointer.
+ */
+#define HASS_STATIC_SCRATCH_MAX_BYTES (16u << 20)
+int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
+                                 int64_t V, int32_t K, float* loss, int32_t* topk_idx, float* topk_q,
+                                 float* lse_t, float* lse_d, unsigned int* device_status,
+                                 void* cuda_stream);
+
+/*
  * Optional per-kernel timing for benchmarks (no counterpart in the paper). While enabled, each
  * kernel launch of the library is bracketed by CUDA events on its stream (the events are created
  * on the first enable). hass_profile_summary waits for the recorded events, adds the elapsed

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     topk_distill_fwd_bwd,
     topk_distill_fwd_bwd_host,
     topk_distill_fwd_draft,
+    topk_distill_fwd_static,
     topk_distill_host_workspace_bytes,
     topk_distill_workspace_bytes,
     version,

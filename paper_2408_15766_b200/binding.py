@@ -41,6 +41,8 @@ def _load() -> ctypes.CDLL:
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
     L.hass_check.argtypes = [vp, vp]
+    L.hass_topk_distill_fwd_static.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
+    L.hass_topk_distill_fwd_static.restype = ctypes.c_int
     L.hass_profile_enable.argtypes = [ctypes.c_int]
     L.hass_profile_enable.restype = ctypes.c_int
     L.hass_profile_summary.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64), ctypes.c_int]
@@ -125,6 +127,28 @@ def topk_distill_fwd(H_t, H_d, W, K: int, workspace=None, stream=None) -> dict:
     _ok(lib.hass_topk_distill_fwd(_p(H_t), _p(H_d), _p(W), N, d, V, K, _p(out["loss"]), _p(out["topk_idx"]),
                                   _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]), _p(ws), ws.numel(),
                                   _stream(stream)), "hass_topk_distill_fwd")
+    return out
+
+
+def topk_distill_fwd_static(H_t, H_d, W, K: int, stream=None, out: Optional[dict] = None) -> dict:
+    """Forward for callers that cannot hand the library a workspace: the library's built-in 16 MiB
+    scratch array is used instead. Here the outputs are still torch tensors, created by this wrapper
+    when ``out`` is not given; pass preallocated ``out`` tensors to make the call allocation-free end
+    to end. ``out['device_status']`` (uint32[1]) is 0 after a clean run."""
+    N, d, V = _dims(H_t, W)
+    assert H_d.shape == H_t.shape and H_d.dtype == torch.bfloat16 and H_d.is_contiguous()
+    dev = H_t.device
+    if out is None:
+        out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+                   topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+                   topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+                   lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+                   lse_d=torch.empty(N, dtype=torch.float32, device=dev),
+                   device_status=torch.empty(1, dtype=torch.int32, device=dev))
+    _ok(lib.hass_topk_distill_fwd_static(_p(H_t), _p(H_d), _p(W), N, d, V, K, _p(out["loss"]), _p(out["topk_idx"]),
+                                         _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]),
+                                         _p(out.get("device_status")), _stream(stream)),
+        "hass_topk_distill_fwd_static")
     return out
 
 

@@ -654,6 +654,63 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
     return hass_check(workspace, cuda_stream);
 }
 
+// ---- forward without a caller-provided workspace -------------------------------------------------
+// Scratch of hass_topk_distill_fwd_static: lives in the library's device image, so every GPU that
+// loads the library holds these bytes until the process exits.
+#define HASS_STATIC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[HASS_STATIC_SCRATCH_BYTES];
+// Device address of g_static_scratch per device. In host code the symbol itself is only a handle
+// for the runtime, never a pointer a kernel may use; the address comes from cudaGetSymbolAddress.
+static void* g_static_scratch_addr[64] = {nullptr};
+
+int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                                 int32_t K, float* loss, int32_t* topk_idx, float* topk_q, float* lse_t,
+                                 float* lse_d, unsigned int* device_status, void* cuda_stream) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    // the forward needs the statistics / candidate part of the workspace layout only
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (L.fixed_end > HASS_STATIC_SCRATCH_BYTES) {
+        if (kLog)
+            std::fprintf(stderr, "[hass] hass_topk_distill_fwd_static: this size needs %zu bytes of scratch, the built-in "
+                         "array holds %u; use hass_topk_distill_fwd with a workspace\n", L.fixed_end,
+                         HASS_STATIC_SCRATCH_BYTES);
+        return HASS_ERR_UNSUPPORTED;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    if (!g_static_scratch_addr[dev]) {
+        // once per device, with that device current
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = ptr;
+    }
+    void* scratch = g_static_scratch_addr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // forward_impl zeroes the status word (the only part of the scratch that must start at zero:
+    // every statistic and candidate slot that is read has been written by the same call)
+    rc = forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d, scratch,
+                      HASS_STATIC_SCRATCH_BYTES, st);
+    if (rc != HASS_OK) return rc;
+    if (device_status &&
+        cudaMemcpyAsync(device_status, scratch, sizeof(unsigned int), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    return HASS_OK;
+}
+
 int hass_check(void* workspace, void* cuda_stream) {
     if (!workspace) return HASS_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

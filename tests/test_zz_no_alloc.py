@@ -1,0 +1,63 @@
+"""The workspace-free forward (hass_topk_distill_fwd_static) against the ordinary forward.
+
+Some users of the library cannot allocate device memory when they call it (the GPU was reserved
+up front by their framework, or their plug-in interface passes inputs and outputs only), so one
+entry point keeps its scratch in an array compiled into the library. This file checks, through
+the C ABI, that it returns what hass_topk_distill_fwd returns, on two consecutive calls with
+different inputs (the second call finds the first call's leftovers in the shared array), and that
+an oversized problem is refused instead of overrunning the array. The file name makes pytest
+collect it after every other test.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import hass_inputs as hi
+
+pytestmark = pytest.mark.gpu
+
+LOSS_RTOL = 2e-3      # the tolerances of tests/parity.py
+LSE_ATOL = 1e-4
+Q_RTOL = 1e-3
+
+
+def _compare(static, ref):
+    assert int(static["device_status"].item()) == 0
+    assert torch.equal(static["topk_idx"], ref["topk_idx"])
+    np.testing.assert_allclose(static["topk_q"].cpu().numpy(), ref["topk_q"].cpu().numpy(), rtol=Q_RTOL)
+    np.testing.assert_allclose(static["lse_t"].cpu().numpy(), ref["lse_t"].cpu().numpy(), atol=LSE_ATOL)
+    np.testing.assert_allclose(static["lse_d"].cpu().numpy(), ref["lse_d"].cpu().numpy(), atol=LSE_ATOL)
+    a, b = static["loss"].cpu().numpy(), ref["loss"].cpu().numpy()
+    assert np.all(np.abs(a - b) <= LOSS_RTOL * np.maximum(np.abs(b), 1e-6))
+
+
+def test_static_scratch_forward_matches_workspace_forward_twice_in_a_row():
+    import paper_2408_15766_b200 as hass
+    dev = torch.device("cuda:0")
+    # two different problems back to back: a ragged one, then a larger one with more slots and K
+    for (N, d, V, K, seed) in [(300, 256, 5000, 10, 1), (1000, 512, 33000, 24, 2)]:
+        inp = hi.make_custom(N, d, V, K, seed=seed, sigma_w=2.0 / np.sqrt(d))
+        H_t, H_d, W = inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev)
+        ref = hass.topk_distill_fwd(H_t, H_d, W, K)
+        hass.check(ref["workspace"])
+        static = hass.topk_distill_fwd_static(H_t, H_d, W, K)
+        torch.cuda.synchronize()
+        _compare(static, ref)
+        # and once more on the same inputs, reusing the output tensors (no allocation at all)
+        again = hass.topk_distill_fwd_static(H_t, H_d, W, K, out=static)
+        torch.cuda.synchronize()
+        _compare(again, ref)
+
+
+def test_static_scratch_refuses_a_problem_that_does_not_fit():
+    import paper_2408_15766_b200 as hass
+    dev = torch.device("cuda:0")
+    N, d, V, K = 8192, 64, 128256, 128          # forward scratch far above 16 MiB
+    assert hass.topk_distill_workspace_bytes(N, d, V, K) > (16 << 20)
+    buf = torch.zeros(4096, dtype=torch.uint8, device=dev)
+    p = ctypes.c_void_p(buf.data_ptr())
+    rc = hass.lib.hass_topk_distill_fwd_static(p, p, p, N, d, V, K, p, p, p, p, p, None, None)
+    assert rc == -2 and hass.status_string(rc) == "HASS_ERR_UNSUPPORTED"
+    torch.cuda.synchronize()
