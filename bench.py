@@ -295,7 +295,7 @@ def main():
                 "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
                 "flops_per_launch": flops_per_launch, "avg_launch_ms": dom_ms / dom_cnt}
     step_tflops = flops_credit / (ms_step * 1e-3) / 1e12
-    executed = sum(kinds.values())
+    executed = sum(f for k, f in kinds.items() if prof[k][1] > 0)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",

@@ -47,7 +47,8 @@ typedef enum {
     HASS_ERR_WORKSPACE = -3,   /* workspace missing or too small */
     HASS_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed, or no CUDA device */
     HASS_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (see hass_check) */
-    HASS_ERR_ARCH = -6         /* device is not sm_100 */
+    HASS_ERR_ARCH = -6,        /* device is not sm_100 */
+    HASS_ERR_RANGE = -7        /* fused path: a row's logits spread too far (see hass_topk_distill_fwd_bwd) */
 } hass_status;
 
 typedef enum { HASS_BF16 = 0, HASS_FP32 = 1 } hass_dtype; /* element type of dH_d */
@@ -123,14 +124,35 @@ int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, 
                           size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Forward and backward in one call (the whole hot path of one aligning step): same outputs as
- * hass_topk_distill_fwd followed by hass_topk_distill_bwd with the same arguments.
+ * Forward and backward in one call (the whole hot path of one aligning step): the same results as
+ * hass_topk_distill_fwd followed by hass_topk_distill_bwd, up to rounding, but no logit is
+ * computed twice. Rows are processed in bounded chunks; while a chunk's draft logits are swept
+ * for the forward statistics they are also written to the workspace as bf16 values
+ * 2^(z_d log2(e) - ref2), ref2 a per-row exponent fixed from the row's largest logit among the
+ * first 256 tokens, and dH_d = coef (spill W) - sum_{x in Omega_hat} g q(x) W[x,:] is formed by
+ * the second GEMM, whose epilogue applies the per-row scale coef = g S_q 2^ref2 / sum_v e^{z_d}
+ * and the sparse term.
+ * Range condition: the fixed exponent holds as long as no draft logit of a row exceeds that
+ * row's largest logit among tokens 0..255 by more than about 130 (natural-log units; a probability
+ * ratio of e^130). If it does, hass_check reports HASS_ERR_RANGE: topk_idx, topk_q and lse_t are
+ * still valid, loss, lse_d and dH_d are not; hass_topk_distill_fwd followed by hass_topk_distill_bwd
+ * has no such condition and gives them.
  */
 int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                               int64_t V, int32_t K, const float* grad_loss, float* loss,
                               int32_t* topk_idx, float* topk_q, float* lse_t, float* lse_d,
                               void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes,
                               void* cuda_stream);
+
+/*
+ * hass_topk_distill_fwd_bwd for aligning steps j >= 2: topk_idx / topk_q are inputs (as for
+ * hass_topk_distill_fwd_draft), only the draft projection, its loss and dH_d are computed.
+ */
+int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                                    int32_t K, const int32_t* topk_idx, const float* topk_q,
+                                    const float* grad_loss, float* loss, float* lse_d, void* dH_d,
+                                    int dH_dtype, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream);
 
 /*
  * The same forward + backward for callers whose features live in HOST memory (the training

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     topk_distill_bwd,
     topk_distill_fwd,
     topk_distill_fwd_bwd,
+    topk_distill_fwd_bwd_draft,
     topk_distill_fwd_bwd_host,
     topk_distill_fwd_draft,
     topk_distill_fwd_static,

@@ -38,6 +38,9 @@ def _load() -> ctypes.CDLL:
     L.hass_topk_distill_bwd.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
     L.hass_topk_distill_fwd_bwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp,
                                             ctypes.c_int, vp, sz, vp]
+    L.hass_topk_distill_fwd_bwd_draft.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, ctypes.c_int,
+                                                  vp, sz, vp]
+    L.hass_topk_distill_fwd_bwd_draft.restype = ctypes.c_int
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
     L.hass_check.argtypes = [vp, vp]
@@ -201,6 +204,26 @@ def topk_distill_fwd_bwd(H_t, H_d, W, K: int, grad_loss=None, dH_dtype: int = HA
                                       _p(out["topk_idx"]), _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]),
                                       _p(out["dH_d"]), dH_dtype, _p(ws), ws.numel(), _stream(stream)),
         "hass_topk_distill_fwd_bwd")
+    return out
+
+
+def topk_distill_fwd_bwd_draft(H_d, W, topk_idx, topk_q, grad_loss=None, dH_dtype: int = HASS_BF16, workspace=None,
+                               stream=None, out: Optional[dict] = None) -> dict:
+    N, d, V = _dims(H_d, W)
+    K = topk_idx.shape[1]
+    assert topk_idx.dtype == torch.int32 and topk_q.dtype == torch.float32
+    assert topk_idx.is_contiguous() and topk_q.is_contiguous() and topk_idx.shape == topk_q.shape == (N, K)
+    assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
+    dev = H_d.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    if out is None:
+        out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+                   lse_d=torch.empty(N, dtype=torch.float32, device=dev),
+                   dH_d=torch.empty(N, d, dtype=_dh_dtype(dH_dtype), device=dev))
+    out["workspace"] = ws
+    _ok(lib.hass_topk_distill_fwd_bwd_draft(_p(H_d), _p(W), N, d, V, K, _p(topk_idx), _p(topk_q), _p(grad_loss),
+                                            _p(out["loss"]), _p(out["lse_d"]), _p(out["dH_d"]), dH_dtype, _p(ws),
+                                            ws.numel(), _stream(stream)), "hass_topk_distill_fwd_bwd_draft")
     return out
 
 

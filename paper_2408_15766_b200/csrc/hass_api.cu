@@ -2,6 +2,7 @@
 // descriptors, workspace layout and kernel launches. No allocation, no synchronisation except in
 // hass_check and the *_host entry.
 #include <atomic>
+#include <climits>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -179,6 +180,7 @@ struct Layout {
     size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
     long long p_pitch;
     int pref_chunk_tiles;
+    int slot_cap;
     size_t total_pref;
 };
 
@@ -191,10 +193,28 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     int rc = plan_schedule(2 * RT, CT, sms, &s);
     if (rc != HASS_OK) return rc;
     if (fwd_sched) *fwd_sched = s;
+    int pref = sms / 4;
+    if (pref < 1) pref = 1;
+    if (pref > RT) pref = RT;
+    // partial-statistics slots: enough for the whole-batch forward and for the per-chunk forward
+    // sweeps of the fused path (target + draft tiles, or draft tiles only, of a full or last chunk)
+    int slot_cap = s.total_slots;
+    {
+        const int rem = RT % pref;
+        const int cands[5] = {RT, 2 * pref, pref, 2 * rem, rem};
+        for (int i = 0; i < 5; ++i) {
+            if (cands[i] < 1) continue;
+            Schedule t;
+            rc = plan_schedule(cands[i], CT, sms, &t);
+            if (rc != HASS_OK) return rc;
+            if (t.total_slots > slot_cap) slot_cap = t.total_slots;
+        }
+    }
+    L->slot_cap = slot_cap;
     size_t off = 0;
     L->status = off;
     off += 256;
-    const size_t slots = static_cast<size_t>(s.total_slots);
+    const size_t slots = static_cast<size_t>(slot_cap);
     L->part_m = off;
     off = align256(off + slots * BM * 4);
     L->part_s = off;
@@ -215,9 +235,6 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     L->fixed_end = off;
     L->p_pitch = static_cast<long long>(CT) * BN;
     L->scratch_row_tile_bytes = static_cast<size_t>(BM) * L->p_pitch * 2;
-    int pref = sms / 4;
-    if (pref < 1) pref = 1;
-    if (pref > RT) pref = RT;
     L->pref_chunk_tiles = pref;
     L->total_pref = off + L->scratch_row_tile_bytes * pref;
     return HASS_OK;
@@ -297,7 +314,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     } else {
         rc = plan_schedule(RT, CT, di.sms, &p.sched);   // never needs more slots than the full schedule
         if (rc != HASS_OK) return rc;
-        if (p.sched.total_slots > full.total_slots) return HASS_ERR_WORKSPACE;
+        if (p.sched.total_slots > L.slot_cap) return HASS_ERR_WORKSPACE;
         p.row_tiles0 = RT;
         p.topk_row_tiles = 0;
         rc = make_tmap(&p.tmA0, H_d, N, d, d, BK, BM);
@@ -306,6 +323,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     if (rc == HASS_OK) rc = make_tmap(&p.tmB, W, V, d, d, BK, BN);
     if (rc != HASS_OK) return rc;
     log_schedule(with_target ? "fwd stats" : "fwd stats (draft)", p.sched);
+    p.spill_begin = INT_MAX;
     p.a_row_offset = 0;
     p.row_global_offset = 0;
     p.rows_valid = static_cast<int>(N);
@@ -324,7 +342,8 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     FinalizeParams f;
     std::memset(&f, 0, sizeof(f));
     f.sched = p.sched;
-    f.N = static_cast<int>(N);
+    f.row_begin = 0;
+    f.rows = static_cast<int>(N);
     f.d = static_cast<int>(d);
     f.K = K;
     f.row_tiles_t = with_target ? RT : 0;
@@ -456,6 +475,151 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
     return HASS_OK;
 }
 
+// ---- fused forward + backward -------------------------------------------------------------------
+// Per chunk of row tiles: (1) one sweep computes the logits of the chunk's target and draft rows,
+// their statistics and Top-K candidates, and spills the draft tiles as 2^(z log2e - ref2) in bf16;
+// (2) finalize gives loss, Omega_hat, lse and the per-row scale of the spilled tiles; (3) the second
+// GEMM contracts the spilled tiles with W and applies scale and sparse term in its epilogue. No
+// logit is computed twice. with_target = false: Omega_hat is an input (aligning steps >= 2).
+static int fused_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
+                      long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
+                      int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
+                      void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
+        return HASS_ERR_INVALID_ARG;
+    if (with_target && (!H_t || !idx_out || !q_out || !lse_t || !aligned16(H_t))) return HASS_ERR_INVALID_ARG;
+    if (!with_target && (!idx_in || !q_in)) return HASS_ERR_INVALID_ARG;
+    if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.fixed_end + L.scratch_row_tile_bytes) return HASS_ERR_WORKSPACE;
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN), DT = ceil_div(d, BN);
+    long long fit = static_cast<long long>((workspace_bytes - L.fixed_end) / L.scratch_row_tile_bytes);
+    int chunk_tiles = L.pref_chunk_tiles;
+    if (fit < chunk_tiles) chunk_tiles = static_cast<int>(fit);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* gq = reinterpret_cast<float*>(ws + L.sgq);
+    float* coef = reinterpret_cast<float*>(ws + L.coef);
+    __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(ws + L.scratch);
+    unsigned int* status = reinterpret_cast<unsigned int*>(ws + L.status);
+    if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    CUtensorMap tmHt, tmHd, tmWk, tmWn, tmP;
+    rc = make_tmap(&tmHd, H_d, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = with_target ? make_tmap(&tmHt, H_t, N, d, d, BK, BM) : make_tmap(&tmHt, H_d, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = make_tmap(&tmWk, W, V, d, d, BK, BN);
+    if (rc == HASS_OK) rc = make_tmap(&tmWn, W, V, d, d, 64, BK);
+    if (rc == HASS_OK) rc = make_tmap(&tmP, P, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
+    if (rc != HASS_OK) return rc;
+
+    for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
+        const int tiles = (RT - t0 < chunk_tiles) ? RT - t0 : chunk_tiles;
+        const int rows = static_cast<int>((N - static_cast<long long>(t0) * BM < static_cast<long long>(tiles) * BM)
+                                              ? N - static_cast<long long>(t0) * BM
+                                              : static_cast<long long>(tiles) * BM);
+        // (1) logits sweep with statistics, candidates and spill
+        GemmParams p;
+        std::memset(&p, 0, sizeof(p));
+        rc = plan_schedule(with_target ? 2 * tiles : tiles, CT, di.sms, &p.sched);
+        if (rc != HASS_OK) return rc;
+        if (p.sched.total_slots > L.slot_cap) return HASS_ERR_WORKSPACE;
+        log_schedule("fused stats", p.sched);
+        p.tmA0 = tmHt;
+        p.tmA1 = tmHd;
+        p.tmB = tmWk;
+        p.row_tiles0 = tiles;
+        p.topk_row_tiles = with_target ? tiles : 0;
+        p.spill_begin = with_target ? tiles : 0;
+        p.a_row_offset = t0 * BM;
+        p.row_global_offset = t0 * BM;
+        p.rows_valid = static_cast<int>(N);
+        p.n_cols = static_cast<int>(V);
+        p.col_tiles = CT;
+        p.k_blocks = ceil_div(d, BK);
+        p.K = K;
+        p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+        p.part_s = reinterpret_cast<float*>(ws + L.part_s);
+        p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
+        p.cand_i = reinterpret_cast<int*>(ws + L.cand_i);
+        p.P = P;
+        p.p_pitch = L.p_pitch;
+        p.status = status;
+        rc = launch_gemm<MODE_STATS>(p, st);
+        if (rc != HASS_OK) return rc;
+        // (2) statistics -> loss, Omega_hat, per-row scale
+        FinalizeParams f;
+        std::memset(&f, 0, sizeof(f));
+        f.sched = p.sched;
+        f.d = static_cast<int>(d);
+        f.K = K;
+        f.row_begin = t0 * BM;
+        f.rows = rows;
+        f.row_tiles_t = with_target ? tiles : 0;
+        f.part_m = p.part_m;
+        f.part_s = p.part_s;
+        f.cand_v = p.cand_v;
+        f.cand_i = p.cand_i;
+        f.H_d = static_cast<const __nv_bfloat16*>(H_d);
+        f.W = static_cast<const __nv_bfloat16*>(W);
+        f.idx_in = idx_in;
+        f.q_in = q_in;
+        f.loss = loss;
+        f.idx_out = idx_out;
+        f.q_out = q_out;
+        f.lse_t = lse_t;
+        f.lse_d = lse_d;
+        f.grad_loss = grad_loss;
+        f.coef_out = coef;
+        f.gq_out = gq;
+        {
+            KernelTimer timer(KIND_FINALIZE, st);
+            finalize_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(f);
+        }
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+        // (3) dH_d rows of the chunk
+        GemmParams o;
+        std::memset(&o, 0, sizeof(o));
+        rc = plan_schedule(tiles, DT, di.sms, &o.sched);
+        if (rc != HASS_OK) return rc;
+        log_schedule("fused dH_d", o.sched);
+        o.tmA0 = tmP;
+        o.tmA1 = tmP;
+        o.tmB = tmWn;
+        o.row_tiles0 = tiles;
+        o.spill_begin = INT_MAX;
+        o.a_row_offset = 0;
+        o.row_global_offset = t0 * BM;
+        o.rows_valid = static_cast<int>(N);
+        o.n_cols = static_cast<int>(d);
+        o.col_tiles = DT;
+        o.k_blocks = ceil_div(V, BK);
+        o.K = K;
+        o.coef = coef;
+        o.sidx = with_target ? idx_out : idx_in;
+        o.sgq = gq;
+        o.Wg = static_cast<const __nv_bfloat16*>(W);
+        o.out = dH_d;
+        o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+        o.out_pitch = d;
+        o.status = status;
+        rc = launch_gemm<MODE_OUT>(o, st);
+        if (rc != HASS_OK) return rc;
+    }
+    return HASS_OK;
+}
+
 }  // namespace hass
 
 using namespace hass;
@@ -471,6 +635,7 @@ const char* hass_status_string(int status) {
         case HASS_ERR_CUDA: return "HASS_ERR_CUDA";
         case HASS_ERR_TIMEOUT: return "HASS_ERR_TIMEOUT";
         case HASS_ERR_ARCH: return "HASS_ERR_ARCH";
+        case HASS_ERR_RANGE: return "HASS_ERR_RANGE";
         default: return "HASS_ERR_UNKNOWN";
     }
 }
@@ -554,13 +719,16 @@ int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, i
                               int32_t K, const float* grad_loss, float* loss, int32_t* topk_idx, float* topk_q,
                               float* lse_t, float* lse_d, void* dH_d, int dH_dtype, void* workspace,
                               size_t workspace_bytes, void* cuda_stream) {
-    // validate the backward's own arguments before anything is launched
-    if (!dH_d || !aligned16(dH_d) || (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32)) return HASS_ERR_INVALID_ARG;
-    int rc = forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
-                          workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
-    if (rc != HASS_OK) return rc;
-    return backward_impl(H_d, W, N, d, V, K, topk_idx, topk_q, lse_d, grad_loss, dH_d, dH_dtype, workspace,
-                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream), false);
+    return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
+                      dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
+                                    const int32_t* topk_idx, const float* topk_q, const float* grad_loss, float* loss,
+                                    float* lse_d, void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes,
+                                    void* cuda_stream) {
+    return fused_impl(false, nullptr, H_d, W, N, d, V, K, grad_loss, topk_idx, topk_q, loss, nullptr, nullptr, nullptr,
+                      lse_d, dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Device staging appended to the normal workspace by the *_host entry.
@@ -726,7 +894,7 @@ int hass_check(void* workspace, void* cuda_stream) {
     if (word != 0) {
         cudaMemset(workspace, 0, 4);
         if (kLog) std::fprintf(stderr, "[hass] device status word 0x%x\n", word);
-        return HASS_ERR_TIMEOUT;
+        return (word & 0xffu) == 2u ? HASS_ERR_RANGE : HASS_ERR_TIMEOUT;
     }
     return HASS_OK;
 }

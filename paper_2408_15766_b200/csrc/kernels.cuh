@@ -59,6 +59,8 @@ struct GemmParams {
     int col_tiles;
     int k_blocks;          // ceil(contraction extent / BK)
     int K;                 // Top-K
+    int spill_begin;       // MODE_STATS: row tiles >= spill_begin also write the tile 2^(z log2e - ref2) in bf16 to
+                           // P (row tile index - spill_begin); INT_MAX: none
     // MODE_STATS outputs (per slot)
     float* part_m;
     float* part_s;
@@ -71,7 +73,9 @@ struct GemmParams {
     const float* sgq;      // [N, K] g * q in the same order
     __nv_bfloat16* P;      // [chunk rows, p_pitch]
     long long p_pitch;
-    // MODE_OUT
+    // MODE_OUT. With Wg != nullptr the epilogue computes coef[row] * acc - sum_k sgq[row,k] * Wg[sidx[row,k], :]
+    // (row scale and the sparse Omega_hat term of dz_d W); otherwise it stores the accumulator.
+    const __nv_bfloat16* Wg;
     void* out;
     int out_fp32;
     long long out_pitch;   // elements
@@ -187,8 +191,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             for_each_item([&](int rt, int ln, int S, int) {
                 const bool second = (MODE == MODE_STATS) && rt >= p.row_tiles0;
                 const CUtensorMap* tmA = second ? &p.tmA1 : &p.tmA0;
-                const int row0 = second ? (rt - p.row_tiles0) * BM : p.a_row_offset + rt * BM;
-                for (int ct = ln; ct < p.col_tiles; ct += S) {
+                const int row0 = p.a_row_offset + (second ? rt - p.row_tiles0 : rt) * BM;
+                const int t0 = (MODE == MODE_STATS && rt >= p.spill_begin && ln != 0) ? -1 : 0;
+                const int nt = (p.col_tiles - ln + S - 1) / S;
+                for (int t = t0; t < nt; ++t) {
+                    const int ct = t < 0 ? 0 : ln + t * S;   // t = -1: column tile 0, for the row references only
                     for (int kb = 0; kb < p.k_blocks; ++kb) {
                         if (!wait_barrier(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) return false;
                         mbar_arrive_expect_tx(full_bar(stage), A_STAGE_BYTES + B_STAGE_BYTES);
@@ -220,8 +227,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             uint32_t phase = 0;
             int ab = 0;
             uint32_t aphase = 0;
-            for_each_item([&](int, int ln, int S, int) {
-                for (int ct = ln; ct < p.col_tiles; ct += S) {
+            for_each_item([&](int rt, int ln, int S, int) {
+                const int t0 = (MODE == MODE_STATS && rt >= p.spill_begin && ln != 0) ? -1 : 0;
+                const int nt = (p.col_tiles - ln + S - 1) / S;
+                for (int t = t0; t < nt; ++t) {
                     if (!wait_barrier(tempty_bar(ab), aphase ^ 1u, abort_flag, p.status, 2)) return false;
                     tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + ab * BN;
@@ -272,7 +281,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             // ---- per-item state ----
             float m = -INFINITY, s = 0.f, thr = -INFINITY;        // MODE_STATS
             bool want_topk = false;
-            float lse2 = 0.f, coef = 0.f;                         // MODE_PROBS
+            const bool spill = MODE == MODE_STATS && rt >= p.spill_begin;
+            float ref2 = 0.f;                                     // spill rows: exponent offset (log2 units)
+            float lse2 = 0.f, coef = 0.f;                         // MODE_PROBS / fused MODE_OUT
             const int* si = nullptr;
             const float* sg = nullptr;
             int cur = 0, nxt = INT_MAX;
@@ -288,15 +299,43 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 sg = p.sgq + static_cast<long long>(g_row) * p.K;
                 nxt = si[0];
             }
-            for (int ct = ln; ct < p.col_tiles; ct += S) {
+            if (MODE == MODE_OUT && p.Wg != nullptr && row_ok) {
+                coef = p.coef[g_row];
+                si = p.sidx + static_cast<long long>(g_row) * p.K;
+                sg = p.sgq + static_cast<long long>(g_row) * p.K;
+            }
+            const int t0 = (spill && ln != 0) ? -1 : 0;
+            const int nt = (p.col_tiles - ln + S - 1) / S;
+            for (int t = t0; t < nt; ++t) {
+                const int ct = t < 0 ? 0 : ln + t * S;
                 // the whole warp must agree before the warp-collective TMEM loads below
                 const bool ready = wait_barrier(tfull_bar(ab), aphase, abort_flag, p.status, 4);
                 if (!__all_sync(0xffffffffu, ready)) return false;
                 tc_fence_after_sync();
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + ab * BN;
                 const int col_base = ct * BN;
+                bool skip_tile = false;
+                if (MODE == MODE_STATS && spill && t == t0) {
+                    // Reference exponent of this row: its largest logit in column tile 0. Every lane of
+                    // the row tile computes tile 0 first and so derives the same value.
+                    float mx = -INFINITY;
 #pragma unroll 1
-                for (int ch = 0; ch < BN / 32; ++ch) {
+                    for (int ch = 0; ch < BN / 32; ++ch) {
+                        uint32_t r[32];
+                        tmem_ld32(t_row + ch * 32, r);
+                        tmem_ld_wait(r);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (ch * 32 + j < p.n_cols) mx = fmaxf(mx, __uint_as_float(r[j]));
+                    }
+                    // spilled values are 2^(z log2e - ref2) <= about 2^-64 for typical rows, which leaves
+                    // 2^191 of headroom above the reference before bf16 / fp32 overflow
+                    ref2 = fmaf(mx, LOG2E, 64.f);
+                    m = ref2 * (1.0f / LOG2E);
+                    skip_tile = t < 0;
+                }
+#pragma unroll 1
+                for (int ch = 0; ch < BN / 32 && !skip_tile; ++ch) {
                     uint32_t r[32];
                     tmem_ld32(t_row + ch * 32, r);
                     tmem_ld_wait(r);
@@ -307,23 +346,46 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             for (int j = 0; j < 32; ++j)
                                 if (col0 + j >= p.n_cols) r[j] = __float_as_uint(-INFINITY);
                         }
-                        float cm = __uint_as_float(r[0]);
+                        if (!spill) {
+                            float cm = __uint_as_float(r[0]);
 #pragma unroll
-                        for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
-                        if (cm > m) {
-                            s *= ex2((m - cm) * LOG2E);
-                            m = cm;
-                        }
-                        const float mneg = -m * LOG2E;
-                        float acc = 0.f;
+                            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
+                            if (cm > m) {
+                                s *= ex2((m - cm) * LOG2E);
+                                m = cm;
+                            }
+                            const float mneg = -m * LOG2E;
+                            float acc = 0.f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), LOG2E, mneg));
-                        s += acc;
-                        if (want_topk && cm > thr) {
+                            for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), LOG2E, mneg));
+                            s += acc;
+                            if (want_topk && cm > thr) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const float x = __uint_as_float(r[j]);
+                                    if (x > thr) thr = topk_insert(lv, li, cnt_minpos, p.K, x, col0 + j);
+                                }
+                            }
+                        } else {
+                            // one exponential per logit serves both the row's sum and the spilled tile
+                            float e[32];
+                            float acc = 0.f;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                const float x = __uint_as_float(r[j]);
-                                if (x > thr) thr = topk_insert(lv, li, cnt_minpos, p.K, x, col0 + j);
+                                e[j] = ex2(fminf(fmaf(__uint_as_float(r[j]), LOG2E, -ref2), 127.f));
+                                acc += e[j];
+                            }
+                            s += acc;
+                            uint4* dst = reinterpret_cast<uint4*>(
+                                p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch + col0);
+#pragma unroll
+                            for (int g8 = 0; g8 < 4; ++g8) {
+                                uint4 w;
+                                w.x = pack_bf16x2(e[8 * g8 + 0], e[8 * g8 + 1]);
+                                w.y = pack_bf16x2(e[8 * g8 + 2], e[8 * g8 + 3]);
+                                w.z = pack_bf16x2(e[8 * g8 + 4], e[8 * g8 + 5]);
+                                w.w = pack_bf16x2(e[8 * g8 + 6], e[8 * g8 + 7]);
+                                dst[g8] = w;
                             }
                         }
                     } else if (MODE == MODE_PROBS) {
@@ -358,30 +420,50 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             w.w = pack_bf16x2(e[8 * g8 + 6], e[8 * g8 + 7]);
                             dst[g8] = w;
                         }
-                    } else {
-                        if (row_ok) {
-                            if (p.out_fp32) {
-                                float* dst = reinterpret_cast<float*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+                    } else if (row_ok) {
+                        float o[32];
 #pragma unroll
-                                for (int g4 = 0; g4 < 8; ++g4) {
-                                    if (col0 + 4 * g4 < p.n_cols) {
-                                        *reinterpret_cast<float4*>(dst + 4 * g4) =
-                                            make_float4(__uint_as_float(r[4 * g4]), __uint_as_float(r[4 * g4 + 1]),
-                                                        __uint_as_float(r[4 * g4 + 2]), __uint_as_float(r[4 * g4 + 3]));
-                                    }
-                                }
-                            } else {
-                                __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+                        for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(r[j]);
+                        if (p.Wg != nullptr) {
+                            // dH_d = coef * (spilled tile x W) - sum_{x in Omega_hat} g q(x) W[x, :]
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) o[j] *= coef;
+                            for (int k = 0; k < p.K; ++k) {
+                                const float gq = sg[k];
+                                const __nv_bfloat16* wr = p.Wg + static_cast<long long>(si[k]) * p.out_pitch + col0;
 #pragma unroll
                                 for (int g8 = 0; g8 < 4; ++g8) {
                                     if (col0 + 8 * g8 < p.n_cols) {
-                                        uint4 w;
-                                        w.x = pack_bf16x2(__uint_as_float(r[8 * g8 + 0]), __uint_as_float(r[8 * g8 + 1]));
-                                        w.y = pack_bf16x2(__uint_as_float(r[8 * g8 + 2]), __uint_as_float(r[8 * g8 + 3]));
-                                        w.z = pack_bf16x2(__uint_as_float(r[8 * g8 + 4]), __uint_as_float(r[8 * g8 + 5]));
-                                        w.w = pack_bf16x2(__uint_as_float(r[8 * g8 + 6]), __uint_as_float(r[8 * g8 + 7]));
-                                        *reinterpret_cast<uint4*>(dst + 8 * g8) = w;
+                                        const uint4 wv = *reinterpret_cast<const uint4*>(wr + 8 * g8);
+                                        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                                        for (int u = 0; u < 4; ++u) {
+                                            const float2 w2 = __bfloat1622float2(wp[u]);
+                                            o[8 * g8 + 2 * u] = fmaf(-gq, w2.x, o[8 * g8 + 2 * u]);
+                                            o[8 * g8 + 2 * u + 1] = fmaf(-gq, w2.y, o[8 * g8 + 2 * u + 1]);
+                                        }
                                     }
+                                }
+                            }
+                        }
+                        if (p.out_fp32) {
+                            float* dst = reinterpret_cast<float*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+#pragma unroll
+                            for (int g4 = 0; g4 < 8; ++g4)
+                                if (col0 + 4 * g4 < p.n_cols)
+                                    *reinterpret_cast<float4*>(dst + 4 * g4) =
+                                        make_float4(o[4 * g4], o[4 * g4 + 1], o[4 * g4 + 2], o[4 * g4 + 3]);
+                        } else {
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+#pragma unroll
+                            for (int g8 = 0; g8 < 4; ++g8) {
+                                if (col0 + 8 * g8 < p.n_cols) {
+                                    uint4 w;
+                                    w.x = pack_bf16x2(o[8 * g8 + 0], o[8 * g8 + 1]);
+                                    w.y = pack_bf16x2(o[8 * g8 + 2], o[8 * g8 + 3]);
+                                    w.z = pack_bf16x2(o[8 * g8 + 4], o[8 * g8 + 5]);
+                                    w.w = pack_bf16x2(o[8 * g8 + 6], o[8 * g8 + 7]);
+                                    *reinterpret_cast<uint4*>(dst + 8 * g8) = w;
                                 }
                             }
                         }
@@ -398,6 +480,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 const long long so = static_cast<long long>(slot) * BM + r_local;
                 p.part_m[so] = m;
                 p.part_s[so] = s;
+                // a spilled value reached the top of the fp32 range: the row's logits spread too far
+                // above its reference for the fixed-exponent spill
+                if (spill && !(s < 1e38f)) atomicCAS(p.status, 0u, (5u << 8) | 2u);
                 if (want_topk) {
                     const int cnt = cnt_minpos[0];
                     for (int k = 0; k < p.K; ++k) {
@@ -431,7 +516,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 // Omega_hat with K dot products, and evaluates Eq. 1.
 struct FinalizeParams {
     Schedule sched;
-    int N, d, K;
+    int d, K;
+    int row_begin, rows;   // global rows [row_begin, row_begin + rows) = local row tiles 0.. of the schedule
     int row_tiles_t;       // row tiles of the target matrix in the schedule (0: Omega_hat is an input)
     const float* part_m;
     const float* part_s;
@@ -446,6 +532,10 @@ struct FinalizeParams {
     float* q_out;
     float* lse_t;
     float* lse_d;
+    // fused backward (all nullable): per-row scale of the spilled tiles and g * q of Omega_hat
+    const float* grad_loss;
+    float* coef_out;       // [N]   g * S_q * exp(m_spill - lse_d), m_spill = the row's spill reference
+    float* gq_out;         // [N,K] g * q, in the order of topk_idx
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -478,9 +568,10 @@ __device__ __forceinline__ float warp_lse(const float* pm, const float* ps, int 
 
 __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ FinalizeParams p) {
     const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (row >= p.N) return;
-    const int rt = row / BM, r = row % BM;
+    const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (local >= p.rows) return;
+    const int row = p.row_begin + local;
+    const int rt = local / BM, r = local % BM;
     const int K = p.K;
     int slot0, S;
 
@@ -488,6 +579,9 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     find_slots(p.sched, p.row_tiles_t + rt, slot0, S);
     const float lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
     if (lane == 0) p.lse_d[row] = lse_d;
+    const float m_spill = p.part_m[static_cast<long long>(slot0) * BM + r];
+    const float g = p.grad_loss ? p.grad_loss[row] : 1.f;
+    float S_q = 0.f;
 
     float lse_t = 0.f;
     if (p.row_tiles_t > 0) {
@@ -560,8 +654,13 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
+        S_q += qv;
+        if (lane == 0 && p.gq_out) p.gq_out[static_cast<long long>(row) * K + j] = g * qv;
     }
-    if (lane == 0) p.loss[row] = loss;
+    if (lane == 0) {
+        p.loss[row] = loss;
+        if (p.coef_out) p.coef_out[row] = g * S_q * expf(m_spill - lse_d);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
