@@ -8,7 +8,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libhass_b200.so")
+# HASS_LIBRARY_PATH selects another build of the same library (e.g. a tuning variant)
+_LIB_PATH = os.environ.get("HASS_LIBRARY_PATH") or os.path.join(_HERE, "libhass_b200.so")
 
 HASS_BF16, HASS_FP32 = 0, 1
 K_MAX = 128
