@@ -176,7 +176,7 @@ static int make_tmap(CUtensorMap* tm, const void* base, long long rows, long lon
 static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 struct Layout {
-    size_t status, part_m, part_s, cand_v, cand_i, sidx, sgq, coef, lse2, scratch, fixed_end;
+    size_t status, part_m, part_s, cand_v, cand_i, fwd_end, sidx, sgq, coef, lse2, sparse, scratch, fixed_end;
     size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
     long long p_pitch;
     int pref_chunk_tiles;
@@ -219,10 +219,12 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     off = align256(off + slots * BM * 4);
     L->part_s = off;
     off = align256(off + slots * BM * 4);
+    const int Kc = K > K_REG ? K : K_REG;   // candidates per (row, slot)
     L->cand_v = off;
-    off = align256(off + slots * BM * 4 * K);
+    off = align256(off + slots * BM * 4 * Kc);
     L->cand_i = off;
-    off = align256(off + slots * BM * 4 * K);
+    off = align256(off + slots * BM * 4 * Kc);
+    L->fwd_end = off;                       // what the forward-only entry points use
     L->sidx = off;
     off = align256(off + static_cast<size_t>(N) * K * 4);
     L->sgq = off;
@@ -231,6 +233,8 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     off = align256(off + static_cast<size_t>(N) * 4);
     L->lse2 = off;
     off = align256(off + static_cast<size_t>(N) * 4);
+    L->sparse = off;                        // fused path: Omega_hat term of one chunk of rows, fp32 [chunk rows, d]
+    off = align256(off + static_cast<size_t>(pref) * BM * d * 4);
     L->scratch = off;
     L->fixed_end = off;
     L->p_pitch = static_cast<long long>(CT) * BN;
@@ -294,7 +298,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     Schedule full;
     rc = make_layout(N, d, V, K, di.sms, &L, &full);
     if (rc != HASS_OK) return rc;
-    if (workspace_bytes < L.fixed_end) return HASS_ERR_WORKSPACE;
+    if (workspace_bytes < L.fwd_end) return HASS_ERR_WORKSPACE;
     const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     // every public call starts with a clean status word
@@ -331,6 +335,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     p.col_tiles = CT;
     p.k_blocks = ceil_div(d, BK);
     p.K = K;
+    p.Kc = K > K_REG ? K : K_REG;
     p.part_m = reinterpret_cast<float*>(ws + L.part_m);
     p.part_s = reinterpret_cast<float*>(ws + L.part_s);
     p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
@@ -346,6 +351,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.rows = static_cast<int>(N);
     f.d = static_cast<int>(d);
     f.K = K;
+    f.Kc = K > K_REG ? K : K_REG;
     f.row_tiles_t = with_target ? RT : 0;
     f.part_m = p.part_m;
     f.part_s = p.part_s;
@@ -509,6 +515,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     float* gq = reinterpret_cast<float*>(ws + L.sgq);
     float* coef = reinterpret_cast<float*>(ws + L.coef);
+    float* sparse = reinterpret_cast<float*>(ws + L.sparse);
     __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(ws + L.scratch);
     unsigned int* status = reinterpret_cast<unsigned int*>(ws + L.status);
     if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) {
@@ -548,6 +555,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.col_tiles = CT;
         p.k_blocks = ceil_div(d, BK);
         p.K = K;
+        p.Kc = K > K_REG ? K : K_REG;
         p.part_m = reinterpret_cast<float*>(ws + L.part_m);
         p.part_s = reinterpret_cast<float*>(ws + L.part_s);
         p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
@@ -563,6 +571,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.sched = p.sched;
         f.d = static_cast<int>(d);
         f.K = K;
+        f.Kc = K > K_REG ? K : K_REG;
         f.row_begin = t0 * BM;
         f.rows = rows;
         f.row_tiles_t = with_target ? tiles : 0;
@@ -582,6 +591,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.grad_loss = grad_loss;
         f.coef_out = coef;
         f.gq_out = gq;
+        f.sparse_out = sparse;
         {
             KernelTimer timer(KIND_FINALIZE, st);
             finalize_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(f);
@@ -607,9 +617,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         o.k_blocks = ceil_div(V, BK);
         o.K = K;
         o.coef = coef;
-        o.sidx = with_target ? idx_out : idx_in;
-        o.sgq = gq;
-        o.Wg = static_cast<const __nv_bfloat16*>(W);
+        o.sparse = sparse;
         o.out = dH_d;
         o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
         o.out_pitch = d;
@@ -843,10 +851,10 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
     Layout L;
     rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
     if (rc != HASS_OK) return rc;
-    if (L.fixed_end > HASS_STATIC_SCRATCH_BYTES) {
+    if (L.fwd_end > HASS_STATIC_SCRATCH_BYTES) {
         if (kLog)
             std::fprintf(stderr, "[hass] hass_topk_distill_fwd_static: this size needs %zu bytes of scratch, the built-in "
-                         "array holds %u; use hass_topk_distill_fwd with a workspace\n", L.fixed_end,
+                         "array holds %u; use hass_topk_distill_fwd with a workspace\n", L.fwd_end,
                          HASS_STATIC_SCRATCH_BYTES);
         return HASS_ERR_UNSUPPORTED;
     }

@@ -27,6 +27,7 @@ constexpr int NUM_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, war
 constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
 constexpr int MAX_PHASES = 48;
 constexpr int K_CAP = 128;         // == HASS_K_MAX
+constexpr int K_REG = 16;          // Top-K lists up to this length live in registers
 constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -59,6 +60,7 @@ struct GemmParams {
     int col_tiles;
     int k_blocks;          // ceil(contraction extent / BK)
     int K;                 // Top-K
+    int Kc;                // candidates kept per (row, slot): max(K, K_REG)
     int spill_begin;       // MODE_STATS: row tiles >= spill_begin also write the tile 2^(z log2e - ref2) in bf16 to
                            // P (row tile index - spill_begin); INT_MAX: none
     // MODE_STATS outputs (per slot)
@@ -73,9 +75,9 @@ struct GemmParams {
     const float* sgq;      // [N, K] g * q in the same order
     __nv_bfloat16* P;      // [chunk rows, p_pitch]
     long long p_pitch;
-    // MODE_OUT. With Wg != nullptr the epilogue computes coef[row] * acc - sum_k sgq[row,k] * Wg[sidx[row,k], :]
-    // (row scale and the sparse Omega_hat term of dz_d W); otherwise it stores the accumulator.
-    const __nv_bfloat16* Wg;
+    // MODE_OUT. With sparse != nullptr the epilogue computes coef[row] * acc - sparse[local row, :] (row scale
+    // and the Omega_hat term of dz_d W, precomputed by finalize); otherwise it stores the accumulator.
+    const float* sparse;   // [chunk rows, out_pitch]
     void* out;
     int out_fp32;
     long long out_pitch;   // elements
@@ -274,6 +276,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         float lv[MODE == MODE_STATS ? K_CAP : 1];
         int li[MODE == MODE_STATS ? K_CAP : 1];
         int cnt_minpos[2];
+        // K <= K_REG: the K_REG largest logits seen so far, sorted descending, in registers
+        float tv[MODE == MODE_STATS ? K_REG : 1];
+        int ti[MODE == MODE_STATS ? K_REG : 1];
+        // logits of the current 32-column chunk that beat the admission threshold (local memory)
+        float pend_v[MODE == MODE_STATS ? 32 : 1];
+        int pend_i[MODE == MODE_STATS ? 32 : 1];
+        const bool reg_list = p.K <= K_REG;
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
@@ -291,6 +300,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 want_topk = rt < p.topk_row_tiles;
                 cnt_minpos[0] = 0;
                 cnt_minpos[1] = 0;
+#pragma unroll
+                for (int i = 0; i < K_REG; ++i) {
+                    tv[i] = -INFINITY;
+                    ti[i] = -1;
+                }
             }
             if (MODE == MODE_PROBS && row_ok) {
                 lse2 = p.lse2[g_row];
@@ -299,11 +313,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 sg = p.sgq + static_cast<long long>(g_row) * p.K;
                 nxt = si[0];
             }
-            if (MODE == MODE_OUT && p.Wg != nullptr && row_ok) {
-                coef = p.coef[g_row];
-                si = p.sidx + static_cast<long long>(g_row) * p.K;
-                sg = p.sgq + static_cast<long long>(g_row) * p.K;
-            }
+            if (MODE == MODE_OUT && p.sparse != nullptr && row_ok) coef = p.coef[g_row];
             const int t0 = (spill && ln != 0) ? -1 : 0;
             const int nt = (p.col_tiles - ln + S - 1) / S;
             for (int t = t0; t < nt; ++t) {
@@ -360,10 +370,39 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), LOG2E, mneg));
                             s += acc;
                             if (want_topk && cm > thr) {
+                                // collect the chunk's candidates, then admit them one by one (the
+                                // threshold only rises, so each is re-checked against the current one)
+                                int np = 0;
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) {
                                     const float x = __uint_as_float(r[j]);
-                                    if (x > thr) thr = topk_insert(lv, li, cnt_minpos, p.K, x, col0 + j);
+                                    if (x > thr) {
+                                        pend_v[np] = x;
+                                        pend_i[np] = col0 + j;
+                                        ++np;
+                                    }
+                                }
+                                for (int q = 0; q < np; ++q) {
+                                    const float x = pend_v[q];
+                                    const int id = pend_i[q];
+                                    if (!(x > thr)) continue;
+                                    if (reg_list) {
+                                        // sorted insertion; equal logits stay behind earlier (lower) token ids
+#pragma unroll
+                                        for (int i = K_REG - 1; i >= 1; --i) {
+                                            const bool shift = x > tv[i - 1];
+                                            const bool here = !shift && x > tv[i];
+                                            tv[i] = shift ? tv[i - 1] : (here ? x : tv[i]);
+                                            ti[i] = shift ? ti[i - 1] : (here ? id : ti[i]);
+                                        }
+                                        if (x > tv[0]) {
+                                            tv[0] = x;
+                                            ti[0] = id;
+                                        }
+                                        thr = tv[K_REG - 1];
+                                    } else {
+                                        thr = topk_insert(lv, li, cnt_minpos, p.K, x, id);
+                                    }
                                 }
                             }
                         } else {
@@ -424,25 +463,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                         float o[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(r[j]);
-                        if (p.Wg != nullptr) {
+                        if (p.sparse != nullptr) {
                             // dH_d = coef * (spilled tile x W) - sum_{x in Omega_hat} g q(x) W[x, :]
+                            const float* sp = p.sparse + static_cast<long long>(rt * BM + r_local) * p.out_pitch + col0;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) o[j] *= coef;
-                            for (int k = 0; k < p.K; ++k) {
-                                const float gq = sg[k];
-                                const __nv_bfloat16* wr = p.Wg + static_cast<long long>(si[k]) * p.out_pitch + col0;
-#pragma unroll
-                                for (int g8 = 0; g8 < 4; ++g8) {
-                                    if (col0 + 8 * g8 < p.n_cols) {
-                                        const uint4 wv = *reinterpret_cast<const uint4*>(wr + 8 * g8);
-                                        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
-#pragma unroll
-                                        for (int u = 0; u < 4; ++u) {
-                                            const float2 w2 = __bfloat1622float2(wp[u]);
-                                            o[8 * g8 + 2 * u] = fmaf(-gq, w2.x, o[8 * g8 + 2 * u]);
-                                            o[8 * g8 + 2 * u + 1] = fmaf(-gq, w2.y, o[8 * g8 + 2 * u + 1]);
-                                        }
-                                    }
+                            for (int g4 = 0; g4 < 8; ++g4) {
+                                if (col0 + 4 * g4 < p.n_cols) {
+                                    const float4 v = *reinterpret_cast<const float4*>(sp + 4 * g4);
+                                    o[4 * g4 + 0] = fmaf(coef, o[4 * g4 + 0], -v.x);
+                                    o[4 * g4 + 1] = fmaf(coef, o[4 * g4 + 1], -v.y);
+                                    o[4 * g4 + 2] = fmaf(coef, o[4 * g4 + 2], -v.z);
+                                    o[4 * g4 + 3] = fmaf(coef, o[4 * g4 + 3], -v.w);
                                 }
                             }
                         }
@@ -484,11 +515,20 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 // above its reference for the fixed-exponent spill
                 if (spill && !(s < 1e38f)) atomicCAS(p.status, 0u, (5u << 8) | 2u);
                 if (want_topk) {
-                    const int cnt = cnt_minpos[0];
-                    for (int k = 0; k < p.K; ++k) {
-                        const long long co = (static_cast<long long>(slot) * p.K + k) * BM + r_local;
-                        p.cand_v[co] = k < cnt ? lv[k] : -INFINITY;
-                        p.cand_i[co] = k < cnt ? li[k] : -1;
+                    if (reg_list) {
+#pragma unroll
+                        for (int k = 0; k < K_REG; ++k) {
+                            const long long co = (static_cast<long long>(slot) * K_REG + k) * BM + r_local;
+                            p.cand_v[co] = tv[k];
+                            p.cand_i[co] = ti[k];
+                        }
+                    } else {
+                        const int cnt = cnt_minpos[0];
+                        for (int k = 0; k < p.K; ++k) {
+                            const long long co = (static_cast<long long>(slot) * p.K + k) * BM + r_local;
+                            p.cand_v[co] = k < cnt ? lv[k] : -INFINITY;
+                            p.cand_i[co] = k < cnt ? li[k] : -1;
+                        }
                     }
                 }
             }
@@ -517,6 +557,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 struct FinalizeParams {
     Schedule sched;
     int d, K;
+    int Kc;                // candidates per (row, slot) written by the sweep
     int row_begin, rows;   // global rows [row_begin, row_begin + rows) = local row tiles 0.. of the schedule
     int row_tiles_t;       // row tiles of the target matrix in the schedule (0: Omega_hat is an input)
     const float* part_m;
@@ -536,6 +577,7 @@ struct FinalizeParams {
     const float* grad_loss;
     float* coef_out;       // [N]   g * S_q * exp(m_spill - lse_d), m_spill = the row's spill reference
     float* gq_out;         // [N,K] g * q, in the order of topk_idx
+    float* sparse_out;     // [rows, d] sum_{x in Omega_hat} g q(x) W[x, :], indexed by local row
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -594,7 +636,11 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     float loss = 0.f;
     float prev_v = INFINITY;
     int prev_i = -1;
-    const int C = S * K;   // candidates of this row (target path)
+    const int Kc = p.Kc;
+    const int C = S * Kc;  // candidates of this row (target path)
+    __shared__ int sh_tok[8][K_CAP];
+    __shared__ float sh_gq[8][K_CAP];
+    const int wib = threadIdx.x >> 5;
     for (int j = 0; j < K; ++j) {
         int tok;
         float qv;
@@ -603,7 +649,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             float bv = -INFINITY;
             int bi = INT_MAX;
             for (int c = lane; c < C; c += 32) {
-                const long long co = (static_cast<long long>(slot0 + c / K) * K + (c % K)) * BM + r;
+                const long long co = (static_cast<long long>(slot0 + c / Kc) * Kc + (c % Kc)) * BM + r;
                 const float v = p.cand_v[co];
                 const int i = p.cand_i[co];
                 if (i < 0) continue;
@@ -655,7 +701,32 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
         S_q += qv;
-        if (lane == 0 && p.gq_out) p.gq_out[static_cast<long long>(row) * K + j] = g * qv;
+        if (lane == 0) {
+            if (p.gq_out) p.gq_out[static_cast<long long>(row) * K + j] = g * qv;
+            sh_tok[wib][j] = tok;
+            sh_gq[wib][j] = g * qv;
+        }
+    }
+    if (p.sparse_out) {
+        // the Omega_hat term of dz_d W for this row, 256 columns (8 per lane) at a time
+        __syncwarp();
+        float* so = p.sparse_out + static_cast<long long>(local) * p.d;
+        for (int k0 = lane * 8; k0 < p.d; k0 += 256) {
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < K; ++j) {
+                const float gq = sh_gq[wib][j];
+                const uint4 wv = *reinterpret_cast<const uint4*>(p.W + static_cast<long long>(sh_tok[wib][j]) * p.d + k0);
+                const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float2 b = __bfloat1622float2(wp[t]);
+                    a[2 * t] = fmaf(gq, b.x, a[2 * t]);
+                    a[2 * t + 1] = fmaf(gq, b.y, a[2 * t + 1]);
+                }
+            }
+            *reinterpret_cast<float4*>(so + k0) = make_float4(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<float4*>(so + k0 + 4) = make_float4(a[4], a[5], a[6], a[7]);
+        }
     }
     if (lane == 0) {
         p.loss[row] = loss;

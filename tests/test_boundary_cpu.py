@@ -37,7 +37,7 @@ def test_workspace_bytes_is_bounded_in_N(hass):
     a = hass.topk_distill_workspace_bytes(8192, 4096, 128256, 10)
     b = hass.topk_distill_workspace_bytes(65536, 4096, 128256, 10)
     scratch = 37 * 128 * 128256 * 2          # one chunk of dz_d rows, independent of N
-    assert scratch <= a < scratch + (64 << 20)
+    assert scratch <= a < scratch + (160 << 20)   # + statistics, lists and the fp32 Omega_hat term of one chunk
     assert b - a < (256 << 20)               # grows only by O(N K) lists and partial statistics
     assert a < 8192 * 128256 * 2             # less than one N x V bf16 matrix
 
