@@ -473,6 +473,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
         o.K = K;
         o.out = dH_d;
         o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+        o.out_align32 = ((reinterpret_cast<uintptr_t>(dH_d) | static_cast<uintptr_t>(d * (dH_dtype == HASS_FP32 ? 4 : 2))) & 31u) == 0 ? 1 : 0;
         o.out_pitch = d;
         o.status = p.status;
         rc = launch_gemm<MODE_OUT>(o, st);
@@ -620,6 +621,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         o.sparse = sparse;
         o.out = dH_d;
         o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+        o.out_align32 = ((reinterpret_cast<uintptr_t>(dH_d) | static_cast<uintptr_t>(d * (dH_dtype == HASS_FP32 ? 4 : 2))) & 31u) == 0 ? 1 : 0;
         o.out_pitch = d;
         o.status = status;
         rc = launch_gemm<MODE_OUT>(o, st);

@@ -80,6 +80,7 @@ struct GemmParams {
     const float* sparse;   // [chunk rows, out_pitch]
     void* out;
     int out_fp32;
+    int out_align32;       // out base and row pitch are multiples of 32 bytes (256-bit stores allowed)
     long long out_pitch;   // elements
     unsigned int* status;
 };
@@ -406,26 +407,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 }
                             }
                         } else {
-                            // one exponential per logit serves both the row's sum and the spilled tile
+                            // one exponential per logit serves both the row's sum and the spilled tile; a
+                            // logit beyond the exponent range gives inf here and is reported at the item's end
                             float e[32];
                             float acc = 0.f;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                e[j] = ex2(fminf(fmaf(__uint_as_float(r[j]), LOG2E, -ref2), 127.f));
+                                e[j] = ex2(fmaf(__uint_as_float(r[j]), LOG2E, -ref2));
                                 acc += e[j];
                             }
                             s += acc;
-                            uint4* dst = reinterpret_cast<uint4*>(
-                                p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch + col0);
+                            __nv_bfloat16* dst =
+                                p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch + col0;
 #pragma unroll
-                            for (int g8 = 0; g8 < 4; ++g8) {
-                                uint4 w;
-                                w.x = pack_bf16x2(e[8 * g8 + 0], e[8 * g8 + 1]);
-                                w.y = pack_bf16x2(e[8 * g8 + 2], e[8 * g8 + 3]);
-                                w.z = pack_bf16x2(e[8 * g8 + 4], e[8 * g8 + 5]);
-                                w.w = pack_bf16x2(e[8 * g8 + 6], e[8 * g8 + 7]);
-                                dst[g8] = w;
-                            }
+                            for (int g16 = 0; g16 < 2; ++g16)
+                                st_global_v8(dst + 16 * g16, pack_bf16x2(e[16 * g16 + 0], e[16 * g16 + 1]),
+                                             pack_bf16x2(e[16 * g16 + 2], e[16 * g16 + 3]),
+                                             pack_bf16x2(e[16 * g16 + 4], e[16 * g16 + 5]),
+                                             pack_bf16x2(e[16 * g16 + 6], e[16 * g16 + 7]),
+                                             pack_bf16x2(e[16 * g16 + 8], e[16 * g16 + 9]),
+                                             pack_bf16x2(e[16 * g16 + 10], e[16 * g16 + 11]),
+                                             pack_bf16x2(e[16 * g16 + 12], e[16 * g16 + 13]),
+                                             pack_bf16x2(e[16 * g16 + 14], e[16 * g16 + 15]));
                         }
                     } else if (MODE == MODE_PROBS) {
                         while (nxt < col0) {
@@ -463,38 +466,71 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                         float o[32];
 #pragma unroll
                         for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(r[j]);
+                        const bool full = col0 + 32 <= p.n_cols;
                         if (p.sparse != nullptr) {
                             // dH_d = coef * (spilled tile x W) - sum_{x in Omega_hat} g q(x) W[x, :]
                             const float* sp = p.sparse + static_cast<long long>(rt * BM + r_local) * p.out_pitch + col0;
+                            if (full) {
 #pragma unroll
-                            for (int g4 = 0; g4 < 8; ++g4) {
-                                if (col0 + 4 * g4 < p.n_cols) {
-                                    const float4 v = *reinterpret_cast<const float4*>(sp + 4 * g4);
-                                    o[4 * g4 + 0] = fmaf(coef, o[4 * g4 + 0], -v.x);
-                                    o[4 * g4 + 1] = fmaf(coef, o[4 * g4 + 1], -v.y);
-                                    o[4 * g4 + 2] = fmaf(coef, o[4 * g4 + 2], -v.z);
-                                    o[4 * g4 + 3] = fmaf(coef, o[4 * g4 + 3], -v.w);
+                                for (int g8 = 0; g8 < 4; ++g8) {
+                                    float v[8];
+                                    ld_global_v8(sp + 8 * g8, v);
+#pragma unroll
+                                    for (int u = 0; u < 8; ++u) o[8 * g8 + u] = fmaf(coef, o[8 * g8 + u], -v[u]);
+                                }
+                            } else {
+#pragma unroll
+                                for (int g4 = 0; g4 < 8; ++g4) {
+                                    if (col0 + 4 * g4 < p.n_cols) {
+                                        const float4 v = *reinterpret_cast<const float4*>(sp + 4 * g4);
+                                        o[4 * g4 + 0] = fmaf(coef, o[4 * g4 + 0], -v.x);
+                                        o[4 * g4 + 1] = fmaf(coef, o[4 * g4 + 1], -v.y);
+                                        o[4 * g4 + 2] = fmaf(coef, o[4 * g4 + 2], -v.z);
+                                        o[4 * g4 + 3] = fmaf(coef, o[4 * g4 + 3], -v.w);
+                                    }
                                 }
                             }
                         }
                         if (p.out_fp32) {
                             float* dst = reinterpret_cast<float*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+                            if (full && p.out_align32) {
 #pragma unroll
-                            for (int g4 = 0; g4 < 8; ++g4)
-                                if (col0 + 4 * g4 < p.n_cols)
-                                    *reinterpret_cast<float4*>(dst + 4 * g4) =
-                                        make_float4(o[4 * g4], o[4 * g4 + 1], o[4 * g4 + 2], o[4 * g4 + 3]);
+                                for (int g8 = 0; g8 < 4; ++g8)
+                                    st_global_v8(dst + 8 * g8, __float_as_uint(o[8 * g8]), __float_as_uint(o[8 * g8 + 1]),
+                                                 __float_as_uint(o[8 * g8 + 2]), __float_as_uint(o[8 * g8 + 3]),
+                                                 __float_as_uint(o[8 * g8 + 4]), __float_as_uint(o[8 * g8 + 5]),
+                                                 __float_as_uint(o[8 * g8 + 6]), __float_as_uint(o[8 * g8 + 7]));
+                            } else {
+#pragma unroll
+                                for (int g4 = 0; g4 < 8; ++g4)
+                                    if (col0 + 4 * g4 < p.n_cols)
+                                        *reinterpret_cast<float4*>(dst + 4 * g4) =
+                                            make_float4(o[4 * g4], o[4 * g4 + 1], o[4 * g4 + 2], o[4 * g4 + 3]);
+                            }
                         } else {
                             __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
+                            if (full && p.out_align32) {
 #pragma unroll
-                            for (int g8 = 0; g8 < 4; ++g8) {
-                                if (col0 + 8 * g8 < p.n_cols) {
-                                    uint4 w;
-                                    w.x = pack_bf16x2(o[8 * g8 + 0], o[8 * g8 + 1]);
-                                    w.y = pack_bf16x2(o[8 * g8 + 2], o[8 * g8 + 3]);
-                                    w.z = pack_bf16x2(o[8 * g8 + 4], o[8 * g8 + 5]);
-                                    w.w = pack_bf16x2(o[8 * g8 + 6], o[8 * g8 + 7]);
-                                    *reinterpret_cast<uint4*>(dst + 8 * g8) = w;
+                                for (int g16 = 0; g16 < 2; ++g16)
+                                    st_global_v8(dst + 16 * g16, pack_bf16x2(o[16 * g16 + 0], o[16 * g16 + 1]),
+                                                 pack_bf16x2(o[16 * g16 + 2], o[16 * g16 + 3]),
+                                                 pack_bf16x2(o[16 * g16 + 4], o[16 * g16 + 5]),
+                                                 pack_bf16x2(o[16 * g16 + 6], o[16 * g16 + 7]),
+                                                 pack_bf16x2(o[16 * g16 + 8], o[16 * g16 + 9]),
+                                                 pack_bf16x2(o[16 * g16 + 10], o[16 * g16 + 11]),
+                                                 pack_bf16x2(o[16 * g16 + 12], o[16 * g16 + 13]),
+                                                 pack_bf16x2(o[16 * g16 + 14], o[16 * g16 + 15]));
+                            } else {
+#pragma unroll
+                                for (int g8 = 0; g8 < 4; ++g8) {
+                                    if (col0 + 8 * g8 < p.n_cols) {
+                                        uint4 w;
+                                        w.x = pack_bf16x2(o[8 * g8 + 0], o[8 * g8 + 1]);
+                                        w.y = pack_bf16x2(o[8 * g8 + 2], o[8 * g8 + 3]);
+                                        w.z = pack_bf16x2(o[8 * g8 + 4], o[8 * g8 + 5]);
+                                        w.w = pack_bf16x2(o[8 * g8 + 6], o[8 * g8 + 7]);
+                                        *reinterpret_cast<uint4*>(dst + 8 * g8) = w;
+                                    }
                                 }
                             }
                         }

@@ -142,6 +142,28 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
                    "+r"(r[29]), "+r"(r[30]), "+r"(r[31])::"memory");
 }
 
+// ---- 256-bit global accesses (address must be 32-byte aligned) ---------------------------------
+__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
+                                             uint32_t f, uint32_t g, uint32_t h) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(a), "r"(b), "r"(c), "r"(d),
+                 "r"(e), "r"(f), "r"(g), "r"(h)
+                 : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const void* ptr, float (&v)[8]) {
+    uint32_t a, b, c, d, e, f, g, h;
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(a), "=r"(b), "=r"(c), "=r"(d), "=r"(e), "=r"(f), "=r"(g), "=r"(h)
+                 : "l"(ptr));
+    v[0] = __uint_as_float(a);
+    v[1] = __uint_as_float(b);
+    v[2] = __uint_as_float(c);
+    v[3] = __uint_as_float(d);
+    v[4] = __uint_as_float(e);
+    v[5] = __uint_as_float(f);
+    v[6] = __uint_as_float(g);
+    v[7] = __uint_as_float(h);
+}
+
 // ---- descriptors ------------------------------------------------------------------------------
 // Shared-memory matrix descriptor (tcgen05): start address, leading/stride byte offsets (all >> 4),
 // descriptor version 1, 128-byte swizzle.
