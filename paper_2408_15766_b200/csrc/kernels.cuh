@@ -358,18 +358,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 if (col0 + j >= p.n_cols) r[j] = __float_as_uint(-INFINITY);
                         }
                         if (!spill) {
-                            float cm = __uint_as_float(r[0]);
+                            float cm = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1]));
 #pragma unroll
-                            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
+                            for (int j = 2; j < 32; j += 2) cm = fmax3(cm, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
                             if (cm > m) {
                                 s *= ex2((m - cm) * LOG2E);
                                 m = cm;
                             }
                             const float mneg = -m * LOG2E;
-                            float acc = 0.f;
+                            float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) acc += ex2(fmaf(__uint_as_float(r[j]), LOG2E, mneg));
-                            s += acc;
+                            for (int j = 0; j < 32; j += 2) {
+                                float t0, t1;
+                                ffma2(t0, t1, __uint_as_float(r[j]), __uint_as_float(r[j + 1]), LOG2E, LOG2E, mneg, mneg);
+                                fadd2(acc0, acc1, acc0, acc1, ex2(t0), ex2(t1));
+                            }
+                            s += acc0 + acc1;
                             if (want_topk && cm > thr) {
                                 // collect the chunk's candidates, then admit them one by one (the
                                 // threshold only rises, so each is re-checked against the current one)
@@ -410,13 +414,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             // one exponential per logit serves both the row's sum and the spilled tile; a
                             // logit beyond the exponent range gives inf here and is reported at the item's end
                             float e[32];
-                            float acc = 0.f;
+                            float acc0 = 0.f, acc1 = 0.f;
+                            const float nref2 = -ref2;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                e[j] = ex2(fmaf(__uint_as_float(r[j]), LOG2E, -ref2));
-                                acc += e[j];
+                            for (int j = 0; j < 32; j += 2) {
+                                float t0, t1;
+                                ffma2(t0, t1, __uint_as_float(r[j]), __uint_as_float(r[j + 1]), LOG2E, LOG2E, nref2, nref2);
+                                e[j] = ex2(t0);
+                                e[j + 1] = ex2(t1);
+                                fadd2(acc0, acc1, acc0, acc1, e[j], e[j + 1]);
                             }
-                            s += acc;
+                            s += acc0 + acc1;
                             __nv_bfloat16* dst =
                                 p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch + col0;
 #pragma unroll
