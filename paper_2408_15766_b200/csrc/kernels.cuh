@@ -28,7 +28,6 @@ constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
 constexpr int MAX_PHASES = 48;
 constexpr int K_CAP = 128;         // == HASS_K_MAX
 constexpr int K_REG = 16;          // Top-K lists up to this length live in registers
-constexpr int PEND_CAP = 64;       // pending Top-K candidates per row between two admission passes
 constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -281,11 +280,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         // K <= K_REG: the K_REG largest logits seen so far, sorted descending, in registers
         float tv[MODE == MODE_STATS ? K_REG : 1];
         int ti[MODE == MODE_STATS ? K_REG : 1];
-        // logits of the current tile that beat the admission threshold, waiting to be admitted (local memory)
-        float pend_v[MODE == MODE_STATS ? PEND_CAP : 1];
-        int pend_i[MODE == MODE_STATS ? PEND_CAP : 1];
+        // logits of the current 32-column chunk that beat the admission threshold (local memory)
+        float pend_v[MODE == MODE_STATS ? 32 : 1];
+        int pend_i[MODE == MODE_STATS ? 32 : 1];
         const bool reg_list = p.K <= K_REG;
-        const int lo = reg_list ? K_REG - p.K : 0;   // the register list occupies slots lo .. K_REG-1
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
@@ -317,37 +315,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 nxt = si[0];
             }
             if (MODE == MODE_OUT && p.sparse != nullptr && row_ok) coef = p.coef[g_row];
-            int np = 0;   // pending candidates of this row
-            // Admits the pending candidates in order. The threshold only rises, so each one is checked
-            // again; equal logits stay behind earlier (lower) token ids. With K <= K_REG the list is
-            // sorted descending in registers tv[lo .. K_REG-1], so the K-th largest is always tv[K_REG-1].
-            auto flush_pending = [&]() {
-                for (int q = 0; q < np; ++q) {
-                    const float x = pend_v[q];
-                    const int id = pend_i[q];
-                    if (!(x > thr)) continue;
-                    if (reg_list) {
-#pragma unroll
-                        for (int i = K_REG - 1; i >= 0; --i) {
-                            if (i > 0 && i > lo) {
-                                const bool shift = x > tv[i > 0 ? i - 1 : 0];
-                                const bool here = !shift && x > tv[i];
-                                tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
-                                ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
-                            } else if (i == lo) {
-                                if (x > tv[i]) {
-                                    tv[i] = x;
-                                    ti[i] = id;
-                                }
-                            }
-                        }
-                        thr = tv[K_REG - 1];
-                    } else {
-                        thr = topk_insert(lv, li, cnt_minpos, p.K, x, id);
-                    }
-                }
-                np = 0;
-            };
             const int t0 = (spill && ln != 0) ? -1 : 0;
             const int nt = (p.col_tiles - ln + S - 1) / S;
             for (int t = t0; t < nt; ++t) {
@@ -385,8 +352,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     tmem_ld_wait(r);
                     const int col0 = col_base + ch * 32;
                     if (MODE == MODE_STATS) {
-                        // room for a whole chunk in every row's pending buffer
-                        if (want_topk && __any_sync(0xffffffffu, np > PEND_CAP - 32)) flush_pending();
                         if (col0 + 32 > p.n_cols) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -410,7 +375,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             }
                             s += acc0 + acc1;
                             if (want_topk && cm > thr) {
-                                // collect the chunk's candidates; they are admitted in batches (flush_pending)
+                                // collect the chunk's candidates, then admit them one by one (the
+                                // threshold only rises, so each is re-checked against the current one)
+                                int np = 0;
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) {
                                     const float x = __uint_as_float(r[j]);
@@ -418,6 +385,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                         pend_v[np] = x;
                                         pend_i[np] = col0 + j;
                                         ++np;
+                                    }
+                                }
+                                for (int q = 0; q < np; ++q) {
+                                    const float x = pend_v[q];
+                                    const int id = pend_i[q];
+                                    if (!(x > thr)) continue;
+                                    if (reg_list) {
+                                        // sorted insertion; equal logits stay behind earlier (lower) token ids
+#pragma unroll
+                                        for (int i = K_REG - 1; i >= 1; --i) {
+                                            const bool shift = x > tv[i - 1];
+                                            const bool here = !shift && x > tv[i];
+                                            tv[i] = shift ? tv[i - 1] : (here ? x : tv[i]);
+                                            ti[i] = shift ? ti[i - 1] : (here ? id : ti[i]);
+                                        }
+                                        if (x > tv[0]) {
+                                            tv[0] = x;
+                                            ti[0] = id;
+                                        }
+                                        thr = tv[K_REG - 1];
+                                    } else {
+                                        thr = topk_insert(lv, li, cnt_minpos, p.K, x, id);
                                     }
                                 }
                             }
@@ -561,7 +550,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 if (lane == 0) mbar_arrive(tempty_bar(ab));
                 ab ^= 1;
                 if (ab == 0) aphase ^= 1u;
-                if (MODE == MODE_STATS && want_topk) flush_pending();
             }
             if (MODE == MODE_STATS) {
                 const long long so = static_cast<long long>(slot) * BM + r_local;
