@@ -96,36 +96,56 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Replace-the-minimum insertion into an unsorted K-list kept in local memory. Returns the new
-// admission threshold: -inf while the list is not full, else its smallest value. Among equal
-// smallest values the one with the highest token id is the next to be evicted, and admission is
-// strict (x > threshold) with token ids visited in increasing order, so equal logits resolve to
-// the lower token id.
+// Top-K list for K > K_REG: a binary min-heap in local memory, ordered so that the root is the entry
+// to evict next (smallest logit; among equal logits the highest token id). Returns the new admission
+// threshold: -inf while the list is not full, else the root's logit. Admission is strict (x > threshold)
+// and token ids arrive in increasing order, so equal logits resolve to the lower token id.
+__device__ __forceinline__ bool heap_before(float av, int ai, float bv, int bi) {
+    return av < bv || (av == bv && ai > bi);
+}
 __device__ __noinline__ float topk_insert(float* lv, int* li, int* cnt_minpos, int K, float x, int idx) {
     int cnt = cnt_minpos[0];
     if (cnt < K) {
-        lv[cnt] = x;
-        li[cnt] = idx;
-        cnt_minpos[0] = ++cnt;
-        if (cnt < K) return -INFINITY;
-    } else {
-        const int mp = cnt_minpos[1];
-        lv[mp] = x;
-        li[mp] = idx;
-    }
-    float mn = lv[0];
-    int mi = li[0], mp = 0;
-    for (int j = 1; j < K; ++j) {
-        const float a = lv[j];
-        const int b = li[j];
-        if (a < mn || (a == mn && b > mi)) {
-            mn = a;
-            mi = b;
-            mp = j;
+        // sift up from the new leaf
+        int pos = cnt;
+        while (pos > 0) {
+            const int par = (pos - 1) >> 1;
+            const float pv = lv[par];
+            const int pi = li[par];
+            if (!heap_before(x, idx, pv, pi)) break;
+            lv[pos] = pv;
+            li[pos] = pi;
+            pos = par;
         }
+        lv[pos] = x;
+        li[pos] = idx;
+        cnt_minpos[0] = ++cnt;
+        return cnt < K ? -INFINITY : lv[0];
     }
-    cnt_minpos[1] = mp;
-    return mn;
+    // replace the root and sift down
+    int pos = 0;
+    while (true) {
+        int c = 2 * pos + 1;
+        if (c >= K) break;
+        float cv = lv[c];
+        int ci = li[c];
+        if (c + 1 < K) {
+            const float rv = lv[c + 1];
+            const int ri = li[c + 1];
+            if (heap_before(rv, ri, cv, ci)) {
+                cv = rv;
+                ci = ri;
+                ++c;
+            }
+        }
+        if (!heap_before(cv, ci, x, idx)) break;
+        lv[pos] = cv;
+        li[pos] = ci;
+        pos = c;
+    }
+    lv[pos] = x;
+    li[pos] = idx;
+    return lv[0];
 }
 
 template <int MODE>
@@ -284,6 +304,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         float pend_v[MODE == MODE_STATS ? 32 : 1];
         int pend_i[MODE == MODE_STATS ? 32 : 1];
         const bool reg_list = p.K <= K_REG;
+        const int lo = reg_list ? K_REG - p.K : 0;   // the register list occupies slots lo .. K_REG-1
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
@@ -392,17 +413,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                     const int id = pend_i[q];
                                     if (!(x > thr)) continue;
                                     if (reg_list) {
-                                        // sorted insertion; equal logits stay behind earlier (lower) token ids
+                                        // sorted insertion into tv[lo .. K_REG-1] (descending), so the K-th largest
+                                        // is always tv[K_REG-1]; equal logits stay behind earlier (lower) token ids
 #pragma unroll
-                                        for (int i = K_REG - 1; i >= 1; --i) {
-                                            const bool shift = x > tv[i - 1];
-                                            const bool here = !shift && x > tv[i];
-                                            tv[i] = shift ? tv[i - 1] : (here ? x : tv[i]);
-                                            ti[i] = shift ? ti[i - 1] : (here ? id : ti[i]);
-                                        }
-                                        if (x > tv[0]) {
-                                            tv[0] = x;
-                                            ti[0] = id;
+                                        for (int i = K_REG - 1; i >= 0; --i) {
+                                            if (i > 0 && i > lo) {
+                                                const bool shift = x > tv[i > 0 ? i - 1 : 0];
+                                                const bool here = !shift && x > tv[i];
+                                                tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
+                                                ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
+                                            } else if (i == lo) {
+                                                if (x > tv[i]) {
+                                                    tv[i] = x;
+                                                    ti[i] = id;
+                                                }
+                                            }
                                         }
                                         thr = tv[K_REG - 1];
                                     } else {
