@@ -32,6 +32,10 @@ import hass_inputs as hi  # noqa: E402
 
 METRIC = "tokens/sec fused top-K distill fwd+bwd"
 UNIT = "tokens/s"
+# dram__bytes_read + dram__bytes_write of the dominant kernel (the logits sweep) per launch, from the ncu
+# capture summarised in profiles/gemm_kernel_l2-7b_ncu_full.md (l2-7b shape, mean of the two chunk launches),
+# scaled to the bench shape by the vocabulary ratio; valid for the library version it was taken with.
+TRAFFIC_CAPTURE = {"version": 10100, "workload": "l3-8b", "bytes_per_launch": 1.11e9 * 128256 / 32000}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -290,7 +294,10 @@ def main():
     achieved = flops_per_launch / (dom_ms / dom_cnt * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops_sustained"])
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak,
+                "traffic": (TRAFFIC_CAPTURE["bytes_per_launch"]
+                            if dom == "stats_gemm" and wl.name == TRAFFIC_CAPTURE["workload"]
+                            and hass.version() == TRAFFIC_CAPTURE["version"] else None),
                 "peak_kind": f"bf16_tflops_sustained, of {peak_kind} (kernel timed inside a long step)",
                 "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
                 "flops_per_launch": flops_per_launch, "avg_launch_ms": dom_ms / dom_cnt}
@@ -302,7 +309,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "N": N, "d": d, "V": V, "K": K, "rows_per_gpu": N,
                        "l2": "inputs larger than L2 (W alone is %.0f MB)" % (V * d * 2 / 1e6),
-                       "dH_dtype": "bf16", "target_stats": "recomputed every step"},
+                       "dH_dtype": "bf16", "target_stats": "recomputed every step", "path": "hass_topk_distill_fwd_bwd (no logit recompute)"},
             "clocks": clocks, "gpu_launches": launches,
             "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
                        "executed_tflops": executed / (ms_step * 1e-3) / 1e12, "executed_flops_per_step": executed,
