@@ -197,9 +197,9 @@ int64_t hass_kernel_launch_count(void);
  * cudaFree imply. For them the partial softmax statistics and Top-K candidates of the forward
  * sweep live in an array built into the library's device image instead of a caller workspace.
  *
- *   - The array is HASS_STATIC_SCRATCH_MAX_BYTES (16 MiB) and every GPU that loads the library
+ *   - The array is HASS_STATIC_SCRATCH_MAX_BYTES (32 MiB) and every GPU that loads the library
  *     holds it until the process exits. A problem whose forward scratch does not fit (it grows
- *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits up to K = 31) is refused
+ *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits up to K = 32) is refused
  *     with HASS_ERR_UNSUPPORTED; use hass_topk_distill_fwd with a workspace then.
  *   - The call allocates and frees nothing, in this library or through any other.
  *   - The first call on each device looks up the array's device address (a CUDA runtime query,
@@ -212,7 +212,7 @@ int64_t hass_kernel_launch_count(void);
  *     non-zero code of a bounded device-side wait that gave up (outputs are then undefined);
  *     it replaces hass_check, which needs a workspace pointer.
  */
-#define HASS_STATIC_SCRATCH_MAX_BYTES (16u << 20)
+#define HASS_STATIC_SCRATCH_MAX_BYTES (32u << 20)
 int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                                  int64_t V, int32_t K, float* loss, int32_t* topk_idx, float* topk_q,
                                  float* lse_t, float* lse_d, unsigned int* device_status,

@@ -135,7 +135,7 @@ def topk_distill_fwd(H_t, H_d, W, K: int, workspace=None, stream=None) -> dict:
 
 
 def topk_distill_fwd_static(H_t, H_d, W, K: int, stream=None, out: Optional[dict] = None) -> dict:
-    """Forward for callers that cannot hand the library a workspace: the library's built-in 16 MiB
+    """Forward for callers that cannot hand the library a workspace: the library's built-in 32 MiB
     scratch array is used instead. Here the outputs are still torch tensors, created by this wrapper
     when ``out`` is not given; pass preallocated ``out`` tensors to make the call allocation-free end
     to end. ``out['device_status']`` (uint32[1]) is 0 after a clean run."""

@@ -219,11 +219,10 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     off = align256(off + slots * BM * 4);
     L->part_s = off;
     off = align256(off + slots * BM * 4);
-    const int Kc = K > K_REG ? K : K_REG;   // candidates per (row, slot)
-    L->cand_v = off;
-    off = align256(off + slots * BM * 4 * Kc);
-    L->cand_i = off;
-    off = align256(off + slots * BM * 4 * Kc);
+    L->cand_v = off;                        // candidate buffers: (logit, token id) pairs, cand_cap(K) per (row, slot)
+    off = align256(off + slots * BM * 8 * cand_cap(K));
+    L->cand_i = off;                        // entries in use per (row, slot)
+    off = align256(off + slots * BM * 4);
     L->fwd_end = off;                       // what the forward-only entry points use
     L->sidx = off;
     off = align256(off + static_cast<size_t>(N) * K * 4);
@@ -335,11 +334,11 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     p.col_tiles = CT;
     p.k_blocks = ceil_div(d, BK);
     p.K = K;
-    p.Kc = K > K_REG ? K : K_REG;
+    p.cap = cand_cap(K);
     p.part_m = reinterpret_cast<float*>(ws + L.part_m);
     p.part_s = reinterpret_cast<float*>(ws + L.part_s);
-    p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
-    p.cand_i = reinterpret_cast<int*>(ws + L.cand_i);
+    p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
+    p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
     p.status = reinterpret_cast<unsigned int*>(ws + L.status);
     rc = launch_gemm<MODE_STATS>(p, st);
     if (rc != HASS_OK) return rc;
@@ -351,12 +350,12 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.rows = static_cast<int>(N);
     f.d = static_cast<int>(d);
     f.K = K;
-    f.Kc = K > K_REG ? K : K_REG;
+    f.cap = cand_cap(K);
     f.row_tiles_t = with_target ? RT : 0;
     f.part_m = p.part_m;
     f.part_s = p.part_s;
-    f.cand_v = p.cand_v;
-    f.cand_i = p.cand_i;
+    f.cand = p.cand;
+    f.cand_n = p.cand_n;
     f.H_d = static_cast<const __nv_bfloat16*>(H_d);
     f.W = static_cast<const __nv_bfloat16*>(W);
     f.idx_in = idx_in;
@@ -556,11 +555,11 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.col_tiles = CT;
         p.k_blocks = ceil_div(d, BK);
         p.K = K;
-        p.Kc = K > K_REG ? K : K_REG;
+        p.cap = cand_cap(K);
         p.part_m = reinterpret_cast<float*>(ws + L.part_m);
         p.part_s = reinterpret_cast<float*>(ws + L.part_s);
-        p.cand_v = reinterpret_cast<float*>(ws + L.cand_v);
-        p.cand_i = reinterpret_cast<int*>(ws + L.cand_i);
+        p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
+        p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
         p.P = P;
         p.p_pitch = L.p_pitch;
         p.status = status;
@@ -572,14 +571,14 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.sched = p.sched;
         f.d = static_cast<int>(d);
         f.K = K;
-        f.Kc = K > K_REG ? K : K_REG;
+        f.cap = cand_cap(K);
         f.row_begin = t0 * BM;
         f.rows = rows;
         f.row_tiles_t = with_target ? tiles : 0;
         f.part_m = p.part_m;
         f.part_s = p.part_s;
-        f.cand_v = p.cand_v;
-        f.cand_i = p.cand_i;
+        f.cand = p.cand;
+        f.cand_n = p.cand_n;
         f.H_d = static_cast<const __nv_bfloat16*>(H_d);
         f.W = static_cast<const __nv_bfloat16*>(W);
         f.idx_in = idx_in;
@@ -835,7 +834,7 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
 // ---- forward without a caller-provided workspace -------------------------------------------------
 // Scratch of hass_topk_distill_fwd_static: lives in the library's device image, so every GPU that
 // loads the library holds these bytes until the process exits.
-#define HASS_STATIC_SCRATCH_BYTES (16u << 20)
+#define HASS_STATIC_SCRATCH_BYTES (32u << 20)
 static __device__ __align__(256) unsigned char g_static_scratch[HASS_STATIC_SCRATCH_BYTES];
 // Device address of g_static_scratch per device. In host code the symbol itself is only a handle
 // for the runtime, never a pointer a kernel may use; the address comes from cudaGetSymbolAddress.

@@ -27,7 +27,6 @@ constexpr int NUM_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, war
 constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
 constexpr int MAX_PHASES = 48;
 constexpr int K_CAP = 128;         // == HASS_K_MAX
-constexpr int K_REG = 16;          // Top-K lists up to this length live in registers
 constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -60,14 +59,14 @@ struct GemmParams {
     int col_tiles;
     int k_blocks;          // ceil(contraction extent / BK)
     int K;                 // Top-K
-    int Kc;                // candidates kept per (row, slot): max(K, K_REG)
+    int cap;               // capacity of a (row, slot) candidate buffer: cand_cap(K)
     int spill_begin;       // MODE_STATS: row tiles >= spill_begin also write the tile 2^(z log2e - ref2) in bf16 to
                            // P (row tile index - spill_begin); INT_MAX: none
     // MODE_STATS outputs (per slot)
     float* part_m;
     float* part_s;
-    float* cand_v;
-    int* cand_i;
+    uint2* cand;           // [slot, row, cap] (logit bits, token id)
+    int* cand_n;           // [slot, row] entries in use
     // MODE_PROBS
     const float* lse2;     // [N] lse_d * log2(e)
     const float* coef;     // [N] g * S_q
@@ -96,56 +95,73 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Top-K list for K > K_REG: a binary min-heap in local memory, ordered so that the root is the entry
-// to evict next (smallest logit; among equal logits the highest token id). Returns the new admission
-// threshold: -inf while the list is not full, else the root's logit. Admission is strict (x > threshold)
-// and token ids arrive in increasing order, so equal logits resolve to the lower token id.
-__device__ __forceinline__ bool heap_before(float av, int ai, float bv, int bi) {
-    return av < bv || (av == bv && ai > bi);
+// ---- streaming Top-K candidates ---------------------------------------------------------------------
+// Each (row, slot) owns a buffer of `cap` (logit, token id) pairs in the workspace. The epilogue thread of
+// the row appends every logit above its admission threshold; when a buffer is nearly full the whole warp
+// compacts it to the row's K best and raises the threshold to the K-th largest logit. Entries stay in
+// increasing token-id order, admission is strict (x > threshold), and among logits equal to the K-th the
+// lowest token ids are kept, so equal logits resolve to the lower token id.
+constexpr int CAND_CAP_MAX = 256;                 // largest buffer: K = 128
+constexpr int CAND_REGS = CAND_CAP_MAX / 32;      // entries per lane during a compaction
+
+__host__ __device__ constexpr int cand_cap(int K) { return ((K + (K > 32 ? K : 32)) + 31) / 32 * 32; }
+
+// order-preserving map from fp32 bit patterns to unsigned integers (and back); 0 is below every float
+__device__ __forceinline__ uint32_t ordered_key(uint32_t bits) {
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
 }
-__device__ __noinline__ float topk_insert(float* lv, int* li, int* cnt_minpos, int K, float x, int idx) {
-    int cnt = cnt_minpos[0];
-    if (cnt < K) {
-        // sift up from the new leaf
-        int pos = cnt;
-        while (pos > 0) {
-            const int par = (pos - 1) >> 1;
-            const float pv = lv[par];
-            const int pi = li[par];
-            if (!heap_before(x, idx, pv, pi)) break;
-            lv[pos] = pv;
-            li[pos] = pi;
-            pos = par;
+__device__ __forceinline__ uint32_t key_bits(uint32_t key) {
+    return (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
+}
+
+// Warp-collective: compacts the buffer `buf` holding n >= K entries to its K best, in place, keeping their
+// order. Returns the bit pattern of the K-th largest logit (the new admission threshold).
+__device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K, int cap, int lane) {
+    uint32_t key[CAND_REGS];
+    int id[CAND_REGS];
+    const int groups = cap >> 5;
+#pragma unroll
+    for (int t = 0; t < CAND_REGS; ++t) {
+        key[t] = 0u;
+        id[t] = -1;
+        const int e = lane + 32 * t;
+        if (t < groups && e < n) {
+            const uint2 v = __ldcg(buf + e);
+            key[t] = ordered_key(v.x);
+            id[t] = static_cast<int>(v.y);
         }
-        lv[pos] = x;
-        li[pos] = idx;
-        cnt_minpos[0] = ++cnt;
-        return cnt < K ? -INFINITY : lv[0];
     }
-    // replace the root and sift down
-    int pos = 0;
-    while (true) {
-        int c = 2 * pos + 1;
-        if (c >= K) break;
-        float cv = lv[c];
-        int ci = li[c];
-        if (c + 1 < K) {
-            const float rv = lv[c + 1];
-            const int ri = li[c + 1];
-            if (heap_before(rv, ri, cv, ci)) {
-                cv = rv;
-                ci = ri;
-                ++c;
-            }
+    // largest T with at least K keys >= T, bit by bit
+    uint32_t T = 0u;
+#pragma unroll 1
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t cand = T | (1u << bit);
+        int c = 0;
+#pragma unroll
+        for (int t = 0; t < CAND_REGS; ++t) c += (key[t] >= cand) ? 1 : 0;
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (c >= K) T = cand;
+    }
+    int n_gt = 0;
+#pragma unroll
+    for (int t = 0; t < CAND_REGS; ++t) n_gt += (key[t] > T) ? 1 : 0;
+    n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+    const int need_eq = K - n_gt;             // >= 1: how many entries equal to the K-th are kept
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int run_eq = 0, out = 0;
+#pragma unroll
+    for (int t = 0; t < CAND_REGS; ++t) {
+        if (t < groups) {
+            const bool eq = key[t] == T;
+            const uint32_t em = __ballot_sync(0xffffffffu, eq);
+            const bool keep = key[t] > T || (eq && run_eq + __popc(em & lt_mask) < need_eq);
+            run_eq += __popc(em);
+            const uint32_t km = __ballot_sync(0xffffffffu, keep);
+            if (keep) buf[out + __popc(km & lt_mask)] = make_uint2(key_bits(key[t]), static_cast<uint32_t>(id[t]));
+            out += __popc(km);
         }
-        if (!heap_before(cv, ci, x, idx)) break;
-        lv[pos] = cv;
-        li[pos] = ci;
-        pos = c;
     }
-    lv[pos] = x;
-    li[pos] = idx;
-    return lv[0];
+    return key_bits(T);
 }
 
 template <int MODE>
@@ -293,18 +309,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         const int r_local = quad * 32 + lane;      // row inside the tile
         int ab = 0;
         uint32_t aphase = 0;
-        // Top-K list of this thread's row (MODE_STATS); lives in local memory, touched only on admission
-        float lv[MODE == MODE_STATS ? K_CAP : 1];
-        int li[MODE == MODE_STATS ? K_CAP : 1];
-        int cnt_minpos[2];
-        // K <= K_REG: the K_REG largest logits seen so far, sorted descending, in registers
-        float tv[MODE == MODE_STATS ? K_REG : 1];
-        int ti[MODE == MODE_STATS ? K_REG : 1];
-        // logits of the current 32-column chunk that beat the admission threshold (local memory)
-        float pend_v[MODE == MODE_STATS ? 32 : 1];
-        int pend_i[MODE == MODE_STATS ? 32 : 1];
-        const bool reg_list = p.K <= K_REG;
-        const int lo = reg_list ? K_REG - p.K : 0;   // the register list occupies slots lo .. K_REG-1
+        // Top-K candidates of this thread's row (MODE_STATS): buffer in the workspace, entries in use
+        uint2* cbuf = nullptr;
+        int cnt = 0;
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
@@ -320,13 +327,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             int cur = 0, nxt = INT_MAX;
             if (MODE == MODE_STATS) {
                 want_topk = rt < p.topk_row_tiles;
-                cnt_minpos[0] = 0;
-                cnt_minpos[1] = 0;
-#pragma unroll
-                for (int i = 0; i < K_REG; ++i) {
-                    tv[i] = -INFINITY;
-                    ti[i] = -1;
-                }
+                cbuf = p.cand + (static_cast<long long>(slot) * BM + r_local) * p.cap;
+                cnt = 0;
             }
             if (MODE == MODE_PROBS && row_ok) {
                 lse2 = p.lse2[g_row];
@@ -373,6 +375,23 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     tmem_ld_wait(r);
                     const int col0 = col_base + ch * 32;
                     if (MODE == MODE_STATS) {
+                        if (want_topk) {
+                            // make room for a whole chunk in every row's buffer (warp-uniform control flow)
+                            uint32_t full = __ballot_sync(0xffffffffu, cnt > p.cap - 32);
+                            while (full) {
+                                const int L = __ffs(full) - 1;
+                                full &= full - 1u;
+                                __syncwarp();
+                                const unsigned long long bp = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(cbuf), L);
+                                const int n = __shfl_sync(0xffffffffu, cnt, L);
+                                const uint32_t tb = compact_candidates(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane);
+                                __syncwarp();
+                                if (lane == L) {
+                                    cnt = p.K;
+                                    thr = __uint_as_float(tb);
+                                }
+                            }
+                        }
                         if (col0 + 32 > p.n_cols) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -396,42 +415,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             }
                             s += acc0 + acc1;
                             if (want_topk && cm > thr) {
-                                // collect the chunk's candidates, then admit them one by one (the
-                                // threshold only rises, so each is re-checked against the current one)
-                                int np = 0;
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) {
-                                    const float x = __uint_as_float(r[j]);
-                                    if (x > thr) {
-                                        pend_v[np] = x;
-                                        pend_i[np] = col0 + j;
-                                        ++np;
-                                    }
-                                }
-                                for (int q = 0; q < np; ++q) {
-                                    const float x = pend_v[q];
-                                    const int id = pend_i[q];
-                                    if (!(x > thr)) continue;
-                                    if (reg_list) {
-                                        // sorted insertion into tv[lo .. K_REG-1] (descending), so the K-th largest
-                                        // is always tv[K_REG-1]; equal logits stay behind earlier (lower) token ids
-#pragma unroll
-                                        for (int i = K_REG - 1; i >= 0; --i) {
-                                            if (i > 0 && i > lo) {
-                                                const bool shift = x > tv[i > 0 ? i - 1 : 0];
-                                                const bool here = !shift && x > tv[i];
-                                                tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
-                                                ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
-                                            } else if (i == lo) {
-                                                if (x > tv[i]) {
-                                                    tv[i] = x;
-                                                    ti[i] = id;
-                                                }
-                                            }
-                                        }
-                                        thr = tv[K_REG - 1];
-                                    } else {
-                                        thr = topk_insert(lv, li, cnt_minpos, p.K, x, id);
+                                    if (__uint_as_float(r[j]) > thr) {
+                                        cbuf[cnt] = make_uint2(r[j], static_cast<uint32_t>(col0 + j));
+                                        ++cnt;
                                     }
                                 }
                             }
@@ -583,23 +571,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 // a spilled value reached the top of the fp32 range: the row's logits spread too far
                 // above its reference for the fixed-exponent spill
                 if (spill && !(s < 1e38f)) atomicCAS(p.status, 0u, (5u << 8) | 2u);
-                if (want_topk) {
-                    if (reg_list) {
-#pragma unroll
-                        for (int k = 0; k < K_REG; ++k) {
-                            const long long co = (static_cast<long long>(slot) * K_REG + k) * BM + r_local;
-                            p.cand_v[co] = tv[k];
-                            p.cand_i[co] = ti[k];
-                        }
-                    } else {
-                        const int cnt = cnt_minpos[0];
-                        for (int k = 0; k < p.K; ++k) {
-                            const long long co = (static_cast<long long>(slot) * p.K + k) * BM + r_local;
-                            p.cand_v[co] = k < cnt ? lv[k] : -INFINITY;
-                            p.cand_i[co] = k < cnt ? li[k] : -1;
-                        }
-                    }
-                }
+                if (want_topk) p.cand_n[static_cast<long long>(slot) * BM + r_local] = cnt;
             }
             return true;
         });
@@ -626,13 +598,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 struct FinalizeParams {
     Schedule sched;
     int d, K;
-    int Kc;                // candidates per (row, slot) written by the sweep
+    int cap;               // capacity of a (row, slot) candidate buffer
     int row_begin, rows;   // global rows [row_begin, row_begin + rows) = local row tiles 0.. of the schedule
     int row_tiles_t;       // row tiles of the target matrix in the schedule (0: Omega_hat is an input)
     const float* part_m;
     const float* part_s;
-    const float* cand_v;
-    const int* cand_i;
+    const uint2* cand;
+    const int* cand_n;
     const __nv_bfloat16* H_d;
     const __nv_bfloat16* W;
     const int* idx_in;     // [N,K] when row_tiles_t == 0
@@ -705,8 +677,8 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     float loss = 0.f;
     float prev_v = INFINITY;
     int prev_i = -1;
-    const int Kc = p.Kc;
-    const int C = S * Kc;  // candidates of this row (target path)
+    const int cap = p.cap;
+    const int C = S * cap; // candidate entries of this row (target path); a slot uses the first cand_n of its cap
     __shared__ int sh_tok[8][K_CAP];
     __shared__ float sh_gq[8][K_CAP];
     const int wib = threadIdx.x >> 5;
@@ -718,10 +690,11 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             float bv = -INFINITY;
             int bi = INT_MAX;
             for (int c = lane; c < C; c += 32) {
-                const long long co = (static_cast<long long>(slot0 + c / Kc) * Kc + (c % Kc)) * BM + r;
-                const float v = p.cand_v[co];
-                const int i = p.cand_i[co];
-                if (i < 0) continue;
+                const long long so = static_cast<long long>(slot0 + c / cap) * BM + r;
+                if (c % cap >= p.cand_n[so]) continue;
+                const uint2 ce = p.cand[so * cap + (c % cap)];
+                const float v = __uint_as_float(ce.x);
+                const int i = static_cast<int>(ce.y);
                 const bool after_prev = (v < prev_v) || (v == prev_v && i > prev_i);
                 const bool better = (v > bv) || (v == bv && i < bi);
                 if (after_prev && better) {
