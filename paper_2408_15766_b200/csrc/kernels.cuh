@@ -104,7 +104,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 constexpr int CAND_CAP_MAX = 256;                 // largest buffer: K = 128
 constexpr int CAND_REGS = CAND_CAP_MAX / 32;      // entries per lane during a compaction
 
-__host__ __device__ constexpr int cand_cap(int K) { return ((K + (K > 32 ? K : 32)) + 31) / 32 * 32; }
+// K + at least 96 spare entries (a compaction is triggered 32 entries before the end), multiple of 32
+__host__ __device__ constexpr int cand_cap(int K) { return ((K + (K > 96 ? K : 96)) + 31) / 32 * 32; }
 
 // order-preserving map from fp32 bit patterns to unsigned integers (and back); 0 is below every float
 __device__ __forceinline__ uint32_t ordered_key(uint32_t bits) {
