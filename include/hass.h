@@ -199,7 +199,7 @@ int64_t hass_kernel_launch_count(void);
  *
  *   - The array is HASS_STATIC_SCRATCH_MAX_BYTES (32 MiB) and every GPU that loads the library
  *     holds it until the process exits. A problem whose forward scratch does not fit (it grows
- *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits up to K = 32) is refused
+ *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits for K <= 16; larger K use much larger candidate buffers) is refused
  *     with HASS_ERR_UNSUPPORTED; use hass_topk_distill_fwd with a workspace then.
  *   - The call allocates and frees nothing, in this library or through any other.
  *   - The first call on each device looks up the array's device address (a CUDA runtime query,

@@ -71,7 +71,8 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e0 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<MODE_PROBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-            if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess) {
+            cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
                 cudaGetLastError();
                 return HASS_ERR_CUDA;
             }
@@ -172,6 +173,9 @@ static int make_tmap(CUtensorMap* tm, const void* base, long long rows, long lon
     return r == CUDA_SUCCESS ? HASS_OK : HASS_ERR_CUDA;
 }
 
+// capacity of a (row, slot) candidate buffer for this K
+static int topk_cap(int K) { return K <= K_REG ? K_REG : cand_cap(K); }
+
 // ---- workspace layout -------------------------------------------------------------------------
 static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
@@ -220,7 +224,7 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     L->part_s = off;
     off = align256(off + slots * BM * 4);
     L->cand_v = off;                        // candidate buffers: (logit, token id) pairs, cand_cap(K) per (row, slot)
-    off = align256(off + slots * BM * 8 * cand_cap(K));
+    off = align256(off + slots * BM * 8 * topk_cap(K));
     L->cand_i = off;                        // entries in use per (row, slot)
     off = align256(off + slots * BM * 4);
     L->fwd_end = off;                       // what the forward-only entry points use
@@ -270,7 +274,10 @@ static void log_schedule(const char* what, const Schedule& s) {
 template <int MODE>
 static int launch_gemm(const GemmParams& p, cudaStream_t st) {
     KernelTimer timer(MODE, st);
-    gemm_kernel<MODE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    if (MODE == MODE_STATS && p.K <= K_REG)
+        gemm_kernel<MODE_STATS, TOPK_REG><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    else
+        gemm_kernel<MODE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
     g_launches.fetch_add(1);
     return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
 }
@@ -334,7 +341,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     p.col_tiles = CT;
     p.k_blocks = ceil_div(d, BK);
     p.K = K;
-    p.cap = cand_cap(K);
+    p.cap = topk_cap(K);
     p.part_m = reinterpret_cast<float*>(ws + L.part_m);
     p.part_s = reinterpret_cast<float*>(ws + L.part_s);
     p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
@@ -350,7 +357,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.rows = static_cast<int>(N);
     f.d = static_cast<int>(d);
     f.K = K;
-    f.cap = cand_cap(K);
+    f.cap = topk_cap(K);
     f.row_tiles_t = with_target ? RT : 0;
     f.part_m = p.part_m;
     f.part_s = p.part_s;
@@ -555,7 +562,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.col_tiles = CT;
         p.k_blocks = ceil_div(d, BK);
         p.K = K;
-        p.cap = cand_cap(K);
+        p.cap = topk_cap(K);
         p.part_m = reinterpret_cast<float*>(ws + L.part_m);
         p.part_s = reinterpret_cast<float*>(ws + L.part_s);
         p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
@@ -571,7 +578,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.sched = p.sched;
         f.d = static_cast<int>(d);
         f.K = K;
-        f.cap = cand_cap(K);
+        f.cap = topk_cap(K);
         f.row_begin = t0 * BM;
         f.rows = rows;
         f.row_tiles_t = with_target ? tiles : 0;

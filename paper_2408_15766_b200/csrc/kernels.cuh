@@ -165,7 +165,13 @@ __device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K,
     return key_bits(T);
 }
 
-template <int MODE>
+// TOPK selects how MODE_STATS keeps a row's Top-K candidates: TOPK_REG (K <= K_REG) a sorted list in
+// registers, all lanes inserting in parallel - best while most rows still admit logits; TOPK_BUF (any K)
+// append buffers with warp-cooperative compaction - cost nearly independent of K.
+enum { TOPK_REG = 0, TOPK_BUF = 1 };
+constexpr int K_REG = 16;
+
+template <int MODE, int TOPK = TOPK_BUF>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
     constexpr bool B_MN_MAJOR = (MODE == MODE_OUT);
     extern __shared__ uint8_t smem_raw[];
@@ -313,6 +319,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         // Top-K candidates of this thread's row (MODE_STATS): buffer in the workspace, entries in use
         uint2* cbuf = nullptr;
         int cnt = 0;
+        // TOPK_REG: the K largest logits so far sorted descending in tv[lo .. K_REG-1] (so the K-th largest is
+        // always tv[K_REG-1]), and the current chunk's admitted logits waiting in a small local-memory buffer
+        constexpr bool USE_REG = MODE == MODE_STATS && TOPK == TOPK_REG;
+        float tv[USE_REG ? K_REG : 1];
+        int ti[USE_REG ? K_REG : 1];
+        float pend_v[USE_REG ? 32 : 1];
+        int pend_i[USE_REG ? 32 : 1];
+        const int lo = K_REG - p.K;
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
@@ -330,6 +344,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 want_topk = rt < p.topk_row_tiles;
                 cbuf = p.cand + (static_cast<long long>(slot) * BM + r_local) * p.cap;
                 cnt = 0;
+                if (USE_REG) {
+#pragma unroll
+                    for (int i = 0; i < (USE_REG ? K_REG : 1); ++i) {
+                        tv[i] = -INFINITY;
+                        ti[i] = -1;
+                    }
+                }
             }
             if (MODE == MODE_PROBS && row_ok) {
                 lse2 = p.lse2[g_row];
@@ -376,7 +397,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     tmem_ld_wait(r);
                     const int col0 = col_base + ch * 32;
                     if (MODE == MODE_STATS) {
-                        if (want_topk) {
+                        if (!USE_REG && want_topk) {
                             // make room for a whole chunk in every row's buffer (warp-uniform control flow)
                             uint32_t full = __ballot_sync(0xffffffffu, cnt > p.cap - 32);
                             while (full) {
@@ -415,13 +436,48 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 fadd2(acc0, acc1, acc0, acc1, ex2(t0), ex2(t1));
                             }
                             s += acc0 + acc1;
-                            if (want_topk && cm > thr) {
+                            if (!USE_REG && want_topk && cm > thr) {
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) {
                                     if (__uint_as_float(r[j]) > thr) {
                                         cbuf[cnt] = make_uint2(r[j], static_cast<uint32_t>(col0 + j));
                                         ++cnt;
                                     }
+                                }
+                            }
+                            if (USE_REG && want_topk && cm > thr) {
+                                // collect the chunk's candidates, then admit them one by one (the
+                                // threshold only rises, so each is re-checked against the current one)
+                                int np = 0;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) {
+                                    const float x = __uint_as_float(r[j]);
+                                    if (x > thr) {
+                                        pend_v[USE_REG ? np : 0] = x;
+                                        pend_i[USE_REG ? np : 0] = col0 + j;
+                                        ++np;
+                                    }
+                                }
+                                for (int q = 0; q < np; ++q) {
+                                    const float x = pend_v[USE_REG ? q : 0];
+                                    const int id = pend_i[USE_REG ? q : 0];
+                                    if (!(x > thr)) continue;
+                                    // sorted insertion; equal logits stay behind earlier (lower) token ids
+#pragma unroll
+                                    for (int i = (USE_REG ? K_REG : 1) - 1; i >= 0; --i) {
+                                        if (i > 0 && i > lo) {
+                                            const bool shift = x > tv[i > 0 ? i - 1 : 0];
+                                            const bool here = !shift && x > tv[i];
+                                            tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
+                                            ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
+                                        } else if (i == lo) {
+                                            if (x > tv[i]) {
+                                                tv[i] = x;
+                                                ti[i] = id;
+                                            }
+                                        }
+                                    }
+                                    thr = tv[(USE_REG ? K_REG : 1) - 1];
                                 }
                             }
                         } else {
@@ -572,6 +628,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 // a spilled value reached the top of the fp32 range: the row's logits spread too far
                 // above its reference for the fixed-exponent spill
                 if (spill && !(s < 1e38f)) atomicCAS(p.status, 0u, (5u << 8) | 2u);
+                if (USE_REG && want_topk) {
+                    // the register list goes out as a full buffer of K_REG entries (unused ones carry id -1)
+#pragma unroll
+                    for (int k = 0; k < (USE_REG ? K_REG : 1); ++k)
+                        cbuf[k] = make_uint2(__float_as_uint(tv[k]), static_cast<uint32_t>(ti[k]));
+                    cnt = K_REG;
+                }
                 if (want_topk) p.cand_n[static_cast<long long>(slot) * BM + r_local] = cnt;
             }
             return true;
@@ -679,7 +742,6 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     float prev_v = INFINITY;
     int prev_i = -1;
     const int cap = p.cap;
-    const int C = S * cap; // candidate entries of this row (target path); a slot uses the first cand_n of its cap
     __shared__ int sh_tok[8][K_CAP];
     __shared__ float sh_gq[8][K_CAP];
     const int wib = threadIdx.x >> 5;
@@ -690,17 +752,20 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             // next candidate after (prev_v, prev_i) in the order: logit descending, then token id ascending
             float bv = -INFINITY;
             int bi = INT_MAX;
-            for (int c = lane; c < C; c += 32) {
-                const long long so = static_cast<long long>(slot0 + c / cap) * BM + r;
-                if (c % cap >= p.cand_n[so]) continue;
-                const uint2 ce = p.cand[so * cap + (c % cap)];
-                const float v = __uint_as_float(ce.x);
-                const int i = static_cast<int>(ce.y);
-                const bool after_prev = (v < prev_v) || (v == prev_v && i > prev_i);
-                const bool better = (v > bv) || (v == bv && i < bi);
-                if (after_prev && better) {
-                    bv = v;
-                    bi = i;
+            for (int sl = 0; sl < S; ++sl) {
+                const long long so = static_cast<long long>(slot0 + sl) * BM + r;
+                const int n = p.cand_n[so];
+                for (int e = lane; e < n; e += 32) {
+                    const uint2 ce = p.cand[so * cap + e];
+                    const float v = __uint_as_float(ce.x);
+                    const int i = static_cast<int>(ce.y);
+                    if (i < 0) continue;
+                    const bool after_prev = (v < prev_v) || (v == prev_v && i > prev_i);
+                    const bool better = (v > bv) || (v == bv && i < bi);
+                    if (after_prev && better) {
+                        bv = v;
+                        bi = i;
+                    }
                 }
             }
 #pragma unroll
