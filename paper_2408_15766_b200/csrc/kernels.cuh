@@ -319,14 +319,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         // Top-K candidates of this thread's row (MODE_STATS): buffer in the workspace, entries in use
         uint2* cbuf = nullptr;
         int cnt = 0;
-        // TOPK_REG: the K largest logits so far sorted descending in tv[lo .. K_REG-1] (so the K-th largest is
-        // always tv[K_REG-1]), and the current chunk's admitted logits waiting in a small local-memory buffer
+        // TOPK_REG: the K_REG largest logits so far sorted descending in tv[] (the admission threshold is the
+        // K_REG-th largest: a list of exactly K entries with its K-th as threshold measured slower), and the
+        // current chunk's admitted logits waiting in a small local-memory buffer
         constexpr bool USE_REG = MODE == MODE_STATS && TOPK == TOPK_REG;
         float tv[USE_REG ? K_REG : 1];
         int ti[USE_REG ? K_REG : 1];
         float pend_v[USE_REG ? 32 : 1];
         int pend_i[USE_REG ? 32 : 1];
-        const int lo = K_REG - p.K;
+        constexpr int lo = 0;
 
         for_each_item([&](int rt, int ln, int S, int slot) {
             const int g_row = p.row_global_offset + rt * BM + r_local;
