@@ -714,6 +714,8 @@ __device__ __forceinline__ float warp_lse(const float* pm, const float* ps, int 
     return m + logf(s);
 }
 
+constexpr int FIN_GRP = 16;   // tokens of Omega_hat whose W rows finalize reads together
+
 __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ FinalizeParams p) {
     const int lane = threadIdx.x & 31;
     const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -744,7 +746,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     int prev_i = -1;
     const int cap = p.cap;
     __shared__ int sh_tok[8][K_CAP];
-    __shared__ float sh_gq[8][K_CAP];
+    __shared__ float sh_q[8][K_CAP];
     const int wib = threadIdx.x >> 5;
     for (int j = 0; j < K; ++j) {
         int tok;
@@ -790,51 +792,67 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             tok = p.idx_in[static_cast<long long>(row) * K + j];
             qv = p.q_in[static_cast<long long>(row) * K + j];
         }
-        // draft logit of this token: <H_d[row], W[tok]>
-        const __nv_bfloat16* wrow = p.W + static_cast<long long>(tok) * p.d;
-        float acc = 0.f;
-        for (int k = lane * 8; k < p.d; k += 256) {
-            const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k);
-            const uint4 wv = *reinterpret_cast<const uint4*>(wrow + k);
-            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
-            const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const float2 a = __bfloat1622float2(hp[t]);
-                const float2 b = __bfloat1622float2(wp[t]);
-                acc = fmaf(a.x, b.x, acc);
-                acc = fmaf(a.y, b.y, acc);
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
         S_q += qv;
         if (lane == 0) {
             if (p.gq_out) p.gq_out[static_cast<long long>(row) * K + j] = g * qv;
             sh_tok[wib][j] = tok;
-            sh_gq[wib][j] = g * qv;
+            sh_q[wib][j] = qv;
         }
     }
-    if (p.sparse_out) {
-        // the Omega_hat term of dz_d W for this row, 256 columns (8 per lane) at a time
-        __syncwarp();
-        float* so = p.sparse_out + static_cast<long long>(local) * p.d;
-        for (int k0 = lane * 8; k0 < p.d; k0 += 256) {
-            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int j = 0; j < K; ++j) {
-                const float gq = sh_gq[wib][j];
-                const uint4 wv = *reinterpret_cast<const uint4*>(p.W + static_cast<long long>(sh_tok[wib][j]) * p.d + k0);
-                const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+    __syncwarp();
+    // Draft logits at Omega_hat (K dot products with rows of W) and, for the fused backward, the row
+    // sum_{x in Omega_hat} g q(x) W[x, :]. The W rows are read once: FIN_GRP tokens at a time, 256 columns
+    // (8 per lane) per step; the fp32 row is accumulated across token groups.
+    float* so = p.sparse_out ? p.sparse_out + static_cast<long long>(local) * p.d : nullptr;
+    for (int g0 = 0; g0 < K; g0 += FIN_GRP) {
+        const int ng = K - g0 < FIN_GRP ? K - g0 : FIN_GRP;
+        float dot[FIN_GRP];
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const float2 b = __bfloat1622float2(wp[t]);
-                    a[2 * t] = fmaf(gq, b.x, a[2 * t]);
-                    a[2 * t + 1] = fmaf(gq, b.y, a[2 * t + 1]);
+        for (int jj = 0; jj < FIN_GRP; ++jj) dot[jj] = 0.f;
+        for (int k0 = lane * 8; k0 < p.d; k0 += 256) {
+            const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0);
+            const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+            float h[8];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const float2 f2 = __bfloat1622float2(hp[t]);
+                h[2 * t] = f2.x;
+                h[2 * t + 1] = f2.y;
+            }
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (so && g0 > 0) {
+                const float4 a0 = *reinterpret_cast<const float4*>(so + k0);
+                const float4 a1 = *reinterpret_cast<const float4*>(so + k0 + 4);
+                a[0] = a0.x; a[1] = a0.y; a[2] = a0.z; a[3] = a0.w;
+                a[4] = a1.x; a[5] = a1.y; a[6] = a1.z; a[7] = a1.w;
+            }
+#pragma unroll
+            for (int jj = 0; jj < FIN_GRP; ++jj) {
+                if (jj < ng) {
+                    const float gq = g * sh_q[wib][g0 + jj];
+                    const uint4 wv = *reinterpret_cast<const uint4*>(p.W + static_cast<long long>(sh_tok[wib][g0 + jj]) * p.d + k0);
+                    const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float2 b = __bfloat1622float2(wp[t]);
+                        dot[jj] = fmaf(h[2 * t], b.x, dot[jj]);
+                        dot[jj] = fmaf(h[2 * t + 1], b.y, dot[jj]);
+                        a[2 * t] = fmaf(gq, b.x, a[2 * t]);
+                        a[2 * t + 1] = fmaf(gq, b.y, a[2 * t + 1]);
+                    }
                 }
             }
-            *reinterpret_cast<float4*>(so + k0) = make_float4(a[0], a[1], a[2], a[3]);
-            *reinterpret_cast<float4*>(so + k0 + 4) = make_float4(a[4], a[5], a[6], a[7]);
+            if (so) {
+                *reinterpret_cast<float4*>(so + k0) = make_float4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<float4*>(so + k0 + 4) = make_float4(a[4], a[5], a[6], a[7]);
+            }
+        }
+#pragma unroll
+        for (int jj = 0; jj < FIN_GRP; ++jj) {
+            float acc = dot[jj];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (jj < ng) loss += sh_q[wib][g0 + jj] * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
         }
     }
     if (lane == 0) {
