@@ -214,6 +214,7 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
             if (t.total_slots > slot_cap) slot_cap = t.total_slots;
         }
     }
+    if (slot_cap < sms) slot_cap = sms;     // any single-phase schedule (a caller-limited, smaller chunk) fits
     L->slot_cap = slot_cap;
     size_t off = 0;
     L->status = off;

@@ -42,6 +42,8 @@ def test_tiny_config_all_rows():
 @pytest.mark.parametrize("N,d,V,K", [
     (1, 64, 64, 1), (64, 256, 1000, 2), (127, 264, 1024, 10), (129, 64, 32003, 10),
     (300, 256, 5000, 64), (200, 128, 777, 100), (130, 512, 300, 128), (5, 8, 9, 9),
+    (4800, 64, 700, 5),       # two row chunks, the second one ragged
+    (260, 72, 20000, 17),     # smallest K on the buffered Top-K path, d not a multiple of 64
 ])
 def test_awkward_shapes(N, d, V, K):
     inp = hi.make_custom(N, d, V, K, seed=N + V, sigma_w=0.5 / np.sqrt(d) * 4)
@@ -111,6 +113,33 @@ def test_fused_path_reports_rows_beyond_its_exponent_range():
     hass.check(out["workspace"])
     assert torch.equal(out["topk_idx"], f["topk_idx"]) and torch.equal(out["lse_t"], f["lse_t"])
     print(compare(inp.H_t, H_d, W, K, dict(_to_cpu(f), dH_d=dH.cpu())))
+
+
+def test_smaller_workspace_means_smaller_row_chunks_same_results():
+    hass = _hass()
+    N, d, V, K = 1000, 128, 3000, 10
+    inp = hi.make_custom(N, d, V, K, seed=21, sigma_w=0.2)
+    dev = torch.device("cuda:0")
+    H_t, H_d, W = inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev)
+    full = hass.topk_distill_workspace_bytes(N, d, V, K)
+    tile_bytes = 128 * (-(-V // 256) * 256) * 2          # dz_d / spill scratch of one 128-row tile
+    row_tiles = -(-N // 128)
+    small = torch.empty(full - (row_tiles - 2) * tile_bytes, dtype=torch.uint8, device=dev)   # room for 2 row tiles
+    a = hass.topk_distill_fwd_bwd(H_t, H_d, W, K)
+    b = hass.topk_distill_fwd_bwd(H_t, H_d, W, K, workspace=small)
+    hass.check(a["workspace"])
+    hass.check(small)
+    for k in ("topk_idx", "topk_q", "lse_t"):
+        assert torch.equal(a[k], b[k]), k
+    print(compare(inp.H_t, inp.H_d[0], inp.W, K, _to_cpu(b)))
+    dH = hass.topk_distill_bwd(H_d, W, b["topk_idx"], b["topk_q"], b["lse_d"], workspace=small)
+    hass.check(small)
+    print(compare(inp.H_t, inp.H_d[0], inp.W, K, dict(_to_cpu(b), dH_d=dH.cpu())))
+    # a workspace without room for even one row tile of scratch is refused
+    tiny = torch.empty(full - row_tiles * tile_bytes, dtype=torch.uint8, device=dev)
+    with pytest.raises(hass.HassError) as e:
+        hass.topk_distill_fwd_bwd(H_t, H_d, W, K, workspace=tiny)
+    assert e.value.status == -3
 
 
 def test_host_buffer_entry_matches_device_entry():
