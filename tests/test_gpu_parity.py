@@ -129,8 +129,10 @@ def test_smaller_workspace_means_smaller_row_chunks_same_results():
     b = hass.topk_distill_fwd_bwd(H_t, H_d, W, K, workspace=small)
     hass.check(a["workspace"])
     hass.check(small)
-    for k in ("topk_idx", "topk_q", "lse_t"):
-        assert torch.equal(a[k], b[k]), k
+    # a different chunking splits the vocabulary sweep differently: same sets, sums in another order
+    assert torch.equal(a["topk_idx"], b["topk_idx"])
+    assert torch.allclose(a["lse_t"], b["lse_t"], atol=1e-5, rtol=0)
+    assert torch.allclose(a["topk_q"], b["topk_q"], rtol=1e-5, atol=0)
     print(compare(inp.H_t, inp.H_d[0], inp.W, K, _to_cpu(b)))
     dH = hass.topk_distill_bwd(H_d, W, b["topk_idx"], b["topk_q"], b["lse_d"], workspace=small)
     hass.check(small)
