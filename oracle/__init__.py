@@ -48,6 +48,13 @@ def _load():
         lib.hass_oracle_features.restype = ctypes.c_int
         lib.hass_oracle_features.argtypes = [c_vp, c_vp, c_vp, ctypes.c_int, c_i64, c_i64, c_i64, c_i32,
                                              c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
+        lib.hass_oracle_row_objective.restype = ctypes.c_int
+        lib.hass_oracle_row_objective.argtypes = [c_vp, c_vp, c_i64, c_i32, c_dbl, c_dbl, c_dbl, c_vp,
+                                                  c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
+        lib.hass_oracle_features_objective.restype = ctypes.c_int
+        lib.hass_oracle_features_objective.argtypes = [c_vp, c_vp, c_vp, ctypes.c_int, c_i64, c_i64, c_i64, c_i32,
+                                                       c_dbl, c_dbl, c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp,
+                                                       c_vp, c_vp, c_vp, c_vp]
         lib.hass_oracle_logits_at.restype = ctypes.c_int
         lib.hass_oracle_logits_at.argtypes = [c_vp, c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_i64, c_vp]
         _lib = lib
@@ -83,6 +90,31 @@ def from_logits(z_t, z_d, K: int, g: float = 1.0, forced_idx=None, want_dz: bool
     return dict(loss=float(loss[0]), idx=idx, q_k=q_k, lse_t=float(lse_t[0]), lse_d=float(lse_d[0]), dz_d=dz)
 
 
+def objective_from_logits(z_t, z_d, K: int, w_ce: float, w_topk: float, g: float = 1.0) -> dict:
+    """One row of logits: cross-entropy over the whole vocabulary, Top-K loss, and the derivative of
+    w_ce * L_CE + w_topk * L_TopK with respect to the draft logits."""
+    z_t = np.ascontiguousarray(z_t, dtype=np.float64)
+    z_d = np.ascontiguousarray(z_d, dtype=np.float64)
+    V = z_t.shape[0]
+    loss, ce, lse_t, lse_d = np.zeros(1), np.zeros(1), np.zeros(1), np.zeros(1)
+    idx = np.zeros(K, dtype=np.int32)
+    q_k = np.zeros(K)
+    dz = np.zeros(V)
+    rc = _load().hass_oracle_row_objective(_ptr(z_t), _ptr(z_d), V, K, float(g), float(w_ce), float(w_topk), None,
+                                           _ptr(ce), _ptr(loss), _ptr(idx), _ptr(q_k), _ptr(lse_t), _ptr(lse_d),
+                                           _ptr(dz))
+    if rc != 0:
+        raise ValueError("oracle: bad arguments")
+    return dict(loss_ce=float(ce[0]), loss=float(loss[0]), idx=idx, q_k=q_k, lse_t=float(lse_t[0]),
+                lse_d=float(lse_d[0]), dz_d=dz)
+
+
+def objective_from_features(H_t, H_d, W, K: int, w_ce: float, w_topk: float, rows=None, grad_loss=None,
+                            forced_idx=None, want_dH: bool = True) -> dict:
+    """from_features for the objective w_ce * L_CE + w_topk * L_TopK; also returns loss_ce."""
+    return _features(H_t, H_d, W, K, rows, grad_loss, forced_idx, want_dH, float(w_ce), float(w_topk), True)
+
+
 def from_features(H_t, H_d, W, K: int, rows=None, grad_loss=None, forced_idx=None,
                   want_dH: bool = True) -> dict:
     """Steps 1-5 on feature rows.
@@ -91,6 +123,10 @@ def from_features(H_t, H_d, W, K: int, rows=None, grad_loss=None, forced_idx=Non
     the GPU receives) or float64 arrays (used by the finite-difference pin).
     ``rows`` selects a subset; outputs are indexed by position in ``rows``.
     """
+    return _features(H_t, H_d, W, K, rows, grad_loss, forced_idx, want_dH, 0.0, 1.0, False)
+
+
+def _features(H_t, H_d, W, K, rows, grad_loss, forced_idx, want_dH, w_ce, w_topk, want_ce) -> dict:
     H_t = np.ascontiguousarray(H_t)
     H_d = np.ascontiguousarray(H_d)
     W = np.ascontiguousarray(W)
@@ -115,12 +151,16 @@ def from_features(H_t, H_d, W, K: int, rows=None, grad_loss=None, forced_idx=Non
     idx = np.zeros((n, K), dtype=np.int32)
     q_k = np.zeros((n, K))
     dH = np.zeros((n, d)) if want_dH else None
-    rc = _load().hass_oracle_features(_ptr(H_t), _ptr(H_d), _ptr(W), H_t.dtype.itemsize, N, d, V, K,
-                                      _ptr(gl), _ptr(rows_a), n, _ptr(f), _ptr(loss), _ptr(idx),
-                                      _ptr(q_k), _ptr(lse_t), _ptr(lse_d), _ptr(dH))
+    ce = np.zeros(n) if want_ce else None
+    rc = _load().hass_oracle_features_objective(_ptr(H_t), _ptr(H_d), _ptr(W), H_t.dtype.itemsize, N, d, V, K,
+                                                w_ce, w_topk, _ptr(gl), _ptr(rows_a), n, _ptr(f), _ptr(ce),
+                                                _ptr(loss), _ptr(idx), _ptr(q_k), _ptr(lse_t), _ptr(lse_d), _ptr(dH))
     if rc != 0:
         raise ValueError("oracle: bad arguments")
-    return dict(loss=loss, idx=idx, q_k=q_k, lse_t=lse_t, lse_d=lse_d, dH_d=dH)
+    out = dict(loss=loss, idx=idx, q_k=q_k, lse_t=lse_t, lse_d=lse_d, dH_d=dH)
+    if want_ce:
+        out["loss_ce"] = ce
+    return out
 
 
 def logits_at(H, W, row, tok) -> np.ndarray:

@@ -25,6 +25,14 @@
  *           (derivative of Eq. 1 with q and Omega_hat constant: the target side needs no
  *            gradient, Appendix "Training Overhead"; g is the upstream weight of row i)
  *
+ * Combined objective (Section 3.2: the training objective of one aligning step is the cross-entropy
+ * between the target's and the draft's next-token distributions plus auxiliary terms, one of which is the
+ * Top-K loss with weight w, Section 4.1): the *_objective entries also return
+ *   L_CE = - sum_{x in Omega} q(x) log p(x)
+ * and differentiate  w_ce L_CE + w_topk L_TopK:
+ *   dL/dz_d[v] = g ( w_ce (p[v] - q[v]) + w_topk (S_q p[v] - q[v] [v in Omega_hat]) ).
+ * The plain entries are the case w_ce = 0, w_topk = 1.
+ *
  * Inputs of the feature-level entry are bf16 bit patterns widened exactly to fp64.
  * The only liberty taken with summation order is SIMD reassociation of the inner
  * dot-product loop (omp simd reduction), i.e. rounding order.
@@ -121,9 +129,9 @@ static double log_sum_exp(const double* z, int64_t V) {
  *   dz_d        [V] out or NULL.
  * Returns 0, or -1 on bad arguments.
  */
-int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V, int32_t K, double g,
-                                const int32_t* forced_idx, double* loss, int32_t* idx, double* q_k,
-                                double* lse_t_out, double* lse_d_out, double* dz_d) {
+int hass_oracle_row_objective(const double* z_t, const double* z_d, int64_t V, int32_t K, double g, double w_ce,
+                              double w_topk, const int32_t* forced_idx, double* loss_ce, double* loss, int32_t* idx,
+                              double* q_k, double* lse_t_out, double* lse_d_out, double* dz_d) {
     if (V < 1 || K < 1 || K > V) return -1;
     const double lse_t = log_sum_exp(z_t, V);
     const double lse_d = log_sum_exp(z_d, V);
@@ -162,13 +170,30 @@ int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V,
     *loss = L;
     if (lse_t_out) *lse_t_out = lse_t;
     if (lse_d_out) *lse_d_out = lse_d;
+    if (loss_ce) {
+        /* full-vocabulary cross-entropy between q and p */
+        double ce = 0.0;
+        for (int64_t v = 0; v < V; ++v) ce -= exp(z_t[v] - lse_t) * (z_d[v] - lse_d);
+        *loss_ce = ce;
+    }
 
     if (dz_d) {
-        for (int64_t v = 0; v < V; ++v) dz_d[v] = g * S_q * exp(z_d[v] - lse_d);
-        for (int32_t j = 0; j < K; ++j) dz_d[idx[j]] -= g * q_k[j];
+        for (int64_t v = 0; v < V; ++v) {
+            const double p = exp(z_d[v] - lse_d);
+            const double q = exp(z_t[v] - lse_t);
+            dz_d[v] = g * (w_ce * (p - q) + w_topk * S_q * p);
+        }
+        for (int32_t j = 0; j < K; ++j) dz_d[idx[j]] -= g * w_topk * q_k[j];
     }
     free(order);
     return 0;
+}
+
+int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V, int32_t K, double g,
+                                const int32_t* forced_idx, double* loss, int32_t* idx, double* q_k,
+                                double* lse_t_out, double* lse_d_out, double* dz_d) {
+    return hass_oracle_row_objective(z_t, z_d, V, K, g, 0.0, 1.0, forced_idx, NULL, loss, idx, q_k, lse_t_out,
+                                     lse_d_out, dz_d);
 }
 
 /* ---- feature-level entries -------------------------------------------------------- */
@@ -182,10 +207,11 @@ int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V,
  * Outputs are indexed by position in `rows`: loss, lse_t, lse_d [n_rows]; idx, q_k [n_rows, K];
  * dH_d [n_rows, d] (may be NULL to skip step 5's back-projection).
  */
-int hass_oracle_features(const void* H_t, const void* H_d, const void* W, int elem_bytes, int64_t N,
-                         int64_t d, int64_t V, int32_t K, const double* grad_loss, const int64_t* rows,
-                         int64_t n_rows, const int32_t* forced_idx, double* loss, int32_t* idx,
-                         double* q_k, double* lse_t, double* lse_d, double* dH_d) {
+int hass_oracle_features_objective(const void* H_t, const void* H_d, const void* W, int elem_bytes, int64_t N,
+                                   int64_t d, int64_t V, int32_t K, double w_ce, double w_topk,
+                                   const double* grad_loss, const int64_t* rows, int64_t n_rows,
+                                   const int32_t* forced_idx, double* loss_ce, double* loss, int32_t* idx,
+                                   double* q_k, double* lse_t, double* lse_d, double* dH_d) {
     if (N < 1 || d < 1 || V < 1 || K < 1 || K > V || n_rows < 0) return -1;
     if (elem_bytes != 2 && elem_bytes != 8) return -1;
     if (!rows && n_rows != N) return -1;
@@ -225,9 +251,9 @@ int hass_oracle_features(const void* H_t, const void* H_d, const void* W, int el
                 dot2(ht, hd, w, d, &zt[v], &zd[v]);
             }
             /* steps 2-5 on the logits */
-            int rc = hass_oracle_row_from_logits(zt, zd, V, K, g, forced_idx ? forced_idx + r * K : NULL,
-                                                 &loss[r], idx + r * K, q_k + r * K, &lse_t[r], &lse_d[r],
-                                                 dH_d ? dz : NULL);
+            int rc = hass_oracle_row_objective(zt, zd, V, K, g, w_ce, w_topk, forced_idx ? forced_idx + r * K : NULL,
+                                               loss_ce ? &loss_ce[r] : NULL, &loss[r], idx + r * K, q_k + r * K,
+                                               &lse_t[r], &lse_d[r], dH_d ? dz : NULL);
             if (rc != 0) {
 #pragma omp atomic write
                 status = -1;
@@ -257,6 +283,14 @@ int hass_oracle_features(const void* H_t, const void* H_d, const void* W, int el
         free(dz);
     }
     return status;
+}
+
+int hass_oracle_features(const void* H_t, const void* H_d, const void* W, int elem_bytes, int64_t N,
+                         int64_t d, int64_t V, int32_t K, const double* grad_loss, const int64_t* rows,
+                         int64_t n_rows, const int32_t* forced_idx, double* loss, int32_t* idx,
+                         double* q_k, double* lse_t, double* lse_d, double* dH_d) {
+    return hass_oracle_features_objective(H_t, H_d, W, elem_bytes, N, d, V, K, 0.0, 1.0, grad_loss, rows, n_rows,
+                                          forced_idx, NULL, loss, idx, q_k, lse_t, lse_d, dH_d);
 }
 
 /* Step 1 for selected (row, token) pairs: z[j] = sum_k H[row_j, k] W[tok_j, k], bf16 inputs.

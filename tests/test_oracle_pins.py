@@ -276,3 +276,66 @@ def test_expected_magnitudes_on_tiny_config():
     r = oracle.from_features(hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W), wl.K,
                              want_dH=False)
     assert abs(r["lse_t"].mean() - (np.log(wl.V) + 0.32 ** 2 / 2)) < 0.05
+
+
+# ---- combined objective: cross-entropy over the vocabulary + w * Top-K (Section 3.2) ---------------
+
+def test_objective_ce_only_is_soft_target_cross_entropy_with_autograd_gradient():
+    V, K = 90, 7
+    z_t, z_d = _rand_logits(V, seed=31)
+    r = oracle.objective_from_logits(z_t, z_d, K, w_ce=1.0, w_topk=0.0, g=1.7)
+    zd = torch.tensor(z_d, requires_grad=True)
+    q = torch.softmax(torch.tensor(z_t), 0)
+    ce = torch.nn.functional.cross_entropy(zd[None], q[None])        # soft (probability) targets
+    (1.7 * ce).backward()
+    assert r["loss_ce"] == pytest.approx(float(ce), rel=1e-12)
+    np.testing.assert_allclose(r["dz_d"], zd.grad.numpy(), atol=1e-14)
+    # the Top-K loss and set are unaffected by the weights
+    base = oracle.from_logits(z_t, z_d, K)
+    assert r["loss"] == pytest.approx(base["loss"], rel=1e-13) and np.array_equal(r["idx"], base["idx"])
+
+
+def test_objective_gradient_is_linear_in_the_two_weights_and_matches_finite_differences():
+    V, K = 60, 6
+    z_t, z_d = _rand_logits(V, seed=33)
+    a = oracle.objective_from_logits(z_t, z_d, K, 1.0, 0.0)
+    b = oracle.objective_from_logits(z_t, z_d, K, 0.0, 1.0)
+    c = oracle.objective_from_logits(z_t, z_d, K, 0.6, 2.5, g=0.5)
+    np.testing.assert_allclose(c["dz_d"], 0.5 * (0.6 * a["dz_d"] + 2.5 * b["dz_d"]), atol=1e-15)
+    np.testing.assert_allclose(b["dz_d"], oracle.from_logits(z_t, z_d, K)["dz_d"], atol=0)
+    h = 1e-6
+    for v in (0, 17, int(c["idx"][0]), 59):
+        e = np.zeros(V)
+        e[v] = h
+        up = oracle.objective_from_logits(z_t, z_d + e, K, 0.6, 2.5)
+        dn = oracle.objective_from_logits(z_t, z_d - e, K, 0.6, 2.5)
+        fd = 0.5 * ((0.6 * up["loss_ce"] + 2.5 * up["loss"]) - (0.6 * dn["loss_ce"] + 2.5 * dn["loss"])) / (2 * h)
+        assert c["dz_d"][v] == pytest.approx(fd, rel=1e-6, abs=1e-10)
+
+
+def test_objective_k_equals_v_makes_both_losses_equal():
+    V = 40
+    z_t, z_d = _rand_logits(V, seed=35)
+    r = oracle.objective_from_logits(z_t, z_d, V, 1.0, 1.0)
+    assert r["loss"] == pytest.approx(r["loss_ce"], rel=1e-12)
+    np.testing.assert_allclose(r["dz_d"], 2 * oracle.objective_from_logits(z_t, z_d, V, 1.0, 0.0)["dz_d"], atol=1e-15)
+
+
+def test_objective_features_level_autograd_restatement():
+    N, d, V, K, w = 5, 24, 80, 6, 0.5
+    Ht, Hd, W, inp = _feat(N, d, V, seed=37, sigma_w=0.3)
+    g = np.array([1.0, 0.0, 2.0, -1.0, 0.5])
+    r = oracle.objective_from_features(Ht, Hd, W, K, 1.0, w, grad_loss=g)
+    Htt, Wt = inp.H_t.double(), inp.W.double()
+    Hdt = inp.H_d[0].double().requires_grad_(True)
+    q = torch.softmax(Htt @ Wt.T, -1)
+    logp = torch.log_softmax(Hdt @ Wt.T, -1)
+    ce = -(q * logp).sum(-1)
+    qk, idx = torch.topk(q, K, dim=-1)
+    tk = -(qk * logp.gather(-1, idx)).sum(-1)
+    ((ce + w * tk) * torch.tensor(g)).sum().backward()
+    np.testing.assert_allclose(r["loss_ce"], ce.detach().numpy(), rtol=1e-12)
+    np.testing.assert_allclose(r["loss"], tk.detach().numpy(), rtol=1e-12)
+    np.testing.assert_allclose(r["dH_d"], Hdt.grad.numpy(), atol=1e-13)
+    plain = oracle.from_features(Ht, Hd, W, K, grad_loss=g)
+    np.testing.assert_allclose(plain["dH_d"], oracle.objective_from_features(Ht, Hd, W, K, 0.0, 1.0, grad_loss=g)["dH_d"], atol=0)
