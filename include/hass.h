@@ -155,6 +155,31 @@ int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, i
                                     void* cuda_stream);
 
 /*
+ * Combined training objective of one aligning step (Section 3.2: the cross-entropy between the
+ * target's and the draft's next-token distributions plus the Top-K loss of Section 3.1 with
+ * weight w, Section 4.1 uses w = 1.0), forward and backward in one call:
+ *
+ *   loss_ce[i]   = - sum_{v in Omega}     q_i(v) log p_i(v)        (full vocabulary)
+ *   loss_topk[i] = - sum_{x in Omega_hat} q_i(x) log p_i(x)        (Eq. 1)
+ *   dz_d[i,v]    = grad_loss[i] * ( (1 + w S_q) p(v) - q(v) - w q(v) [v in Omega_hat] )
+ *   dH_d         = dz_d W
+ *
+ * i.e. the gradient of sum_i grad_loss[i] (loss_ce[i] + w loss_topk[i]) with respect to H_d. The
+ * sweep spills the target tiles as well, a second GEMM forms q W per row, from which both the
+ * cross-entropy, lse_d - <H_d[i], (q W)[i]>, and its gradient term follow; 8 N d V tensor FLOPs
+ * are executed. Range condition and HASS_ERR_RANGE as for hass_topk_distill_fwd_bwd, for target
+ * and draft logits alike. The other outputs are those of hass_topk_distill_fwd.
+ * Workspace: hass_combined_distill_workspace_bytes (the normal workspace plus the target spill and
+ * a q W buffer for one chunk of rows).
+ */
+int hass_combined_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes);
+int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
+                                  int64_t V, int32_t K, float w_topk, const float* grad_loss,
+                                  float* loss_ce, float* loss_topk, int32_t* topk_idx, float* topk_q,
+                                  float* lse_t, float* lse_d, void* dH_d, int dH_dtype, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The same forward + backward for callers whose features live in HOST memory (the training
  * listing reads precomputed target hidden states per batch): H_t_host, H_d_host [N,d] bf16 are
  * copied to the device, the path runs, and loss_host [N] (fp32) and dH_d_host [N,d] (dH_dtype)

@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     HASS_FP32,
     K_MAX,
     check,
+    combined_distill_fwd_bwd,
+    combined_distill_workspace_bytes,
     kernel_launch_count,
     lib,
     PROFILE_KINDS,

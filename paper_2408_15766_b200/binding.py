@@ -42,6 +42,11 @@ def _load() -> ctypes.CDLL:
     L.hass_topk_distill_fwd_bwd_draft.argtypes = [vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, ctypes.c_int,
                                                   vp, sz, vp]
     L.hass_topk_distill_fwd_bwd_draft.restype = ctypes.c_int
+    L.hass_combined_distill_workspace_bytes.argtypes = [i64, i64, i64, i32, ctypes.POINTER(sz)]
+    L.hass_combined_distill_workspace_bytes.restype = ctypes.c_int
+    L.hass_combined_distill_fwd_bwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp,
+                                                vp, vp, ctypes.c_int, vp, sz, vp]
+    L.hass_combined_distill_fwd_bwd.restype = ctypes.c_int
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
     L.hass_check.argtypes = [vp, vp]
@@ -225,6 +230,36 @@ def topk_distill_fwd_bwd_draft(H_d, W, topk_idx, topk_q, grad_loss=None, dH_dtyp
     _ok(lib.hass_topk_distill_fwd_bwd_draft(_p(H_d), _p(W), N, d, V, K, _p(topk_idx), _p(topk_q), _p(grad_loss),
                                             _p(out["loss"]), _p(out["lse_d"]), _p(out["dH_d"]), dH_dtype, _p(ws),
                                             ws.numel(), _stream(stream)), "hass_topk_distill_fwd_bwd_draft")
+    return out
+
+
+def combined_distill_workspace_bytes(N: int, d: int, V: int, K: int) -> int:
+    out = ctypes.c_size_t(0)
+    _ok(lib.hass_combined_distill_workspace_bytes(N, d, V, K, ctypes.byref(out)), "hass_combined_distill_workspace_bytes")
+    return int(out.value)
+
+
+def combined_distill_fwd_bwd(H_t, H_d, W, K: int, w_topk: float = 1.0, grad_loss=None, dH_dtype: int = HASS_BF16,
+                             workspace=None, stream=None, out: Optional[dict] = None) -> dict:
+    """Cross-entropy over the full vocabulary plus w times the Top-K loss, forward and backward."""
+    N, d, V = _dims(H_t, W)
+    assert H_d.shape == H_t.shape and H_d.dtype == torch.bfloat16 and H_d.is_contiguous()
+    assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
+    dev = H_t.device
+    ws = _workspace(workspace, combined_distill_workspace_bytes(N, d, V, K), dev)
+    if out is None:
+        out = dict(loss_ce=torch.empty(N, dtype=torch.float32, device=dev),
+                   loss=torch.empty(N, dtype=torch.float32, device=dev),
+                   topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+                   topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+                   lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+                   lse_d=torch.empty(N, dtype=torch.float32, device=dev),
+                   dH_d=torch.empty(N, d, dtype=_dh_dtype(dH_dtype), device=dev))
+    out["workspace"] = ws
+    _ok(lib.hass_combined_distill_fwd_bwd(_p(H_t), _p(H_d), _p(W), N, d, V, K, ctypes.c_float(w_topk), _p(grad_loss),
+                                          _p(out["loss_ce"]), _p(out["loss"]), _p(out["topk_idx"]), _p(out["topk_q"]),
+                                          _p(out["lse_t"]), _p(out["lse_d"]), _p(out["dH_d"]), dH_dtype, _p(ws),
+                                          ws.numel(), _stream(stream)), "hass_combined_distill_fwd_bwd")
     return out
 
 

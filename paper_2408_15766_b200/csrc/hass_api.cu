@@ -495,10 +495,19 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
 // (2) finalize gives loss, Omega_hat, lse and the per-row scale of the spilled tiles; (3) the second
 // GEMM contracts the spilled tiles with W and applies scale and sparse term in its epilogue. No
 // logit is computed twice. with_target = false: Omega_hat is an input (aligning steps >= 2).
+// Extra buffers and outputs of the combined objective CE(q, p) + w * Top-K (nullptr: Top-K loss alone).
+struct Combined {
+    float w;               // weight of the Top-K term
+    float* loss_ce;        // [N] out: full-vocabulary cross-entropy per row
+    float* coef_t;         // [N] scratch: scale of the target spill
+    float* T;              // [chunk rows, d] scratch: q W of the chunk's rows
+    __nv_bfloat16* Pt;     // [chunk rows, p_pitch] scratch: spill of the target tiles
+};
+
 static int fused_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
                       long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
                       int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
-                      void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                      void* workspace, size_t workspace_bytes, cudaStream_t st, const Combined* cmb = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
@@ -536,6 +545,8 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     if (rc == HASS_OK) rc = make_tmap(&tmWk, W, V, d, d, BK, BN);
     if (rc == HASS_OK) rc = make_tmap(&tmWn, W, V, d, d, 64, BK);
     if (rc == HASS_OK) rc = make_tmap(&tmP, P, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
+    CUtensorMap tmPt;
+    if (rc == HASS_OK && cmb) rc = make_tmap(&tmPt, cmb->Pt, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
     if (rc != HASS_OK) return rc;
 
     for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
@@ -569,6 +580,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
         p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
         p.P = P;
+        p.Pt = cmb ? cmb->Pt : nullptr;
         p.p_pitch = L.p_pitch;
         p.status = status;
         rc = launch_gemm<MODE_STATS>(p, st);
@@ -600,6 +612,8 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.coef_out = coef;
         f.gq_out = gq;
         f.sparse_out = sparse;
+        f.w_topk = cmb ? cmb->w : 1.f;
+        f.coef_t_out = cmb ? cmb->coef_t : nullptr;
         {
             KernelTimer timer(KIND_FINALIZE, st);
             finalize_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(f);
@@ -612,6 +626,37 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         rc = plan_schedule(tiles, DT, di.sms, &o.sched);
         if (rc != HASS_OK) return rc;
         log_schedule("fused dH_d", o.sched);
+        if (cmb) {
+            // (2b) q W of the chunk's rows from the target spill, then the cross-entropy and its gradient term
+            GemmParams t = o;
+            t.tmA0 = tmPt;
+            t.tmA1 = tmPt;
+            t.tmB = tmWn;
+            t.row_tiles0 = tiles;
+            t.spill_begin = INT_MAX;
+            t.row_global_offset = 0;
+            t.rows_valid = rows;
+            t.n_cols = static_cast<int>(d);
+            t.col_tiles = DT;
+            t.k_blocks = ceil_div(V, BK);
+            t.K = K;
+            t.coef = cmb->coef_t + static_cast<long long>(t0) * BM;
+            t.out = cmb->T;
+            t.out_fp32 = 1;
+            t.out_align32 = 1;
+            t.out_pitch = d;
+            t.status = status;
+            rc = launch_gemm<MODE_OUT>(t, st);
+            if (rc != HASS_OK) return rc;
+            {
+                KernelTimer timer(KIND_FINALIZE, st);
+                ce_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(rows, t0 * BM, static_cast<int>(d),
+                                                             static_cast<const __nv_bfloat16*>(H_d), cmb->T, lse_d, grad_loss,
+                                                             cmb->loss_ce, sparse);
+            }
+            g_launches.fetch_add(1);
+            if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+        }
         o.tmA0 = tmP;
         o.tmA1 = tmP;
         o.tmB = tmWn;
@@ -746,6 +791,63 @@ int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, i
                                     void* cuda_stream) {
     return fused_impl(false, nullptr, H_d, W, N, d, V, K, grad_loss, topk_idx, topk_q, loss, nullptr, nullptr, nullptr,
                       lse_d, dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Buffers appended to the normal workspace by the combined-objective entry.
+struct CombinedStage {
+    size_t coef_t, T, Pt, total;
+};
+static int combined_stage(int64_t N, int64_t d, int64_t V, int32_t K, size_t base, CombinedStage* c) {
+    Layout L;
+    int rc = make_layout(N, d, V, K, sm_count_or_default(), &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    size_t off = align256(base);
+    c->coef_t = off;
+    off = align256(off + static_cast<size_t>(N) * 4);
+    c->T = off;
+    off = align256(off + static_cast<size_t>(L.pref_chunk_tiles) * BM * d * 4);
+    c->Pt = off;
+    off = align256(off + L.scratch_row_tile_bytes * L.pref_chunk_tiles);
+    c->total = off;
+    return HASS_OK;
+}
+
+int hass_combined_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes) {
+    if (!bytes) return HASS_ERR_INVALID_ARG;
+    size_t base = 0;
+    int rc = hass_topk_distill_workspace_bytes(N, d, V, K, &base);
+    if (rc != HASS_OK) return rc;
+    CombinedStage c;
+    rc = combined_stage(N, d, V, K, base, &c);
+    if (rc != HASS_OK) return rc;
+    *bytes = c.total;
+    return HASS_OK;
+}
+
+int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                                  int32_t K, float w_topk, const float* grad_loss, float* loss_ce, float* loss_topk,
+                                  int32_t* topk_idx, float* topk_q, float* lse_t, float* lse_d, void* dH_d,
+                                  int dH_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!loss_ce || !(w_topk == w_topk)) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    size_t base = 0;
+    rc = hass_topk_distill_workspace_bytes(N, d, V, K, &base);
+    if (rc != HASS_OK) return rc;
+    CombinedStage c;
+    rc = combined_stage(N, d, V, K, base, &c);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < c.total) return HASS_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    Combined cmb;
+    cmb.w = w_topk;
+    cmb.loss_ce = loss_ce;
+    cmb.coef_t = reinterpret_cast<float*>(ws + c.coef_t);
+    cmb.T = reinterpret_cast<float*>(ws + c.T);
+    cmb.Pt = reinterpret_cast<__nv_bfloat16*>(ws + c.Pt);
+    return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss_topk, topk_idx, topk_q, lse_t,
+                      lse_d, dH_d, dH_dtype, workspace, base, static_cast<cudaStream_t>(cuda_stream), &cmb);
 }
 
 // Device staging appended to the normal workspace by the *_host entry.

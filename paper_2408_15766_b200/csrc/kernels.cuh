@@ -73,9 +73,11 @@ struct GemmParams {
     const int* sidx;       // [N, K] Omega_hat sorted by token id
     const float* sgq;      // [N, K] g * q in the same order
     __nv_bfloat16* P;      // [chunk rows, p_pitch]
+    __nv_bfloat16* Pt;     // [chunk rows, p_pitch] spill of the target tiles, or nullptr
     long long p_pitch;
     // MODE_OUT. With sparse != nullptr the epilogue computes coef[row] * acc - sparse[local row, :] (row scale
-    // and the Omega_hat term of dz_d W, precomputed by finalize); otherwise it stores the accumulator.
+    // and the Omega_hat term of dz_d W, precomputed by finalize); with coef alone coef[row] * acc; with neither
+    // it stores the accumulator.
     const float* sparse;   // [chunk rows, out_pitch]
     void* out;
     int out_fp32;
@@ -83,6 +85,12 @@ struct GemmParams {
     long long out_pitch;   // elements
     unsigned int* status;
 };
+
+// MODE_STATS: does this row tile also write its tiles 2^(z log2e - ref2) as bf16? Draft tiles from spill_begin
+// on go to P; with Pt set, the target tiles (the leading topk_row_tiles) go to Pt (combined objective).
+__device__ __forceinline__ bool spills(const GemmParams& p, int rt) {
+    return rt >= p.spill_begin || (p.Pt != nullptr && rt < p.topk_row_tiles);
+}
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -238,7 +246,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 const bool second = (MODE == MODE_STATS) && rt >= p.row_tiles0;
                 const CUtensorMap* tmA = second ? &p.tmA1 : &p.tmA0;
                 const int row0 = p.a_row_offset + (second ? rt - p.row_tiles0 : rt) * BM;
-                const int t0 = (MODE == MODE_STATS && rt >= p.spill_begin && ln != 0) ? -1 : 0;
+                const int t0 = (MODE == MODE_STATS && spills(p, rt) && ln != 0) ? -1 : 0;
                 const int nt = (p.col_tiles - ln + S - 1) / S;
                 for (int t = t0; t < nt; ++t) {
                     const int ct = t < 0 ? 0 : ln + t * S;   // t = -1: column tile 0, for the row references only
@@ -274,7 +282,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             int ab = 0;
             uint32_t aphase = 0;
             for_each_item([&](int rt, int ln, int S, int) {
-                const int t0 = (MODE == MODE_STATS && rt >= p.spill_begin && ln != 0) ? -1 : 0;
+                const int t0 = (MODE == MODE_STATS && spills(p, rt) && ln != 0) ? -1 : 0;
                 const int nt = (p.col_tiles - ln + S - 1) / S;
                 for (int t = t0; t < nt; ++t) {
                     if (!wait_barrier(tempty_bar(ab), aphase ^ 1u, abort_flag, p.status, 2)) return false;
@@ -335,7 +343,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             // ---- per-item state ----
             float m = -INFINITY, s = 0.f, thr = -INFINITY;        // MODE_STATS
             bool want_topk = false;
-            const bool spill = MODE == MODE_STATS && rt >= p.spill_begin;
+            const bool spill = MODE == MODE_STATS && spills(p, rt);
             float ref2 = 0.f;                                     // spill rows: exponent offset (log2 units)
             float lse2 = 0.f, coef = 0.f;                         // MODE_PROBS / fused MODE_OUT
             const int* si = nullptr;
@@ -360,7 +368,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 sg = p.sgq + static_cast<long long>(g_row) * p.K;
                 nxt = si[0];
             }
-            if (MODE == MODE_OUT && p.sparse != nullptr && row_ok) coef = p.coef[g_row];
+            if (MODE == MODE_OUT && p.coef != nullptr && row_ok) coef = p.coef[g_row];
             const int t0 = (spill && ln != 0) ? -1 : 0;
             const int nt = (p.col_tiles - ln + S - 1) / S;
             for (int t = t0; t < nt; ++t) {
@@ -420,10 +428,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             for (int j = 0; j < 32; ++j)
                                 if (col0 + j >= p.n_cols) r[j] = __float_as_uint(-INFINITY);
                         }
-                        if (!spill) {
-                            float cm = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1]));
+                        float cm = -INFINITY;     // the chunk's largest logit (not needed by a spill row without Top-K)
+                        if (!spill || want_topk) {
+                            cm = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1]));
 #pragma unroll
                             for (int j = 2; j < 32; j += 2) cm = fmax3(cm, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+                        }
+                        if (!spill) {
                             if (cm > m) {
                                 s *= ex2((m - cm) * LOG2E);
                                 m = cm;
@@ -437,50 +448,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 fadd2(acc0, acc1, acc0, acc1, ex2(t0), ex2(t1));
                             }
                             s += acc0 + acc1;
-                            if (!USE_REG && want_topk && cm > thr) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    if (__uint_as_float(r[j]) > thr) {
-                                        cbuf[cnt] = make_uint2(r[j], static_cast<uint32_t>(col0 + j));
-                                        ++cnt;
-                                    }
-                                }
-                            }
-                            if (USE_REG && want_topk && cm > thr) {
-                                // collect the chunk's candidates, then admit them one by one (the
-                                // threshold only rises, so each is re-checked against the current one)
-                                int np = 0;
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const float x = __uint_as_float(r[j]);
-                                    if (x > thr) {
-                                        pend_v[USE_REG ? np : 0] = x;
-                                        pend_i[USE_REG ? np : 0] = col0 + j;
-                                        ++np;
-                                    }
-                                }
-                                for (int q = 0; q < np; ++q) {
-                                    const float x = pend_v[USE_REG ? q : 0];
-                                    const int id = pend_i[USE_REG ? q : 0];
-                                    if (!(x > thr)) continue;
-                                    // sorted insertion; equal logits stay behind earlier (lower) token ids
-#pragma unroll
-                                    for (int i = (USE_REG ? K_REG : 1) - 1; i >= 0; --i) {
-                                        if (i > 0 && i > lo) {
-                                            const bool shift = x > tv[i > 0 ? i - 1 : 0];
-                                            const bool here = !shift && x > tv[i];
-                                            tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
-                                            ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
-                                        } else if (i == lo) {
-                                            if (x > tv[i]) {
-                                                tv[i] = x;
-                                                ti[i] = id;
-                                            }
-                                        }
-                                    }
-                                    thr = tv[(USE_REG ? K_REG : 1) - 1];
-                                }
-                            }
                         } else {
                             // one exponential per logit serves both the row's sum and the spilled tile; a
                             // logit beyond the exponent range gives inf here and is reported at the item's end
@@ -496,8 +463,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 fadd2(acc0, acc1, acc0, acc1, e[j], e[j + 1]);
                             }
                             s += acc0 + acc1;
-                            __nv_bfloat16* dst =
-                                p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch + col0;
+                            __nv_bfloat16* dst = (rt >= p.spill_begin
+                                                      ? p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch
+                                                      : p.Pt + static_cast<long long>(rt * BM + r_local) * p.p_pitch) + col0;
 #pragma unroll
                             for (int g16 = 0; g16 < 2; ++g16)
                                 st_global_v8(dst + 16 * g16, pack_bf16x2(e[16 * g16 + 0], e[16 * g16 + 1]),
@@ -508,6 +476,50 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                              pack_bf16x2(e[16 * g16 + 10], e[16 * g16 + 11]),
                                              pack_bf16x2(e[16 * g16 + 12], e[16 * g16 + 13]),
                                              pack_bf16x2(e[16 * g16 + 14], e[16 * g16 + 15]));
+                        }
+                        if (!USE_REG && want_topk && cm > thr) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                if (__uint_as_float(r[j]) > thr) {
+                                    cbuf[cnt] = make_uint2(r[j], static_cast<uint32_t>(col0 + j));
+                                    ++cnt;
+                                }
+                            }
+                        }
+                        if (USE_REG && want_topk && cm > thr) {
+                            // collect the chunk's candidates, then admit them one by one (the
+                            // threshold only rises, so each is re-checked against the current one)
+                            int np = 0;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const float x = __uint_as_float(r[j]);
+                                if (x > thr) {
+                                    pend_v[USE_REG ? np : 0] = x;
+                                    pend_i[USE_REG ? np : 0] = col0 + j;
+                                    ++np;
+                                }
+                            }
+                            for (int q = 0; q < np; ++q) {
+                                const float x = pend_v[USE_REG ? q : 0];
+                                const int id = pend_i[USE_REG ? q : 0];
+                                if (!(x > thr)) continue;
+                                // sorted insertion; equal logits stay behind earlier (lower) token ids
+#pragma unroll
+                                for (int i = (USE_REG ? K_REG : 1) - 1; i >= 0; --i) {
+                                    if (i > 0 && i > lo) {
+                                        const bool shift = x > tv[i > 0 ? i - 1 : 0];
+                                        const bool here = !shift && x > tv[i];
+                                        tv[i] = shift ? tv[i > 0 ? i - 1 : 0] : (here ? x : tv[i]);
+                                        ti[i] = shift ? ti[i > 0 ? i - 1 : 0] : (here ? id : ti[i]);
+                                    } else if (i == lo) {
+                                        if (x > tv[i]) {
+                                            tv[i] = x;
+                                            ti[i] = id;
+                                        }
+                                    }
+                                }
+                                thr = tv[(USE_REG ? K_REG : 1) - 1];
+                            }
                         }
                     } else if (MODE == MODE_PROBS) {
                         while (nxt < col0) {
@@ -569,6 +581,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                     }
                                 }
                             }
+                        }
+                        if (p.sparse == nullptr && p.coef != nullptr) {
+                            // row scale only (the target side's q W of the combined objective)
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) o[j] *= coef;
                         }
                         if (p.out_fp32) {
                             float* dst = reinterpret_cast<float*>(p.out) + static_cast<long long>(g_row) * p.out_pitch + col0;
@@ -684,6 +701,9 @@ struct FinalizeParams {
     float* coef_out;       // [N]   g * S_q * exp(m_spill - lse_d), m_spill = the row's spill reference
     float* gq_out;         // [N,K] g * q, in the order of topk_idx
     float* sparse_out;     // [rows, d] sum_{x in Omega_hat} g q(x) W[x, :], indexed by local row
+    // combined objective CE(q, p) + w * Top-K (coef_t_out != nullptr): the target tiles were spilled as well
+    float w_topk;          // weight w of the Top-K term
+    float* coef_t_out;     // [N] e^(m_spill_t - lse_t): scale that turns (target spill x W) into q W
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -737,8 +757,13 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     if (p.row_tiles_t > 0) {
         find_slots(p.sched, rt, slot0, S);
         lse_t = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
-        if (lane == 0) p.lse_t[row] = lse_t;
+        if (lane == 0) {
+            p.lse_t[row] = lse_t;
+            if (p.coef_t_out) p.coef_t_out[row] = expf(p.part_m[static_cast<long long>(slot0) * BM + r] - lse_t);
+        }
     }
+    const bool combined = p.coef_t_out != nullptr;
+    const float gw = combined ? g * p.w_topk : g;     // weight of the Omega_hat term q 1[Omega_hat] in dz_d
 
     const __nv_bfloat16* hrow = p.H_d + static_cast<long long>(row) * p.d;
     float loss = 0.f;
@@ -829,7 +854,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
 #pragma unroll
             for (int jj = 0; jj < FIN_GRP; ++jj) {
                 if (jj < ng) {
-                    const float gq = g * sh_q[wib][g0 + jj];
+                    const float gq = gw * sh_q[wib][g0 + jj];
                     const uint4 wv = *reinterpret_cast<const uint4*>(p.W + static_cast<long long>(sh_tok[wib][g0 + jj]) * p.d + k0);
                     const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
 #pragma unroll
@@ -857,8 +882,46 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     }
     if (lane == 0) {
         p.loss[row] = loss;
-        if (p.coef_out) p.coef_out[row] = g * S_q * expf(m_spill - lse_d);
+        // dense part of dz_d: g S_q p (Top-K loss) or g (1 + w S_q) p (combined objective)
+        if (p.coef_out) p.coef_out[row] = (combined ? g * (1.f + p.w_topk * S_q) : g * S_q) * expf(m_spill - lse_d);
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// ce_kernel (combined objective): one warp per row of a chunk. T[local, :] = q W of the row (from the second
+// GEMM over the target spill). Full-vocabulary cross-entropy -sum_v q log p = lse_d - <H_d[row], q W>, and the
+// q W row joins the row's Omega_hat term so that dH_d = coef (draft spill x W) - sparse.
+__global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d, const __nv_bfloat16* __restrict__ H_d,
+                                                 const float* __restrict__ T, const float* __restrict__ lse_d,
+                                                 const float* __restrict__ grad_loss, float* __restrict__ loss_ce,
+                                                 float* __restrict__ sparse) {
+    const int lane = threadIdx.x & 31;
+    const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (local >= rows) return;
+    const int row = row_begin + local;
+    const float g = grad_loss ? grad_loss[row] : 1.f;
+    const __nv_bfloat16* hrow = H_d + static_cast<long long>(row) * d;
+    const float* trow = T + static_cast<long long>(local) * d;
+    float* srow = sparse + static_cast<long long>(local) * d;
+    float dot = 0.f;
+    for (int k0 = lane * 8; k0 < d; k0 += 256) {
+        const uint4 hv = *reinterpret_cast<const uint4*>(hrow + k0);
+        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+        const float4 t0 = *reinterpret_cast<const float4*>(trow + k0);
+        const float4 t1 = *reinterpret_cast<const float4*>(trow + k0 + 4);
+        float4 s0 = *reinterpret_cast<const float4*>(srow + k0);
+        float4 s1 = *reinterpret_cast<const float4*>(srow + k0 + 4);
+        const float2 h0 = __bfloat1622float2(hp[0]), h1 = __bfloat1622float2(hp[1]);
+        const float2 h2 = __bfloat1622float2(hp[2]), h3 = __bfloat1622float2(hp[3]);
+        dot += h0.x * t0.x + h0.y * t0.y + h1.x * t0.z + h1.y * t0.w + h2.x * t1.x + h2.y * t1.y + h3.x * t1.z + h3.y * t1.w;
+        s0.x = fmaf(g, t0.x, s0.x); s0.y = fmaf(g, t0.y, s0.y); s0.z = fmaf(g, t0.z, s0.z); s0.w = fmaf(g, t0.w, s0.w);
+        s1.x = fmaf(g, t1.x, s1.x); s1.y = fmaf(g, t1.y, s1.y); s1.z = fmaf(g, t1.z, s1.z); s1.w = fmaf(g, t1.w, s1.w);
+        *reinterpret_cast<float4*>(srow + k0) = s0;
+        *reinterpret_cast<float4*>(srow + k0 + 4) = s1;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (lane == 0) loss_ce[row] = lse_d[row] - dot;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -223,3 +223,32 @@ def test_l3_70b_k_sweep_sampled_rows(K):
     rows = hi.sample_rows(wl.N, max(FULL_ROWS // 3, 32), seed=wl.seed)
     stats, _ = _run_and_compare(inp, K, rows=rows)
     print("l3-70b K", K, stats)
+
+
+@pytest.mark.parametrize("N,d,V,K,w", [(64, 256, 1024, 10, 1.0), (300, 128, 5000, 5, 0.5), (4800, 64, 700, 20, 2.0)])
+def test_combined_objective_matches_oracle(N, d, V, K, w):
+    """Cross-entropy over the vocabulary + w * Top-K loss, forward and backward in one call."""
+    import oracle
+    hass = _hass()
+    inp = hi.make_custom(N, d, V, K, seed=N + K, sigma_w=2.0 / np.sqrt(d))
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(1)
+    grad = rng.uniform(0.5, 1.5, size=N)
+    grad[-1] = 0.0
+    out = hass.combined_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), K, w_topk=w,
+                                        grad_loss=torch.tensor(grad, dtype=torch.float32, device=dev),
+                                        dH_dtype=hass.HASS_FP32)
+    hass.check(out["workspace"])
+    # Top-K loss, Omega_hat, lse: the usual comparison (dH_d is that of the combined objective, checked below)
+    cpu = _to_cpu(out)
+    print(compare(inp.H_t, inp.H_d[0], inp.W, K, cpu, check_dH=False))
+    rows = hi.sample_rows(N, 256, seed=3)
+    ref = oracle.objective_from_features(hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W), K,
+                                         1.0, w, rows=rows, grad_loss=grad,
+                                         forced_idx=cpu["topk_idx"].numpy()[rows].astype(np.int32))
+    ce = cpu["loss_ce"].numpy()[rows]
+    assert np.all(np.abs(ce - ref["loss_ce"]) <= 2e-3 * np.maximum(np.abs(ref["loss_ce"]), 1e-6))
+    scale = np.abs(ref["dH_d"]).max()
+    err = np.abs(cpu["dH_d"].numpy()[rows].astype(np.float64) - ref["dH_d"]).max()
+    print("combined: loss_ce rel", float((np.abs(ce - ref["loss_ce"]) / np.abs(ref["loss_ce"])).max()), "dH rel", err / scale)
+    assert err <= 1e-2 * scale
