@@ -614,6 +614,9 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.sparse_out = sparse;
         f.w_topk = cmb ? cmb->w : 1.f;
         f.coef_t_out = cmb ? cmb->coef_t : nullptr;
+        f.Pt = cmb ? cmb->Pt : nullptr;
+        f.p_pitch = L.p_pitch;
+        f.ce_corr_out = reinterpret_cast<float*>(ws + L.lse2);    // [N] floats, otherwise used by the split backward
         {
             KernelTimer timer(KIND_FINALIZE, st);
             finalize_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(f);
@@ -652,7 +655,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
                 KernelTimer timer(KIND_FINALIZE, st);
                 ce_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(rows, t0 * BM, static_cast<int>(d),
                                                              static_cast<const __nv_bfloat16*>(H_d), cmb->T, lse_d, grad_loss,
-                                                             cmb->loss_ce, sparse);
+                                                             reinterpret_cast<const float*>(ws + L.lse2), cmb->loss_ce, sparse);
             }
             g_launches.fetch_add(1);
             if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;

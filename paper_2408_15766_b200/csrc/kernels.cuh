@@ -704,6 +704,10 @@ struct FinalizeParams {
     // combined objective CE(q, p) + w * Top-K (coef_t_out != nullptr): the target tiles were spilled as well
     float w_topk;          // weight w of the Top-K term
     float* coef_t_out;     // [N] e^(m_spill_t - lse_t): scale that turns (target spill x W) into q W
+    const __nv_bfloat16* Pt;   // target spill of the chunk [rows, p_pitch]
+    long long p_pitch;
+    float* ce_corr_out;    // [N] sum_{x in Omega_hat} (q(x) - bf16 q(x)) z_d(x): the cross-entropy is formed from
+                           // the bf16 spill; its largest terms are put back in fp32
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -763,6 +767,8 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
         }
     }
     const bool combined = p.coef_t_out != nullptr;
+    const float coef_t = combined ? expf(p.part_m[static_cast<long long>(slot0) * BM + r] - lse_t) : 0.f;
+    float ce_corr = 0.f;
     const float gw = combined ? g * p.w_topk : g;     // weight of the Omega_hat term q 1[Omega_hat] in dz_d
 
     const __nv_bfloat16* hrow = p.H_d + static_cast<long long>(row) * p.d;
@@ -877,10 +883,18 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             float acc = dot[jj];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (jj < ng) loss += sh_q[wib][g0 + jj] * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
+            if (jj < ng) {
+                const float qv = sh_q[wib][g0 + jj];
+                loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
+                if (combined) {
+                    const float q_spill = __bfloat162float(p.Pt[static_cast<long long>(local) * p.p_pitch + sh_tok[wib][g0 + jj]]) * coef_t;
+                    ce_corr += (qv - q_spill) * acc;
+                }
+            }
         }
     }
     if (lane == 0) {
+        if (combined) p.ce_corr_out[row] = ce_corr;
         p.loss[row] = loss;
         // dense part of dz_d: g S_q p (Top-K loss) or g (1 + w S_q) p (combined objective)
         if (p.coef_out) p.coef_out[row] = (combined ? g * (1.f + p.w_topk * S_q) : g * S_q) * expf(m_spill - lse_d);
@@ -890,11 +904,11 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
 // ---------------------------------------------------------------------------------------------
 // ce_kernel (combined objective): one warp per row of a chunk. T[local, :] = q W of the row (from the second
 // GEMM over the target spill). Full-vocabulary cross-entropy -sum_v q log p = lse_d - <H_d[row], q W>, and the
-// q W row joins the row's Omega_hat term so that dH_d = coef (draft spill x W) - sparse.
+// (with the fp32 correction of the Omega_hat terms from finalize) the q W row joins the row's Omega_hat term so that dH_d = coef (draft spill x W) - sparse.
 __global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d, const __nv_bfloat16* __restrict__ H_d,
                                                  const float* __restrict__ T, const float* __restrict__ lse_d,
-                                                 const float* __restrict__ grad_loss, float* __restrict__ loss_ce,
-                                                 float* __restrict__ sparse) {
+                                                 const float* __restrict__ grad_loss, const float* __restrict__ ce_corr,
+                                                 float* __restrict__ loss_ce, float* __restrict__ sparse) {
     const int lane = threadIdx.x & 31;
     const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (local >= rows) return;
@@ -921,7 +935,7 @@ __global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d,
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    if (lane == 0) loss_ce[row] = lse_d[row] - dot;
+    if (lane == 0) loss_ce[row] = lse_d[row] - dot - ce_corr[row];
 }
 
 // ---------------------------------------------------------------------------------------------
