@@ -190,6 +190,9 @@ def main():
     ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--K", type=int, default=None)
+    ap.add_argument("--objective", default="topk", choices=["topk", "combined"],
+                    help="topk: Eq. 1 alone (the headline metric); combined: cross-entropy over the vocabulary "
+                         "+ w * Top-K in one call (8 N d V tensor FLOPs)")
     ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -216,13 +219,18 @@ def main():
     H_t, W = inp.H_t.to(dev), inp.W.to(dev)
     H_d_steps = [h.to(dev) for h in inp.H_d]      # one draft-feature tensor per aligning step
     H_d = H_d_steps[0]
-    ws = torch.empty(hass.topk_distill_host_workspace_bytes(N, d, V, K), dtype=torch.uint8, device=dev)
+    combined = args.objective == "combined"
+    ws_bytes = max(hass.topk_distill_host_workspace_bytes(N, d, V, K),
+                   hass.combined_distill_workspace_bytes(N, d, V, K) if combined else 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
                topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
                topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
                lse_t=torch.empty(N, dtype=torch.float32, device=dev),
                lse_d=torch.empty(N, dtype=torch.float32, device=dev),
                dH_d=torch.empty(N, d, dtype=torch.bfloat16, device=dev))
+    if combined:
+        out["loss_ce"] = torch.empty(N, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
 
     counts = {"full": 0, "draft": 0, "i": 0}
@@ -232,7 +240,10 @@ def main():
         # reuse Omega_hat and q (the workload's `steps`; 1 for the default workload, so every step is full).
         j = counts["i"] % wl.steps
         counts["i"] += 1
-        if j == 0:
+        if combined:
+            counts["full"] += 1
+            hass.combined_distill_fwd_bwd(H_t, H_d_steps[j], W, K, w_topk=1.0, workspace=ws, out=out, stream=stream)
+        elif j == 0:
             counts["full"] += 1
             hass.topk_distill_fwd_bwd(H_t, H_d_steps[0], W, K, workspace=ws, out=out, stream=stream)
         else:
@@ -270,7 +281,7 @@ def main():
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not combined:
         Ht_h, Hd_h = inp.H_t.pin_memory(), inp.H_d[0].pin_memory()
         loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
         dH_h = torch.empty(N, d, dtype=torch.bfloat16).pin_memory()
@@ -294,10 +305,11 @@ def main():
         return
 
     # ---- roofline of the dominant kernel (tensor-core bound) ----
-    flops_credit = 6.0 * N * d * V                 # three d x V products per token
+    # three d x V products per token (z_t, z_d, dH_d); the combined objective needs a fourth (q W)
+    flops_credit = (8.0 if combined else 6.0) * N * d * V
     # executed tensor work per step, averaged over the timed steps (a draft-only step skips the target product)
     kinds = {"stats_gemm": (4.0 * n_full + 2.0 * n_draft) / args.steps * N * d * V, "dz_gemm": 2.0 * N * d * V,
-             "dH_gemm": 2.0 * N * d * V}
+             "dH_gemm": (4.0 if combined else 2.0) * N * d * V}
     total_ms = sum(v[0] for v in prof.values())
     kernel_rows = {}
     for k, (ms, cnt) in prof.items():
@@ -327,10 +339,11 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "N": N, "d": d, "V": V, "K": K, "rows_per_gpu": N,
                        "l2": "inputs larger than L2 (W alone is %.0f MB)" % (V * d * 2 / 1e6),
-                       "dH_dtype": "bf16", "aligning_steps": wl.steps,
+                       "dH_dtype": "bf16", "aligning_steps": wl.steps, "objective": args.objective,
                        "target_stats": ("recomputed every step" if wl.steps == 1 else
                                         "computed in aligning step 1, reused in steps 2..%d" % wl.steps),
-                       "path": "hass_topk_distill_fwd_bwd (no logit recompute)"},
+                       "path": ("hass_combined_distill_fwd_bwd" if combined else
+                                "hass_topk_distill_fwd_bwd (no logit recompute)")},
             "clocks": clocks, "gpu_launches": launches,
             "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
                        "executed_tflops": executed / (ms_step * 1e-3) / 1e12, "executed_flops_per_step": executed,

@@ -252,3 +252,24 @@ def test_combined_objective_matches_oracle(N, d, V, K, w):
     err = np.abs(cpu["dH_d"].numpy()[rows].astype(np.float64) - ref["dH_d"]).max()
     print("combined: loss_ce rel", float((np.abs(ce - ref["loss_ce"]) / np.abs(ref["loss_ce"])).max()), "dH rel", err / scale)
     assert err <= 1e-2 * scale
+
+
+def test_combined_objective_l2_7b_sampled_rows():
+    import oracle
+    hass = _hass()
+    wl = hi.WORKLOADS["l2-7b"]
+    inp = hi.make_inputs(wl)
+    dev = torch.device("cuda:0")
+    out = hass.combined_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), wl.K, w_topk=1.0)
+    hass.check(out["workspace"])
+    cpu = _to_cpu(out)
+    rows = hi.sample_rows(wl.N, max(FULL_ROWS // 2, 32), seed=1)
+    print(compare(inp.H_t, inp.H_d[0], inp.W, wl.K, cpu, rows=rows, check_dH=False))
+    ref = oracle.objective_from_features(hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W), wl.K,
+                                         1.0, 1.0, rows=rows, forced_idx=cpu["topk_idx"].numpy()[rows].astype(np.int32))
+    ce = cpu["loss_ce"].numpy()[rows]
+    assert np.all(np.abs(ce - ref["loss_ce"]) <= 2e-3 * np.abs(ref["loss_ce"]))
+    scale = np.abs(ref["dH_d"]).max()
+    err = np.abs(cpu["dH_d"].float().numpy()[rows].astype(np.float64) - ref["dH_d"]).max()
+    print("l2-7b combined: loss_ce rel", float((np.abs(ce - ref["loss_ce"]) / np.abs(ref["loss_ce"])).max()), "dH rel", err / scale)
+    assert err <= 1e-2 * scale
