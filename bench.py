@@ -326,7 +326,7 @@ def main():
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak,
                 "traffic": (TRAFFIC_CAPTURE["bytes_per_launch"]
-                            if dom == "stats_gemm" and wl.name == TRAFFIC_CAPTURE["workload"]
+                            if dom == "stats_gemm" and not combined and wl.name == TRAFFIC_CAPTURE["workload"]
                             and hass.version() == TRAFFIC_CAPTURE["version"] else None),
                 "peak_kind": f"bf16_tflops_sustained, of {peak_kind} (kernel timed inside a long step)",
                 "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
