@@ -55,6 +55,12 @@ def _load():
         lib.hass_oracle_features_objective.argtypes = [c_vp, c_vp, c_vp, ctypes.c_int, c_i64, c_i64, c_i64, c_i32,
                                                        c_dbl, c_dbl, c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp,
                                                        c_vp, c_vp, c_vp, c_vp]
+        lib.hass_oracle_row_variant.restype = ctypes.c_int
+        lib.hass_oracle_row_variant.argtypes = [c_vp, c_vp, c_i64, c_i32, c_dbl, ctypes.c_int, c_dbl, c_vp, c_vp, c_vp,
+                                                c_vp, c_vp, c_vp, c_vp]
+        lib.hass_oracle_features_variant.restype = ctypes.c_int
+        lib.hass_oracle_features_variant.argtypes = [c_vp, c_vp, c_vp, c_i64, c_i64, c_i64, c_i32, ctypes.c_int, c_dbl,
+                                                     c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
         lib.hass_oracle_logits_at.restype = ctypes.c_int
         lib.hass_oracle_logits_at.argtypes = [c_vp, c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_i64, c_vp]
         _lib = lib
@@ -88,6 +94,49 @@ def from_logits(z_t, z_d, K: int, g: float = 1.0, forced_idx=None, want_dz: bool
     if rc != 0:
         raise ValueError("oracle: bad arguments")
     return dict(loss=float(loss[0]), idx=idx, q_k=q_k, lse_t=float(lse_t[0]), lse_d=float(lse_d[0]), dz_d=dz)
+
+
+VARIANT_TOPK, VARIANT_TOP_P, VARIANT_NORMED = 0, 1, 2
+
+
+def variant_from_logits(z_t, z_d, K: int, variant: int, param: float = 0.0, g: float = 1.0) -> dict:
+    """One row of logits under a loss variant of Section 4.3 (Top-P, Normed Top-K) or Eq. 1."""
+    z_t = np.ascontiguousarray(z_t, dtype=np.float64)
+    z_d = np.ascontiguousarray(z_d, dtype=np.float64)
+    V = z_t.shape[0]
+    loss, lse_t, lse_d = np.zeros(1), np.zeros(1), np.zeros(1)
+    idx = np.zeros(K, dtype=np.int32)
+    q_k = np.zeros(K)
+    n = np.zeros(1, dtype=np.int32)
+    dz = np.zeros(V)
+    rc = _load().hass_oracle_row_variant(_ptr(z_t), _ptr(z_d), V, K, float(g), int(variant), float(param), _ptr(loss),
+                                         _ptr(idx), _ptr(q_k), _ptr(n), _ptr(lse_t), _ptr(lse_d), _ptr(dz))
+    if rc != 0:
+        raise ValueError("oracle: bad arguments")
+    return dict(loss=float(loss[0]), idx=idx, q_k=q_k, n=int(n[0]), lse_t=float(lse_t[0]), lse_d=float(lse_d[0]),
+                dz_d=dz)
+
+
+def variant_from_features(H_t, H_d, W, K: int, variant: int, param: float = 0.0, rows=None, grad_loss=None) -> dict:
+    """Feature-level loss variants on bf16 bit patterns; outputs indexed by position in ``rows``."""
+    H_t, H_d, W = np.ascontiguousarray(H_t), np.ascontiguousarray(H_d), np.ascontiguousarray(W)
+    assert H_t.dtype == H_d.dtype == W.dtype == np.uint16
+    N, d = H_t.shape
+    V = W.shape[0]
+    rows_a = np.arange(N, dtype=np.int64) if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = rows_a.shape[0]
+    gl = None if grad_loss is None else np.ascontiguousarray(grad_loss, dtype=np.float64)
+    loss, lse_t, lse_d = np.zeros(n), np.zeros(n), np.zeros(n)
+    idx = np.zeros((n, K), dtype=np.int32)
+    q_k = np.zeros((n, K))
+    cnt = np.zeros(n, dtype=np.int32)
+    dH = np.zeros((n, d))
+    rc = _load().hass_oracle_features_variant(_ptr(H_t), _ptr(H_d), _ptr(W), N, d, V, K, int(variant), float(param),
+                                              _ptr(gl), _ptr(rows_a), n, _ptr(loss), _ptr(idx), _ptr(q_k), _ptr(cnt),
+                                              _ptr(lse_t), _ptr(lse_d), _ptr(dH))
+    if rc != 0:
+        raise ValueError("oracle: bad arguments")
+    return dict(loss=loss, idx=idx, q_k=q_k, n=cnt, lse_t=lse_t, lse_d=lse_d, dH_d=dH)
 
 
 def objective_from_logits(z_t, z_d, K: int, w_ce: float, w_topk: float, g: float = 1.0) -> dict:

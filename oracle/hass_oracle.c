@@ -33,6 +33,15 @@
  *   dL/dz_d[v] = g ( w_ce (p[v] - q[v]) + w_topk (S_q p[v] - q[v] [v in Omega_hat]) ).
  * The plain entries are the case w_ce = 0, w_topk = 1.
  *
+ * Loss variants of Section 4.3 (the paper describes them in one sentence each; the readings are this
+ * file's), selected by `variant` in the *_variant entries, all with q and Omega_hat constant:
+ *   1  Top-P:        Omega_hat = the shortest prefix of the tokens sorted by descending q whose cumulative
+ *                    probability is larger than P, at most K tokens; loss and gradient as Eq. 1 on that set.
+ *   2  Normed Top-K: q and p are both renormalised over Omega_hat (linear normalisation of the
+ *                    probabilities, which equals a softmax over the logits restricted to Omega_hat):
+ *                    L = - sum_{x in Omega_hat} qn(x) log pn(x), qn = q / S_q, pn = p / S_p;
+ *                    dL/dz_d[x] = g (pn(x) - qn(x)) on Omega_hat and 0 elsewhere.
+ *
  * Inputs of the feature-level entry are bf16 bit patterns widened exactly to fp64.
  * The only liberty taken with summation order is SIMD reassociation of the inner
  * dot-product loop (omp simd reduction), i.e. rounding order.
@@ -187,6 +196,122 @@ int hass_oracle_row_objective(const double* z_t, const double* z_d, int64_t V, i
     }
     free(order);
     return 0;
+}
+
+/*
+ * Loss variants (see the header). variant 0 = Eq. 1, 1 = Top-P (param = P, K = cap), 2 = Normed Top-K.
+ * n_out receives |Omega_hat|; idx / q_k beyond it are -1 / 0.
+ */
+int hass_oracle_row_variant(const double* z_t, const double* z_d, int64_t V, int32_t K, double g, int variant,
+                            double param, double* loss, int32_t* idx, double* q_k, int32_t* n_out,
+                            double* lse_t_out, double* lse_d_out, double* dz_d) {
+    if (variant < 0 || variant > 2) return -1;
+    int rc = hass_oracle_row_objective(z_t, z_d, V, K, g, 0.0, 1.0, NULL, NULL, loss, idx, q_k, lse_t_out, lse_d_out,
+                                       variant == 0 ? dz_d : NULL);
+    if (rc != 0) return rc;
+    int32_t n = K;
+    if (variant == 0) {
+        if (n_out) *n_out = n;
+        return 0;
+    }
+    const double lse_d = log_sum_exp(z_d, V);
+    if (variant == 1) {
+        /* shortest sorted prefix whose cumulative target probability is larger than P */
+        double cum = 0.0;
+        n = 0;
+        while (n < K) {
+            cum += q_k[n];
+            ++n;
+            if (cum > param) break;
+        }
+        double S_q = 0.0, L = 0.0;
+        for (int32_t j = 0; j < n; ++j) {
+            S_q += q_k[j];
+            L -= q_k[j] * (z_d[idx[j]] - lse_d);
+        }
+        *loss = L;
+        if (dz_d) {
+            for (int64_t v = 0; v < V; ++v) dz_d[v] = g * S_q * exp(z_d[v] - lse_d);
+            for (int32_t j = 0; j < n; ++j) dz_d[idx[j]] -= g * q_k[j];
+        }
+        for (int32_t j = n; j < K; ++j) {
+            idx[j] = -1;
+            q_k[j] = 0.0;
+        }
+    } else {
+        /* both distributions renormalised over Omega_hat */
+        double S_q = 0.0, m = z_d[idx[0]];
+        for (int32_t j = 0; j < K; ++j) {
+            S_q += q_k[j];
+            if (z_d[idx[j]] > m) m = z_d[idx[j]];
+        }
+        double se = 0.0;
+        for (int32_t j = 0; j < K; ++j) se += exp(z_d[idx[j]] - m);
+        const double lse_k = m + log(se);
+        double L = 0.0;
+        for (int32_t j = 0; j < K; ++j) L -= (q_k[j] / S_q) * (z_d[idx[j]] - lse_k);
+        *loss = L;
+        if (dz_d) {
+            for (int64_t v = 0; v < V; ++v) dz_d[v] = 0.0;
+            for (int32_t j = 0; j < K; ++j) dz_d[idx[j]] = g * (exp(z_d[idx[j]] - lse_k) - q_k[j] / S_q);
+        }
+    }
+    if (n_out) *n_out = n;
+    return 0;
+}
+
+/* Feature-level loss variants for a set of rows (bf16 bit patterns); outputs as hass_oracle_features plus n. */
+int hass_oracle_features_variant(const uint16_t* H_t, const uint16_t* H_d, const uint16_t* W, int64_t N, int64_t d,
+                                 int64_t V, int32_t K, int variant, double param, const double* grad_loss,
+                                 const int64_t* rows, int64_t n_rows, double* loss, int32_t* idx, double* q_k,
+                                 int32_t* n_out, double* lse_t, double* lse_d, double* dH_d) {
+    if (N < 1 || d < 1 || V < 1 || K < 1 || K > V || n_rows < 0 || !rows) return -1;
+    int status = 0;
+#pragma omp parallel
+    {
+        double* ht = (double*)malloc(sizeof(double) * (size_t)d);
+        double* hd = (double*)malloc(sizeof(double) * (size_t)d);
+        double* wr = (double*)malloc(sizeof(double) * (size_t)d);
+        double* zt = (double*)malloc(sizeof(double) * (size_t)V);
+        double* zd = (double*)malloc(sizeof(double) * (size_t)V);
+        double* dz = (double*)malloc(sizeof(double) * (size_t)V);
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            const int64_t i = rows[r];
+            if (i < 0 || i >= N) {
+#pragma omp atomic write
+                status = -1;
+                continue;
+            }
+            const double g = grad_loss ? grad_loss[i] : 1.0;
+            widen_bf16(H_t + i * d, ht, d);
+            widen_bf16(H_d + i * d, hd, d);
+            for (int64_t v = 0; v < V; ++v) {
+                widen_bf16(W + v * d, wr, d);
+                dot2(ht, hd, wr, d, &zt[v], &zd[v]);
+            }
+            if (hass_oracle_row_variant(zt, zd, V, K, g, variant, param, &loss[r], idx + r * K, q_k + r * K, &n_out[r],
+                                        &lse_t[r], &lse_d[r], dz) != 0) {
+#pragma omp atomic write
+                status = -1;
+                continue;
+            }
+            double* out = dH_d + r * d;
+            for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+            for (int64_t v = 0; v < V; ++v) {
+                if (dz[v] == 0.0) continue;
+                widen_bf16(W + v * d, wr, d);
+                axpy(dz[v], wr, out, d);
+            }
+        }
+        free(ht);
+        free(hd);
+        free(wr);
+        free(zt);
+        free(zd);
+        free(dz);
+    }
+    return status;
 }
 
 int hass_oracle_row_from_logits(const double* z_t, const double* z_d, int64_t V, int32_t K, double g,

@@ -339,3 +339,69 @@ def test_objective_features_level_autograd_restatement():
     np.testing.assert_allclose(r["dH_d"], Hdt.grad.numpy(), atol=1e-13)
     plain = oracle.from_features(Ht, Hd, W, K, grad_loss=g)
     np.testing.assert_allclose(plain["dH_d"], oracle.objective_from_features(Ht, Hd, W, K, 0.0, 1.0, grad_loss=g)["dH_d"], atol=0)
+
+
+# ---- loss variants of Section 4.3: Top-P and Normed Top-K ---------------------------------------------
+
+def test_top_p_is_the_shortest_sorted_prefix_and_reduces_to_top_k():
+    V, cap = 50, 12
+    z_t, z_d = _rand_logits(V, seed=41, scale=2.0)
+    q = np.exp(z_t) / np.exp(z_t).sum()
+    p = np.exp(z_d) / np.exp(z_d).sum()
+    order = np.argsort(-q, kind="stable")
+    for P in (0.05, 0.3, 0.6, 0.9):
+        n = int(np.searchsorted(np.cumsum(q[order]), P, side="right")) + 1      # literal: first prefix with cum > P
+        n = min(n, cap)
+        r = oracle.variant_from_logits(z_t, z_d, cap, oracle.VARIANT_TOP_P, P)
+        assert r["n"] == n and np.array_equal(r["idx"][:n], order[:n]) and np.all(r["idx"][n:] == -1)
+        assert r["loss"] == pytest.approx(-(q[order[:n]] * np.log(p[order[:n]])).sum(), rel=1e-12)
+        same = oracle.from_logits(z_t, z_d, n)           # Eq. 1 with K = n is the same loss and gradient
+        assert r["loss"] == pytest.approx(same["loss"], rel=1e-13)
+        np.testing.assert_allclose(r["dz_d"], same["dz_d"], atol=1e-16)
+    full = oracle.variant_from_logits(z_t, z_d, cap, oracle.VARIANT_TOP_P, 2.0)     # P never reached: all cap tokens
+    assert full["n"] == cap and full["loss"] == pytest.approx(oracle.from_logits(z_t, z_d, cap)["loss"], rel=1e-13)
+    one = oracle.variant_from_logits(z_t, z_d, cap, oracle.VARIANT_TOP_P, 0.0)
+    assert one["n"] == 1 and one["loss"] == pytest.approx(oracle.from_logits(z_t, z_d, 1)["loss"], rel=1e-13)
+
+
+def test_normed_top_k_closed_forms_and_autograd():
+    V, K = 70, 8
+    z_t, z_d = _rand_logits(V, seed=43, scale=1.5)
+    r = oracle.variant_from_logits(z_t, z_d, K, oracle.VARIANT_NORMED, g=1.3)
+    zd = torch.tensor(z_d, requires_grad=True)
+    q = torch.softmax(torch.tensor(z_t), 0)
+    qk, idx = torch.topk(q, K)
+    logpn = torch.log_softmax(zd[idx], 0)                # softmax over the logits restricted to Omega_hat
+    loss = -((qk / qk.sum()) * logpn).sum()
+    (1.3 * loss).backward()
+    assert np.array_equal(r["idx"], idx.numpy())
+    assert r["loss"] == pytest.approx(float(loss), rel=1e-12)
+    np.testing.assert_allclose(r["dz_d"], zd.grad.numpy(), atol=1e-15)
+    # linear normalisation of the probabilities gives the same thing
+    p = torch.softmax(torch.tensor(z_d), 0)
+    lin = -((qk / qk.sum()) * torch.log(p[idx] / p[idx].sum())).sum()
+    assert r["loss"] == pytest.approx(float(lin), rel=1e-12)
+    # K = V: nothing to renormalise, plain cross-entropy; K = 1: the loss and its gradient vanish
+    allv = oracle.variant_from_logits(z_t, z_d, V, oracle.VARIANT_NORMED)
+    assert allv["loss"] == pytest.approx(float(-(q * torch.log_softmax(torch.tensor(z_d), 0)).sum()), rel=1e-12)
+    k1 = oracle.variant_from_logits(z_t, z_d, 1, oracle.VARIANT_NORMED)
+    assert abs(k1["loss"]) < 1e-15 and np.abs(k1["dz_d"]).max() < 1e-15
+    # invariant to shifting the draft logits, gradient sums to zero, non-negative
+    sh = oracle.variant_from_logits(z_t, z_d + 4.0, K, oracle.VARIANT_NORMED, g=1.3)
+    assert sh["loss"] == pytest.approx(r["loss"], rel=1e-12) and abs(r["dz_d"].sum()) < 1e-15 and r["loss"] >= 0
+
+
+def test_variants_at_features_level_match_the_row_entry():
+    N, d, V, K = 4, 16, 60, 5
+    Ht, Hd, W, _ = _feat(N, d, V, seed=45, sigma_w=0.3)
+    zt, zd = _z(Ht, W), _z(Hd, W)
+    Wd = torch.from_numpy(W.view(np.int16).copy()).view(torch.bfloat16).double().numpy()
+    g = np.array([1.0, 0.5, 0.0, 2.0])
+    for variant, param in ((oracle.VARIANT_TOPK, 0.0), (oracle.VARIANT_TOP_P, 0.2), (oracle.VARIANT_NORMED, 0.0)):
+        f = oracle.variant_from_features(Ht, Hd, W, K, variant, param, grad_loss=g)
+        for i in range(N):
+            r = oracle.variant_from_logits(zt[i], zd[i], K, variant, param, g=g[i])
+            assert f["loss"][i] == pytest.approx(r["loss"], rel=1e-12) and f["n"][i] == r["n"]
+            np.testing.assert_allclose(f["dH_d"][i], r["dz_d"] @ Wd, atol=1e-13)
+    plain = oracle.from_features(Ht, Hd, W, K, grad_loss=g)
+    np.testing.assert_allclose(oracle.variant_from_features(Ht, Hd, W, K, 0, grad_loss=g)["dH_d"], plain["dH_d"], atol=1e-15)
