@@ -180,6 +180,29 @@ int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* 
                                   size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Loss variants that the paper compares with the Top-K loss (Section 4.3, one sentence each; the exact
+ * formulas below are this library's readings), forward and backward in one call:
+ *
+ *   HASS_LOSS_TOPK         Eq. 1; the same as hass_topk_distill_fwd_bwd.
+ *   HASS_LOSS_TOP_P        Omega_hat = the shortest prefix of the tokens sorted by descending q whose
+ *                          cumulative probability is larger than param = P, at most K tokens; loss and
+ *                          gradient as Eq. 1 on that set. topk_idx / topk_q beyond the prefix are -1 / 0.
+ *   HASS_LOSS_NORMED_TOPK  q and p both renormalised over Omega_hat (the K most probable tokens):
+ *                          L = - sum qn log pn, qn = q / S_q, pn = p / S_p (a softmax of the draft
+ *                          logits restricted to Omega_hat), dz_d = g (pn - qn) on Omega_hat, 0 elsewhere.
+ *                          Only the target rows are swept; lse_d is not written (may be NULL).
+ *
+ * topk_n [N] (nullable) receives |Omega_hat| per row. The other arguments are those of
+ * hass_topk_distill_fwd_bwd. The Bi-directional, Recall@k and BiLD losses of that section are not built.
+ */
+typedef enum { HASS_LOSS_TOPK = 0, HASS_LOSS_TOP_P = 1, HASS_LOSS_NORMED_TOPK = 2 } hass_loss_variant;
+int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
+                                 int64_t V, int32_t K, int variant, float param, const float* grad_loss,
+                                 float* loss, int32_t* topk_idx, float* topk_q, int32_t* topk_n,
+                                 float* lse_t, float* lse_d, void* dH_d, int dH_dtype, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The same forward + backward for callers whose features live in HOST memory (the training
  * listing reads precomputed target hidden states per batch): H_t_host, H_d_host [N,d] bf16 are
  * copied to the device, the path runs, and loss_host [N] (fp32) and dH_d_host [N,d] (dH_dtype)

@@ -29,4 +29,8 @@ from .binding import (  # noqa: F401
     topk_distill_host_workspace_bytes,
     topk_distill_workspace_bytes,
     version,
+    variant_distill_fwd_bwd,
+    LOSS_TOPK,
+    LOSS_TOP_P,
+    LOSS_NORMED_TOPK,
 )

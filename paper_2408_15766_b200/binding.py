@@ -47,6 +47,9 @@ def _load() -> ctypes.CDLL:
     L.hass_combined_distill_fwd_bwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp,
                                                 vp, vp, ctypes.c_int, vp, sz, vp]
     L.hass_combined_distill_fwd_bwd.restype = ctypes.c_int
+    L.hass_variant_distill_fwd_bwd.argtypes = [vp, vp, vp, i64, i64, i64, i32, ctypes.c_int, ctypes.c_float, vp, vp, vp,
+                                               vp, vp, vp, vp, vp, ctypes.c_int, vp, sz, vp]
+    L.hass_variant_distill_fwd_bwd.restype = ctypes.c_int
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
     L.hass_check.argtypes = [vp, vp]
@@ -260,6 +263,31 @@ def combined_distill_fwd_bwd(H_t, H_d, W, K: int, w_topk: float = 1.0, grad_loss
                                           _p(out["loss_ce"]), _p(out["loss"]), _p(out["topk_idx"]), _p(out["topk_q"]),
                                           _p(out["lse_t"]), _p(out["lse_d"]), _p(out["dH_d"]), dH_dtype, _p(ws),
                                           ws.numel(), _stream(stream)), "hass_combined_distill_fwd_bwd")
+    return out
+
+
+LOSS_TOPK, LOSS_TOP_P, LOSS_NORMED_TOPK = 0, 1, 2
+
+
+def variant_distill_fwd_bwd(H_t, H_d, W, K: int, variant: int, param: float = 0.0, grad_loss=None,
+                            dH_dtype: int = HASS_BF16, workspace=None, stream=None) -> dict:
+    """Top-P / Normed Top-K / Top-K loss, forward and backward. See hass_variant_distill_fwd_bwd."""
+    N, d, V = _dims(H_t, W)
+    assert H_d.shape == H_t.shape and H_d.dtype == torch.bfloat16 and H_d.is_contiguous()
+    assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
+    dev = H_t.device
+    ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
+               topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
+               topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+               topk_n=torch.empty(N, dtype=torch.int32, device=dev),
+               lse_t=torch.empty(N, dtype=torch.float32, device=dev),
+               lse_d=torch.zeros(N, dtype=torch.float32, device=dev),
+               dH_d=torch.empty(N, d, dtype=_dh_dtype(dH_dtype), device=dev), workspace=ws)
+    _ok(lib.hass_variant_distill_fwd_bwd(_p(H_t), _p(H_d), _p(W), N, d, V, K, int(variant), ctypes.c_float(param),
+                                         _p(grad_loss), _p(out["loss"]), _p(out["topk_idx"]), _p(out["topk_q"]),
+                                         _p(out["topk_n"]), _p(out["lse_t"]), _p(out["lse_d"]), _p(out["dH_d"]),
+                                         dH_dtype, _p(ws), ws.numel(), _stream(stream)), "hass_variant_distill_fwd_bwd")
     return out
 
 

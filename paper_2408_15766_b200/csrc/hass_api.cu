@@ -507,7 +507,8 @@ struct Combined {
 static int fused_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
                       long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
                       int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
-                      void* workspace, size_t workspace_bytes, cudaStream_t st, const Combined* cmb = nullptr) {
+                      void* workspace, size_t workspace_bytes, cudaStream_t st, const Combined* cmb = nullptr,
+                      float top_p = 0.f, int* topk_n = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
@@ -612,6 +613,8 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.coef_out = coef;
         f.gq_out = gq;
         f.sparse_out = sparse;
+        f.top_p = top_p;
+        f.n_out = topk_n;
         f.w_topk = cmb ? cmb->w : 1.f;
         f.coef_t_out = cmb ? cmb->coef_t : nullptr;
         f.Pt = cmb ? cmb->Pt : nullptr;
@@ -683,6 +686,92 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         if (rc != HASS_OK) return rc;
     }
     return HASS_OK;
+}
+
+// ---- Normed Top-K variant -----------------------------------------------------------------------------
+// Both distributions are renormalised over Omega_hat, so the loss and its gradient involve the draft
+// logits on Omega_hat only: one sweep over the TARGET rows (statistics + Top-K), then finalize computes the
+// K draft logits per row, the loss and the gradient row directly. No draft sweep, no second GEMM.
+static int normed_impl(const void* H_t, const void* H_d, const void* W, long long N, long long d, long long V, int K,
+                       const float* grad_loss, float* loss, int* idx_out, float* q_out, int* topk_n, float* lse_t,
+                       void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_t || !H_d || !W || !loss || !idx_out || !q_out || !lse_t || !dH_d) return HASS_ERR_INVALID_ARG;
+    if (!aligned16(H_t) || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d)) return HASS_ERR_INVALID_ARG;
+    if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.fwd_end) return HASS_ERR_WORKSPACE;
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    rc = plan_schedule(RT, CT, di.sms, &p.sched);
+    if (rc != HASS_OK) return rc;
+    if (p.sched.total_slots > L.slot_cap) return HASS_ERR_WORKSPACE;
+    log_schedule("normed stats (target)", p.sched);
+    rc = make_tmap(&p.tmA0, H_t, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = make_tmap(&p.tmA1, H_t, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = make_tmap(&p.tmB, W, V, d, d, BK, BN);
+    if (rc != HASS_OK) return rc;
+    p.row_tiles0 = RT;
+    p.topk_row_tiles = RT;
+    p.spill_begin = INT_MAX;
+    p.rows_valid = static_cast<int>(N);
+    p.n_cols = static_cast<int>(V);
+    p.col_tiles = CT;
+    p.k_blocks = ceil_div(d, BK);
+    p.K = K;
+    p.cap = topk_cap(K);
+    p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+    p.part_s = reinterpret_cast<float*>(ws + L.part_s);
+    p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
+    p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
+    p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    rc = launch_gemm<MODE_STATS>(p, st);
+    if (rc != HASS_OK) return rc;
+    FinalizeParams f;
+    std::memset(&f, 0, sizeof(f));
+    f.sched = p.sched;
+    f.d = static_cast<int>(d);
+    f.K = K;
+    f.cap = p.cap;
+    f.row_begin = 0;
+    f.rows = static_cast<int>(N);
+    f.row_tiles_t = RT;
+    f.part_m = p.part_m;
+    f.part_s = p.part_s;
+    f.cand = p.cand;
+    f.cand_n = p.cand_n;
+    f.H_d = static_cast<const __nv_bfloat16*>(H_d);
+    f.W = static_cast<const __nv_bfloat16*>(W);
+    f.loss = loss;
+    f.idx_out = idx_out;
+    f.q_out = q_out;
+    f.lse_t = lse_t;
+    f.grad_loss = grad_loss;
+    f.n_out = topk_n;
+    f.normed = 1;
+    f.dH_out = dH_d;
+    f.dH_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+    {
+        KernelTimer timer(KIND_FINALIZE, st);
+        finalize_kernel<<<ceil_div(N, 8), 256, 0, st>>>(f);
+    }
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
 }
 
 }  // namespace hass
@@ -794,6 +883,28 @@ int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, i
                                     void* cuda_stream) {
     return fused_impl(false, nullptr, H_d, W, N, d, V, K, grad_loss, topk_idx, topk_q, loss, nullptr, nullptr, nullptr,
                       lse_d, dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
+                                 int32_t K, int variant, float param, const float* grad_loss, float* loss,
+                                 int32_t* topk_idx, float* topk_q, int32_t* topk_n, float* lse_t, float* lse_d,
+                                 void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    switch (variant) {
+        case HASS_LOSS_TOPK:
+            return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
+                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, 0.f, topk_n);
+        case HASS_LOSS_TOP_P:
+            if (!(param > 0.f)) return HASS_ERR_INVALID_ARG;
+            return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
+                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, param, topk_n);
+        case HASS_LOSS_NORMED_TOPK:
+            return normed_impl(H_t, H_d, W, N, d, V, K, grad_loss, loss, topk_idx, topk_q, topk_n, lse_t, dH_d, dH_dtype,
+                               workspace, workspace_bytes, st);
+        default:
+            return HASS_ERR_INVALID_ARG;
+    }
 }
 
 // Buffers appended to the normal workspace by the combined-objective entry.

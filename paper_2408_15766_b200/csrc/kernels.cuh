@@ -708,6 +708,13 @@ struct FinalizeParams {
     long long p_pitch;
     float* ce_corr_out;    // [N] sum_{x in Omega_hat} (q(x) - bf16 q(x)) z_d(x): the cross-entropy is formed from
                            // the bf16 spill; its largest terms are put back in fp32
+    // loss variants of Section 4.3
+    float top_p;           // > 0: Omega_hat is cut to the shortest sorted prefix with cumulative q > top_p (Top-P)
+    int* n_out;            // [N] |Omega_hat| (nullable)
+    int normed;            // 1: Normed Top-K - q, p renormalised over Omega_hat; no draft sweep exists, and the
+                           // gradient row sum_x g (pn(x) - qn(x)) W[x,:] goes straight to dH_out
+    void* dH_out;          // [N, d] (normed only)
+    int dH_fp32;
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -749,11 +756,14 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     const int K = p.K;
     int slot0, S;
 
-    // draft statistics
-    find_slots(p.sched, p.row_tiles_t + rt, slot0, S);
-    const float lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
-    if (lane == 0) p.lse_d[row] = lse_d;
-    const float m_spill = p.part_m[static_cast<long long>(slot0) * BM + r];
+    // draft statistics (the Normed Top-K variant has none: it needs the draft logits on Omega_hat only)
+    float lse_d = 0.f, m_spill = 0.f;
+    if (!p.normed) {
+        find_slots(p.sched, p.row_tiles_t + rt, slot0, S);
+        lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
+        if (lane == 0) p.lse_d[row] = lse_d;
+        m_spill = p.part_m[static_cast<long long>(slot0) * BM + r];
+    }
     const float g = p.grad_loss ? p.grad_loss[row] : 1.f;
     float S_q = 0.f;
 
@@ -778,6 +788,9 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     const int cap = p.cap;
     __shared__ int sh_tok[8][K_CAP];
     __shared__ float sh_q[8][K_CAP];
+    __shared__ float sh_dot[8][K_CAP];
+    float cum_q = 0.f;
+    int n_sel = 0;
     const int wib = threadIdx.x >> 5;
     for (int j = 0; j < K; ++j) {
         int tok;
@@ -815,8 +828,22 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             prev_i = bi;
             tok = bi == INT_MAX ? 0 : bi;     // cannot happen for K <= V; keeps the gather in range
             qv = expf(bv - lse_t);
+            int tok_out = tok;
+            if (p.top_p > 0.f) {
+                // Top-P: a token belongs to Omega_hat while the probability of those before it is <= P
+                if (cum_q > p.top_p) {
+                    tok_out = -1;
+                    tok = 0;
+                    qv = 0.f;
+                } else {
+                    ++n_sel;
+                }
+                cum_q += qv;
+            } else {
+                ++n_sel;
+            }
             if (lane == 0) {
-                p.idx_out[static_cast<long long>(row) * K + j] = tok;
+                p.idx_out[static_cast<long long>(row) * K + j] = tok_out;
                 p.q_out[static_cast<long long>(row) * K + j] = qv;
             }
         } else {
@@ -834,7 +861,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     // Draft logits at Omega_hat (K dot products with rows of W) and, for the fused backward, the row
     // sum_{x in Omega_hat} g q(x) W[x, :]. The W rows are read once: FIN_GRP tokens at a time, 256 columns
     // (8 per lane) per step; the fp32 row is accumulated across token groups.
-    float* so = p.sparse_out ? p.sparse_out + static_cast<long long>(local) * p.d : nullptr;
+    float* so = (p.sparse_out && !p.normed) ? p.sparse_out + static_cast<long long>(local) * p.d : nullptr;
     for (int g0 = 0; g0 < K; g0 += FIN_GRP) {
         const int ng = K - g0 < FIN_GRP ? K - g0 : FIN_GRP;
         float dot[FIN_GRP];
@@ -885,11 +912,63 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
             if (jj < ng) {
                 const float qv = sh_q[wib][g0 + jj];
+                if (lane == 0) sh_dot[wib][g0 + jj] = acc;
                 loss += qv * (lse_d - acc);     // -q log p,  log p = z_d - lse_d
                 if (combined) {
                     const float q_spill = __bfloat162float(p.Pt[static_cast<long long>(local) * p.p_pitch + sh_tok[wib][g0 + jj]]) * coef_t;
                     ce_corr += (qv - q_spill) * acc;
                 }
+            }
+        }
+    }
+    if (lane == 0 && p.n_out) p.n_out[row] = n_sel;
+    if (p.normed) {
+        // Normed Top-K: qn = q / S_q, pn = softmax of the draft logits restricted to Omega_hat
+        __syncwarp();
+        float mx = -INFINITY;
+        for (int j = lane; j < K; j += 32) mx = fmaxf(mx, sh_dot[wib][j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int j = lane; j < K; j += 32) se += expf(sh_dot[wib][j] - mx);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float lse_k = mx + logf(se);
+        float ln = 0.f;
+        for (int j = lane; j < K; j += 32) {
+            const float qn = sh_q[wib][j] / S_q;
+            const float zj = sh_dot[wib][j];
+            ln += qn * (lse_k - zj);
+            sh_dot[wib][j] = g * (expf(zj - lse_k) - qn);      // dL/dz_d on Omega_hat
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ln += __shfl_xor_sync(0xffffffffu, ln, o);
+        loss = ln;
+        __syncwarp();
+        for (int k0 = lane * 8; k0 < p.d; k0 += 256) {
+            float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < K; ++j) {
+                const float c = sh_dot[wib][j];
+                const uint4 wv = *reinterpret_cast<const uint4*>(p.W + static_cast<long long>(sh_tok[wib][j]) * p.d + k0);
+                const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float2 b = __bfloat1622float2(wp[t]);
+                    a[2 * t] = fmaf(c, b.x, a[2 * t]);
+                    a[2 * t + 1] = fmaf(c, b.y, a[2 * t + 1]);
+                }
+            }
+            if (p.dH_fp32) {
+                float* o = reinterpret_cast<float*>(p.dH_out) + static_cast<long long>(row) * p.d + k0;
+                *reinterpret_cast<float4*>(o) = make_float4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<float4*>(o + 4) = make_float4(a[4], a[5], a[6], a[7]);
+            } else {
+                uint4 w;
+                w.x = pack_bf16x2(a[0], a[1]);
+                w.y = pack_bf16x2(a[2], a[3]);
+                w.z = pack_bf16x2(a[4], a[5]);
+                w.w = pack_bf16x2(a[6], a[7]);
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dH_out) + static_cast<long long>(row) * p.d + k0) = w;
             }
         }
     }

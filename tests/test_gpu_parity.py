@@ -273,3 +273,60 @@ def test_combined_objective_l2_7b_sampled_rows():
     err = np.abs(cpu["dH_d"].float().numpy()[rows].astype(np.float64) - ref["dH_d"]).max()
     print("l2-7b combined: loss_ce rel", float((np.abs(ce - ref["loss_ce"]) / np.abs(ref["loss_ce"])).max()), "dH rel", err / scale)
     assert err <= 1e-2 * scale
+
+
+@pytest.mark.parametrize("N,d,V,K", [(64, 256, 1024, 10), (300, 128, 5000, 24), (4800, 64, 700, 8)])
+def test_normed_top_k_variant_matches_oracle(N, d, V, K):
+    import oracle
+    hass = _hass()
+    inp = hi.make_custom(N, d, V, K, seed=N + K + 1, sigma_w=2.0 / np.sqrt(d))
+    dev = torch.device("cuda:0")
+    grad = np.random.default_rng(2).uniform(-1.0, 2.0, size=N)
+    out = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), K, hass.LOSS_NORMED_TOPK,
+                                       grad_loss=torch.tensor(grad, dtype=torch.float32, device=dev),
+                                       dH_dtype=hass.HASS_FP32)
+    hass.check(out["workspace"])
+    cpu = _to_cpu(out)
+    ref = oracle.variant_from_features(hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W), K,
+                                       oracle.VARIANT_NORMED, grad_loss=grad)
+    same = (np.sort(cpu["topk_idx"].numpy(), 1) == np.sort(ref["idx"], 1)).all(1)      # rows without a near-tie at rank K
+    assert same.mean() > 0.97
+    assert np.all(cpu["topk_n"].numpy() == K)
+    np.testing.assert_allclose(cpu["lse_t"].numpy(), ref["lse_t"], atol=1e-4)
+    l, lr = cpu["loss"].numpy()[same], ref["loss"][same]
+    assert np.all(np.abs(l - lr) <= 2e-3 * np.maximum(np.abs(lr), 1e-6))
+    scale = np.abs(ref["dH_d"]).max()
+    err = np.abs(cpu["dH_d"].numpy()[same].astype(np.float64) - ref["dH_d"][same]).max()
+    print("normed: loss rel", float((np.abs(l - lr) / np.maximum(np.abs(lr), 1e-6)).max()), "dH rel", err / scale)
+    assert err <= 1e-2 * scale
+
+
+@pytest.mark.parametrize("N,d,V,K,P", [(64, 256, 1024, 10, 0.01), (300, 128, 5000, 24, 0.3), (4800, 64, 700, 16, 0.5)])
+def test_top_p_variant_matches_oracle(N, d, V, K, P):
+    import oracle
+    hass = _hass()
+    inp = hi.make_custom(N, d, V, K, seed=N + K + 2, sigma_w=2.0 / np.sqrt(d))
+    dev = torch.device("cuda:0")
+    out = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev), K, hass.LOSS_TOP_P, P,
+                                       dH_dtype=hass.HASS_FP32)
+    hass.check(out["workspace"])
+    cpu = _to_cpu(out)
+    ref = oracle.variant_from_features(hi.bf16_bits(inp.H_t), hi.bf16_bits(inp.H_d[0]), hi.bf16_bits(inp.W), K,
+                                       oracle.VARIANT_TOP_P, P)
+    n_gpu, n_ref = cpu["topk_n"].numpy(), ref["n"]
+    assert n_gpu.min() >= 1 and n_gpu.max() <= K and len(np.unique(n_ref)) > 1
+    # the prefix length is decided by comparing a running sum with P: rows whose sum comes within 1e-5 of P
+    # at the cut may legitimately stop one token earlier or later in fp32
+    cum = np.cumsum(ref["q_k"], 1)
+    near = np.abs(cum - P).min(1) < 1e-5
+    ok = (n_gpu == n_ref) & (np.sort(np.where(cpu["topk_idx"].numpy() < 0, 1 << 30, cpu["topk_idx"].numpy()), 1)
+                             == np.sort(np.where(ref["idx"] < 0, 1 << 30, ref["idx"]), 1)).all(1)
+    assert np.all(ok | near) and ok.mean() > 0.97
+    idx = cpu["topk_idx"].numpy()
+    assert np.all((idx >= 0) == (np.arange(K)[None, :] < n_gpu[:, None]))
+    l, lr = cpu["loss"].numpy()[ok], ref["loss"][ok]
+    assert np.all(np.abs(l - lr) <= 2e-3 * np.maximum(np.abs(lr), 1e-6))
+    scale = np.abs(ref["dH_d"]).max()
+    err = np.abs(cpu["dH_d"].numpy()[ok].astype(np.float64) - ref["dH_d"][ok]).max()
+    print("top-p: mean n", n_gpu.mean(), "loss rel", float((np.abs(l - lr) / np.maximum(np.abs(lr), 1e-6)).max()), "dH rel", err / scale)
+    assert err <= 1e-2 * scale
