@@ -301,7 +301,7 @@ def test_normed_top_k_variant_matches_oracle(N, d, V, K):
     assert err <= 1e-2 * scale
 
 
-@pytest.mark.parametrize("N,d,V,K,P", [(64, 256, 1024, 10, 0.01), (300, 128, 5000, 24, 0.3), (4800, 64, 700, 16, 0.5)])
+@pytest.mark.parametrize("N,d,V,K,P", [(64, 256, 1024, 10, 0.2), (300, 128, 5000, 24, 0.3), (4800, 64, 700, 16, 0.5)])
 def test_top_p_variant_matches_oracle(N, d, V, K, P):
     import oracle
     hass = _hass()
