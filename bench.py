@@ -190,9 +190,10 @@ def main():
     ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--K", type=int, default=None)
-    ap.add_argument("--objective", default="topk", choices=["topk", "combined"],
+    ap.add_argument("--objective", default="topk", choices=["topk", "combined", "top_p", "normed"],
                     help="topk: Eq. 1 alone (the headline metric); combined: cross-entropy over the vocabulary "
-                         "+ w * Top-K in one call (8 N d V tensor FLOPs)")
+                         "+ w * Top-K in one call (8 N d V tensor FLOPs); top_p (P = 0.5, at most K tokens) and "
+                         "normed (Normed Top-K: only the target product, 2 N d V) are the loss variants of Section 4.3")
     ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -243,6 +244,10 @@ def main():
         if combined:
             counts["full"] += 1
             hass.combined_distill_fwd_bwd(H_t, H_d_steps[j], W, K, w_topk=1.0, workspace=ws, out=out, stream=stream)
+        elif args.objective in ("top_p", "normed"):
+            counts["full"] += 1
+            hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, hass.LOSS_TOP_P if args.objective == "top_p"
+                                         else hass.LOSS_NORMED_TOPK, 0.5, workspace=ws, stream=stream)
         elif j == 0:
             counts["full"] += 1
             hass.topk_distill_fwd_bwd(H_t, H_d_steps[0], W, K, workspace=ws, out=out, stream=stream)
@@ -281,7 +286,7 @@ def main():
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
-    if not args.no_e2e and not combined:
+    if not args.no_e2e and args.objective == "topk":
         Ht_h, Hd_h = inp.H_t.pin_memory(), inp.H_d[0].pin_memory()
         loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
         dH_h = torch.empty(N, d, dtype=torch.bfloat16).pin_memory()
@@ -306,9 +311,11 @@ def main():
 
     # ---- roofline of the dominant kernel (tensor-core bound) ----
     # three d x V products per token (z_t, z_d, dH_d); the combined objective needs a fourth (q W)
-    flops_credit = (8.0 if combined else 6.0) * N * d * V
+    normed = args.objective == "normed"
+    flops_credit = (8.0 if combined else 2.0 if normed else 6.0) * N * d * V
     # executed tensor work per step, averaged over the timed steps (a draft-only step skips the target product)
-    kinds = {"stats_gemm": (4.0 * n_full + 2.0 * n_draft) / args.steps * N * d * V, "dz_gemm": 2.0 * N * d * V,
+    kinds = {"stats_gemm": (2.0 * n_full if normed else 4.0 * n_full + 2.0 * n_draft) / args.steps * N * d * V,
+             "dz_gemm": 2.0 * N * d * V,
              "dH_gemm": (4.0 if combined else 2.0) * N * d * V}
     total_ms = sum(v[0] for v in prof.values())
     kernel_rows = {}
@@ -326,7 +333,7 @@ def main():
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak,
                 "traffic": (TRAFFIC_CAPTURE["bytes_per_launch"]
-                            if dom == "stats_gemm" and not combined and wl.name == TRAFFIC_CAPTURE["workload"]
+                            if dom == "stats_gemm" and args.objective == "topk" and wl.name == TRAFFIC_CAPTURE["workload"]
                             and hass.version() == TRAFFIC_CAPTURE["version"] else None),
                 "peak_kind": f"bf16_tflops_sustained, of {peak_kind} (kernel timed inside a long step)",
                 "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
@@ -342,8 +349,9 @@ def main():
                        "dH_dtype": "bf16", "aligning_steps": wl.steps, "objective": args.objective,
                        "target_stats": ("recomputed every step" if wl.steps == 1 else
                                         "computed in aligning step 1, reused in steps 2..%d" % wl.steps),
-                       "path": ("hass_combined_distill_fwd_bwd" if combined else
-                                "hass_topk_distill_fwd_bwd (no logit recompute)")},
+                       "path": {"combined": "hass_combined_distill_fwd_bwd", "top_p": "hass_variant_distill_fwd_bwd (Top-P)",
+                                "normed": "hass_variant_distill_fwd_bwd (Normed Top-K)",
+                                "topk": "hass_topk_distill_fwd_bwd (no logit recompute)"}[args.objective]},
             "clocks": clocks, "gpu_launches": launches,
             "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
                        "executed_tflops": executed / (ms_step * 1e-3) / 1e12, "executed_flops_per_step": executed,
