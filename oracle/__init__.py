@@ -96,7 +96,7 @@ def from_logits(z_t, z_d, K: int, g: float = 1.0, forced_idx=None, want_dz: bool
     return dict(loss=float(loss[0]), idx=idx, q_k=q_k, lse_t=float(lse_t[0]), lse_d=float(lse_d[0]), dz_d=dz)
 
 
-VARIANT_TOPK, VARIANT_TOP_P, VARIANT_NORMED = 0, 1, 2
+VARIANT_TOPK, VARIANT_TOP_P, VARIANT_NORMED, VARIANT_BIDIR = 0, 1, 2, 3
 
 
 def variant_from_logits(z_t, z_d, K: int, variant: int, param: float = 0.0, g: float = 1.0) -> dict:
@@ -105,8 +105,9 @@ def variant_from_logits(z_t, z_d, K: int, variant: int, param: float = 0.0, g: f
     z_d = np.ascontiguousarray(z_d, dtype=np.float64)
     V = z_t.shape[0]
     loss, lse_t, lse_d = np.zeros(1), np.zeros(1), np.zeros(1)
-    idx = np.zeros(K, dtype=np.int32)
-    q_k = np.zeros(K)
+    kk = 2 * K if variant == VARIANT_BIDIR else K
+    idx = np.zeros(kk, dtype=np.int32)
+    q_k = np.zeros(kk)
     n = np.zeros(1, dtype=np.int32)
     dz = np.zeros(V)
     rc = _load().hass_oracle_row_variant(_ptr(z_t), _ptr(z_d), V, K, float(g), int(variant), float(param), _ptr(loss),
@@ -127,8 +128,9 @@ def variant_from_features(H_t, H_d, W, K: int, variant: int, param: float = 0.0,
     n = rows_a.shape[0]
     gl = None if grad_loss is None else np.ascontiguousarray(grad_loss, dtype=np.float64)
     loss, lse_t, lse_d = np.zeros(n), np.zeros(n), np.zeros(n)
-    idx = np.zeros((n, K), dtype=np.int32)
-    q_k = np.zeros((n, K))
+    kk = 2 * K if variant == VARIANT_BIDIR else K
+    idx = np.zeros((n, kk), dtype=np.int32)
+    q_k = np.zeros((n, kk))
     cnt = np.zeros(n, dtype=np.int32)
     dH = np.zeros((n, d))
     rc = _load().hass_oracle_features_variant(_ptr(H_t), _ptr(H_d), _ptr(W), N, d, V, K, int(variant), float(param),

@@ -41,6 +41,11 @@
  *                    probabilities, which equals a softmax over the logits restricted to Omega_hat):
  *                    L = - sum_{x in Omega_hat} qn(x) log pn(x), qn = q / S_q, pn = p / S_p;
  *                    dL/dz_d[x] = g (pn(x) - qn(x)) on Omega_hat and 0 elsewhere.
+ *   3  Bi-directional Top-K: Omega_hat = (K most probable tokens under q) united with (K most probable
+ *                    under p); loss and gradient as Eq. 1 on that set, the set being a constant:
+ *                    L = - sum_{x in U} q(x) log p(x), dL/dz_d[v] = g (S_U p[v] - q[v] [v in U]).
+ *                    idx / q_k then hold up to 2K entries: the target's K in descending q, followed by the
+ *                    draft's tokens that are not among them in descending p.
  *
  * Inputs of the feature-level entry are bf16 bit patterns widened exactly to fp64.
  * The only liberty taken with summation order is SIMD reassociation of the inner
@@ -205,7 +210,48 @@ int hass_oracle_row_objective(const double* z_t, const double* z_d, int64_t V, i
 int hass_oracle_row_variant(const double* z_t, const double* z_d, int64_t V, int32_t K, double g, int variant,
                             double param, double* loss, int32_t* idx, double* q_k, int32_t* n_out,
                             double* lse_t_out, double* lse_d_out, double* dz_d) {
-    if (variant < 0 || variant > 2) return -1;
+    if (variant < 0 || variant > 3) return -1;
+    if (variant == 3) {
+        /* union of the two Top-K sets; idx and q_k have room for 2K entries */
+        double l0, lt, ld;
+        int32_t* it = (int32_t*)malloc(sizeof(int32_t) * (size_t)K * 2);
+        double* qt = (double*)malloc(sizeof(double) * (size_t)K * 2);
+        int rc3 = hass_oracle_row_objective(z_t, z_d, V, K, g, 0.0, 1.0, NULL, NULL, &l0, it, qt, &lt, &ld, NULL);
+        if (rc3 == 0) /* the draft's own Top-K: the same selection with the roles of the logits exchanged */
+            rc3 = hass_oracle_row_objective(z_d, z_d, V, K, g, 0.0, 1.0, NULL, NULL, &l0, it + K, qt + K, NULL, NULL, NULL);
+        if (rc3 != 0) {
+            free(it);
+            free(qt);
+            return rc3;
+        }
+        int32_t n = 0;
+        double S_U = 0.0, L = 0.0;
+        for (int32_t j = 0; j < 2 * K; ++j) {
+            int dup = 0;
+            for (int32_t i = 0; i < n; ++i) dup |= (idx[i] == it[j]);
+            if (dup) continue;
+            idx[n] = it[j];
+            q_k[n] = exp(z_t[it[j]] - lt);
+            S_U += q_k[n];
+            L -= q_k[n] * (z_d[it[j]] - ld);
+            ++n;
+        }
+        for (int32_t j = n; j < 2 * K; ++j) {
+            idx[j] = -1;
+            q_k[j] = 0.0;
+        }
+        *loss = L;
+        if (lse_t_out) *lse_t_out = lt;
+        if (lse_d_out) *lse_d_out = ld;
+        if (dz_d) {
+            for (int64_t v = 0; v < V; ++v) dz_d[v] = g * S_U * exp(z_d[v] - ld);
+            for (int32_t j = 0; j < n; ++j) dz_d[idx[j]] -= g * q_k[j];
+        }
+        if (n_out) *n_out = n;
+        free(it);
+        free(qt);
+        return 0;
+    }
     int rc = hass_oracle_row_objective(z_t, z_d, V, K, g, 0.0, 1.0, NULL, NULL, loss, idx, q_k, lse_t_out, lse_d_out,
                                        variant == 0 ? dz_d : NULL);
     if (rc != 0) return rc;
@@ -290,7 +336,8 @@ int hass_oracle_features_variant(const uint16_t* H_t, const uint16_t* H_d, const
                 widen_bf16(W + v * d, wr, d);
                 dot2(ht, hd, wr, d, &zt[v], &zd[v]);
             }
-            if (hass_oracle_row_variant(zt, zd, V, K, g, variant, param, &loss[r], idx + r * K, q_k + r * K, &n_out[r],
+            const int64_t kk = variant == 3 ? 2 * (int64_t)K : K;   /* entries per row of idx / q_k */
+            if (hass_oracle_row_variant(zt, zd, V, K, g, variant, param, &loss[r], idx + r * kk, q_k + r * kk, &n_out[r],
                                         &lse_t[r], &lse_d[r], dz) != 0) {
 #pragma omp atomic write
                 status = -1;

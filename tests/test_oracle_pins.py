@@ -405,3 +405,38 @@ def test_variants_at_features_level_match_the_row_entry():
             np.testing.assert_allclose(f["dH_d"][i], r["dz_d"] @ Wd, atol=1e-13)
     plain = oracle.from_features(Ht, Hd, W, K, grad_loss=g)
     np.testing.assert_allclose(oracle.variant_from_features(Ht, Hd, W, K, 0, grad_loss=g)["dH_d"], plain["dH_d"], atol=1e-15)
+
+
+def test_bidirectional_top_k_is_eq1_on_the_union_of_both_top_k_sets():
+    V, K = 64, 5
+    z_t, z_d = _rand_logits(V, seed=47, scale=1.5)
+    r = oracle.variant_from_logits(z_t, z_d, K, oracle.VARIANT_BIDIR, g=0.7)
+    zd = torch.tensor(z_d, requires_grad=True)
+    q = torch.softmax(torch.tensor(z_t), 0)
+    logp = torch.log_softmax(zd, 0)
+    top_t = torch.topk(q, K).indices.tolist()
+    top_d = torch.topk(logp.detach(), K).indices.tolist()
+    union = top_t + [x for x in top_d if x not in top_t]
+    loss = -(q[union] * logp[union]).sum()
+    (0.7 * loss).backward()
+    assert r["n"] == len(union) and list(r["idx"][:r["n"]]) == union and np.all(r["idx"][r["n"]:] == -1)
+    assert K < r["n"] <= 2 * K                      # this seed has draft tokens outside the target's set
+    assert r["loss"] == pytest.approx(float(loss), rel=1e-12)
+    np.testing.assert_allclose(r["dz_d"], zd.grad.numpy(), atol=1e-15)
+    # identical logits: the two sets coincide and the variant is Eq. 1
+    same = oracle.variant_from_logits(z_t, z_t, K, oracle.VARIANT_BIDIR)
+    base = oracle.from_logits(z_t, z_t, K)
+    assert same["n"] == K and same["loss"] == pytest.approx(base["loss"], rel=1e-13)
+    np.testing.assert_allclose(same["dz_d"], base["dz_d"], atol=1e-16)
+    # K = V: every token, plain cross-entropy
+    allv = oracle.variant_from_logits(z_t, z_d, V, oracle.VARIANT_BIDIR)
+    assert allv["n"] == V and allv["loss"] == pytest.approx(float(-(q * torch.log_softmax(torch.tensor(z_d), 0)).sum()), rel=1e-12)
+    # feature level agrees with the row entry
+    Ht, Hd, W, _ = _feat(3, 16, 50, seed=49, sigma_w=0.3)
+    f = oracle.variant_from_features(Ht, Hd, W, 4, oracle.VARIANT_BIDIR)
+    zt, zdd = _z(Ht, W), _z(Hd, W)
+    Wd = torch.from_numpy(W.view(np.int16).copy()).view(torch.bfloat16).double().numpy()
+    for i in range(3):
+        ri = oracle.variant_from_logits(zt[i], zdd[i], 4, oracle.VARIANT_BIDIR)
+        assert f["n"][i] == ri["n"] and np.array_equal(f["idx"][i], ri["idx"]) and f["loss"][i] == pytest.approx(ri["loss"], rel=1e-12)
+        np.testing.assert_allclose(f["dH_d"][i], ri["dz_d"] @ Wd, atol=1e-13)
