@@ -191,11 +191,21 @@ int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* 
  *                          L = - sum qn log pn, qn = q / S_q, pn = p / S_p (a softmax of the draft
  *                          logits restricted to Omega_hat), dz_d = g (pn - qn) on Omega_hat, 0 elsewhere.
  *                          Only the target rows are swept; lse_d is not written (may be NULL).
+ *   HASS_LOSS_BIDIR_TOPK   Omega_hat = the K most probable tokens under q united with the K most probable
+ *                          under p (taken as a constant set); loss and gradient as Eq. 1 on the union.
+ *                          topk_idx / topk_q must hold 2K entries per row: the target's K in descending q,
+ *                          then the draft's tokens not among them in descending p, then -1 / 0. K <= 64.
  *
  * topk_n [N] (nullable) receives |Omega_hat| per row. The other arguments are those of
- * hass_topk_distill_fwd_bwd. The Bi-directional, Recall@k and BiLD losses of that section are not built.
+ * hass_topk_distill_fwd_bwd. The Recall@k surrogate and BiLD losses of that section are not built (the
+ * paper does not define them).
  */
-typedef enum { HASS_LOSS_TOPK = 0, HASS_LOSS_TOP_P = 1, HASS_LOSS_NORMED_TOPK = 2 } hass_loss_variant;
+typedef enum {
+    HASS_LOSS_TOPK = 0,
+    HASS_LOSS_TOP_P = 1,
+    HASS_LOSS_NORMED_TOPK = 2,
+    HASS_LOSS_BIDIR_TOPK = 3
+} hass_loss_variant;
 int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                                  int64_t V, int32_t K, int variant, float param, const float* grad_loss,
                                  float* loss, int32_t* topk_idx, float* topk_q, int32_t* topk_n,

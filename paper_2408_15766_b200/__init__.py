@@ -33,4 +33,5 @@ from .binding import (  # noqa: F401
     LOSS_TOPK,
     LOSS_TOP_P,
     LOSS_NORMED_TOPK,
+    LOSS_BIDIR_TOPK,
 )

@@ -266,7 +266,7 @@ def combined_distill_fwd_bwd(H_t, H_d, W, K: int, w_topk: float = 1.0, grad_loss
     return out
 
 
-LOSS_TOPK, LOSS_TOP_P, LOSS_NORMED_TOPK = 0, 1, 2
+LOSS_TOPK, LOSS_TOP_P, LOSS_NORMED_TOPK, LOSS_BIDIR_TOPK = 0, 1, 2, 3
 
 
 def variant_distill_fwd_bwd(H_t, H_d, W, K: int, variant: int, param: float = 0.0, grad_loss=None,
@@ -277,9 +277,10 @@ def variant_distill_fwd_bwd(H_t, H_d, W, K: int, variant: int, param: float = 0.
     assert grad_loss is None or (grad_loss.dtype == torch.float32 and grad_loss.shape == (N,))
     dev = H_t.device
     ws = _workspace(workspace, topk_distill_workspace_bytes(N, d, V, K), dev)
+    kk = 2 * K if variant == LOSS_BIDIR_TOPK else K      # the bi-directional set holds up to 2K tokens
     out = dict(loss=torch.empty(N, dtype=torch.float32, device=dev),
-               topk_idx=torch.empty(N, K, dtype=torch.int32, device=dev),
-               topk_q=torch.empty(N, K, dtype=torch.float32, device=dev),
+               topk_idx=torch.empty(N, kk, dtype=torch.int32, device=dev),
+               topk_q=torch.empty(N, kk, dtype=torch.float32, device=dev),
                topk_n=torch.empty(N, dtype=torch.int32, device=dev),
                lse_t=torch.empty(N, dtype=torch.float32, device=dev),
                lse_d=torch.zeros(N, dtype=torch.float32, device=dev),

@@ -508,7 +508,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
                       long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
                       int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
                       void* workspace, size_t workspace_bytes, cudaStream_t st, const Combined* cmb = nullptr,
-                      float top_p = 0.f, int* topk_n = nullptr) {
+                      float top_p = 0.f, int* topk_n = nullptr, bool bidir = false) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
@@ -516,6 +516,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     if (with_target && (!H_t || !idx_out || !q_out || !lse_t || !aligned16(H_t))) return HASS_ERR_INVALID_ARG;
     if (!with_target && (!idx_in || !q_in)) return HASS_ERR_INVALID_ARG;
     if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (bidir && (!with_target || 2 * K > K_CAP)) return HASS_ERR_UNSUPPORTED;   // the union holds up to 2K tokens
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
     DeviceInfo di;
     rc = device_info(&di);
@@ -531,7 +532,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     int chunk_tiles = L.pref_chunk_tiles;
     if (fit < chunk_tiles) chunk_tiles = static_cast<int>(fit);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    float* gq = reinterpret_cast<float*>(ws + L.sgq);
+    float* gq = bidir ? nullptr : reinterpret_cast<float*>(ws + L.sgq);    // [N, K]: too small for the 2K-token union
     float* coef = reinterpret_cast<float*>(ws + L.coef);
     float* sparse = reinterpret_cast<float*>(ws + L.sparse);
     __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(ws + L.scratch);
@@ -566,7 +567,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.tmA1 = tmHd;
         p.tmB = tmWk;
         p.row_tiles0 = tiles;
-        p.topk_row_tiles = with_target ? tiles : 0;
+        p.topk_row_tiles = with_target ? (bidir ? 2 * tiles : tiles) : 0;
         p.spill_begin = with_target ? tiles : 0;
         p.a_row_offset = t0 * BM;
         p.row_global_offset = t0 * BM;
@@ -615,6 +616,8 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.sparse_out = sparse;
         f.top_p = top_p;
         f.n_out = topk_n;
+        f.bidir = bidir ? 1 : 0;
+        f.H_t = static_cast<const __nv_bfloat16*>(H_t);
         f.w_topk = cmb ? cmb->w : 1.f;
         f.coef_t_out = cmb ? cmb->coef_t : nullptr;
         f.Pt = cmb ? cmb->Pt : nullptr;
@@ -899,6 +902,9 @@ int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W
             if (!(param > 0.f)) return HASS_ERR_INVALID_ARG;
             return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
                               lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, param, topk_n);
+        case HASS_LOSS_BIDIR_TOPK:
+            return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
+                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, 0.f, topk_n, true);
         case HASS_LOSS_NORMED_TOPK:
             return normed_impl(H_t, H_d, W, N, d, V, K, grad_loss, loss, topk_idx, topk_q, topk_n, lse_t, dH_d, dH_dtype,
                                workspace, workspace_bytes, st);

@@ -715,6 +715,9 @@ struct FinalizeParams {
                            // gradient row sum_x g (pn(x) - qn(x)) W[x,:] goes straight to dH_out
     void* dH_out;          // [N, d] (normed only)
     int dH_fp32;
+    int bidir;             // 1: Bi-directional Top-K - Omega_hat also takes the draft's K most probable tokens (the draft
+                           // rows collected candidates too); idx_out / q_out then have 2K entries per row
+    const __nv_bfloat16* H_t;   // target features (bidir: target logits of the draft's tokens)
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -758,8 +761,11 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
 
     // draft statistics (the Normed Top-K variant has none: it needs the draft logits on Omega_hat only)
     float lse_d = 0.f, m_spill = 0.f;
+    int slot0_d = 0, S_d = 0;
     if (!p.normed) {
         find_slots(p.sched, p.row_tiles_t + rt, slot0, S);
+        slot0_d = slot0;
+        S_d = S;
         lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
         if (lane == 0) p.lse_d[row] = lse_d;
         m_spill = p.part_m[static_cast<long long>(slot0) * BM + r];
@@ -786,44 +792,51 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
     float prev_v = INFINITY;
     int prev_i = -1;
     const int cap = p.cap;
-    __shared__ int sh_tok[8][K_CAP];
+    __shared__ int sh_tok[8][K_CAP];      // Omega_hat of the warp's row (the bi-directional set needs 2K <= K_CAP)
     __shared__ float sh_q[8][K_CAP];
     __shared__ float sh_dot[8][K_CAP];
     float cum_q = 0.f;
     int n_sel = 0;
     const int wib = threadIdx.x >> 5;
+    // next candidate of the slots [sl0, sl0 + nS) after (pv, pi) in the order: logit descending, then token id
+    // ascending (warp-collective; every lane gets the result)
+    auto select_next = [&](int sl0, int nS, float pv, int pi, float& bv, int& bi) {
+        bv = -INFINITY;
+        bi = INT_MAX;
+        for (int sl = 0; sl < nS; ++sl) {
+            const long long so = static_cast<long long>(sl0 + sl) * BM + r;
+            const int n = p.cand_n[so];
+            for (int e = lane; e < n; e += 32) {
+                const uint2 ce = p.cand[so * cap + e];
+                const float v = __uint_as_float(ce.x);
+                const int i = static_cast<int>(ce.y);
+                if (i < 0) continue;
+                const bool after_prev = (v < pv) || (v == pv && i > pi);
+                const bool better = (v > bv) || (v == bv && i < bi);
+                if (after_prev && better) {
+                    bv = v;
+                    bi = i;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+            }
+        }
+    };
+    const int ostride = p.bidir ? 2 * K : K;     // entries per row of idx_out / q_out
     for (int j = 0; j < K; ++j) {
         int tok;
         float qv;
         if (p.row_tiles_t > 0) {
-            // next candidate after (prev_v, prev_i) in the order: logit descending, then token id ascending
-            float bv = -INFINITY;
-            int bi = INT_MAX;
-            for (int sl = 0; sl < S; ++sl) {
-                const long long so = static_cast<long long>(slot0 + sl) * BM + r;
-                const int n = p.cand_n[so];
-                for (int e = lane; e < n; e += 32) {
-                    const uint2 ce = p.cand[so * cap + e];
-                    const float v = __uint_as_float(ce.x);
-                    const int i = static_cast<int>(ce.y);
-                    if (i < 0) continue;
-                    const bool after_prev = (v < prev_v) || (v == prev_v && i > prev_i);
-                    const bool better = (v > bv) || (v == bv && i < bi);
-                    if (after_prev && better) {
-                        bv = v;
-                        bi = i;
-                    }
-                }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                if (ov > bv || (ov == bv && oi < bi)) {
-                    bv = ov;
-                    bi = oi;
-                }
-            }
+            float bv;
+            int bi;
+            select_next(slot0, S, prev_v, prev_i, bv, bi);
             prev_v = bv;
             prev_i = bi;
             tok = bi == INT_MAX ? 0 : bi;     // cannot happen for K <= V; keeps the gather in range
@@ -843,8 +856,8 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
                 ++n_sel;
             }
             if (lane == 0) {
-                p.idx_out[static_cast<long long>(row) * K + j] = tok_out;
-                p.q_out[static_cast<long long>(row) * K + j] = qv;
+                p.idx_out[static_cast<long long>(row) * ostride + j] = tok_out;
+                p.q_out[static_cast<long long>(row) * ostride + j] = qv;
             }
         } else {
             tok = p.idx_in[static_cast<long long>(row) * K + j];
@@ -858,12 +871,63 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
         }
     }
     __syncwarp();
+    int Ku = K;                                   // |Omega_hat| slots in use (2K at most for the bi-directional set)
+    if (p.bidir) {
+        // the draft's own K most probable tokens, in descending p; those not in the target's set join Omega_hat
+        float pv = INFINITY;
+        int pi = -1;
+        for (int j = 0; j < K; ++j) {
+            float bv;
+            int bi;
+            select_next(slot0_d, S_d, pv, pi, bv, bi);
+            pv = bv;
+            pi = bi;
+            if (bi == INT_MAX) break;
+            bool dup = false;
+            for (int t = lane; t < K; t += 32) dup |= (sh_tok[wib][t] == bi);
+            if (__any_sync(0xffffffffu, dup)) continue;
+            // target probability of this token: q = exp(<H_t[row], W[tok]> - lse_t)
+            const __nv_bfloat16* trow = p.H_t + static_cast<long long>(row) * p.d;
+            const __nv_bfloat16* wrow = p.W + static_cast<long long>(bi) * p.d;
+            float acc = 0.f;
+            for (int k0 = lane * 8; k0 < p.d; k0 += 256) {
+                const uint4 hv = *reinterpret_cast<const uint4*>(trow + k0);
+                const uint4 wv = *reinterpret_cast<const uint4*>(wrow + k0);
+                const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+                const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float2 a2 = __bfloat1622float2(hp[t]);
+                    const float2 b2 = __bfloat1622float2(wp[t]);
+                    acc = fmaf(a2.x, b2.x, acc);
+                    acc = fmaf(a2.y, b2.y, acc);
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            const float qv = expf(acc - lse_t);
+            S_q += qv;
+            if (lane == 0) {
+                sh_tok[wib][Ku] = bi;
+                sh_q[wib][Ku] = qv;
+                p.idx_out[static_cast<long long>(row) * ostride + Ku] = bi;
+                p.q_out[static_cast<long long>(row) * ostride + Ku] = qv;
+            }
+            ++Ku;
+        }
+        for (int u = Ku + lane; u < 2 * K; u += 32) {
+            p.idx_out[static_cast<long long>(row) * ostride + u] = -1;
+            p.q_out[static_cast<long long>(row) * ostride + u] = 0.f;
+        }
+        n_sel = Ku;
+        __syncwarp();
+    }
     // Draft logits at Omega_hat (K dot products with rows of W) and, for the fused backward, the row
     // sum_{x in Omega_hat} g q(x) W[x, :]. The W rows are read once: FIN_GRP tokens at a time, 256 columns
     // (8 per lane) per step; the fp32 row is accumulated across token groups.
     float* so = (p.sparse_out && !p.normed) ? p.sparse_out + static_cast<long long>(local) * p.d : nullptr;
-    for (int g0 = 0; g0 < K; g0 += FIN_GRP) {
-        const int ng = K - g0 < FIN_GRP ? K - g0 : FIN_GRP;
+    for (int g0 = 0; g0 < Ku; g0 += FIN_GRP) {
+        const int ng = Ku - g0 < FIN_GRP ? Ku - g0 : FIN_GRP;
         float dot[FIN_GRP];
 #pragma unroll
         for (int jj = 0; jj < FIN_GRP; ++jj) dot[jj] = 0.f;
