@@ -190,10 +190,11 @@ def main():
     ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--K", type=int, default=None)
-    ap.add_argument("--objective", default="topk", choices=["topk", "combined", "top_p", "normed"],
+    ap.add_argument("--objective", default="topk", choices=["topk", "combined", "top_p", "normed", "bidir"],
                     help="topk: Eq. 1 alone (the headline metric); combined: cross-entropy over the vocabulary "
                          "+ w * Top-K in one call (8 N d V tensor FLOPs); top_p (P = 0.5, at most K tokens) and "
-                         "normed (Normed Top-K: only the target product, 2 N d V) are the loss variants of Section 4.3")
+                         "normed (Normed Top-K: only the target product, 2 N d V) and bidir (Bi-directional "
+                         "Top-K) are the loss variants of Section 4.3")
     ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -244,10 +245,11 @@ def main():
         if combined:
             counts["full"] += 1
             hass.combined_distill_fwd_bwd(H_t, H_d_steps[j], W, K, w_topk=1.0, workspace=ws, out=out, stream=stream)
-        elif args.objective in ("top_p", "normed"):
+        elif args.objective in ("top_p", "normed", "bidir"):
             counts["full"] += 1
-            hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, hass.LOSS_TOP_P if args.objective == "top_p"
-                                         else hass.LOSS_NORMED_TOPK, 0.5, workspace=ws, stream=stream)
+            variant = {"top_p": hass.LOSS_TOP_P, "normed": hass.LOSS_NORMED_TOPK, "bidir": hass.LOSS_BIDIR_TOPK}
+            hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, variant[args.objective], 0.5, workspace=ws,
+                                         stream=stream)
         elif j == 0:
             counts["full"] += 1
             hass.topk_distill_fwd_bwd(H_t, H_d_steps[0], W, K, workspace=ws, out=out, stream=stream)
@@ -351,6 +353,7 @@ def main():
                                         "computed in aligning step 1, reused in steps 2..%d" % wl.steps),
                        "path": {"combined": "hass_combined_distill_fwd_bwd", "top_p": "hass_variant_distill_fwd_bwd (Top-P)",
                                 "normed": "hass_variant_distill_fwd_bwd (Normed Top-K)",
+                                "bidir": "hass_variant_distill_fwd_bwd (Bi-directional Top-K)",
                                 "topk": "hass_topk_distill_fwd_bwd (no logit recompute)"}[args.objective]},
             "clocks": clocks, "gpu_launches": launches,
             "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
