@@ -201,12 +201,13 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
-    rank, world, local = dist_setup(args.gpus)
     if args.impl == "reference":
+        # the CPU oracle needs no process group: rank 0 alone works, the other ranks leave at once
         if args.oracle_rows is None:
             args.oracle_rows = 64
-        run_reference(args, rank, world)
+        run_reference(args, int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")))
         return
+    rank, world, local = dist_setup(args.gpus)
 
     import paper_2408_15766_b200 as hass   # fails loudly if the CUDA library is missing
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
@@ -382,5 +383,5 @@ if __name__ == "__main__":
     main()
     if int(os.environ.get("WORLD_SIZE", "1")) > 1:
         import torch.distributed as dist
-        if dist.is_initialized():
+        if dist.is_available() and dist.is_initialized():
             dist.destroy_process_group()
