@@ -61,10 +61,12 @@ int hass_version(void);
 
 /*
  * Bytes of workspace that every entry point below accepts for this problem size.
- * The figure covers: a status block, per-CTA partial softmax statistics and Top-K candidates of
- * the forward sweep, the index-sorted Top-K lists of the backward, and a bounded scratch for one
- * chunk of rows of the gradient with respect to the draft logits (bf16, chunk_rows x V; the
- * chunk is a fixed number of 128-row tiles that does not grow with N).
+ * The figure covers: a status block, per-CTA partial softmax statistics and Top-K candidate
+ * buffers of the forward sweep, the index-sorted Top-K lists of the split backward, and two
+ * bounded scratch areas for one chunk of rows (a fixed number of 128-row tiles that does not grow
+ * with N): the bf16 un-normalised draft probabilities (fused call) or dz_d (split backward),
+ * chunk_rows x V, and the fp32 Omega_hat term of dH_d, chunk_rows x d. A smaller workspace is
+ * accepted down to room for one 128-row tile of scratch; the calls then work in smaller chunks.
  * Needs no GPU (assumes 148 SMs if none is present).
  */
 int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes);
