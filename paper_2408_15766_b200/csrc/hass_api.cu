@@ -180,7 +180,7 @@ static int topk_cap(int K) { return K <= K_REG ? K_REG : cand_cap(K); }
 static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 struct Layout {
-    size_t status, part_m, part_s, cand_v, cand_i, fwd_end, sidx, sgq, coef, lse2, sparse, scratch, fixed_end;
+    size_t status, part_m, part_s, cand_v, cand_i, thr_share, fwd_end, sidx, sgq, coef, lse2, sparse, scratch, fixed_end;
     size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
     long long p_pitch;
     int pref_chunk_tiles;
@@ -227,6 +227,8 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     L->cand_v = off;                        // candidate buffers: (logit, token id) pairs, cand_cap(K) per (row, slot)
     off = align256(off + slots * BM * 8 * topk_cap(K));
     L->cand_i = off;                        // entries in use per (row, slot)
+    off = align256(off + slots * BM * 4);
+    L->thr_share = off;                     // admission thresholds the lanes of a row tile publish to each other
     off = align256(off + slots * BM * 4);
     L->fwd_end = off;                       // what the forward-only entry points use
     L->sidx = off;
@@ -348,6 +350,11 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
     p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
     p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    p.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+    if (cudaMemsetAsync(p.thr_share, 0xff, static_cast<size_t>(p.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
     rc = launch_gemm<MODE_STATS>(p, st);
     if (rc != HASS_OK) return rc;
 
@@ -585,7 +592,12 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.Pt = cmb ? cmb->Pt : nullptr;
         p.p_pitch = L.p_pitch;
         p.status = status;
-        rc = launch_gemm<MODE_STATS>(p, st);
+        p.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+    if (cudaMemsetAsync(p.thr_share, 0xff, static_cast<size_t>(p.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    rc = launch_gemm<MODE_STATS>(p, st);
         if (rc != HASS_OK) return rc;
         // (2) statistics -> loss, Omega_hat, per-row scale
         FinalizeParams f;
@@ -743,6 +755,11 @@ static int normed_impl(const void* H_t, const void* H_d, const void* W, long lon
     p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
     p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
     p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    p.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+    if (cudaMemsetAsync(p.thr_share, 0xff, static_cast<size_t>(p.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
     rc = launch_gemm<MODE_STATS>(p, st);
     if (rc != HASS_OK) return rc;
     FinalizeParams f;

@@ -67,6 +67,8 @@ struct GemmParams {
     float* part_s;
     uint2* cand;           // [slot, row, cap] (logit bits, token id)
     int* cand_n;           // [slot, row] entries in use
+    float* thr_share;      // [slot, row] each lane's current threshold, read by the other lanes of its row tile
+                           // (initialised to NaN = "nothing published"; nullptr: no sharing)
     // MODE_PROBS
     const float* lse2;     // [N] lse_d * log2(e)
     const float* coef;     // [N] g * S_q
@@ -341,7 +343,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             const int g_row = p.row_global_offset + rt * BM + r_local;
             const bool row_ok = g_row < p.rows_valid;
             // ---- per-item state ----
-            float m = -INFINITY, s = 0.f, thr = -INFINITY;        // MODE_STATS
+            float m = -INFINITY, s = 0.f, thr = -INFINITY;        // MODE_STATS; thr = admission threshold in force
+            float thr_own = -INFINITY;                            // K-th (K_REG-th) largest logit of this lane's own list
+            float thr_sh = -INFINITY;                             // just below the best threshold published by the other lanes
             bool want_topk = false;
             const bool spill = MODE == MODE_STATS && spills(p, rt);
             float ref2 = 0.f;                                     // spill rows: exponent offset (log2 units)
@@ -419,7 +423,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 __syncwarp();
                                 if (lane == L) {
                                     cnt = p.K;
-                                    thr = __uint_as_float(tb);
+                                    thr_own = __uint_as_float(tb);
+                                    thr = fmaxf(thr_own, thr_sh);
                                 }
                             }
                         }
@@ -518,7 +523,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                         }
                                     }
                                 }
-                                thr = tv[(USE_REG ? K_REG : 1) - 1];
+                                thr_own = tv[(USE_REG ? K_REG : 1) - 1];
+                                thr = fmaxf(thr_own, thr_sh);
                             }
                         }
                     } else if (MODE == MODE_PROBS) {
@@ -638,6 +644,21 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 if (lane == 0) mbar_arrive(tempty_bar(ab));
                 ab ^= 1;
                 if (ab == 0) aphase ^= 1u;
+                if (MODE == MODE_STATS && want_topk && p.thr_share != nullptr && S > 1) {
+                    // The K-th largest logit of ANY lane's part of the row is a lower bound of the row's K-th
+                    // largest, so a lane may adopt the other lanes' thresholds: publish ours, read up to three
+                    // neighbours. A logit equal to a foreign threshold must still be admitted (ties are settled
+                    // by token id when the lists are merged), hence the step just below it. Stale or missing
+                    // (NaN) values only leave the threshold lower than it could be.
+                    volatile float* sh = p.thr_share + static_cast<long long>(slot - ln) * BM + r_local;
+                    sh[static_cast<long long>(ln) * BM] = thr_own;
+                    const int nn = S - 1 < 3 ? S - 1 : 3;
+                    for (int q = 1; q <= nn; ++q) {
+                        const float v = sh[static_cast<long long>((ln + q) % S) * BM];
+                        thr_sh = fmaxf(thr_sh, nextafterf(v, -INFINITY));
+                    }
+                    thr = fmaxf(thr, thr_sh);
+                }
             }
             if (MODE == MODE_STATS) {
                 const long long so = static_cast<long long>(slot) * BM + r_local;
