@@ -136,9 +136,12 @@ int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, 
  * and the sparse term.
  * Range condition: the fixed exponent holds as long as no draft logit of a row exceeds that
  * row's largest logit among tokens 0..255 by more than about 130 (natural-log units; a probability
- * ratio of e^130). If it does, hass_check reports HASS_ERR_RANGE: topk_idx, topk_q and lse_t are
- * still valid, loss, lse_d and dH_d are not; hass_topk_distill_fwd followed by hass_topk_distill_bwd
- * has no such condition and gives them.
+ * ratio of e^130). The sweep detects a violation; the call therefore also enqueues the separate
+ * forward and the recomputing backward as conditional launches that return at once unless a
+ * violation was detected, in which case they redo the whole call exactly. The result is correct
+ * either way; the conditional launches cost about 0.1 % when they have nothing to do.
+ * (hass_combined_distill_fwd_bwd and the Top-P / Bi-directional variants have no such second route:
+ * there hass_check reports HASS_ERR_RANGE and loss, lse_d and dH_d are invalid.)
  */
 int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                               int64_t V, int32_t K, const float* grad_loss, float* loss,

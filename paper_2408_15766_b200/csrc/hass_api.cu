@@ -290,7 +290,7 @@ static int launch_gemm(const GemmParams& p, cudaStream_t st) {
 static int forward_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
                         long long V, int K, const int* idx_in, const float* q_in, float* loss, int* idx_out,
                         float* q_out, float* lse_t, float* lse_d, void* workspace, size_t workspace_bytes,
-                        cudaStream_t st) {
+                        cudaStream_t st, const unsigned int* only_if_range = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !aligned16(H_d) || !aligned16(W)) return HASS_ERR_INVALID_ARG;
@@ -310,8 +310,8 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     if (workspace_bytes < L.fwd_end) return HASS_ERR_WORKSPACE;
     const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    // every public call starts with a clean status word
-    if (cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
+    // every public call starts with a clean status word (a conditional follow-up keeps the one it reads)
+    if (!only_if_range && cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
         cudaGetLastError();
         return HASS_ERR_CUDA;
     }
@@ -350,6 +350,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
     p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
     p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    p.only_if_range = only_if_range;
     p.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
     if (cudaMemsetAsync(p.thr_share, 0xff, static_cast<size_t>(p.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
         cudaGetLastError();
@@ -380,6 +381,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.q_out = q_out;
     f.lse_t = lse_t;
     f.lse_d = lse_d;
+    f.only_if_range = only_if_range;
     const int warps_per_block = 8;
     {
         KernelTimer timer(KIND_FINALIZE, st);
@@ -393,7 +395,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
 static int backward_impl(const void* H_d, const void* W, long long N, long long d, long long V, int K,
                          const int* topk_idx, const float* topk_q, const float* lse_d, const float* grad_loss,
                          void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes, cudaStream_t st,
-                         bool clear_status) {
+                         bool clear_status, const unsigned int* only_if_range = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !topk_idx || !topk_q || !lse_d || !dH_d) return HASS_ERR_INVALID_ARG;
@@ -428,7 +430,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
     {
         KernelTimer timer(KIND_PREP, st);
         bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss,
-                                                           sidx, sgq, coef, lse2);
+                                                           sidx, sgq, coef, lse2, only_if_range);
     }
     g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
@@ -466,6 +468,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
         p.P = P;
         p.p_pitch = L.p_pitch;
         p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+        p.only_if_range = only_if_range;
         rc = launch_gemm<MODE_PROBS>(p, st);
         if (rc != HASS_OK) return rc;
         // (2) dH_d rows of this chunk = dz_d chunk x W
@@ -490,6 +493,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
         o.out_align32 = ((reinterpret_cast<uintptr_t>(dH_d) | static_cast<uintptr_t>(d * (dH_dtype == HASS_FP32 ? 4 : 2))) & 31u) == 0 ? 1 : 0;
         o.out_pitch = d;
         o.status = p.status;
+        o.only_if_range = only_if_range;
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
     }
@@ -699,6 +703,20 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         o.status = status;
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
+    }
+    if (!cmb && !(top_p > 0.f) && !bidir) {
+        // Exact route, enqueued behind every plain fused call: if the sweep reported a row beyond its exponent
+        // range, the separate forward and the recomputing backward (which have no such limit) redo the call
+        // and the report is withdrawn; otherwise each of these launches returns at once.
+        rc = forward_impl(with_target, H_t, H_d, W, N, d, V, K, idx_in, q_in, loss, idx_out, q_out, lse_t, lse_d,
+                          workspace, workspace_bytes, st, status);
+        if (rc != HASS_OK) return rc;
+        rc = backward_impl(H_d, W, N, d, V, K, with_target ? idx_out : idx_in, with_target ? q_out : q_in, lse_d,
+                           grad_loss, dH_d, dH_dtype, workspace, workspace_bytes, st, false, status);
+        if (rc != HASS_OK) return rc;
+        range_handled_kernel<<<1, 1, 0, st>>>(status);
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     }
     return HASS_OK;
 }

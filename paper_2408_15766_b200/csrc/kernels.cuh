@@ -86,6 +86,7 @@ struct GemmParams {
     int out_align32;       // out base and row pitch are multiples of 32 bytes (256-bit stores allowed)
     long long out_pitch;   // elements
     unsigned int* status;
+    const unsigned int* only_if_range;   // nullptr, or: run only if this status word reports a range overflow
 };
 
 // MODE_STATS: does this row tile also write its tiles 2^(z log2e - ref2) as bf16? Draft tiles from spill_begin
@@ -184,6 +185,9 @@ constexpr int K_REG = 16;
 template <int MODE, int TOPK = TOPK_BUF>
 __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
     constexpr bool B_MN_MAJOR = (MODE == MODE_OUT);
+    // conditional launch (the exact route that follows a fused call): nothing to do unless the fused sweep
+    // reported a row beyond its exponent range
+    if (p.only_if_range != nullptr && ((*p.only_if_range) & 0xffu) != 2u) return;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t smemA = smem_base;
@@ -739,6 +743,7 @@ struct FinalizeParams {
     int bidir;             // 1: Bi-directional Top-K - Omega_hat also takes the draft's K most probable tokens (the draft
                            // rows collected candidates too); idx_out / q_out then have 2K entries per row
     const __nv_bfloat16* H_t;   // target features (bidir: target logits of the draft's tokens)
+    const unsigned int* only_if_range;   // as in GemmParams
 };
 
 __device__ __forceinline__ void find_slots(const Schedule& sc, int row_tile, int& slot0, int& S) {
@@ -772,6 +777,7 @@ __device__ __forceinline__ float warp_lse(const float* pm, const float* ps, int 
 constexpr int FIN_GRP = 16;   // tokens of Omega_hat whose W rows finalize reads together
 
 __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ FinalizeParams p) {
+    if (p.only_if_range != nullptr && ((*p.only_if_range) & 0xffu) != 2u) return;
     const int lane = threadIdx.x & 31;
     const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (local >= p.rows) return;
@@ -1102,13 +1108,19 @@ __global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d,
     if (lane == 0) loss_ce[row] = lse_d[row] - dot - ce_corr[row];
 }
 
+// Ends the exact route after a fused call: the range report has been dealt with.
+__global__ void range_handled_kernel(unsigned int* status) {
+    if (((*status) & 0xffu) == 2u) *status = 0u;
+}
+
 // ---------------------------------------------------------------------------------------------
 // bwd_prep: one thread per row. Sorts Omega_hat by token id (the MODE_PROBS epilogue walks the
 // vocabulary in increasing order) and precomputes g * q, g * S_q and lse_d * log2(e).
 __global__ void bwd_prep_kernel(int N, int K, const int* __restrict__ idx, const float* __restrict__ q,
                                 const float* __restrict__ lse_d, const float* __restrict__ grad_loss,
                                 int* __restrict__ sidx, float* __restrict__ sgq, float* __restrict__ coef,
-                                float* __restrict__ lse2) {
+                                float* __restrict__ lse2, const unsigned int* __restrict__ only_if_range) {
+    if (only_if_range != nullptr && ((*only_if_range) & 0xffu) != 2u) return;
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
     if (row >= N) return;
     const float g = grad_loss ? grad_loss[row] : 1.f;

@@ -93,7 +93,7 @@ def test_split_calls_match_fused_call_and_draft_only_forward():
     print("step 2 fused", compare(inp.H_t, inp.H_d[1], inp.W, wl.K, gpu, grad_loss=g.cpu().numpy()))
 
 
-def test_fused_path_reports_rows_beyond_its_exponent_range():
+def test_rows_beyond_the_exponent_range_of_the_spill_are_redone_exactly():
     hass = _hass()
     N, d, V, K = 40, 64, 700, 3
     inp = hi.make_custom(N, d, V, K, seed=3, sigma_w=0.1)
@@ -102,17 +102,19 @@ def test_fused_path_reports_rows_beyond_its_exponent_range():
     W[:256] = -2.0                    # draft logits of the first 256 tokens: -128
     W[300] = 2.0                      # one later token at +128: 256 above the row reference
     dev = torch.device("cuda:0")
-    out = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K)
-    with pytest.raises(hass.HassError) as e:
-        hass.check(out["workspace"])
-    assert e.value.status == -7 and hass.status_string(-7) == "HASS_ERR_RANGE"
-    # the split calls have no range condition
-    f = hass.topk_distill_fwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, workspace=out["workspace"])
-    dH = hass.topk_distill_bwd(H_d.to(dev), W.to(dev), f["topk_idx"], f["topk_q"], f["lse_d"],
-                               dH_dtype=hass.HASS_FP32, workspace=out["workspace"])
+    # the plain fused call notices and falls back to its exact route on the device
+    out = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, dH_dtype=hass.HASS_FP32)
     hass.check(out["workspace"])
-    assert torch.equal(out["topk_idx"], f["topk_idx"]) and torch.equal(out["lse_t"], f["lse_t"])
-    print(compare(inp.H_t, H_d, W, K, dict(_to_cpu(f), dH_d=dH.cpu())))
+    print(compare(inp.H_t, H_d, W, K, _to_cpu(out)))
+    d2 = hass.topk_distill_fwd_bwd_draft(H_d.to(dev), W.to(dev), out["topk_idx"], out["topk_q"],
+                                         dH_dtype=hass.HASS_FP32, workspace=out["workspace"])
+    hass.check(out["workspace"])
+    assert torch.allclose(d2["loss"], out["loss"], rtol=1e-5) and torch.allclose(d2["dH_d"], out["dH_d"], atol=1e-6)
+    # the variants without a second route report it
+    v = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, hass.LOSS_TOP_P, 0.5)
+    with pytest.raises(hass.HassError) as e:
+        hass.check(v["workspace"])
+    assert e.value.status == -7 and hass.status_string(-7) == "HASS_ERR_RANGE"
 
 
 def test_smaller_workspace_means_smaller_row_chunks_same_results():
