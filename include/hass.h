@@ -287,10 +287,11 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * on the first enable). hass_profile_summary waits for the recorded events, adds the elapsed
  * milliseconds and launch counts per kernel kind into arrays of at least HASS_PROFILE_KINDS
  * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
- * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation.
+ * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
+ * launches of the exact route behind a fused call (they return at once unless it is needed).
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */
-#define HASS_PROFILE_KINDS 5
+#define HASS_PROFILE_KINDS 6
 int hass_profile_enable(int on);
 int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
 

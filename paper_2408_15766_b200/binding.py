@@ -314,7 +314,7 @@ def check(workspace: torch.Tensor, stream=None) -> None:
     _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")
 
 
-PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep")
+PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional")
 
 
 def profile_enable(on: bool) -> None:

@@ -18,7 +18,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, NUM_KINDS = 5 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, NUM_KINDS = 6 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -276,7 +276,7 @@ static void log_schedule(const char* what, const Schedule& s) {
 
 template <int MODE>
 static int launch_gemm(const GemmParams& p, cudaStream_t st) {
-    KernelTimer timer(MODE, st);
+    KernelTimer timer(p.only_if_range ? KIND_CONDITIONAL : MODE, st);
     if (MODE == MODE_STATS && p.K <= K_REG)
         gemm_kernel<MODE_STATS, TOPK_REG><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
     else
@@ -384,7 +384,7 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.only_if_range = only_if_range;
     const int warps_per_block = 8;
     {
-        KernelTimer timer(KIND_FINALIZE, st);
+        KernelTimer timer(only_if_range ? KIND_CONDITIONAL : KIND_FINALIZE, st);
         finalize_kernel<<<ceil_div(N, warps_per_block), warps_per_block * 32, 0, st>>>(f);
     }
     g_launches.fetch_add(1);
@@ -428,7 +428,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
     }
 
     {
-        KernelTimer timer(KIND_PREP, st);
+        KernelTimer timer(only_if_range ? KIND_CONDITIONAL : KIND_PREP, st);
         bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss,
                                                            sidx, sgq, coef, lse2, only_if_range);
     }
@@ -714,7 +714,10 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         rc = backward_impl(H_d, W, N, d, V, K, with_target ? idx_out : idx_in, with_target ? q_out : q_in, lse_d,
                            grad_loss, dH_d, dH_dtype, workspace, workspace_bytes, st, false, status);
         if (rc != HASS_OK) return rc;
-        range_handled_kernel<<<1, 1, 0, st>>>(status);
+        {
+            KernelTimer timer(KIND_CONDITIONAL, st);
+            range_handled_kernel<<<1, 1, 0, st>>>(status);
+        }
         g_launches.fetch_add(1);
         if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     }
