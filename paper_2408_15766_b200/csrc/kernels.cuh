@@ -2,11 +2,16 @@
 //
 // One warp-specialised, persistent GEMM kernel (TMA -> shared memory -> tcgen05.mma -> TMEM ->
 // epilogue warps) is instantiated with three epilogues:
-//   MODE_STATS  logits tile -> running max / sum-exp per row (+ Top-K candidates for target rows)
+//   MODE_STATS  logits tile -> per-row softmax statistics, Top-K candidates (two variants: a sorted register
+//               list for K <= 16, append buffers with warp-cooperative compaction otherwise) and, in the fused
+//               forward+backward, a bf16 spill of 2^(z log2e - ref) that the second GEMM consumes
 //   MODE_PROBS  draft logits tile -> dz_d tile = g (S_q p - q [v in Omega_hat]) in bf16 -> scratch
-//   MODE_OUT    plain store of the accumulator (dH_d = dz_d W)
-// plus two small kernels: finalize (merge partial statistics, pick Omega_hat, Eq. 1) and
-// bwd_prep (index-sorted Top-K lists and per-row coefficients for MODE_PROBS).
+//               (the separate, recomputing backward)
+//   MODE_OUT    dH_d tile: coef * acc - Omega_hat row (fused), coef * acc (q W of the combined objective)
+//               or the accumulator as is (separate backward)
+// plus small kernels: finalize (merge partial statistics, pick Omega_hat, Eq. 1 and its variants, the
+// Omega_hat term of dH_d), ce_kernel (cross-entropy of the combined objective), bwd_prep (index-sorted
+// Top-K lists for MODE_PROBS) and range_handled_kernel.
 #pragma once
 #include <cuda_bf16.h>
 #include <float.h>
