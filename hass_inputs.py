@@ -100,3 +100,58 @@ def sample_rows(N: int, n_rows: int, seed: int = 0) -> np.ndarray:
     middle_pool = np.arange(q, N - q, dtype=np.int64)
     mid = rng.choice(middle_pool, size=n_rows - 2 * q, replace=False)
     return np.unique(np.concatenate([head, mid, tail]))
+
+
+# ---- inputs of the HCA attention of the draft layer (Section 3.2) --------------------------------
+@dataclass(frozen=True)
+class HcaWorkload:
+    name: str
+    B: int            # sequences per batch
+    T: int            # tokens per sequence
+    H: int            # query heads
+    Hkv: int          # key/value heads (H a multiple of it)
+    m: int            # earlier draft passes whose features replace the target's (aligning step m + 1)
+    D: int = 128      # head dimension
+    seed: int = 0
+
+
+# Shapes of the one-layer draft model, which copies its target's attention geometry: a tiny
+# case, a ragged mid-size case, and LLaMA3-8B / LLaMA2-7B geometry at 4 x 2048 tokens (the
+# 8192-token batch of the LM-head workloads) in the third aligning step.
+HCA_WORKLOADS = {
+    "hca-tiny": HcaWorkload("hca-tiny", B=2, T=80, H=2, Hkv=1, m=2),
+    "hca-mid": HcaWorkload("hca-mid", B=2, T=333, H=4, Hkv=2, m=3),
+    "hca-l3-8b": HcaWorkload("hca-l3-8b", B=4, T=2048, H=32, Hkv=8, m=2),
+    "hca-l2-7b": HcaWorkload("hca-l2-7b", B=4, T=2048, H=32, Hkv=32, m=2),
+}
+
+
+@dataclass
+class HcaInputs:
+    """bf16 tensors (CPU, contiguous): Q [B, T, H, D]; K_t, V_t and every K_d[i], V_d[i] [B, T, Hkv, D]."""
+    wl: HcaWorkload
+    Q: torch.Tensor
+    K_t: torch.Tensor
+    V_t: torch.Tensor
+    K_d: List[torch.Tensor] = field(default_factory=list)
+    V_d: List[torch.Tensor] = field(default_factory=list)
+
+
+def make_hca_inputs(wl: HcaWorkload) -> HcaInputs:
+    """Projected queries, keys and values stand in for q_proj/k_proj/v_proj of real features:
+    Q, K_t, V_t ~ N(0, 1); the keys/values of draft pass i are the target's plus 0.5 * N(0, 1),
+    the same closeness the LM-head workloads give draft features. Draw order: Q, K_t, V_t,
+    then (K_d[i], V_d[i]) for i = 0 .. m-1; everything rounded to bf16."""
+    g = torch.Generator(device="cpu")
+    g.manual_seed(wl.seed)
+    shape_q = (wl.B, wl.T, wl.H, wl.D)
+    shape_kv = (wl.B, wl.T, wl.Hkv, wl.D)
+    Q = torch.randn(shape_q, generator=g, dtype=torch.float32)
+    K32 = torch.randn(shape_kv, generator=g, dtype=torch.float32)
+    V32 = torch.randn(shape_kv, generator=g, dtype=torch.float32)
+    K_d, V_d = [], []
+    for _ in range(wl.m):
+        K_d.append((K32 + 0.5 * torch.randn(shape_kv, generator=g, dtype=torch.float32)).to(torch.bfloat16).contiguous())
+        V_d.append((V32 + 0.5 * torch.randn(shape_kv, generator=g, dtype=torch.float32)).to(torch.bfloat16).contiguous())
+    return HcaInputs(wl=wl, Q=Q.to(torch.bfloat16).contiguous(), K_t=K32.to(torch.bfloat16).contiguous(),
+                     V_t=V32.to(torch.bfloat16).contiguous(), K_d=K_d, V_d=V_d)

@@ -1,0 +1,153 @@
+"""Pins of the HCA-attention oracle (Section 3.2 and the appendix's attention listing) against
+things other than itself: a library attention routine, the text's concatenated key/value
+sequence written out query by query, closed forms, invariants and finite differences."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import hca_oracle as ho
+
+
+def _rand(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape)
+
+
+def _case(B=2, T=9, H=2, Hkv=1, D=4, m=2, seed=0):
+    Q = _rand((B, T, H, D), seed)
+    K_t = _rand((B, T, Hkv, D), seed + 1)
+    V_t = _rand((B, T, Hkv, D), seed + 2)
+    K_d = [_rand((B, T, Hkv, D), seed + 10 + i) for i in range(m)]
+    V_d = [_rand((B, T, Hkv, D), seed + 20 + i) for i in range(m)]
+    return Q, K_t, V_t, K_d, V_d
+
+
+def _sdpa(Q, K, V):
+    """torch's causal attention in fp64, [B, T, H, D] in and out."""
+    q, k, v = (torch.from_numpy(x).permute(0, 2, 1, 3) for x in (Q, K, V))
+    if k.shape[1] != q.shape[1]:
+        rep = q.shape[1] // k.shape[1]
+        k, v = k.repeat_interleave(rep, dim=1), v.repeat_interleave(rep, dim=1)
+    return torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True).permute(0, 2, 1, 3).numpy()
+
+
+def test_first_aligning_step_is_causal_attention():
+    # step 1 has no draft features: the listing leaves the causal attention untouched
+    Q, K_t, V_t, _, _ = _case(T=17, H=4, Hkv=2, D=8, m=0)
+    O, lse = ho.hca_attention(Q, K_t, V_t)
+    np.testing.assert_allclose(O, _sdpa(Q, K_t, V_t), rtol=1e-12, atol=1e-12)
+    # the normaliser against a direct evaluation for one row
+    b, h, t = 1, 3, 11
+    s = (K_t[b, :t + 1, h // 2, :] @ Q[b, t, h, :]) / math.sqrt(8)
+    assert abs(lse[b, h, t] - math.log(np.exp(s).sum())) < 1e-12
+
+
+def test_draft_equal_to_target_changes_nothing():
+    Q, K_t, V_t, _, _ = _case(m=0)
+    O0, l0 = ho.hca_attention(Q, K_t, V_t)
+    O3, l3 = ho.hca_attention(Q, K_t, V_t, [K_t] * 3, [V_t] * 3)
+    np.testing.assert_allclose(O3, O0, rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(l3, l0, rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("m", [1, 2, 4])
+def test_equals_concatenated_context_per_query(m):
+    """The text's form: the query of step j = m + 1 at position t sees target features up to
+    position t - m and then one feature from each earlier draft pass, oldest first, the latest
+    pass at position t itself. Written out with plain loops, one query at a time."""
+    B, T, H, Hkv, D = 2, 11, 2, 1, 4
+    Q, K_t, V_t, K_d, V_d = _case(B, T, H, Hkv, D, m, seed=3)
+    O, lse = ho.hca_attention(Q, K_t, V_t, K_d, V_d)
+    # chronological list of passes (s_1 first) as the training loop appends them
+    K_chron, V_chron = K_d[::-1], V_d[::-1]
+    for b in range(B):
+        for h in range(H):
+            for t in range(T):
+                keys, vals = [], []
+                for s in range(0, t - m + 1):
+                    keys.append(K_t[b, s, 0]); vals.append(V_t[b, s, 0])
+                for n, s in enumerate(range(t - m + 1, t + 1)):     # n-th earlier pass, 0 = s_1
+                    if s < 0:
+                        continue
+                    keys.append(K_chron[n][b, s, 0]); vals.append(V_chron[n][b, s, 0])
+                sc = np.array([float(np.dot(Q[b, t, h], k)) for k in keys]) / math.sqrt(D)
+                w = np.exp(sc - sc.max()); z = w.sum(); w /= z
+                ref = sum(wi * vi for wi, vi in zip(w, vals))
+                np.testing.assert_allclose(O[b, t, h], ref, rtol=1e-12, atol=1e-12)
+                assert abs(lse[b, h, t] - (sc.max() + math.log(z))) < 1e-12
+
+
+def test_two_token_closed_form():
+    # T = 2, D = 1, one head, one draft pass on the main diagonal
+    Q = np.array([0.5, -1.5]).reshape(1, 2, 1, 1)
+    K_t = np.array([2.0, 3.0]).reshape(1, 2, 1, 1)
+    V_t = np.array([10.0, 20.0]).reshape(1, 2, 1, 1)
+    K_d = [np.array([-1.0, 0.25]).reshape(1, 2, 1, 1)]
+    V_d = [np.array([7.0, -4.0]).reshape(1, 2, 1, 1)]
+    O, lse = ho.hca_attention(Q, K_t, V_t, K_d, V_d)
+    # query 0 sees only its own position, which comes from the draft pass
+    assert O[0, 0, 0, 0] == pytest.approx(7.0, abs=1e-14)
+    assert lse[0, 0, 0] == pytest.approx(0.5 * -1.0, abs=1e-14)
+    # query 1: target key/value at position 0, draft key/value at position 1
+    a, c = -1.5 * 2.0, -1.5 * 0.25
+    w0 = 1.0 / (1.0 + math.exp(c - a))
+    assert O[0, 1, 0, 0] == pytest.approx(w0 * 10.0 + (1 - w0) * -4.0, rel=1e-14)
+    assert lse[0, 0, 1] == pytest.approx(math.log(math.exp(a) + math.exp(c)), rel=1e-14)
+
+
+def test_rows_are_convex_combinations():
+    Q, K_t, V_t, K_d, V_d = _case(T=13, m=3, seed=5)
+    c = np.array([1.0, -2.0, 0.5, 3.0])
+    V_const = np.broadcast_to(c, V_t.shape)
+    O, _ = ho.hca_attention(10.0 * Q, K_t, V_const, K_d, [V_const] * 3)
+    np.testing.assert_allclose(O, np.broadcast_to(c, O.shape), rtol=1e-12, atol=1e-12)
+
+
+def test_grouped_heads_read_their_group():
+    Q, K_t, V_t, K_d, V_d = _case(H=4, Hkv=2, m=2, seed=7)
+    O, lse = ho.hca_attention(Q, K_t, V_t, K_d, V_d)
+    rep = lambda x: np.repeat(x, 2, axis=2)
+    O2, lse2 = ho.hca_attention(Q, rep(K_t), rep(V_t), [rep(x) for x in K_d], [rep(x) for x in V_d])
+    np.testing.assert_array_equal(O, O2)
+    np.testing.assert_array_equal(lse, lse2)
+
+
+def test_scale_argument():
+    Q, K_t, V_t, K_d, V_d = _case(m=1, seed=9)
+    O1, _ = ho.hca_attention(Q, K_t, V_t, K_d, V_d, scale=0.3)
+    O2, _ = ho.hca_attention(0.3 * math.sqrt(Q.shape[-1]) * Q, K_t, V_t, K_d, V_d)
+    np.testing.assert_allclose(O1, O2, rtol=1e-12, atol=1e-12)
+
+
+def test_gradients_against_finite_differences():
+    Q, K_t, V_t, K_d, V_d = _case(B=1, T=6, H=2, Hkv=1, D=3, m=2, seed=11)
+    dO = _rand(Q.shape, 99)
+    grads = ho.hca_attention_grad(Q, K_t, V_t, K_d, V_d, dO)
+    flat_in = [Q, K_t, V_t] + K_d + V_d
+    flat_g = [grads[0], grads[1], grads[2]] + grads[3] + grads[4]
+
+    def f():
+        return float((ho.hca_attention(Q, K_t, V_t, K_d, V_d)[0] * dO).sum())
+
+    rng = np.random.default_rng(1)
+    eps = 1e-6
+    for x, g in zip(flat_in, flat_g):
+        for _ in range(12):
+            pos = tuple(rng.integers(0, n) for n in x.shape)
+            old = x[pos]
+            x[pos] = old + eps; fp = f()
+            x[pos] = old - eps; fm = f()
+            x[pos] = old
+            assert g[pos] == pytest.approx((fp - fm) / (2 * eps), rel=2e-6, abs=2e-8)
+
+
+def test_first_step_gradients_against_autograd():
+    Q, K_t, V_t, _, _ = _case(B=1, T=10, H=2, Hkv=2, D=4, m=0, seed=13)
+    dO = _rand(Q.shape, 5)
+    dQ, dK, dV, _, _ = ho.hca_attention_grad(Q, K_t, V_t, [], [], dO)
+    q, k, v = (torch.from_numpy(x).permute(0, 2, 1, 3).clone().requires_grad_(True) for x in (Q, K_t, V_t))
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+    o.backward(torch.from_numpy(dO).permute(0, 2, 1, 3))
+    for mine, ref in ((dQ, q.grad), (dK, k.grad), (dV, v.grad)):
+        np.testing.assert_allclose(mine, ref.permute(0, 2, 1, 3).numpy(), rtol=1e-11, atol=1e-12)
