@@ -239,6 +239,39 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
                                    void* cuda_stream);
 
 /*
+ * HCA attention of the draft layer (Section 3.2 "Harmonized Context Alignment" and the attention
+ * listing of the appendix), forward. In aligning step m + 1 the query at position t attends
+ * causally to positions s <= t; the key and value of the pair (t, s) come from the target LLM's
+ * features, except for t - s = i < m, where they come from the i-th most recent earlier draft
+ * pass (i = 0: the latest pass, on the main diagonal):
+ *     w[t, .] = softmax_{s <= t}( scale * <Q[t], k(t, s)> ),   O[t] = sum_s w[t, s] v(t, s).
+ * The weights that multiply the draft values are the normalised ones (the text's concatenated
+ * key/value sequence); m = 0 is plain causal attention (the first aligning step).
+ * The projections q_proj/k_proj/v_proj/o_proj are ordinary GEMMs outside this call.
+ *
+ *   Q            [B, T, H, D]     bf16  projected queries (of the latest draft features, or of the
+ *                                       target features when m = 0)
+ *   K_t, V_t     [B, T, Hkv, D]   bf16  projected target features; H a multiple of Hkv, query head
+ *                                       h reads key/value head h / (H / Hkv)
+ *   K_d, V_d     HOST arrays of m DEVICE pointers, each [B, T, Hkv, D] bf16: entry i replaces the
+ *                i-th sub-diagonal. Read during the call only. 0 <= m <= HASS_HCA_MAX_DRAFTS.
+ *   D            must be 128 (HASS_ERR_UNSUPPORTED otherwise); scale > 0, normally 1/sqrt(D)
+ *   O            [B, T, H, D]     bf16  out (32-byte aligned; inputs 16-byte aligned)
+ *   lse          [B, H, T]        fp32  out, optional: natural-log normaliser of each query row
+ *   workspace    at least hass_hca_attention_workspace_bytes (256) bytes, 256-byte aligned; holds
+ *                the status word hass_check reads
+ * One kernel is enqueued on cuda_stream. Errors as for the other entries: argument problems are
+ * returned before anything is launched; a bounded device wait that gave up is reported by
+ * hass_check as HASS_ERR_TIMEOUT and O is then undefined.
+ */
+#define HASS_HCA_MAX_DRAFTS 8
+int hass_hca_attention_workspace_bytes(size_t* bytes);
+int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,
+                           const void* const* V_d, int32_t m, int64_t B, int64_t T, int64_t H,
+                           int64_t Hkv, int64_t D, float scale, void* O, float* lse, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and returns the status word of `workspace`: HASS_OK, or
  * HASS_ERR_TIMEOUT if a kernel gave up on a bounded wait (its outputs are then undefined), or
  * HASS_ERR_CUDA if the stream reports an error. Clears the status word.
@@ -288,10 +321,11 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * milliseconds and launch counts per kernel kind into arrays of at least HASS_PROFILE_KINDS
  * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
  * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
- * launches of the exact route behind a fused call (they return at once unless it is needed).
+ * launches of the exact route behind a fused call (they return at once unless it is needed),
+ * 6 HCA attention.
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */
-#define HASS_PROFILE_KINDS 6
+#define HASS_PROFILE_KINDS 7
 int hass_profile_enable(int on);
 int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
 

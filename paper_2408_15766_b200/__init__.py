@@ -11,6 +11,9 @@ from .binding import (  # noqa: F401
     HASS_FP32,
     K_MAX,
     check,
+    hca_attention_fwd,
+    hca_attention_workspace_bytes,
+    HCA_MAX_DRAFTS,
     combined_distill_fwd_bwd,
     combined_distill_workspace_bytes,
     kernel_launch_count,

@@ -52,6 +52,11 @@ def _load() -> ctypes.CDLL:
     L.hass_variant_distill_fwd_bwd.restype = ctypes.c_int
     L.hass_topk_distill_fwd_bwd_host.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp,
                                                  ctypes.c_int, vp, sz, vp]
+    L.hass_hca_attention_workspace_bytes.argtypes = [ctypes.POINTER(sz)]
+    L.hass_hca_attention_workspace_bytes.restype = ctypes.c_int
+    L.hass_hca_attention_fwd.argtypes = [vp, vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i64, i64, i64, i64,
+                                         i64, ctypes.c_float, vp, vp, vp, sz, vp]
+    L.hass_hca_attention_fwd.restype = ctypes.c_int
     L.hass_check.argtypes = [vp, vp]
     L.hass_topk_distill_fwd_static.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     L.hass_topk_distill_fwd_static.restype = ctypes.c_int
@@ -309,12 +314,48 @@ def topk_distill_fwd_bwd_host(H_t_host, H_d_host, W, K: int, loss_host, dH_d_hos
         "hass_topk_distill_fwd_bwd_host")
 
 
+HCA_MAX_DRAFTS = 8
+
+
+def hca_attention_workspace_bytes() -> int:
+    n = ctypes.c_size_t(0)
+    _ok(lib.hass_hca_attention_workspace_bytes(ctypes.byref(n)), "hass_hca_attention_workspace_bytes")
+    return int(n.value)
+
+
+def hca_attention_fwd(Q, K_t, V_t, K_d=(), V_d=(), scale: Optional[float] = None, want_lse: bool = True,
+                      workspace=None, stream=None) -> dict:
+    """HCA attention forward. Q [B, T, H, D]; K_t, V_t and every K_d[i], V_d[i] [B, T, Hkv, D], bf16 CUDA
+    tensors; entry i of K_d / V_d replaces the i-th sub-diagonal. See hass_hca_attention_fwd."""
+    B, T, H, D = Q.shape
+    Hkv = K_t.shape[2]
+    m = len(K_d)
+    assert len(V_d) == m
+    for x in (Q, K_t, V_t, *K_d, *V_d):
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    for x in (V_t, *K_d, *V_d):
+        assert x.shape == K_t.shape
+    assert K_t.shape == (B, T, Hkv, D)
+    dev = Q.device
+    ws = _workspace(workspace, hca_attention_workspace_bytes(), dev)
+    out = dict(O=torch.empty_like(Q), lse=torch.empty(B, H, T, dtype=torch.float32, device=dev) if want_lse else None,
+               workspace=ws)
+    kd = (ctypes.c_void_p * max(m, 1))(*[x.data_ptr() for x in K_d])
+    vd = (ctypes.c_void_p * max(m, 1))(*[x.data_ptr() for x in V_d])
+    sc = float(scale) if scale is not None else 1.0 / (D ** 0.5)
+    _ok(lib.hass_hca_attention_fwd(_p(Q), _p(K_t), _p(V_t), kd, vd, m, B, T, H, Hkv, D, ctypes.c_float(sc),
+                                   _p(out["O"]), _p(out["lse"]), _p(ws), ws.numel(), _stream(stream)),
+        "hass_hca_attention_fwd")
+    return out
+
+
 def check(workspace: torch.Tensor, stream=None) -> None:
     """Synchronises the stream and raises HassError if a kernel recorded a device-side problem."""
     _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")
 
 
-PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional")
+PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional",
+                 "hca_attention")
 
 
 def profile_enable(on: bool) -> None:

@@ -10,6 +10,7 @@
 
 #include "../../include/hass.h"
 #include "kernels.cuh"
+#include "hca_kernels.cuh"
 
 namespace hass {
 
@@ -18,7 +19,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, NUM_KINDS = 6 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, NUM_KINDS = 7 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -72,7 +73,8 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<MODE_PROBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-            if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+            cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
+            if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
                 cudaGetLastError();
                 return HASS_ERR_CUDA;
             }
@@ -168,6 +170,19 @@ static int make_tmap(CUtensorMap* tm, const void* base, long long rows, long lon
     cuuint32_t box[2] = {static_cast<cuuint32_t>(box_cols), static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HASS_OK : HASS_ERR_CUDA;
+}
+
+// bf16 tensor [B, T, heads * 128] (dense): box = 64 columns x 128 positions of one sequence, 128-byte
+// swizzle. Positions past T read as zeros, so a ragged last tile never sees the next sequence.
+static int make_tmap_seq(CUtensorMap* tm, const void* base, long long B, long long T, long long cols) {
+    cuuint64_t gdim[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(B)};
+    cuuint64_t gstride[2] = {static_cast<cuuint64_t>(cols) * 2, static_cast<cuuint64_t>(cols) * 2 * static_cast<cuuint64_t>(T)};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? HASS_OK : HASS_ERR_CUDA;
@@ -1153,6 +1168,73 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
         cudaGetLastError();
         return HASS_ERR_CUDA;
     }
+    return HASS_OK;
+}
+
+int hass_hca_attention_workspace_bytes(size_t* bytes) {
+    if (!bytes) return HASS_ERR_INVALID_ARG;
+    *bytes = 256;
+    return HASS_OK;
+}
+
+int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,
+                           const void* const* V_d, int32_t m, int64_t B, int64_t T, int64_t H, int64_t Hkv, int64_t D,
+                           float scale, void* O, float* lse, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream) {
+    if (!Q || !K_t || !V_t || !O) return HASS_ERR_INVALID_ARG;
+    if (m < 0 || m > HASS_HCA_MAX_DRAFTS || (m > 0 && (!K_d || !V_d))) return HASS_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || H < 1 || Hkv < 1 || H % Hkv != 0 || !(scale > 0.f) || !(scale < INFINITY))
+        return HASS_ERR_INVALID_ARG;
+    if (D != hca::HD) return HASS_ERR_UNSUPPORTED;
+    if (B > 65535 || T > (1 << 22) || H > 4096 || B * H * ((T + hca::QT - 1) / hca::QT) > INT_MAX / 2)
+        return HASS_ERR_UNSUPPORTED;
+    auto misaligned = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) != 0; };
+    if (misaligned(Q) || misaligned(K_t) || misaligned(V_t) || (reinterpret_cast<uintptr_t>(O) & 31u) != 0)
+        return HASS_ERR_INVALID_ARG;
+    for (int i = 0; i < m; ++i)
+        if (!K_d[i] || !V_d[i] || misaligned(K_d[i]) || misaligned(V_d[i])) return HASS_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < 256 || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    hca::Params p;
+    std::memset(&p, 0, sizeof(p));
+    rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca::HD);
+    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca::HD);
+    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca::HD);
+    if (rc != HASS_OK) return rc;
+    p.Q = static_cast<const __nv_bfloat16*>(Q);
+    for (int i = 0; i < m; ++i) {
+        p.K_d[i] = static_cast<const __nv_bfloat16*>(K_d[i]);
+        p.V_d[i] = static_cast<const __nv_bfloat16*>(V_d[i]);
+    }
+    p.O = static_cast<__nv_bfloat16*>(O);
+    p.lse = lse;
+    p.B = static_cast<int>(B);
+    p.T = static_cast<int>(T);
+    p.H = static_cast<int>(H);
+    p.Hkv = static_cast<int>(Hkv);
+    p.m = m;
+    p.q_tiles = static_cast<int>((T + hca::QT - 1) / hca::QT);
+    p.items = static_cast<int>(B * H) * p.q_tiles;
+    p.c2 = scale * 1.4426950408889634f;
+    p.status = static_cast<unsigned int*>(workspace);
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    const int grid = p.items < di.sms ? p.items : di.sms;
+    {
+        KernelTimer kt(KIND_HCA, st);
+        hca::hca_attention_kernel<<<grid, hca::NUM_THREADS, hca::SMEM_BYTES, st>>>(p);
+    }
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     return HASS_OK;
 }
 

@@ -1,0 +1,120 @@
+"""GPU parity of the HCA attention kernel (through the C ABI) against the fp64 oracle.
+
+Tolerances (the kernel multiplies bf16 operands exactly, accumulates in fp32, rounds the softmax
+weights to bf16 before the value product and the output to bf16):
+  O    |error| <= 1e-2 * max|O|   (bf16 rounding of weights and output, 2^-9 relative each)
+  lse  |error| <= 2e-3            (fp32 sums, approximate exp2)
+"""
+import numpy as np
+import pytest
+import torch
+
+import hass_inputs as hi
+from oracle import hca_oracle as ho
+
+pytestmark = pytest.mark.gpu
+
+O_TOL = 1e-2
+LSE_TOL = 2e-3
+
+
+def _hass():
+    import paper_2408_15766_b200 as hass
+    return hass
+
+
+def _f64(t):
+    return t.to(torch.float64).numpy()
+
+
+def _run(inp, scale=None, m=None):
+    hass = _hass()
+    dev = torch.device("cuda:0")
+    m = inp.wl.m if m is None else m
+    out = hass.hca_attention_fwd(inp.Q.to(dev), inp.K_t.to(dev), inp.V_t.to(dev), [x.to(dev) for x in inp.K_d[:m]],
+                                 [x.to(dev) for x in inp.V_d[:m]], scale=scale)
+    hass.check(out["workspace"])
+    return out["O"].cpu(), out["lse"].cpu()
+
+
+def _compare(inp, O, lse, scale=None, m=None, pairs=None):
+    """pairs: list of (b, h) to check (all when None)."""
+    wl = inp.wl
+    m = wl.m if m is None else m
+    rep = wl.H // wl.Hkv
+    if pairs is None:
+        pairs = [(b, h) for b in range(wl.B) for h in range(wl.H)]
+    worst_o = worst_l = 0.0
+    for b, h in pairs:
+        g = h // rep
+        sl = lambda x, hh: _f64(x[b:b + 1, :, hh:hh + 1, :])
+        O_ref, lse_ref = ho.hca_attention(sl(inp.Q, h), sl(inp.K_t, g), sl(inp.V_t, g),
+                                          [sl(x, g) for x in inp.K_d[:m]], [sl(x, g) for x in inp.V_d[:m]], scale=scale)
+        err = np.abs(_f64(O[b:b + 1, :, h:h + 1, :]) - O_ref).max() / np.abs(O_ref).max()
+        lerr = np.abs(lse[b, h].to(torch.float64).numpy() - lse_ref[0, 0]).max()
+        worst_o, worst_l = max(worst_o, err), max(worst_l, lerr)
+    assert worst_o <= O_TOL, f"O error {worst_o:.3e} of max|O|"
+    assert worst_l <= LSE_TOL, f"lse error {worst_l:.3e}"
+    return worst_o, worst_l
+
+
+@pytest.mark.parametrize("name", ["hca-tiny", "hca-mid"])
+def test_small_workloads_all_heads(name):
+    inp = hi.make_hca_inputs(hi.HCA_WORKLOADS[name])
+    O, lse = _run(inp)
+    print(_compare(inp, O, lse))
+
+
+@pytest.mark.parametrize("B,T,H,Hkv,m", [
+    (1, 1, 1, 1, 1),          # a single position: the output is the draft value row itself
+    (1, 128, 2, 2, 8),        # exactly one tile, the maximum number of draft passes
+    (1, 129, 2, 1, 8),        # one row in the second tile: its sub-diagonals reach back into the first
+    (2, 256, 3, 3, 0),        # first aligning step: plain causal attention
+    (1, 515, 4, 2, 5),
+    (2, 700, 16, 4, 2),       # more work items than SMs: every CTA takes a second item
+])
+def test_awkward_shapes(B, T, H, Hkv, m):
+    inp = hi.make_hca_inputs(hi.HcaWorkload("custom", B=B, T=T, H=H, Hkv=Hkv, m=m, seed=T + m))
+    O, lse = _run(inp)
+    pairs = None if B * H <= 8 else [(0, 0), (0, H - 1), (B - 1, H // 2), (B - 1, 1)]
+    print(_compare(inp, O, lse, pairs=pairs))
+    if T == 1:
+        assert torch.equal(O, inp.V_d[0])
+
+
+def test_steep_scores_rescale_the_accumulator():
+    # scale 1 instead of 1/sqrt(D): scores spread over +-40, so later tiles push the running reference
+    # up by far more than the lazy-rescale threshold
+    inp = hi.make_hca_inputs(hi.HcaWorkload("steep", B=1, T=640, H=2, Hkv=1, m=2, seed=3))
+    O, lse = _run(inp, scale=1.0)
+    print(_compare(inp, O, lse, scale=1.0))
+
+
+def test_fewer_passes_than_provided_and_determinism():
+    inp = hi.make_hca_inputs(hi.HCA_WORKLOADS["hca-mid"])
+    O1, l1 = _run(inp, m=1)
+    _compare(inp, O1, l1, m=1)
+    O2, l2 = _run(inp, m=1)
+    assert torch.equal(O1, O2) and torch.equal(l1, l2)
+
+
+def test_argument_errors():
+    hass = _hass()
+    inp = hi.make_hca_inputs(hi.HCA_WORKLOADS["hca-tiny"])
+    dev = torch.device("cuda:0")
+    Q, K, V = inp.Q.to(dev), inp.K_t.to(dev), inp.V_t.to(dev)
+    with pytest.raises(hass.HassError):       # head dimension other than 128
+        hass.hca_attention_fwd(Q[..., :64].contiguous(), K[..., :64].contiguous(), V[..., :64].contiguous())
+    with pytest.raises(hass.HassError):       # too many draft passes
+        hass.hca_attention_fwd(Q, K, V, [K] * 9, [V] * 9)
+    with pytest.raises(hass.HassError):
+        hass.hca_attention_fwd(Q, K, V, scale=0.0)
+
+
+@pytest.mark.parametrize("name", ["hca-l3-8b", "hca-l2-7b"])
+def test_full_size_sampled_heads(name):
+    wl = hi.HCA_WORKLOADS[name]
+    inp = hi.make_hca_inputs(wl)
+    O, lse = _run(inp)
+    pairs = [(0, 0), (wl.B - 1, wl.H - 1), (1, 5), (2, wl.H // 2 + 1)]
+    print(_compare(inp, O, lse, pairs=pairs))
