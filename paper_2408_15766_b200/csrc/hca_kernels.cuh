@@ -274,14 +274,51 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             const int gkv = h / rep;
             const int t = qt * QT + r;                        // position in the sequence
             const bool valid = t < p.T;
-            // scores against the draft passes' keys on this row's substituted entries (raw, unscaled)
+            const int t_warp = qt * QT + quad * 32;           // first row of this warp
+            // ---- scores against the draft passes' keys on this row's substituted entries (raw, unscaled).
+            // The warp takes its 32 rows one by one with coalesced 256-byte reads (lane = 4 columns), then a
+            // transposing butterfly leaves row rr's dot product on lane rr.
             float sd[MAX_DRAFTS];
-            const __nv_bfloat16* qrow = p.Q + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
 #pragma unroll
-            for (int i = 0; i < MAX_DRAFTS; ++i) {
-                sd[i] = 0.f;
-                if (i < p.m && valid && t - i >= 0)
-                    sd[i] = dot128(qrow, p.K_d[i] + ((static_cast<size_t>(b) * p.T + (t - i)) * p.Hkv + gkv) * HD);
+            for (int i = 0; i < MAX_DRAFTS; ++i) sd[i] = 0.f;
+            if (p.m > 0) {
+                uint2 qv[32];
+#pragma unroll
+                for (int rr = 0; rr < 32; ++rr) {
+                    const int tr = t_warp + rr;
+                    qv[rr] = make_uint2(0u, 0u);
+                    if (tr < p.T)
+                        qv[rr] = __ldg(reinterpret_cast<const uint2*>(
+                                           p.Q + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane);
+                }
+#pragma unroll
+                for (int i = 0; i < MAX_DRAFTS; ++i) {
+                    if (i < p.m) {
+                        float acc[32];
+#pragma unroll
+                        for (int rr = 0; rr < 32; ++rr) {
+                            const int tr = t_warp + rr;
+                            uint2 kv = make_uint2(0u, 0u);
+                            if (tr < p.T && tr - i >= 0)
+                                kv = __ldg(reinterpret_cast<const uint2*>(
+                                               p.K_d[i] + ((static_cast<size_t>(b) * p.T + (tr - i)) * p.Hkv + gkv) * HD) + lane);
+                            acc[rr] = fmaf(bf16_lo(qv[rr].x), bf16_lo(kv.x),
+                                           fmaf(bf16_hi(qv[rr].x), bf16_hi(kv.x),
+                                                fmaf(bf16_lo(qv[rr].y), bf16_lo(kv.y), bf16_hi(qv[rr].y) * bf16_hi(kv.y))));
+                        }
+#pragma unroll
+                        for (int sft = 16; sft >= 1; sft >>= 1) {
+                            const bool up = (lane & sft) != 0;
+#pragma unroll
+                            for (int k = 0; k < sft; ++k) {
+                                const float keep = up ? acc[k + sft] : acc[k];
+                                const float send = up ? acc[k] : acc[k + sft];
+                                acc[k] = keep + __shfl_xor_sync(0xffffffffu, send, sft);
+                            }
+                        }
+                        sd[i] = acc[0];
+                    }
+                }
             }
             float mref = -INFINITY, l = 0.f;
             for (int j = 0; j <= qt; ++j, ++g) {
@@ -293,40 +330,48 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 const bool diag = (j == qt);
                 const bool subst = p.m > 0 && j + 1 >= qt;    // tiles that can hold substituted entries (m <= 128)
                 const int col_base = j * KT;
-                // masks the diagonal tile and overwrites the substituted entries of a 32-column chunk
-                auto fix = [&](float (&v)[32], int c0) {
-                    if (diag) {
+                // the whole row of S into registers, then the S buffer goes back to the tensor core
+                uint32_t raw[4][32];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) tmem_ld32(tmem_s + 32 * k, raw[k]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty(s));
+                float v[4][32];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) v[k][c] = __uint_as_float(raw[k][c]);
+                    // causal mask of the diagonal tile: chunk k against this warp's 32 rows
+                    if (diag && k >= quad) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c0 + c > r) v[c] = -INFINITY;
+                            if (k > quad || c > lane) v[k][c] = -INFINITY;
                     }
                     if (subst) {
 #pragma unroll
                         for (int i = 0; i < MAX_DRAFTS; ++i) {
-                            const int cs = t - i - col_base - c0;
+                            const int cs = t - i - col_base - 32 * k;
                             if (i < p.m && cs >= 0 && cs < 32) {
 #pragma unroll
                                 for (int c = 0; c < 32; ++c)
-                                    if (c == cs) v[c] = sd[i];
+                                    if (c == cs) v[k][c] = sd[i];
                             }
                         }
                     }
-                };
-                // ---- pass 1: row maximum ----
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c0 = 0; c0 < KT; c0 += 32) {
-                    uint32_t raw[32];
-                    tmem_ld32(tmem_s + c0, raw);
-                    tmem_ld_wait(raw);
-                    float v[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(raw[c]);
-                    fix(v, c0);
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) mx = fmax3(mx, v[c], v[c + 1]);
                 }
-                const float cand = mx * p.c2;
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        mx0 = fmax3(mx0, v[k][c], v[k][c + 1]);
+                        mx1 = fmax3(mx1, v[k][c + 2], v[k][c + 3]);
+                    }
+                }
+                const float cand = fmaxf(mx0, mx1) * p.c2;
                 if (j == 0) {
                     mref = cand;
                 } else {
@@ -343,66 +388,60 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                         tc_fence_after_sync();
 #pragma unroll 1
                         for (int c0 = 0; c0 < HD; c0 += 32) {
-                            uint32_t raw[32];
-                            tmem_ld32(tmem_o + c0, raw);
-                            tmem_ld_wait(raw);
+                            uint32_t o[32];
+                            tmem_ld32(tmem_o + c0, o);
+                            tmem_ld_wait(o);
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) raw[c] = __float_as_uint(__uint_as_float(raw[c]) * f);
-                            tmem_st32(tmem_o + c0, raw);
+                            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * f);
+                            tmem_st32(tmem_o + c0, o);
                         }
                         tmem_st_wait();
+                        tc_fence_before_sync();
                     }
                 }
-                // ---- pass 2: P = 2^(x c2 - ref) as bf16 into shared memory; row sum in fp32 ----
-                if (!wait_barrier(pv_done(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // PV(g-2) has read P[s]
-                const uint32_t p_row = base + SMEM_P + s * TILE_BYTES + r * 128;
+                // ---- P = 2^(x c2 - ref): row sum in fp32, bf16 into shared memory ----
                 const float nref = -mref;
-#pragma unroll 1
-                for (int c0 = 0; c0 < KT; c0 += 32) {
-                    uint32_t raw[32];
-                    tmem_ld32(tmem_s + c0, raw);
-                    tmem_ld_wait(raw);
-                    float v[32];
+                float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(raw[c]);
-                    fix(v, c0);
-                    float ls0 = 0.f, ls1 = 0.f;
+                for (int k = 0; k < 4; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        v[c] = ex2(fmaf(v[c], p.c2, nref));
-                        v[c + 1] = ex2(fmaf(v[c + 1], p.c2, nref));
-                        ls0 += v[c];
-                        ls1 += v[c + 1];
+                        float x0, x1;
+                        ffma2(x0, x1, v[k][c], v[k][c + 1], p.c2, p.c2, nref, nref);
+                        v[k][c] = ex2(x0);
+                        v[k][c + 1] = ex2(x1);
+                        fadd2(ls0, ls1, ls0, ls1, v[k][c], v[k][c + 1]);
                     }
-                    l += ls0 + ls1;
                     if (subst) {
                         // substituted entries meet the draft pass's value row in the epilogue, not V_t here
 #pragma unroll
                         for (int i = 0; i < MAX_DRAFTS; ++i) {
-                            const int cs = t - i - col_base - c0;
+                            const int cs = t - i - col_base - 32 * k;
                             if (i < p.m && cs >= 0 && cs < 32) {
 #pragma unroll
                                 for (int c = 0; c < 32; ++c)
-                                    if (c == cs) v[c] = 0.f;
+                                    if (c == cs) v[k][c] = 0.f;
                             }
                         }
                     }
-                    const uint32_t half = p_row + (c0 >> 6) * HALF_BYTES;
+                }
+                l += ls0 + ls1;
+                if (!wait_barrier(pv_done(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // PV(g-2) has read P[s]
+                const uint32_t p_row = base + SMEM_P + s * TILE_BYTES + r * 128;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t half = p_row + (k >> 1) * HALF_BYTES;
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
-                        const int chunk = ((c0 & 63) >> 3) + q4;           // 16-byte unit inside the 128-byte row
-                        st_shared_v4(half + (((chunk ^ (r & 7)) & 7) << 4), pack_bf16(v[8 * q4], v[8 * q4 + 1]),
-                                     pack_bf16(v[8 * q4 + 2], v[8 * q4 + 3]), pack_bf16(v[8 * q4 + 4], v[8 * q4 + 5]),
-                                     pack_bf16(v[8 * q4 + 6], v[8 * q4 + 7]));
+                        const int chunk = (k & 1) * 4 + q4;                // 16-byte unit inside the 128-byte row
+                        st_shared_v4(half + (((chunk ^ (r & 7)) & 7) << 4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
+                                     pack_bf16(v[k][8 * q4 + 2], v[k][8 * q4 + 3]), pack_bf16(v[k][8 * q4 + 4], v[k][8 * q4 + 5]),
+                                     pack_bf16(v[k][8 * q4 + 6], v[k][8 * q4 + 7]));
                     }
                 }
-                tc_fence_before_sync();        // S reads (and any O rescale) ordered before the arrivals
                 fence_proxy_async_smem();      // P visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(s_empty(s));
-                    mbar_arrive(p_full(s));
-                }
+                if (lane == 0) mbar_arrive(p_full(s));
             }
             if (!ok) break;
             // ---- epilogue: O / l, plus the substituted entries' weight times the draft value rows ----
@@ -415,50 +454,65 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
 #pragma unroll
                 for (int i = 0; i < MAX_DRAFTS; ++i)
                     pd[i] = (i < p.m && valid && t - i >= 0) ? ex2(fmaf(sd[i], p.c2, -mref)) * inv : 0.f;
-                __nv_bfloat16* orow = p.O + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
-#pragma unroll 1
-                for (int c0 = 0; c0 < HD; c0 += 32) {
-                    uint32_t raw[32];
-                    tmem_ld32(tmem_o + c0, raw);
-                    tmem_ld_wait(raw);
-                    float v[32];
+                if (valid && p.lse != nullptr)
+                    p.lse[(static_cast<size_t>(b) * p.H + h) * p.T + t] = (mref + log2f(l)) * 0.6931471805599453f;
+                // Stage this warp's 32 rows of O (fp32, normalised) in shared memory. Both PV products that read
+                // the P buffers are complete, and the bytes used are exactly this warp's own rows of the two
+                // P buffers (4 pieces of 128 bytes per row), which no other warp writes.
+                auto piece = [&](int rr, int k) {   // 128-byte piece k (columns 32k .. 32k+31) of row rr of this warp
+                    return base + SMEM_P + (k >> 1) * TILE_BYTES + (k & 1) * HALF_BYTES + (quad * 32 + rr) * 128;
+                };
+                {
+                    uint32_t raw[4][32];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(raw[c]) * inv;
+                    for (int k = 0; k < 4; ++k) tmem_ld32(tmem_o + 32 * k, raw[k]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(o_free);     // the accumulator may be overwritten by the next item
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                        for (int c8 = 0; c8 < 8; ++c8)
+                            st_shared_v4(piece(lane, k) + (((c8 ^ lane) & 7) << 4),
+                                         __float_as_uint(__uint_as_float(raw[k][4 * c8]) * inv),
+                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 1]) * inv),
+                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 2]) * inv),
+                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 3]) * inv));
+                    }
+                }
+                __syncwarp();
+                // row by row with the warp across the 128 columns (lane = 4 columns): coalesced reads of the draft
+                // value rows and coalesced stores of O
+                const int kq = lane >> 3, cq = lane & 7;
+#pragma unroll 4
+                for (int rr = 0; rr < 32; ++rr) {
+                    const int tr = t_warp + rr;
+                    float4 o;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
+                                 : "r"(piece(rr, kq) + (((cq ^ rr) & 7) << 4)));
 #pragma unroll
                     for (int i = 0; i < MAX_DRAFTS; ++i) {
-                        if (pd[i] != 0.f) {
-                            const uint4* vr = reinterpret_cast<const uint4*>(
-                                p.V_d[i] + ((static_cast<size_t>(b) * p.T + (t - i)) * p.Hkv + gkv) * HD + c0);
-#pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4) {
-                                const uint4 w = __ldg(vr + q4);
-                                v[8 * q4 + 0] = fmaf(pd[i], bf16_lo(w.x), v[8 * q4 + 0]);
-                                v[8 * q4 + 1] = fmaf(pd[i], bf16_hi(w.x), v[8 * q4 + 1]);
-                                v[8 * q4 + 2] = fmaf(pd[i], bf16_lo(w.y), v[8 * q4 + 2]);
-                                v[8 * q4 + 3] = fmaf(pd[i], bf16_hi(w.y), v[8 * q4 + 3]);
-                                v[8 * q4 + 4] = fmaf(pd[i], bf16_lo(w.z), v[8 * q4 + 4]);
-                                v[8 * q4 + 5] = fmaf(pd[i], bf16_hi(w.z), v[8 * q4 + 5]);
-                                v[8 * q4 + 6] = fmaf(pd[i], bf16_lo(w.w), v[8 * q4 + 6]);
-                                v[8 * q4 + 7] = fmaf(pd[i], bf16_hi(w.w), v[8 * q4 + 7]);
+                        if (i < p.m) {
+                            const float w = __shfl_sync(0xffffffffu, pd[i], rr);
+                            if (w != 0.f) {
+                                const uint2 vv = __ldg(reinterpret_cast<const uint2*>(
+                                                           p.V_d[i] + ((static_cast<size_t>(b) * p.T + (tr - i)) * p.Hkv + gkv) * HD) + lane);
+                                o.x = fmaf(w, bf16_lo(vv.x), o.x);
+                                o.y = fmaf(w, bf16_hi(vv.x), o.y);
+                                o.z = fmaf(w, bf16_lo(vv.y), o.z);
+                                o.w = fmaf(w, bf16_hi(vv.y), o.w);
                             }
                         }
                     }
-                    if (valid) {
-#pragma unroll
-                        for (int q8 = 0; q8 < 2; ++q8)
-                            st_global_v8(orow + c0 + 16 * q8, pack_bf16(v[16 * q8], v[16 * q8 + 1]),
-                                         pack_bf16(v[16 * q8 + 2], v[16 * q8 + 3]), pack_bf16(v[16 * q8 + 4], v[16 * q8 + 5]),
-                                         pack_bf16(v[16 * q8 + 6], v[16 * q8 + 7]), pack_bf16(v[16 * q8 + 8], v[16 * q8 + 9]),
-                                         pack_bf16(v[16 * q8 + 10], v[16 * q8 + 11]),
-                                         pack_bf16(v[16 * q8 + 12], v[16 * q8 + 13]),
-                                         pack_bf16(v[16 * q8 + 14], v[16 * q8 + 15]));
+                    if (tr < p.T) {
+                        uint2 outv = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
+                        *(reinterpret_cast<uint2*>(p.O + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane) = outv;
                     }
                 }
-                if (valid && p.lse != nullptr)
-                    p.lse[(static_cast<size_t>(b) * p.H + h) * p.T + t] = (mref + log2f(l)) * 0.6931471805599453f;
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);
+                __syncwarp();      // the staging bytes are this warp's P rows of the next tiles
             }
         }
     }
