@@ -3,14 +3,15 @@
 // One persistent, warp-specialised kernel. A work item is one (sequence, query head, tile of 128
 // query positions); it sweeps the key tiles 0 .. its own (causal). Per key tile:
 //   S = Q K_t^T            tcgen05.mma, 128 x 128 x 128, fp32 in TMEM (two S buffers)
-//   softmax warps          read S (one query row per thread), mask the diagonal tile, overwrite
-//                          the entries (t, t - i), i < m, with the score against the i-th draft
-//                          pass's key (a 128-long dot product the thread computed itself), update
-//                          the row's running reference and sum, write P = 2^(x - ref) as bf16 into
-//                          shared memory in the swizzled layout the tensor core reads
+//   softmax warps          read S (one query row per thread), hide the columns past t - m (the causal
+//                          part and the m substituted entries), update the row's running reference
+//                          and sum, write P = 2^(x - ref) as bf16 into shared memory in the swizzled
+//                          layout the tensor core reads
 //   O += P V_t             tcgen05.mma with V_t as an MN-major operand, fp32 in TMEM
-// The substituted entries are written as zeros into P; their weight times the draft pass's value
-// row is added by the row's thread in the epilogue, which also divides by the row sum.
+// The substituted entries (t, t - i), i < m, never pass through the tensor core: their scores against
+// the i-th draft pass's keys are 128-long dot products the softmax warps compute up front (coalesced,
+// one warp per 32 rows); they join the row maximum and sum at the diagonal tile, and their weight times
+// the draft pass's value row is added in the epilogue, which also divides by the row sum.
 // The running reference moves only when a tile's maximum exceeds it by more than 2^8 (the O
 // accumulator in TMEM is then rescaled in place by the softmax warps), so P stays within bf16
 // range and most tiles skip the rescale.
@@ -285,23 +286,24 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 uint2 qv[32];
 #pragma unroll
                 for (int rr = 0; rr < 32; ++rr) {
-                    const int tr = t_warp + rr;
-                    qv[rr] = make_uint2(0u, 0u);
-                    if (tr < p.T)
-                        qv[rr] = __ldg(reinterpret_cast<const uint2*>(
-                                           p.Q + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane);
+                    int tr = t_warp + rr;
+                    tr = tr >= p.T ? p.T - 1 : tr;
+                    qv[rr] = __ldg(reinterpret_cast<const uint2*>(
+                                       p.Q + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane);
                 }
-#pragma unroll
-                for (int i = 0; i < MAX_DRAFTS; ++i) {
-                    if (i < p.m) {
+#pragma unroll 1
+                for (int i = 0; i < p.m; ++i) {
+                    {
                         float acc[32];
+                        const __nv_bfloat16* kd = p.K_d[i];
 #pragma unroll
                         for (int rr = 0; rr < 32; ++rr) {
-                            const int tr = t_warp + rr;
-                            uint2 kv = make_uint2(0u, 0u);
-                            if (tr < p.T && tr - i >= 0)
-                                kv = __ldg(reinterpret_cast<const uint2*>(
-                                               p.K_d[i] + ((static_cast<size_t>(b) * p.T + (tr - i)) * p.Hkv + gkv) * HD) + lane);
+                            // rows outside the sequence read a clamped row (no branch around the load); their
+                            // result is never used
+                            int ts = t_warp + rr - i;
+                            ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
+                            const uint2 kv = __ldg(reinterpret_cast<const uint2*>(
+                                                       kd + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
                             acc[rr] = fmaf(bf16_lo(qv[rr].x), bf16_lo(kv.x),
                                            fmaf(bf16_hi(qv[rr].x), bf16_hi(kv.x),
                                                 fmaf(bf16_lo(qv[rr].y), bf16_lo(kv.y), bf16_hi(qv[rr].y) * bf16_hi(kv.y))));
@@ -316,7 +318,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                                 acc[k] = keep + __shfl_xor_sync(0xffffffffu, send, sft);
                             }
                         }
-                        sd[i] = acc[0];
+#pragma unroll
+                        for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                            if (ii == i) sd[ii] = acc[0];
                     }
                 }
             }
@@ -328,8 +332,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 tc_fence_after_sync();
                 const uint32_t tmem_s = tmem_base + s * KT + lane_addr;
                 const bool diag = (j == qt);
-                const bool subst = p.m > 0 && j + 1 >= qt;    // tiles that can hold substituted entries (m <= 128)
-                const int col_base = j * KT;
+                // Columns past t - m are hidden in the score tile: the causal part (s > t) and the m substituted
+                // entries (t - m < s <= t), which enter the row's maximum and sum as scalars at the diagonal tile
+                // and meet their value rows in the epilogue. Only the last two tiles can hold such columns.
+                const bool band = diag || (p.m > 0 && j + 1 == qt);
+                const int lim = t - p.m - j * KT;
                 // the whole row of S into registers, then the S buffer goes back to the tensor core
                 uint32_t raw[4][32];
 #pragma unroll
@@ -344,22 +351,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 for (int k = 0; k < 4; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) v[k][c] = __uint_as_float(raw[k][c]);
-                    // causal mask of the diagonal tile: chunk k against this warp's 32 rows
-                    if (diag && k >= quad) {
+                    if (band) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (k > quad || c > lane) v[k][c] = -INFINITY;
-                    }
-                    if (subst) {
-#pragma unroll
-                        for (int i = 0; i < MAX_DRAFTS; ++i) {
-                            const int cs = t - i - col_base - 32 * k;
-                            if (i < p.m && cs >= 0 && cs < 32) {
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == cs) v[k][c] = sd[i];
-                            }
-                        }
+                            if (32 * k + c > lim) v[k][c] = -INFINITY;
                     }
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY;
@@ -370,6 +365,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                         mx0 = fmax3(mx0, v[k][c], v[k][c + 1]);
                         mx1 = fmax3(mx1, v[k][c + 2], v[k][c + 3]);
                     }
+                }
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < MAX_DRAFTS; ++i)
+                        if (i < p.m && t - i >= 0) mx0 = fmaxf(mx0, sd[i]);
                 }
                 const float cand = fmaxf(mx0, mx1) * p.c2;
                 if (j == 0) {
@@ -412,20 +412,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                         v[k][c + 1] = ex2(x1);
                         fadd2(ls0, ls1, ls0, ls1, v[k][c], v[k][c + 1]);
                     }
-                    if (subst) {
-                        // substituted entries meet the draft pass's value row in the epilogue, not V_t here
-#pragma unroll
-                        for (int i = 0; i < MAX_DRAFTS; ++i) {
-                            const int cs = t - i - col_base - 32 * k;
-                            if (i < p.m && cs >= 0 && cs < 32) {
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == cs) v[k][c] = 0.f;
-                            }
-                        }
-                    }
                 }
                 l += ls0 + ls1;
+                if (diag) {
+#pragma unroll
+                    for (int i = 0; i < MAX_DRAFTS; ++i)
+                        if (i < p.m && t - i >= 0) l += ex2(fmaf(sd[i], p.c2, nref));
+                }
                 if (!wait_barrier(pv_done(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // PV(g-2) has read P[s]
                 const uint32_t p_row = base + SMEM_P + s * TILE_BYTES + r * 128;
 #pragma unroll
@@ -486,26 +479,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 // row by row with the warp across the 128 columns (lane = 4 columns): coalesced reads of the draft
                 // value rows and coalesced stores of O
                 const int kq = lane >> 3, cq = lane & 7;
-#pragma unroll 4
+#pragma unroll 2
                 for (int rr = 0; rr < 32; ++rr) {
                     const int tr = t_warp + rr;
                     float4 o;
                     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                  : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
                                  : "r"(piece(rr, kq) + (((cq ^ rr) & 7) << 4)));
+#pragma unroll 1
+                    for (int i = 0; i < p.m; ++i) {
+                        float pdi = 0.f;
 #pragma unroll
-                    for (int i = 0; i < MAX_DRAFTS; ++i) {
-                        if (i < p.m) {
-                            const float w = __shfl_sync(0xffffffffu, pd[i], rr);
-                            if (w != 0.f) {
-                                const uint2 vv = __ldg(reinterpret_cast<const uint2*>(
-                                                           p.V_d[i] + ((static_cast<size_t>(b) * p.T + (tr - i)) * p.Hkv + gkv) * HD) + lane);
-                                o.x = fmaf(w, bf16_lo(vv.x), o.x);
-                                o.y = fmaf(w, bf16_hi(vv.x), o.y);
-                                o.z = fmaf(w, bf16_lo(vv.y), o.z);
-                                o.w = fmaf(w, bf16_hi(vv.y), o.w);
-                            }
-                        }
+                        for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                            if (ii == i) pdi = pd[ii];
+                        const float w = __shfl_sync(0xffffffffu, pdi, rr);    // 0 where the entry does not exist
+                        int ts = tr - i;
+                        ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
+                        const uint2 vv = __ldg(reinterpret_cast<const uint2*>(
+                                                   p.V_d[i] + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
+                        o.x = fmaf(w, bf16_lo(vv.x), o.x);
+                        o.y = fmaf(w, bf16_hi(vv.x), o.y);
+                        o.z = fmaf(w, bf16_lo(vv.y), o.z);
+                        o.w = fmaf(w, bf16_hi(vv.y), o.w);
                     }
                     if (tr < p.T) {
                         uint2 outv = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
