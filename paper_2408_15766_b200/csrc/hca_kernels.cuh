@@ -84,6 +84,9 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ void prefetch_l2(const void* ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -282,6 +285,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             float sd[MAX_DRAFTS];
 #pragma unroll
             for (int i = 0; i < MAX_DRAFTS; ++i) sd[i] = 0.f;
+            if (p.m > 0 && item + static_cast<int>(gridDim.x) < p.items) {
+                // pull the draft rows of this CTA's next item towards L2 while this item is processed
+                int qt2, b2, h2;
+                decode(item + gridDim.x, qt2, b2, h2);
+                const int g2 = h2 / rep;
+#pragma unroll 1
+                for (int i = 0; i < p.m; ++i) {
+                    int ts = qt2 * QT + r - i;
+                    ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
+                    const size_t off = ((static_cast<size_t>(b2) * p.T + ts) * p.Hkv + g2) * HD;
+                    prefetch_l2(p.K_d[i] + off);
+                    prefetch_l2(p.K_d[i] + off + 64);
+                    prefetch_l2(p.V_d[i] + off);
+                    prefetch_l2(p.V_d[i] + off + 64);
+                }
+            }
             if (p.m > 0) {
                 uint2 qv[32];
 #pragma unroll
@@ -479,32 +498,44 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 // row by row with the warp across the 128 columns (lane = 4 columns): coalesced reads of the draft
                 // value rows and coalesced stores of O
                 const int kq = lane >> 3, cq = lane & 7;
-#pragma unroll 2
-                for (int rr = 0; rr < 32; ++rr) {
-                    const int tr = t_warp + rr;
-                    float4 o;
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                 : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
-                                 : "r"(piece(rr, kq) + (((cq ^ rr) & 7) << 4)));
+#pragma unroll 1
+                for (int rr0 = 0; rr0 < 32; rr0 += 16) {
+                    float4 o[16];
+#pragma unroll
+                    for (int u = 0; u < 16; ++u)
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(o[u].x), "=f"(o[u].y), "=f"(o[u].z), "=f"(o[u].w)
+                                     : "r"(piece(rr0 + u, kq) + (((cq ^ (rr0 + u)) & 7) << 4)));
 #pragma unroll 1
                     for (int i = 0; i < p.m; ++i) {
                         float pdi = 0.f;
 #pragma unroll
                         for (int ii = 0; ii < MAX_DRAFTS; ++ii)
                             if (ii == i) pdi = pd[ii];
-                        const float w = __shfl_sync(0xffffffffu, pdi, rr);    // 0 where the entry does not exist
-                        int ts = tr - i;
-                        ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
-                        const uint2 vv = __ldg(reinterpret_cast<const uint2*>(
-                                                   p.V_d[i] + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
-                        o.x = fmaf(w, bf16_lo(vv.x), o.x);
-                        o.y = fmaf(w, bf16_hi(vv.x), o.y);
-                        o.z = fmaf(w, bf16_lo(vv.y), o.z);
-                        o.w = fmaf(w, bf16_hi(vv.y), o.w);
+                        const __nv_bfloat16* vd = p.V_d[i];
+                        uint2 vv[16];
+#pragma unroll
+                        for (int u = 0; u < 16; ++u) {
+                            int ts = t_warp + rr0 + u - i;
+                            ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
+                            vv[u] = __ldg(reinterpret_cast<const uint2*>(
+                                              vd + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 16; ++u) {
+                            const float w = __shfl_sync(0xffffffffu, pdi, rr0 + u);    // 0 where the entry does not exist
+                            o[u].x = fmaf(w, bf16_lo(vv[u].x), o[u].x);
+                            o[u].y = fmaf(w, bf16_hi(vv[u].x), o[u].y);
+                            o[u].z = fmaf(w, bf16_lo(vv[u].y), o[u].z);
+                            o[u].w = fmaf(w, bf16_hi(vv[u].y), o[u].w);
+                        }
                     }
-                    if (tr < p.T) {
-                        uint2 outv = make_uint2(pack_bf16(o.x, o.y), pack_bf16(o.z, o.w));
-                        *(reinterpret_cast<uint2*>(p.O + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane) = outv;
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) {
+                        const int tr = t_warp + rr0 + u;
+                        if (tr < p.T)
+                            *(reinterpret_cast<uint2*>(p.O + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane) =
+                                make_uint2(pack_bf16(o[u].x, o[u].y), pack_bf16(o[u].z, o[u].w));
                     }
                 }
                 __syncwarp();      // the staging bytes are this warp's P rows of the next tiles
