@@ -175,12 +175,13 @@ static int make_tmap(CUtensorMap* tm, const void* base, long long rows, long lon
     return r == CUDA_SUCCESS ? HASS_OK : HASS_ERR_CUDA;
 }
 
-// bf16 tensor [B, T, heads * 128] (dense): box = 64 columns x 128 positions of one sequence, 128-byte
+// bf16 tensor [B, T, heads * 128] (dense): box = 64 columns x box_rows positions of one sequence, 128-byte
 // swizzle. Positions past T read as zeros, so a ragged last tile never sees the next sequence.
-static int make_tmap_seq(CUtensorMap* tm, const void* base, long long B, long long T, long long cols) {
+static int make_tmap_seq(CUtensorMap* tm, const void* base, long long B, long long T, long long cols,
+                         int box_rows = 128) {
     cuuint64_t gdim[3] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(B)};
     cuuint64_t gstride[2] = {static_cast<cuuint64_t>(cols) * 2, static_cast<cuuint64_t>(cols) * 2 * static_cast<cuuint64_t>(T)};
-    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1208,12 +1209,12 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
     if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca::HD);
     if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca::HD);
     if (rc != HASS_OK) return rc;
-    p.Q = static_cast<const __nv_bfloat16*>(Q);
-    for (int i = 0; i < m; ++i) {
-        p.K_d[i] = static_cast<const __nv_bfloat16*>(K_d[i]);
-        p.V_d[i] = static_cast<const __nv_bfloat16*>(V_d[i]);
+    for (int i = 0; i < m && rc == HASS_OK; ++i) {
+        rc = make_tmap_seq(&p.tmKd[i], K_d[i], B, T, Hkv * hca::HD);
+        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmVd[i], V_d[i], B, T, Hkv * hca::HD);
     }
-    p.O = static_cast<__nv_bfloat16*>(O);
+    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmO, O, B, T, H * hca::HD, 32);
+    if (rc != HASS_OK) return rc;
     p.lse = lse;
     p.B = static_cast<int>(B);
     p.T = static_cast<int>(T);

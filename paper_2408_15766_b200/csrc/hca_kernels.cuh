@@ -8,10 +8,15 @@
 //                          and sum, write P = 2^(x - ref) as bf16 into shared memory in the swizzled
 //                          layout the tensor core reads
 //   O += P V_t             tcgen05.mma with V_t as an MN-major operand, fp32 in TMEM
-// The substituted entries (t, t - i), i < m, never pass through the tensor core: their scores against
-// the i-th draft pass's keys are 128-long dot products the softmax warps compute up front (coalesced,
-// one warp per 32 rows); they join the row maximum and sum at the diagonal tile, and their weight times
-// the draft pass's value row is added in the epilogue, which also divides by the row sum.
+// The substituted entries (t, t - i), i < m, ride the same pipeline as extra tiles of the item:
+//   before the key tiles   S_i = Q K_d[i]^T with the K_d[i] tile fetched i rows early, so that the
+//                          wanted scores <Q[t], K_d[i][t - i]> sit on the tile's main diagonal; each
+//                          softmax thread keeps its diagonal element
+//   at the diagonal tile   the m scores join the row maximum and sum
+//   after the key tiles    O += diag(p_i) V_d[i], V_d[i] again fetched i rows early and the P buffer
+//                          holding just the weights on its diagonal
+// so no thread reads global memory; the epilogue divides by the row sum, stages bf16 rows in shared
+// memory and stores them with TMA.
 // The running reference moves only when a tile's maximum exceeds it by more than 2^8 (the O
 // accumulator in TMEM is then rescaled in place by the softmax warps), so P stays within bf16
 // range and most tiles skip the rescale.
@@ -46,10 +51,9 @@ constexpr float RESCALE_LOG2 = 8.f;
 
 struct Params {
     CUtensorMap tmQ, tmK, tmV;     // 3-D maps {heads * 128, T, B}, box {64, 128, 1}, 128-byte swizzle
-    const __nv_bfloat16* Q;        // [B, T, H, 128]
-    const __nv_bfloat16* K_d[MAX_DRAFTS];   // [B, T, Hkv, 128] each; index = sub-diagonal
-    const __nv_bfloat16* V_d[MAX_DRAFTS];
-    __nv_bfloat16* O;              // [B, T, H, 128]
+    CUtensorMap tmKd[MAX_DRAFTS];  // the draft passes' keys and values, same geometry; index = sub-diagonal
+    CUtensorMap tmVd[MAX_DRAFTS];
+    CUtensorMap tmO;               // O [B, T, H * 128], box {64, 32, 1}: one warp's rows of half a tile
     float* lse;                    // [B, H, T] or null
     int B, T, H, Hkv, m;
     int q_tiles;                   // ceil(T / 128)
@@ -84,9 +88,16 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void prefetch_l2(const void* ptr) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+// Tiled store shared -> global (rows past the tensor's extent are clipped), tracked by bulk groups.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t smem_src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(tm)),
+                 "r"(smem_src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
 }
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -96,26 +107,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-// Dot product of two 128-element bf16 rows (16-byte aligned), fp32 accumulation.
-__device__ __forceinline__ float dot128(const __nv_bfloat16* a, const __nv_bfloat16* b) {
-    const uint4* pa = reinterpret_cast<const uint4*>(a);
-    const uint4* pb = reinterpret_cast<const uint4*>(b);
-    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-        const uint4 x = __ldg(pa + i), y = __ldg(pb + i);
-        acc0 = fmaf(bf16_lo(x.x), bf16_lo(y.x), acc0);
-        acc1 = fmaf(bf16_hi(x.x), bf16_hi(y.x), acc1);
-        acc0 = fmaf(bf16_lo(x.y), bf16_lo(y.y), acc0);
-        acc1 = fmaf(bf16_hi(x.y), bf16_hi(y.y), acc1);
-        acc0 = fmaf(bf16_lo(x.z), bf16_lo(y.z), acc0);
-        acc1 = fmaf(bf16_hi(x.z), bf16_hi(y.z), acc1);
-        acc0 = fmaf(bf16_lo(x.w), bf16_lo(y.w), acc0);
-        acc1 = fmaf(bf16_hi(x.w), bf16_hi(y.w), acc1);
-    }
-    return acc0 + acc1;
-}
 
 __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __grid_constant__ Params p) {
     extern __shared__ uint8_t smem_raw[];
@@ -159,6 +150,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         prefetch_tensormap(&p.tmQ);
         prefetch_tensormap(&p.tmK);
         prefetch_tensormap(&p.tmV);
+        prefetch_tensormap(&p.tmO);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_ptr_smem), TMEM_COLS);
@@ -171,6 +163,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
 
     const int BH = p.B * p.H;
     const int rep = p.H / p.Hkv;
+    const int m = p.m;
     // item -> (query tile, sequence, head): the longest items (last query tiles) come first
     auto decode = [&](int item, int& qt, int& b, int& h) {
         qt = p.q_tiles - 1 - item / BH;
@@ -178,33 +171,48 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         b = bh / p.H;
         h = bh - b * p.H;
     };
+    // Per item the tensor core runs two sequences, each with its own ring counter:
+    //   score sequence (K ring, S buffers), length m + qt + 1: draft pass 0 .. m-1, then key tiles 0 .. qt
+    //   value sequence (V ring, P buffers), length qt + 1 + m: key tiles 0 .. qt, then draft pass 0 .. m-1
 
     if (warp == 0) {
         // ===================== TMA producer =====================
         if (lane == 0) {
-            uint32_t g = 0, it = 0;    // key tiles and items done by this CTA
-            for (int item = blockIdx.x; item < p.items; item += gridDim.x, ++it) {
+            uint32_t gk = 0, gv = 0, it = 0;
+            bool ok = true;
+            auto load_k = [&](const CUtensorMap* tm, int col, int row, int b) -> bool {
+                const int s = gk & 1u;
+                if (!wait_barrier(k_empty(s), ((gk >> 1) & 1u) ^ 1u, abort_flag, p.status, 2)) return false;
+                mbar_arrive_expect_tx(k_full(s), TILE_BYTES);
+                tma_load_3d(base + SMEM_K + s * TILE_BYTES, tm, k_full(s), col, row, b);
+                tma_load_3d(base + SMEM_K + s * TILE_BYTES + HALF_BYTES, tm, k_full(s), col + 64, row, b);
+                ++gk;
+                return true;
+            };
+            auto load_v = [&](const CUtensorMap* tm, int col, int row, int b) -> bool {
+                const int s = gv & 1u;
+                if (!wait_barrier(v_empty(s), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 3)) return false;
+                mbar_arrive_expect_tx(v_full(s), TILE_BYTES);
+                tma_load_3d(base + SMEM_V + s * TILE_BYTES, tm, v_full(s), col, row, b);
+                tma_load_3d(base + SMEM_V + s * TILE_BYTES + HALF_BYTES, tm, v_full(s), col + 64, row, b);
+                ++gv;
+                return true;
+            };
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
                 int qt, b, h;
                 decode(item, qt, b, h);
-                const int gkv = h / rep;
+                const int col = (h / rep) * HD;
                 if (!wait_barrier(q_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1)) break;
                 mbar_arrive_expect_tx(q_full, TILE_BYTES);
                 tma_load_3d(base + SMEM_Q, &p.tmQ, q_full, h * HD, qt * QT, b);
                 tma_load_3d(base + SMEM_Q + HALF_BYTES, &p.tmQ, q_full, h * HD + 64, qt * QT, b);
-                bool ok = true;
-                for (int j = 0; j <= qt; ++j, ++g) {
-                    const int s = g & 1u;
-                    const uint32_t ph = (g >> 1) & 1u;
-                    if (!wait_barrier(k_empty(s), ph ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
-                    mbar_arrive_expect_tx(k_full(s), TILE_BYTES);
-                    tma_load_3d(base + SMEM_K + s * TILE_BYTES, &p.tmK, k_full(s), gkv * HD, j * KT, b);
-                    tma_load_3d(base + SMEM_K + s * TILE_BYTES + HALF_BYTES, &p.tmK, k_full(s), gkv * HD + 64, j * KT, b);
-                    if (!wait_barrier(v_empty(s), ph ^ 1u, abort_flag, p.status, 3)) { ok = false; break; }
-                    mbar_arrive_expect_tx(v_full(s), TILE_BYTES);
-                    tma_load_3d(base + SMEM_V + s * TILE_BYTES, &p.tmV, v_full(s), gkv * HD, j * KT, b);
-                    tma_load_3d(base + SMEM_V + s * TILE_BYTES + HALF_BYTES, &p.tmV, v_full(s), gkv * HD + 64, j * KT, b);
+                // draft keys start i rows early: row r of the tile is position qt*128 + r - i (zeros before the sequence)
+                for (int i = 0; i < m && ok; ++i) ok = load_k(&p.tmKd[i], col, qt * QT - i, b);
+                for (int j = 0; j <= qt && ok; ++j) {
+                    ok = load_k(&p.tmK, col, j * KT, b);
+                    if (ok) ok = load_v(&p.tmV, col, j * KT, b);
                 }
-                if (!ok) break;
+                for (int i = 0; i < m && ok; ++i) ok = load_v(&p.tmVd[i], col, qt * QT - i, b);
             }
         }
     } else if (warp == 1) {
@@ -213,12 +221,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
             constexpr uint32_t idesc_o = make_idesc_bf16(QT, HD, 0, 1);
             const uint32_t tmem_o = tmem_base + 2 * KT;
-            uint32_t g = 0, it = 0;
+            uint32_t gk = 0, gv = 0, it = 0;
             bool ok = true;
-            // S(g) = Q K^T into S buffer g & 1
-            auto issue_s = [&](uint32_t gg) -> bool {
-                const int s = gg & 1u;
-                const uint32_t ph = (gg >> 1) & 1u;
+            // next element of the score sequence: S = Q K^T into S buffer gk & 1
+            auto issue_s = [&]() -> bool {
+                const int s = gk & 1u;
+                const uint32_t ph = (gk >> 1) & 1u;
                 if (!wait_barrier(k_full(s), ph, abort_flag, p.status, 4)) return false;
                 if (!wait_barrier(s_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
                 tc_fence_after_sync();
@@ -231,37 +239,46 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 }
                 umma_commit(k_empty(s));
                 umma_commit(s_full(s));
+                ++gk;
+                return true;
+            };
+            // next element of the value sequence: O (+)= P V
+            auto issue_pv = [&](bool first) -> bool {
+                const int s = gv & 1u;
+                const uint32_t ph = (gv >> 1) & 1u;
+                if (!wait_barrier(p_full(s), ph, abort_flag, p.status, 7)) return false;
+                if (!wait_barrier(v_full(s), ph, abort_flag, p.status, 8)) return false;
+                if (first && !wait_barrier(o_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < KT / 16; ++k) {
+                    // A = P: K-major halves of 64 keys. B = V: 16 keys further = 16 rows of 128 bytes.
+                    const uint64_t a_desc = make_smem_desc_sw128(
+                        base + SMEM_P + s * TILE_BYTES + (k >> 2) * HALF_BYTES + (k & 3) * 32, 0, 1024);
+                    const uint64_t b_desc =
+                        make_smem_desc_sw128(base + SMEM_V + s * TILE_BYTES + k * 16 * 128, HALF_BYTES, 1024);
+                    umma_bf16(tmem_o, a_desc, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
+                }
+                umma_commit(v_empty(s));
+                umma_commit(pv_done(s));
+                ++gv;
                 return true;
             };
             for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
                 int qt, b, h;
                 decode(item, qt, b, h);
+                const int n_s = m + qt + 1;
                 if (!wait_barrier(q_full, it & 1u, abort_flag, p.status, 6)) break;
-                if (!issue_s(g)) break;
-                if (qt == 0) umma_commit(q_empty);
-                for (int j = 0; j <= qt; ++j, ++g) {
-                    if (j + 1 <= qt) {
-                        if (!issue_s(g + 1)) { ok = false; break; }
-                        if (j + 1 == qt) umma_commit(q_empty);      // Q is free once the item's last S has read it
+                if (!issue_s()) break;
+                if (n_s == 1) umma_commit(q_empty);
+                for (int a = 0; a < n_s && ok; ++a) {
+                    if (a + 1 < n_s) {
+                        ok = issue_s();
+                        if (ok && a + 2 == n_s) umma_commit(q_empty);      // Q is free once the item's last S has read it
                     }
-                    const int s = g & 1u;
-                    const uint32_t ph = (g >> 1) & 1u;
-                    if (!wait_barrier(p_full(s), ph, abort_flag, p.status, 7)) { ok = false; break; }
-                    if (!wait_barrier(v_full(s), ph, abort_flag, p.status, 8)) { ok = false; break; }
-                    if (j == 0 && !wait_barrier(o_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) { ok = false; break; }
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < KT / 16; ++k) {
-                        // A = P: K-major halves of 64 keys. B = V: 16 keys further = 16 rows of 128 bytes.
-                        const uint64_t a_desc = make_smem_desc_sw128(
-                            base + SMEM_P + s * TILE_BYTES + (k >> 2) * HALF_BYTES + (k & 3) * 32, 0, 1024);
-                        const uint64_t b_desc =
-                            make_smem_desc_sw128(base + SMEM_V + s * TILE_BYTES + k * 16 * 128, HALF_BYTES, 1024);
-                        umma_bf16(tmem_o, a_desc, b_desc, idesc_o, (j | k) != 0 ? 1u : 0u);
-                    }
-                    umma_commit(v_empty(s));
-                    umma_commit(pv_done(s));
+                    if (ok && a >= m) ok = issue_pv(a == m);
                 }
+                for (int i = 0; i < m && ok; ++i) ok = issue_pv(false);
             }
         }
     } else {
@@ -270,92 +287,54 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         const int r = quad * 32 + lane;                       // row of the tile = TMEM lane
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
         const uint32_t tmem_o = tmem_base + 2 * KT + lane_addr;
-        uint32_t g = 0, it = 0;
+        uint32_t gk = 0, gv = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+        bool store_pending = false;      // lane 0: a TMA store of this warp may still be reading its staging rows
+        // 16-byte unit `chunk` (0..15) of this thread's 256-byte row of P buffer s, as the tensor core and TMA see it
+        auto p_addr = [&](int s, int chunk) {
+            return base + SMEM_P + s * TILE_BYTES + (chunk >> 3) * HALF_BYTES + r * 128 + ((((chunk & 7) ^ (r & 7))) << 4);
+        };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
             int qt, b, h;
             decode(item, qt, b, h);
-            const int gkv = h / rep;
             const int t = qt * QT + r;                        // position in the sequence
             const bool valid = t < p.T;
-            const int t_warp = qt * QT + quad * 32;           // first row of this warp
-            // ---- scores against the draft passes' keys on this row's substituted entries (raw, unscaled).
-            // The warp takes its 32 rows one by one with coalesced 256-byte reads (lane = 4 columns), then a
-            // transposing butterfly leaves row rr's dot product on lane rr.
+            // ---- draft passes of the score sequence: keep the diagonal element of each S_i (raw, unscaled) ----
             float sd[MAX_DRAFTS];
 #pragma unroll
             for (int i = 0; i < MAX_DRAFTS; ++i) sd[i] = 0.f;
-            if (p.m > 0 && item + static_cast<int>(gridDim.x) < p.items) {
-                // pull the draft rows of this CTA's next item towards L2 while this item is processed
-                int qt2, b2, h2;
-                decode(item + gridDim.x, qt2, b2, h2);
-                const int g2 = h2 / rep;
 #pragma unroll 1
-                for (int i = 0; i < p.m; ++i) {
-                    int ts = qt2 * QT + r - i;
-                    ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
-                    const size_t off = ((static_cast<size_t>(b2) * p.T + ts) * p.Hkv + g2) * HD;
-                    prefetch_l2(p.K_d[i] + off);
-                    prefetch_l2(p.K_d[i] + off + 64);
-                    prefetch_l2(p.V_d[i] + off);
-                    prefetch_l2(p.V_d[i] + off + 64);
-                }
+            for (int i = 0; i < m; ++i, ++gk) {
+                const int s = gk & 1u;
+                if (!wait_barrier(s_full(s), (gk >> 1) & 1u, abort_flag, p.status, 10)) { ok = false; break; }
+                tc_fence_after_sync();
+                uint32_t raw[32];
+                tmem_ld32(tmem_base + s * KT + lane_addr + 32 * quad, raw);     // columns of this warp's diagonal block
+                tmem_ld_wait(raw);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_empty(s));
+                float dv = 0.f;
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    if (c == lane) dv = __uint_as_float(raw[c]);
+#pragma unroll
+                for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                    if (ii == i) sd[ii] = dv;
             }
-            if (p.m > 0) {
-                uint2 qv[32];
-#pragma unroll
-                for (int rr = 0; rr < 32; ++rr) {
-                    int tr = t_warp + rr;
-                    tr = tr >= p.T ? p.T - 1 : tr;
-                    qv[rr] = __ldg(reinterpret_cast<const uint2*>(
-                                       p.Q + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane);
-                }
-#pragma unroll 1
-                for (int i = 0; i < p.m; ++i) {
-                    {
-                        float acc[32];
-                        const __nv_bfloat16* kd = p.K_d[i];
-#pragma unroll
-                        for (int rr = 0; rr < 32; ++rr) {
-                            // rows outside the sequence read a clamped row (no branch around the load); their
-                            // result is never used
-                            int ts = t_warp + rr - i;
-                            ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
-                            const uint2 kv = __ldg(reinterpret_cast<const uint2*>(
-                                                       kd + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
-                            acc[rr] = fmaf(bf16_lo(qv[rr].x), bf16_lo(kv.x),
-                                           fmaf(bf16_hi(qv[rr].x), bf16_hi(kv.x),
-                                                fmaf(bf16_lo(qv[rr].y), bf16_lo(kv.y), bf16_hi(qv[rr].y) * bf16_hi(kv.y))));
-                        }
-#pragma unroll
-                        for (int sft = 16; sft >= 1; sft >>= 1) {
-                            const bool up = (lane & sft) != 0;
-#pragma unroll
-                            for (int k = 0; k < sft; ++k) {
-                                const float keep = up ? acc[k + sft] : acc[k];
-                                const float send = up ? acc[k] : acc[k + sft];
-                                acc[k] = keep + __shfl_xor_sync(0xffffffffu, send, sft);
-                            }
-                        }
-#pragma unroll
-                        for (int ii = 0; ii < MAX_DRAFTS; ++ii)
-                            if (ii == i) sd[ii] = acc[0];
-                    }
-                }
-            }
+            if (!ok) break;
             float mref = -INFINITY, l = 0.f;
-            for (int j = 0; j <= qt; ++j, ++g) {
-                const int s = g & 1u;
-                const uint32_t ph = (g >> 1) & 1u;
-                if (!wait_barrier(s_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
+            for (int j = 0; j <= qt; ++j, ++gk, ++gv) {
+                const int s = gk & 1u;
+                if (!wait_barrier(s_full(s), (gk >> 1) & 1u, abort_flag, p.status, 10)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t tmem_s = tmem_base + s * KT + lane_addr;
                 const bool diag = (j == qt);
                 // Columns past t - m are hidden in the score tile: the causal part (s > t) and the m substituted
-                // entries (t - m < s <= t), which enter the row's maximum and sum as scalars at the diagonal tile
-                // and meet their value rows in the epilogue. Only the last two tiles can hold such columns.
-                const bool band = diag || (p.m > 0 && j + 1 == qt);
-                const int lim = t - p.m - j * KT;
+                // entries (t - m < s <= t), which enter the row's maximum and sum as scalars at the diagonal tile.
+                // Only the last two tiles can hold such columns.
+                const bool band = diag || (m > 0 && j + 1 == qt);
+                const int lim = t - m - j * KT;
                 // the whole row of S into registers, then the S buffer goes back to the tensor core
                 uint32_t raw[4][32];
 #pragma unroll
@@ -388,7 +367,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 if (diag) {
 #pragma unroll
                     for (int i = 0; i < MAX_DRAFTS; ++i)
-                        if (i < p.m && t - i >= 0) mx0 = fmaxf(mx0, sd[i]);
+                        if (i < m && t - i >= 0) mx0 = fmaxf(mx0, sd[i]);
                 }
                 const float cand = fmaxf(mx0, mx1) * p.c2;
                 if (j == 0) {
@@ -396,13 +375,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 } else {
                     const bool grow = cand > mref + RESCALE_LOG2;
                     if (__any_sync(0xffffffffu, grow)) {
-                        // rescale the accumulator: O of this row *= 2^(old ref - new ref); needs PV(g-1) complete
+                        // rescale the accumulator: O of this row *= 2^(old ref - new ref); needs the previous PV complete
                         const float f = grow ? ex2(mref - cand) : 1.f;
                         if (grow) {
                             mref = cand;
                             l *= f;
                         }
-                        const uint32_t gp = g - 1;
+                        const uint32_t gp = gv - 1;
                         if (!wait_barrier(pv_done(gp & 1u), (gp >> 1) & 1u, abort_flag, p.status, 11)) { ok = false; break; }
                         tc_fence_after_sync();
 #pragma unroll 1
@@ -433,114 +412,92 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                     }
                 }
                 l += ls0 + ls1;
-                if (diag) {
-#pragma unroll
-                    for (int i = 0; i < MAX_DRAFTS; ++i)
-                        if (i < p.m && t - i >= 0) l += ex2(fmaf(sd[i], p.c2, nref));
+                const int ps = gv & 1u;
+                if (!wait_barrier(pv_done(ps), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // P[ps] has been read
+                if (store_pending) {
+                    bulk_wait_read();          // (lane 0) the previous item's O store has read this warp's staging rows
+                    store_pending = false;
                 }
-                if (!wait_barrier(pv_done(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // PV(g-2) has read P[s]
-                const uint32_t p_row = base + SMEM_P + s * TILE_BYTES + r * 128;
+                __syncwarp();
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const uint32_t half = p_row + (k >> 1) * HALF_BYTES;
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const int chunk = (k & 1) * 4 + q4;                // 16-byte unit inside the 128-byte row
-                        st_shared_v4(half + (((chunk ^ (r & 7)) & 7) << 4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        st_shared_v4(p_addr(ps, 4 * k + q4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
                                      pack_bf16(v[k][8 * q4 + 2], v[k][8 * q4 + 3]), pack_bf16(v[k][8 * q4 + 4], v[k][8 * q4 + 5]),
                                      pack_bf16(v[k][8 * q4 + 6], v[k][8 * q4 + 7]));
-                    }
                 }
                 fence_proxy_async_smem();      // P visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full(s));
+                if (lane == 0) mbar_arrive(p_full(ps));
             }
             if (!ok) break;
-            // ---- epilogue: O / l, plus the substituted entries' weight times the draft value rows ----
+            // ---- draft passes of the value sequence: P holds only the weight 2^(sd c2 - ref) on its diagonal ----
+#pragma unroll 1
+            for (int i = 0; i < m; ++i, ++gv) {
+                float sdi = 0.f;
+#pragma unroll
+                for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                    if (ii == i) sdi = sd[ii];
+                const float pi = (t - i >= 0) ? ex2(fmaf(sdi, p.c2, -mref)) : 0.f;
+                l += pi;
+                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // column r sits in word (r & 7) / 2
+                const int ps = gv & 1u;
+                if (!wait_barrier(pv_done(ps), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
+#pragma unroll
+                for (int chunk = 0; chunk < 16; ++chunk) {
+                    const bool here = chunk == (r >> 3);
+                    const int w = (r & 7) >> 1;
+                    st_shared_v4(p_addr(ps, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
+                                 here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full(ps));
+            }
+            if (!ok) break;
+            // ---- epilogue: O / l as bf16, staged in this warp's rows of P buffer 0 and stored with TMA ----
             {
-                const uint32_t gp = g - 1;
+                const uint32_t gp = gv - 1;
                 if (!wait_barrier(pv_done(gp & 1u), (gp >> 1) & 1u, abort_flag, p.status, 13)) break;
                 tc_fence_after_sync();
                 const float inv = 1.f / l;
-                float pd[MAX_DRAFTS];
-#pragma unroll
-                for (int i = 0; i < MAX_DRAFTS; ++i)
-                    pd[i] = (i < p.m && valid && t - i >= 0) ? ex2(fmaf(sd[i], p.c2, -mref)) * inv : 0.f;
                 if (valid && p.lse != nullptr)
                     p.lse[(static_cast<size_t>(b) * p.H + h) * p.T + t] = (mref + log2f(l)) * 0.6931471805599453f;
-                // Stage this warp's 32 rows of O (fp32, normalised) in shared memory. Both PV products that read
-                // the P buffers are complete, and the bytes used are exactly this warp's own rows of the two
-                // P buffers (4 pieces of 128 bytes per row), which no other warp writes.
-                auto piece = [&](int rr, int k) {   // 128-byte piece k (columns 32k .. 32k+31) of row rr of this warp
-                    return base + SMEM_P + (k >> 1) * TILE_BYTES + (k & 1) * HALF_BYTES + (quad * 32 + rr) * 128;
-                };
-                {
-                    uint32_t raw[4][32];
+                uint32_t raw[4][32];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) tmem_ld32(tmem_o + 32 * k, raw[k]);
+                for (int k = 0; k < 4; ++k) tmem_ld32(tmem_o + 32 * k, raw[k]);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(o_free);     // the accumulator may be overwritten by the next item
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-#pragma unroll
-                        for (int c8 = 0; c8 < 8; ++c8)
-                            st_shared_v4(piece(lane, k) + (((c8 ^ lane) & 7) << 4),
-                                         __float_as_uint(__uint_as_float(raw[k][4 * c8]) * inv),
-                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 1]) * inv),
-                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 2]) * inv),
-                                         __float_as_uint(__uint_as_float(raw[k][4 * c8 + 3]) * inv));
-                    }
-                }
+                for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
+                tc_fence_before_sync();
                 __syncwarp();
-                // row by row with the warp across the 128 columns (lane = 4 columns): coalesced reads of the draft
-                // value rows and coalesced stores of O
-                const int kq = lane >> 3, cq = lane & 7;
-#pragma unroll 1
-                for (int rr0 = 0; rr0 < 32; rr0 += 16) {
-                    float4 o[16];
+                if (lane == 0) mbar_arrive(o_free);         // the accumulator may be overwritten by the next item
+                // every PV product of the item is complete, so both P buffers are idle; the bytes used are this
+                // warp's own rows, which no other warp writes
 #pragma unroll
-                    for (int u = 0; u < 16; ++u)
-                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                     : "=f"(o[u].x), "=f"(o[u].y), "=f"(o[u].z), "=f"(o[u].w)
-                                     : "r"(piece(rr0 + u, kq) + (((cq ^ (rr0 + u)) & 7) << 4)));
-#pragma unroll 1
-                    for (int i = 0; i < p.m; ++i) {
-                        float pdi = 0.f;
+                for (int k = 0; k < 4; ++k) {
 #pragma unroll
-                        for (int ii = 0; ii < MAX_DRAFTS; ++ii)
-                            if (ii == i) pdi = pd[ii];
-                        const __nv_bfloat16* vd = p.V_d[i];
-                        uint2 vv[16];
-#pragma unroll
-                        for (int u = 0; u < 16; ++u) {
-                            int ts = t_warp + rr0 + u - i;
-                            ts = ts < 0 ? 0 : (ts >= p.T ? p.T - 1 : ts);
-                            vv[u] = __ldg(reinterpret_cast<const uint2*>(
-                                              vd + ((static_cast<size_t>(b) * p.T + ts) * p.Hkv + gkv) * HD) + lane);
-                        }
-#pragma unroll
-                        for (int u = 0; u < 16; ++u) {
-                            const float w = __shfl_sync(0xffffffffu, pdi, rr0 + u);    // 0 where the entry does not exist
-                            o[u].x = fmaf(w, bf16_lo(vv[u].x), o[u].x);
-                            o[u].y = fmaf(w, bf16_hi(vv[u].x), o[u].y);
-                            o[u].z = fmaf(w, bf16_lo(vv[u].y), o[u].z);
-                            o[u].w = fmaf(w, bf16_hi(vv[u].y), o[u].w);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 16; ++u) {
-                        const int tr = t_warp + rr0 + u;
-                        if (tr < p.T)
-                            *(reinterpret_cast<uint2*>(p.O + ((static_cast<size_t>(b) * p.T + tr) * p.H + h) * HD) + lane) =
-                                make_uint2(pack_bf16(o[u].x, o[u].y), pack_bf16(o[u].z, o[u].w));
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const uint32_t* x = &raw[k][8 * q4];
+                        st_shared_v4(p_addr(0, 4 * k + q4),
+                                     pack_bf16(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv),
+                                     pack_bf16(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv),
+                                     pack_bf16(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv),
+                                     pack_bf16(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv));
                     }
                 }
-                __syncwarp();      // the staging bytes are this warp's P rows of the next tiles
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && qt * QT + quad * 32 < p.T) {
+                    const uint32_t src = base + SMEM_P + quad * 32 * 128;
+                    tma_store_3d(&p.tmO, src, h * HD, qt * QT + quad * 32, b);
+                    tma_store_3d(&p.tmO, src + HALF_BYTES, h * HD + 64, qt * QT + quad * 32, b);
+                    bulk_commit();
+                    store_pending = true;
+                }
             }
         }
+        if (lane == 0) bulk_wait_all();      // O stores complete before the CTA's shared memory goes away
     }
 
     // ---- teardown ----
