@@ -181,13 +181,160 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
+# ---- HCA attention of the draft layer (Section 3.2) ---------------------------------------------------
+HCA_METRIC = "tokens/sec HCA attention fwd"
+
+
+def time_hca_oracle(inp, pairs):
+    """fp64 oracle on whole (sequence, head) pairs; returns token-equivalents per second (a pair is
+    T / H of a sequence's attention work)."""
+    from oracle import hca_oracle as ho
+    wl = inp.wl
+    rep = wl.H // wl.Hkv
+    f = lambda x, b, hh: x[b:b + 1, :, hh:hh + 1, :].to(torch.float64).numpy()
+    t0 = time.perf_counter()
+    for b, h in pairs:
+        g = h // rep
+        ho.hca_attention(f(inp.Q, b, h), f(inp.K_t, b, g), f(inp.V_t, b, g), [f(x, b, g) for x in inp.K_d],
+                         [f(x, b, g) for x in inp.V_d])
+    dt = time.perf_counter() - t0
+    return len(pairs) * wl.T / wl.H / dt, dt
+
+
+def hca_pairs(wl, n, seed=0):
+    rng = np.random.default_rng(seed)
+    return [(int(rng.integers(0, wl.B)), int(rng.integers(0, wl.H))) for _ in range(n)]
+
+
+def main_hca(args):
+    wl = hi.HCA_WORKLOADS[args.workload]
+    tokens = wl.B * wl.T
+    config = {"workload": wl.name, "B": wl.B, "T": wl.T, "heads": wl.H, "kv_heads": wl.Hkv, "head_dim": wl.D,
+              "draft_passes_m": wl.m, "aligning_step": wl.m + 1, "path": "hass_hca_attention_fwd"}
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        inp = hi.make_hca_inputs(wl)
+        n_pairs = args.oracle_rows or 4
+        vals = []
+        for i in range(args.warmup + args.steps):
+            v = time_hca_oracle(inp, hca_pairs(wl, n_pairs, seed=i))
+            if i >= args.warmup:
+                vals.append(v)
+        tps = float(np.mean([v[0] for v in vals]))
+        sample = f"{n_pairs} of {wl.B * wl.H} (sequence, head) pairs per step, all {wl.T} positions"
+        print(json.dumps({"impl": "reference", "metric": HCA_METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+                          "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": float(np.mean([v[1] for v in vals]) * 1e3), "higher_is_better": True,
+                          "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                          "config": dict(config, note="fp64 CPU oracle on sampled (sequence, head) pairs"),
+                          "cpu_baseline": {"value": tps, "unit": UNIT, "cores": torch.get_num_threads(),
+                                           "kind": "oracle", "sample": sample},
+                          "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
+        return
+    rank, world, local = dist_setup(args.gpus)
+    import paper_2408_15766_b200 as hass   # fails loudly if the CUDA library is missing
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    peaks, peak_kind = load_peaks()
+    inp = hi.make_hca_inputs(wl)
+    host = [inp.Q, inp.K_t, inp.V_t, *inp.K_d, *inp.V_d]
+    Q, K_t, V_t = (x.to(dev) for x in host[:3])
+    K_d, V_d = [x.to(dev) for x in inp.K_d], [x.to(dev) for x in inp.V_d]
+    ws = torch.zeros(hass.hca_attention_workspace_bytes(), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    in_bytes = sum(x.numel() * 2 for x in host)
+
+    def step():
+        return hass.hca_attention_fwd(Q, K_t, V_t, K_d, V_d, workspace=ws, stream=stream)
+
+    for _ in range(args.warmup):
+        step()
+    hass.check(ws)
+    barrier(world)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    hass.profile_enable(True)
+    launches0 = hass.kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier(world)
+    launches = hass.kernel_launch_count() - launches0
+    prof = hass.profile_summary()
+    hass.profile_enable(False)
+    clocks = sampler.stop()
+    hass.check(ws)
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
+
+    # end to end: projected features from pinned host memory, O back to host, through the public call
+    e2e = None
+    if not args.no_e2e:
+        pinned = [x.pin_memory() for x in host]
+        O_h = torch.empty_like(inp.Q).pin_memory()
+
+        def step_e2e():
+            d_ = [x.to(dev, non_blocking=True) for x in pinned]
+            out = hass.hca_attention_fwd(d_[0], d_[1], d_[2], d_[3:3 + wl.m], d_[3 + wl.m:], workspace=ws,
+                                         want_lse=False, stream=stream)
+            O_h.copy_(out["O"], non_blocking=True)
+
+        for _ in range(3):
+            step_e2e()
+        barrier(world)
+        torch.cuda.synchronize()
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            step_e2e()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1) / n_e2e, world, dev)
+        e2e = {"value": aggregate(tokens, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": inp.Q.numel() * 2,
+               "note": "Q, K_t, V_t and the draft passes' K/V from pinned host memory, O back to host"}
+    if rank != 0:
+        return
+    # causal attention: two products of 2 * D flops per (query, key) pair with key <= query
+    flops = 4.0 * wl.D * wl.B * wl.H * wl.T * (wl.T + 1) / 2
+    ms_k, cnt = prof["hca_attention"]
+    achieved = flops / (ms_k / cnt * 1e-3) / 1e12
+    peak = float(peaks["bf16_tflops"])
+    line = {"metric": HCA_METRIC, "value": aggregate(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": dict(config, l2="inputs and output (%.0f MB) larger than L2" % ((in_bytes + inp.Q.numel() * 2) / 1e6)),
+            "clocks": clocks, "gpu_launches": launches,
+            "roofline": {"bound": "tensor", "kernel": "hca_attention", "achieved": achieved, "peak": peak,
+                         "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                         "peak_kind": f"bf16_tflops (burst), of {peak_kind} (a sub-millisecond kernel timed alone)",
+                         "flops_per_launch": flops, "avg_launch_ms": ms_k / cnt}}
+    if e2e:
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        n_pairs = args.oracle_rows or 16
+        tps, dt = time_hca_oracle(inp, hca_pairs(wl, n_pairs))
+        line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": f"{n_pairs} of {wl.B * wl.H} (sequence, head) pairs, all {wl.T} positions, {dt:.1f} s"}
+    print(json.dumps(line), flush=True)
+
+
 # ---- main --------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS))
+    ap.add_argument("--workload", default="l3-8b", choices=list(hi.WORKLOADS) + list(hi.HCA_WORKLOADS),
+                    help="hca-*: the HCA attention of the draft layer instead of the LM-head path")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--objective", default="topk", choices=["topk", "combined", "top_p", "normed", "bidir"],
@@ -201,6 +348,9 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.workload in hi.HCA_WORKLOADS:
+        main_hca(args)
+        return
     if args.impl == "reference":
         # the CPU oracle needs no process group: rank 0 alone works, the other ranks leave at once
         if args.oracle_rows is None:
