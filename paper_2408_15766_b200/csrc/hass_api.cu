@@ -74,6 +74,8 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
+            // two CTAs of this kernel share an SM: ask for the largest shared-memory carve-out
+            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
                 cudaGetLastError();
                 return HASS_ERR_CUDA;
@@ -1205,16 +1207,15 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
 
     hca::Params p;
     std::memset(&p, 0, sizeof(p));
-    rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca::HD);
-    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca::HD);
-    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca::HD);
-    if (rc != HASS_OK) return rc;
+    rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca::HD, hca::QT);
+    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca::HD, hca::KT);
+    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca::HD, hca::KT);
     for (int i = 0; i < m && rc == HASS_OK; ++i) {
-        rc = make_tmap_seq(&p.tmKd[i], K_d[i], B, T, Hkv * hca::HD);
-        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmVd[i], V_d[i], B, T, Hkv * hca::HD);
+        rc = make_tmap_seq(&p.tmKd[i], K_d[i], B, T, Hkv * hca::HD, hca::KT);
+        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmVd[i], V_d[i], B, T, Hkv * hca::HD, hca::KT);
     }
-    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmO, O, B, T, H * hca::HD, 32);
     if (rc != HASS_OK) return rc;
+    p.O = static_cast<__nv_bfloat16*>(O);
     p.lse = lse;
     p.B = static_cast<int>(B);
     p.T = static_cast<int>(T);
@@ -1222,6 +1223,7 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
     p.Hkv = static_cast<int>(Hkv);
     p.m = m;
     p.q_tiles = static_cast<int>((T + hca::QT - 1) / hca::QT);
+    p.k_tiles = static_cast<int>((T + hca::KT - 1) / hca::KT);
     p.items = static_cast<int>(B * H) * p.q_tiles;
     p.c2 = scale * 1.4426950408889634f;
     p.status = static_cast<unsigned int*>(workspace);
@@ -1229,7 +1231,7 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
         cudaGetLastError();
         return HASS_ERR_CUDA;
     }
-    const int grid = p.items < di.sms ? p.items : di.sms;
+    const int grid = p.items < 2 * di.sms ? p.items : 2 * di.sms;      // two CTAs per SM
     {
         KernelTimer kt(KIND_HCA, st);
         hca::hca_attention_kernel<<<grid, hca::NUM_THREADS, hca::SMEM_BYTES, st>>>(p);

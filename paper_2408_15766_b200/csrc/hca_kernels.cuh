@@ -1,26 +1,26 @@
 // HCA attention of the draft layer (Section 3.2; the appendix's attention listing) for sm_100a.
 //
-// One persistent, warp-specialised kernel. A work item is one (sequence, query head, tile of 128
-// query positions); it sweeps the key tiles 0 .. its own (causal). Per key tile:
-//   S = Q K_t^T            tcgen05.mma, 128 x 128 x 128, fp32 in TMEM (two S buffers)
+// One persistent, warp-specialised kernel, two CTAs per SM. A work item is one (sequence, query head,
+// tile of 128 query positions); it sweeps its causal key tiles of 64 keys. Per key tile:
+//   S = Q K_t^T            tcgen05.mma, 128 x 64 x 128, fp32 in TMEM (two S buffers)
 //   softmax warps          read S (one query row per thread), hide the columns past t - m (the causal
 //                          part and the m substituted entries), update the row's running reference
 //                          and sum, write P = 2^(x - ref) as bf16 into shared memory in the swizzled
 //                          layout the tensor core reads
 //   O += P V_t             tcgen05.mma with V_t as an MN-major operand, fp32 in TMEM
-// The substituted entries (t, t - i), i < m, ride the same pipeline as extra tiles of the item:
-//   before the key tiles   S_i = Q K_d[i]^T with the K_d[i] tile fetched i rows early, so that the
-//                          wanted scores <Q[t], K_d[i][t - i]> sit on the tile's main diagonal; each
-//                          softmax thread keeps its diagonal element
-//   at the diagonal tile   the m scores join the row maximum and sum
-//   after the key tiles    O += diag(p_i) V_d[i], V_d[i] again fetched i rows early and the P buffer
-//                          holding just the weights on its diagonal
-// so no thread reads global memory; the epilogue divides by the row sum, stages bf16 rows in shared
-// memory and stores them with TMA.
-// The running reference moves only when a tile's maximum exceeds it by more than 2^8 (the O
-// accumulator in TMEM is then rescaled in place by the softmax warps), so P stays within bf16
-// range and most tiles skip the rescale.
+// The substituted entries (t, t - i), i < m, ride the same pipeline as extra half-height tiles:
+//   before the key tiles   S_ih = Q K_d[i]^T for the two 64-key halves h of the K_d[i] tile fetched
+//                          i rows early, so that the wanted scores <Q[t], K_d[i][t - i]> sit on the
+//                          diagonal of half h for the rows of half h; each thread keeps its element
+//   at the last key tile   the m scores join the row maximum and sum
+//   after the key tiles    O += diag_h(p_i) V_d[i] (half h of V_d[i] fetched i rows early; the P
+//                          buffer holds just the weights of the rows of half h on its diagonal)
+// so no thread reads global memory. The running reference moves only when a tile's maximum exceeds it
+// by more than 2^8 (the O accumulator in TMEM is then rescaled in place by the softmax warps), so P
+// stays within bf16 range and most tiles skip the rescale.
 //
+// Two CTAs share an SM (112 KB of shared memory and 256 TMEM columns each): while one CTA's softmax
+// warps wait for the tensor core, TMEM or a barrier, the other's keep the exp2 unit busy.
 // Warps: 0 = TMA producer (Q once per item, K and V tiles through two-stage rings),
 //        1 = MMA issuer and TMEM owner, 2-5 = softmax + epilogue (TMEM lane quadrant = warp % 4).
 // Every wait is bounded (wait_barrier); a wait that gives up sets the status word and all roles leave.
@@ -33,30 +33,35 @@ namespace hass {
 namespace hca {
 
 constexpr int QT = 128;            // query rows per item
-constexpr int KT = 128;            // keys per tile
+constexpr int KT = 64;             // keys per tile
 constexpr int HD = 128;            // head dimension
 constexpr int MAX_DRAFTS = 8;      // m <= 8
 constexpr int NUM_THREADS = 192;
-constexpr int TILE_BYTES = 128 * 128 * 2;           // any 128 x 128 bf16 tile: two 16 KB halves of 64 columns
-constexpr int HALF_BYTES = TILE_BYTES / 2;
+constexpr int Q_BYTES = QT * HD * 2;                 // two halves (64 columns of the head dimension) of 128 rows x 128 B
+constexpr int Q_HALF = Q_BYTES / 2;
+constexpr int KV_BYTES = KT * HD * 2;                // two halves of 64 rows x 128 B
+constexpr int KV_HALF = KV_BYTES / 2;
+constexpr int P_BYTES = QT * KT * 2;                 // 128 rows x 128 B
 constexpr int SMEM_Q = 0;
-constexpr int SMEM_K = SMEM_Q + TILE_BYTES;          // 2 stages
-constexpr int SMEM_V = SMEM_K + 2 * TILE_BYTES;      // 2 stages
-constexpr int SMEM_P = SMEM_V + 2 * TILE_BYTES;      // 2 buffers
-constexpr int SMEM_BAR = SMEM_P + 2 * TILE_BYTES;
-constexpr int NUM_BARS = 19;
-constexpr int SMEM_BYTES = SMEM_BAR + 256 + 1024 /*alignment slack*/;
-constexpr int TMEM_COLS = 512;     // S0 at 0, S1 at 128, O at 256
+constexpr int SMEM_K = SMEM_Q + Q_BYTES;             // 2 stages
+constexpr int SMEM_V = SMEM_K + 2 * KV_BYTES;        // 2 stages
+constexpr int SMEM_P = SMEM_V + 2 * KV_BYTES;        // 1 buffer
+constexpr int SMEM_BAR = SMEM_P + P_BYTES;
+constexpr int NUM_BARS = 17;
+constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 114944: two CTAs fit the SM's 228 KB
+constexpr int TMEM_COLS = 256;     // S0 at 0, S1 at 64, O at 128
 constexpr float RESCALE_LOG2 = 8.f;
 
 struct Params {
-    CUtensorMap tmQ, tmK, tmV;     // 3-D maps {heads * 128, T, B}, box {64, 128, 1}, 128-byte swizzle
+    CUtensorMap tmQ;               // [B, T, H * 128], box {64, 128, 1}, 128-byte swizzle
+    CUtensorMap tmK, tmV;          // [B, T, Hkv * 128], box {64, 64, 1}
     CUtensorMap tmKd[MAX_DRAFTS];  // the draft passes' keys and values, same geometry; index = sub-diagonal
     CUtensorMap tmVd[MAX_DRAFTS];
-    CUtensorMap tmO;               // O [B, T, H * 128], box {64, 32, 1}: one warp's rows of half a tile
+    __nv_bfloat16* O;              // [B, T, H, 128]
     float* lse;                    // [B, H, T] or null
     int B, T, H, Hkv, m;
     int q_tiles;                   // ceil(T / 128)
+    int k_tiles;                   // ceil(T / 64)
     int items;                     // B * H * q_tiles
     float c2;                      // scale * log2(e)
     unsigned int* status;
@@ -88,16 +93,6 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// Tiled store shared -> global (rows past the tensor's extent are clipped), tracked by bulk groups.
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t smem_src, int x, int y, int z) {
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
-                     reinterpret_cast<uint64_t>(tm)),
-                 "r"(smem_src), "r"(x), "r"(y), "r"(z)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -105,13 +100,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
 }
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __grid_constant__ Params p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
+__global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t base = smem_u32(smem_raw);
+    if ((base & 1023u) != 0u) {
+        // the swizzled tiles need a 1024-byte aligned window; report instead of computing garbage
+        if (threadIdx.x == 0) atomicCAS(p.status, 0u, (20u << 8) | 1u);
+        return;
+    }
     const uint32_t bar0 = base + SMEM_BAR;
     // barriers
     const uint32_t q_full = bar0, q_empty = bar0 + 8;
@@ -121,10 +118,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
     auto v_empty = [&](int b) { return bar0 + 8u * (8 + b); };
     auto s_full = [&](int b) { return bar0 + 8u * (10 + b); };
     auto s_empty = [&](int b) { return bar0 + 8u * (12 + b); };
-    auto p_full = [&](int b) { return bar0 + 8u * (14 + b); };
-    auto pv_done = [&](int b) { return bar0 + 8u * (16 + b); };
-    const uint32_t o_free = bar0 + 8u * 18;
-    uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + SMEM_BAR + 8 * NUM_BARS);
+    const uint32_t p_full = bar0 + 8u * 14;
+    const uint32_t pv_done = bar0 + 8u * 15;
+    const uint32_t o_free = bar0 + 8u * 16;
+    uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_raw + SMEM_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -140,9 +137,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             mbar_init(v_empty(b), 1);
             mbar_init(s_full(b), 1);
             mbar_init(s_empty(b), 4);
-            mbar_init(p_full(b), 4);
-            mbar_init(pv_done(b), 1);
         }
+        mbar_init(p_full, 4);
+        mbar_init(pv_done, 1);
         mbar_init(o_free, 4);
         *abort_flag = 0;
         fence_barrier_init();
@@ -150,7 +147,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         prefetch_tensormap(&p.tmQ);
         prefetch_tensormap(&p.tmK);
         prefetch_tensormap(&p.tmV);
-        prefetch_tensormap(&p.tmO);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_ptr_smem), TMEM_COLS);
@@ -171,9 +167,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         b = bh / p.H;
         h = bh - b * p.H;
     };
+    // key tiles of an item: 0 .. 2 qt + 1, cut at the end of the sequence
+    auto key_tiles = [&](int qt) { return min(2 * qt + 2, p.k_tiles); };
     // Per item the tensor core runs two sequences, each with its own ring counter:
-    //   score sequence (K ring, S buffers), length m + qt + 1: draft pass 0 .. m-1, then key tiles 0 .. qt
-    //   value sequence (V ring, P buffers), length qt + 1 + m: key tiles 0 .. qt, then draft pass 0 .. m-1
+    //   score sequence (K ring, S buffers), length 2m + n: draft pass i, half h (element 2i + h), then key tiles 0 .. n-1
+    //   value sequence (V ring, P buffer),  length n + 2m: key tiles 0 .. n-1, then draft pass i, half h
 
     if (warp == 0) {
         // ===================== TMA producer =====================
@@ -183,18 +181,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             auto load_k = [&](const CUtensorMap* tm, int col, int row, int b) -> bool {
                 const int s = gk & 1u;
                 if (!wait_barrier(k_empty(s), ((gk >> 1) & 1u) ^ 1u, abort_flag, p.status, 2)) return false;
-                mbar_arrive_expect_tx(k_full(s), TILE_BYTES);
-                tma_load_3d(base + SMEM_K + s * TILE_BYTES, tm, k_full(s), col, row, b);
-                tma_load_3d(base + SMEM_K + s * TILE_BYTES + HALF_BYTES, tm, k_full(s), col + 64, row, b);
+                mbar_arrive_expect_tx(k_full(s), KV_BYTES);
+                tma_load_3d(base + SMEM_K + s * KV_BYTES, tm, k_full(s), col, row, b);
+                tma_load_3d(base + SMEM_K + s * KV_BYTES + KV_HALF, tm, k_full(s), col + 64, row, b);
                 ++gk;
                 return true;
             };
             auto load_v = [&](const CUtensorMap* tm, int col, int row, int b) -> bool {
                 const int s = gv & 1u;
                 if (!wait_barrier(v_empty(s), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 3)) return false;
-                mbar_arrive_expect_tx(v_full(s), TILE_BYTES);
-                tma_load_3d(base + SMEM_V + s * TILE_BYTES, tm, v_full(s), col, row, b);
-                tma_load_3d(base + SMEM_V + s * TILE_BYTES + HALF_BYTES, tm, v_full(s), col + 64, row, b);
+                mbar_arrive_expect_tx(v_full(s), KV_BYTES);
+                tma_load_3d(base + SMEM_V + s * KV_BYTES, tm, v_full(s), col, row, b);
+                tma_load_3d(base + SMEM_V + s * KV_BYTES + KV_HALF, tm, v_full(s), col + 64, row, b);
                 ++gv;
                 return true;
             };
@@ -202,17 +200,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int col = (h / rep) * HD;
+                const int n = key_tiles(qt);
                 if (!wait_barrier(q_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1)) break;
-                mbar_arrive_expect_tx(q_full, TILE_BYTES);
+                mbar_arrive_expect_tx(q_full, Q_BYTES);
                 tma_load_3d(base + SMEM_Q, &p.tmQ, q_full, h * HD, qt * QT, b);
-                tma_load_3d(base + SMEM_Q + HALF_BYTES, &p.tmQ, q_full, h * HD + 64, qt * QT, b);
-                // draft keys start i rows early: row r of the tile is position qt*128 + r - i (zeros before the sequence)
-                for (int i = 0; i < m && ok; ++i) ok = load_k(&p.tmKd[i], col, qt * QT - i, b);
-                for (int j = 0; j <= qt && ok; ++j) {
+                tma_load_3d(base + SMEM_Q + Q_HALF, &p.tmQ, q_full, h * HD + 64, qt * QT, b);
+                // draft keys start i rows early: row r of half hf is position qt*128 + 64 hf + r - i (zeros before the sequence)
+                for (int e = 0; e < 2 * m && ok; ++e) ok = load_k(&p.tmKd[e >> 1], col, qt * QT + 64 * (e & 1) - (e >> 1), b);
+                for (int j = 0; j < n && ok; ++j) {
                     ok = load_k(&p.tmK, col, j * KT, b);
                     if (ok) ok = load_v(&p.tmV, col, j * KT, b);
                 }
-                for (int i = 0; i < m && ok; ++i) ok = load_v(&p.tmVd[i], col, qt * QT - i, b);
+                for (int e = 0; e < 2 * m && ok; ++e) ok = load_v(&p.tmVd[e >> 1], col, qt * QT + 64 * (e & 1) - (e >> 1), b);
             }
         }
     } else if (warp == 1) {
@@ -232,9 +231,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
-                    const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
-                    const uint64_t a_desc = make_smem_desc_sw128(base + SMEM_Q + off, 0, 1024);
-                    const uint64_t b_desc = make_smem_desc_sw128(base + SMEM_K + s * TILE_BYTES + off, 0, 1024);
+                    const uint64_t a_desc = make_smem_desc_sw128(base + SMEM_Q + (k >> 2) * Q_HALF + (k & 3) * 32, 0, 1024);
+                    const uint64_t b_desc =
+                        make_smem_desc_sw128(base + SMEM_K + s * KV_BYTES + (k >> 2) * KV_HALF + (k & 3) * 32, 0, 1024);
                     umma_bf16(tmem_base + s * KT, a_desc, b_desc, idesc_s, k != 0 ? 1u : 0u);
                 }
                 umma_commit(k_empty(s));
@@ -245,29 +244,28 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
             // next element of the value sequence: O (+)= P V
             auto issue_pv = [&](bool first) -> bool {
                 const int s = gv & 1u;
-                const uint32_t ph = (gv >> 1) & 1u;
-                if (!wait_barrier(p_full(s), ph, abort_flag, p.status, 7)) return false;
-                if (!wait_barrier(v_full(s), ph, abort_flag, p.status, 8)) return false;
+                if (!wait_barrier(p_full, gv & 1u, abort_flag, p.status, 7)) return false;
+                if (!wait_barrier(v_full(s), (gv >> 1) & 1u, abort_flag, p.status, 8)) return false;
                 if (first && !wait_barrier(o_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k) {
-                    // A = P: K-major halves of 64 keys. B = V: 16 keys further = 16 rows of 128 bytes.
-                    const uint64_t a_desc = make_smem_desc_sw128(
-                        base + SMEM_P + s * TILE_BYTES + (k >> 2) * HALF_BYTES + (k & 3) * 32, 0, 1024);
+                    // A = P: K-major, 64 keys = one 128-byte row. B = V: 64-column groups KV_HALF apart, 16 keys
+                    // further = 16 rows of 128 bytes.
+                    const uint64_t a_desc = make_smem_desc_sw128(base + SMEM_P + k * 32, 0, 1024);
                     const uint64_t b_desc =
-                        make_smem_desc_sw128(base + SMEM_V + s * TILE_BYTES + k * 16 * 128, HALF_BYTES, 1024);
+                        make_smem_desc_sw128(base + SMEM_V + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
                     umma_bf16(tmem_o, a_desc, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
                 }
                 umma_commit(v_empty(s));
-                umma_commit(pv_done(s));
+                umma_commit(pv_done);
                 ++gv;
                 return true;
             };
             for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
                 int qt, b, h;
                 decode(item, qt, b, h);
-                const int n_s = m + qt + 1;
+                const int n_s = 2 * m + key_tiles(qt);
                 if (!wait_barrier(q_full, it & 1u, abort_flag, p.status, 6)) break;
                 if (!issue_s()) break;
                 if (n_s == 1) umma_commit(q_empty);
@@ -276,9 +274,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                         ok = issue_s();
                         if (ok && a + 2 == n_s) umma_commit(q_empty);      // Q is free once the item's last S has read it
                     }
-                    if (ok && a >= m) ok = issue_pv(a == m);
+                    if (ok && a >= 2 * m) ok = issue_pv(a == 2 * m);
                 }
-                for (int i = 0; i < m && ok; ++i) ok = issue_pv(false);
+                for (int e = 0; e < 2 * m && ok; ++e) ok = issue_pv(false);
             }
         }
     } else {
@@ -289,64 +287,64 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
         const uint32_t tmem_o = tmem_base + 2 * KT + lane_addr;
         uint32_t gk = 0, gv = 0;
         bool ok = true;
-        bool store_pending = false;      // lane 0: a TMA store of this warp may still be reading its staging rows
-        // 16-byte unit `chunk` (0..15) of this thread's 256-byte row of P buffer s, as the tensor core and TMA see it
-        auto p_addr = [&](int s, int chunk) {
-            return base + SMEM_P + s * TILE_BYTES + (chunk >> 3) * HALF_BYTES + r * 128 + ((((chunk & 7) ^ (r & 7))) << 4);
-        };
+        // 16-byte unit `chunk` (0..7) of this thread's 128-byte row of the P buffer, as the tensor core sees it
+        auto p_addr = [&](int chunk) { return base + SMEM_P + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
         for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
             int qt, b, h;
             decode(item, qt, b, h);
+            const int n = key_tiles(qt);
             const int t = qt * QT + r;                        // position in the sequence
             const bool valid = t < p.T;
-            // ---- draft passes of the score sequence: keep the diagonal element of each S_i (raw, unscaled) ----
+            // ---- draft passes of the score sequence: keep the diagonal element of each S_ih (raw, unscaled) ----
             float sd[MAX_DRAFTS];
 #pragma unroll
             for (int i = 0; i < MAX_DRAFTS; ++i) sd[i] = 0.f;
 #pragma unroll 1
-            for (int i = 0; i < m; ++i, ++gk) {
+            for (int e = 0; e < 2 * m; ++e, ++gk) {
                 const int s = gk & 1u;
                 if (!wait_barrier(s_full(s), (gk >> 1) & 1u, abort_flag, p.status, 10)) { ok = false; break; }
                 tc_fence_after_sync();
-                uint32_t raw[32];
-                tmem_ld32(tmem_base + s * KT + lane_addr + 32 * quad, raw);     // columns of this warp's diagonal block
-                tmem_ld_wait(raw);
+                if ((quad >> 1) == (e & 1)) {                  // this warp's rows lie in half e & 1
+                    uint32_t raw[32];
+                    tmem_ld32(tmem_base + s * KT + lane_addr + 32 * (quad & 1), raw);     // this warp's diagonal block
+                    tmem_ld_wait(raw);
+                    float dv = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (c == lane) dv = __uint_as_float(raw[c]);
+#pragma unroll
+                    for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                        if (ii == (e >> 1)) sd[ii] = dv;
+                }
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty(s));
-                float dv = 0.f;
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                    if (c == lane) dv = __uint_as_float(raw[c]);
-#pragma unroll
-                for (int ii = 0; ii < MAX_DRAFTS; ++ii)
-                    if (ii == i) sd[ii] = dv;
             }
             if (!ok) break;
             float mref = -INFINITY, l = 0.f;
-            for (int j = 0; j <= qt; ++j, ++gk, ++gv) {
+            for (int j = 0; j < n; ++j, ++gk, ++gv) {
                 const int s = gk & 1u;
                 if (!wait_barrier(s_full(s), (gk >> 1) & 1u, abort_flag, p.status, 10)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t tmem_s = tmem_base + s * KT + lane_addr;
-                const bool diag = (j == qt);
+                const bool last = (j == n - 1);
                 // Columns past t - m are hidden in the score tile: the causal part (s > t) and the m substituted
-                // entries (t - m < s <= t), which enter the row's maximum and sum as scalars at the diagonal tile.
-                // Only the last two tiles can hold such columns.
-                const bool band = diag || (m > 0 && j + 1 == qt);
+                // entries (t - m < s <= t), which enter the row's maximum and sum as scalars at the last tile.
+                // Only tiles reaching past the first row's limit can hold such columns.
+                const bool band = j * KT + KT - 1 > qt * QT - m;
                 const int lim = t - m - j * KT;
-                // the whole row of S into registers, then the S buffer goes back to the tensor core
-                uint32_t raw[4][32];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) tmem_ld32(tmem_s + 32 * k, raw[k]);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
+                // the row's 64 scores into registers, then the S buffer goes back to the tensor core
+                uint32_t raw[2][32];
+                tmem_ld32(tmem_s, raw[0]);
+                tmem_ld32(tmem_s + 32, raw[1]);
+                tmem_ld_wait(raw[0]);
+                tmem_ld_wait(raw[1]);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(s_empty(s));
-                float v[4][32];
+                float v[2][32];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) v[k][c] = __uint_as_float(raw[k][c]);
                     if (band) {
@@ -357,14 +355,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
                         mx0 = fmax3(mx0, v[k][c], v[k][c + 1]);
                         mx1 = fmax3(mx1, v[k][c + 2], v[k][c + 3]);
                     }
                 }
-                if (diag) {
+                if (last) {
 #pragma unroll
                     for (int i = 0; i < MAX_DRAFTS; ++i)
                         if (i < m && t - i >= 0) mx0 = fmaxf(mx0, sd[i]);
@@ -373,7 +371,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                 if (j == 0) {
                     mref = cand;
                 } else {
-                    const bool grow = cand > mref + RESCALE_LOG2;
+                    const bool grow = cand > mref + RESCALE_LOG2;      // also true when every earlier column of the row was hidden
                     if (__any_sync(0xffffffffu, grow)) {
                         // rescale the accumulator: O of this row *= 2^(old ref - new ref); needs the previous PV complete
                         const float f = grow ? ex2(mref - cand) : 1.f;
@@ -381,8 +379,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                             mref = cand;
                             l *= f;
                         }
-                        const uint32_t gp = gv - 1;
-                        if (!wait_barrier(pv_done(gp & 1u), (gp >> 1) & 1u, abort_flag, p.status, 11)) { ok = false; break; }
+                        if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
                         tc_fence_after_sync();
 #pragma unroll 1
                         for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -398,10 +395,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                     }
                 }
                 // ---- P = 2^(x c2 - ref): row sum in fp32, bf16 into shared memory ----
-                const float nref = -mref;
+                // (a row whose columns were all hidden so far has ref = -inf; it gets P = 0, not 2^(-inf + inf))
+                const float nref = mref == -INFINITY ? 0.f : -mref;
                 float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
                         float x0, x1;
@@ -412,92 +410,92 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_kernel(const __g
                     }
                 }
                 l += ls0 + ls1;
-                const int ps = gv & 1u;
-                if (!wait_barrier(pv_done(ps), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // P[ps] has been read
-                if (store_pending) {
-                    bulk_wait_read();          // (lane 0) the previous item's O store has read this warp's staging rows
-                    store_pending = false;
-                }
-                __syncwarp();
+                if (last) {
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                    for (int i = 0; i < MAX_DRAFTS; ++i)
+                        if (i < m && t - i >= 0) l += ex2(fmaf(sd[i], p.c2, nref));
+                }
+                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // P has been read
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4)
-                        st_shared_v4(p_addr(ps, 4 * k + q4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
+                        st_shared_v4(p_addr(4 * k + q4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
                                      pack_bf16(v[k][8 * q4 + 2], v[k][8 * q4 + 3]), pack_bf16(v[k][8 * q4 + 4], v[k][8 * q4 + 5]),
                                      pack_bf16(v[k][8 * q4 + 6], v[k][8 * q4 + 7]));
                 }
                 fence_proxy_async_smem();      // P visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full(ps));
+                if (lane == 0) mbar_arrive(p_full);
             }
             if (!ok) break;
-            // ---- draft passes of the value sequence: P holds only the weight 2^(sd c2 - ref) on its diagonal ----
+            // ---- draft passes of the value sequence: P holds only the weights 2^(sd c2 - ref) of the rows of one
+            //      half on its diagonal ----
+            const float nref_f = mref == -INFINITY ? 0.f : -mref;
 #pragma unroll 1
-            for (int i = 0; i < m; ++i, ++gv) {
+            for (int e = 0; e < 2 * m; ++e, ++gv) {
+                const int i = e >> 1;
                 float sdi = 0.f;
 #pragma unroll
                 for (int ii = 0; ii < MAX_DRAFTS; ++ii)
                     if (ii == i) sdi = sd[ii];
-                const float pi = (t - i >= 0) ? ex2(fmaf(sdi, p.c2, -mref)) : 0.f;
-                l += pi;
-                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // column r sits in word (r & 7) / 2
-                const int ps = gv & 1u;
-                if (!wait_barrier(pv_done(ps), ((gv >> 1) & 1u) ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
+                const bool mine = (r >> 6) == (e & 1) && t - i >= 0;
+                const float pi = mine ? ex2(fmaf(sdi, p.c2, nref_f)) : 0.f;
+                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // column r & 63 sits in word (r & 7) / 2
+                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
 #pragma unroll
-                for (int chunk = 0; chunk < 16; ++chunk) {
-                    const bool here = chunk == (r >> 3);
+                for (int chunk = 0; chunk < 8; ++chunk) {
+                    const bool here = chunk == ((r & 63) >> 3);
                     const int w = (r & 7) >> 1;
-                    st_shared_v4(p_addr(ps, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
+                    st_shared_v4(p_addr(chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
                                  here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full(ps));
+                if (lane == 0) mbar_arrive(p_full);
             }
             if (!ok) break;
-            // ---- epilogue: O / l as bf16, staged in this warp's rows of P buffer 0 and stored with TMA ----
+            // ---- epilogue: O / l as bf16, each thread stores its own 256-byte row ----
             {
-                const uint32_t gp = gv - 1;
-                if (!wait_barrier(pv_done(gp & 1u), (gp >> 1) & 1u, abort_flag, p.status, 13)) break;
+                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 13)) break;
                 tc_fence_after_sync();
                 const float inv = 1.f / l;
                 if (valid && p.lse != nullptr)
                     p.lse[(static_cast<size_t>(b) * p.H + h) * p.T + t] = (mref + log2f(l)) * 0.6931471805599453f;
-                uint32_t raw[4][32];
+                __nv_bfloat16* orow = p.O + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) tmem_ld32(tmem_o + 32 * k, raw[k]);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) tmem_ld_wait(raw[k]);
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(o_free);         // the accumulator may be overwritten by the next item
-                // every PV product of the item is complete, so both P buffers are idle; the bytes used are this
-                // warp's own rows, which no other warp writes
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const uint32_t* x = &raw[k][8 * q4];
-                        st_shared_v4(p_addr(0, 4 * k + q4),
-                                     pack_bf16(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv),
-                                     pack_bf16(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv),
-                                     pack_bf16(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv),
-                                     pack_bf16(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv));
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t raw[2][32];
+                    tmem_ld32(tmem_o + 64 * hf, raw[0]);
+                    tmem_ld32(tmem_o + 64 * hf + 32, raw[1]);
+                    tmem_ld_wait(raw[0]);
+                    tmem_ld_wait(raw[1]);
+                    if (hf == 1) {
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(o_free);     // the accumulator may be overwritten by the next item
                     }
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0 && qt * QT + quad * 32 < p.T) {
-                    const uint32_t src = base + SMEM_P + quad * 32 * 128;
-                    tma_store_3d(&p.tmO, src, h * HD, qt * QT + quad * 32, b);
-                    tma_store_3d(&p.tmO, src + HALF_BYTES, h * HD + 64, qt * QT + quad * 32, b);
-                    bulk_commit();
-                    store_pending = true;
+                    if (valid) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                            for (int q8 = 0; q8 < 2; ++q8) {
+                                const uint32_t* x = &raw[k][16 * q8];
+                                st_global_v8(orow + 64 * hf + 32 * k + 16 * q8,
+                                             pack_bf16(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv),
+                                             pack_bf16(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv),
+                                             pack_bf16(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv),
+                                             pack_bf16(__uint_as_float(x[6]) * inv, __uint_as_float(x[7]) * inv),
+                                             pack_bf16(__uint_as_float(x[8]) * inv, __uint_as_float(x[9]) * inv),
+                                             pack_bf16(__uint_as_float(x[10]) * inv, __uint_as_float(x[11]) * inv),
+                                             pack_bf16(__uint_as_float(x[12]) * inv, __uint_as_float(x[13]) * inv),
+                                             pack_bf16(__uint_as_float(x[14]) * inv, __uint_as_float(x[15]) * inv));
+                            }
+                        }
+                    }
                 }
             }
         }
-        if (lane == 0) bulk_wait_all();      // O stores complete before the CTA's shared memory goes away
     }
 
     // ---- teardown ----
