@@ -167,6 +167,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
         b = bh / p.H;
         h = bh - b * p.H;
     };
+    // Items are sorted longest first; round k hands items k*G .. k*G + G-1 to the G CTAs, in alternating
+    // direction, so that a CTA that got a long item in one round gets a short one in the next.
+    auto first_item = [&](uint32_t k) {
+        const int G = gridDim.x, c = blockIdx.x;
+        return static_cast<int>(k) * G + ((k & 1u) ? G - 1 - c : c);
+    };
     // key tiles of an item: 0 .. 2 qt + 1, cut at the end of the sequence
     auto key_tiles = [&](int qt) { return min(2 * qt + 2, p.k_tiles); };
     // Per item the tensor core runs two sequences, each with its own ring counter:
@@ -196,7 +202,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 ++gv;
                 return true;
             };
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            for (int item = first_item(0); item < p.items && ok; item = first_item(++it)) {
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int col = (h / rep) * HD;
@@ -262,7 +268,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 ++gv;
                 return true;
             };
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            for (int item = first_item(0); item < p.items && ok; item = first_item(++it)) {
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int n_s = 2 * m + key_tiles(qt);
@@ -289,7 +295,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
         bool ok = true;
         // 16-byte unit `chunk` (0..7) of this thread's 128-byte row of the P buffer, as the tensor core sees it
         auto p_addr = [&](int chunk) { return base + SMEM_P + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x) {
+        for (int item = first_item(0), it = 0; item < p.items && ok; item = first_item(++it)) {
             int qt, b, h;
             decode(item, qt, b, h);
             const int n = key_tiles(qt);
