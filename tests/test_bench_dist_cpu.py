@@ -48,3 +48,19 @@ def test_reference_arm_prints_one_json_line(tmp_path):
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
+
+
+def test_reference_arm_of_the_hca_workloads(tmp_path):
+    import json
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "hca-tiny",
+                          "--steps", "2", "--warmup", "1", "--oracle-rows", "3"], capture_output=True, text=True,
+                         timeout=300)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["config"]["workload"] == "hca-tiny" and line["value"] > 0 and line["gpu_launches"] == 0
+    # a rank other than 0 leaves without printing
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "hca-tiny",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=300,
+                         env=dict(os.environ, RANK="1", WORLD_SIZE="2"))
+    assert out.returncode == 0 and out.stdout.strip() == ""

@@ -72,6 +72,9 @@ def test_small_workloads_all_heads(name):
     (2, 256, 3, 3, 0),        # first aligning step: plain causal attention
     (1, 515, 4, 2, 5),
     (2, 700, 16, 4, 2),       # more work items than SMs: every CTA takes a second item
+    (1, 4096, 2, 1, 3),       # a long sequence: 64 key tiles in the last items
+    (3, 64, 5, 5, 4),         # one key tile per item, five heads
+    (1, 70, 1, 1, 8),         # the second key tile holds only hidden columns for most rows
 ])
 def test_awkward_shapes(B, T, H, Hkv, m):
     inp = hi.make_hca_inputs(hi.HcaWorkload("custom", B=B, T=T, H=H, Hkv=Hkv, m=m, seed=T + m))
