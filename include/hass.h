@@ -272,6 +272,30 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
                            size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Backward of hass_hca_attention_fwd (Section 3.2; the paper prints the forward only, the gradients are the
+ * chain rule through it): given dO = d(loss)/dO it returns the gradients with respect to every projected
+ * input. With P the softmax weights (recomputed from lse), Dt = <dO[t], O[t]> and
+ * dS[t,s] = P[t,s] (<dO[t], v(t,s)> - Dt) scale:
+ *     dQ[t] = sum_s dS[t,s] k(t,s);   dK_t[s], dV_t[s] collect the pairs with t - s >= m;
+ *     dK_d[i][s], dV_d[i][s] collect the single pair t = s + i of every query head of the group.
+ *
+ *   Q, K_t, V_t, K_d, V_d, m, B, T, H, Hkv, D, scale   as in the forward call
+ *   O [B, T, H, D] bf16, lse [B, H, T] fp32              the forward's outputs (lse is required here)
+ *   dO [B, T, H, D] bf16
+ *   dQ [B, T, H, D], dK_t, dV_t [B, T, Hkv, D] bf16      out (32-byte aligned)
+ *   dK_d, dV_d   HOST arrays of m DEVICE pointers, each [B, T, Hkv, D] bf16, out
+ *   workspace    hass_hca_attention_bwd_workspace_bytes(B, T, H, m) bytes, 256-byte aligned
+ * Four kinds of kernels are enqueued on cuda_stream (row sums, dQ, dK_t/dV_t, one row-scaling kernel per
+ * draft pass). Errors as for the forward.
+ */
+int hass_hca_attention_bwd_workspace_bytes(int64_t B, int64_t T, int64_t H, int32_t m, size_t* bytes);
+int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,
+                           const void* const* V_d, int32_t m, int64_t B, int64_t T, int64_t H,
+                           int64_t Hkv, int64_t D, float scale, const void* O, const float* lse,
+                           const void* dO, void* dQ, void* dK_t, void* dV_t, void* const* dK_d,
+                           void* const* dV_d, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream` and returns the status word of `workspace`: HASS_OK, or
  * HASS_ERR_TIMEOUT if a kernel gave up on a bounded wait (its outputs are then undefined), or
  * HASS_ERR_CUDA if the stream reports an error. Clears the status word.
@@ -322,10 +346,10 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
  * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
  * launches of the exact route behind a fused call (they return at once unless it is needed),
- * 6 HCA attention.
+ * 6 HCA attention forward, 7 HCA attention backward (all its kernels).
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */
-#define HASS_PROFILE_KINDS 7
+#define HASS_PROFILE_KINDS 8
 int hass_profile_enable(int on);
 int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
 

@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     HASS_FP32,
     K_MAX,
     check,
+    hca_attention_bwd,
+    hca_attention_bwd_workspace_bytes,
     hca_attention_fwd,
     hca_attention_workspace_bytes,
     HCA_MAX_DRAFTS,

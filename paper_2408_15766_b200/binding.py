@@ -57,6 +57,12 @@ def _load() -> ctypes.CDLL:
     L.hass_hca_attention_fwd.argtypes = [vp, vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i64, i64, i64, i64,
                                          i64, ctypes.c_float, vp, vp, vp, sz, vp]
     L.hass_hca_attention_fwd.restype = ctypes.c_int
+    L.hass_hca_attention_bwd_workspace_bytes.argtypes = [i64, i64, i64, i32, ctypes.POINTER(sz)]
+    L.hass_hca_attention_bwd_workspace_bytes.restype = ctypes.c_int
+    L.hass_hca_attention_bwd.argtypes = [vp, vp, vp, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i64, i64, i64, i64,
+                                         i64, ctypes.c_float, vp, vp, vp, vp, vp, vp, ctypes.POINTER(vp),
+                                         ctypes.POINTER(vp), vp, sz, vp]
+    L.hass_hca_attention_bwd.restype = ctypes.c_int
     L.hass_check.argtypes = [vp, vp]
     L.hass_topk_distill_fwd_static.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     L.hass_topk_distill_fwd_static.restype = ctypes.c_int
@@ -349,13 +355,44 @@ def hca_attention_fwd(Q, K_t, V_t, K_d=(), V_d=(), scale: Optional[float] = None
     return out
 
 
+def hca_attention_bwd_workspace_bytes(B: int, T: int, H: int, m: int) -> int:
+    n = ctypes.c_size_t(0)
+    _ok(lib.hass_hca_attention_bwd_workspace_bytes(B, T, H, m, ctypes.byref(n)), "hass_hca_attention_bwd_workspace_bytes")
+    return int(n.value)
+
+
+def hca_attention_bwd(Q, K_t, V_t, K_d, V_d, O, lse, dO, scale: Optional[float] = None, workspace=None,
+                      stream=None) -> dict:
+    """HCA attention backward: gradients of every projected input. See hass_hca_attention_bwd."""
+    B, T, H, D = Q.shape
+    Hkv = K_t.shape[2]
+    m = len(K_d)
+    assert len(V_d) == m
+    for x in (Q, K_t, V_t, O, dO, *K_d, *V_d):
+        assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    assert O.shape == Q.shape and dO.shape == Q.shape and V_t.shape == K_t.shape == (B, T, Hkv, D)
+    assert lse.dtype == torch.float32 and lse.shape == (B, H, T) and lse.is_contiguous()
+    dev = Q.device
+    ws = _workspace(workspace, hca_attention_bwd_workspace_bytes(B, T, H, m), dev)
+    out = dict(dQ=torch.empty_like(Q), dK_t=torch.empty_like(K_t), dV_t=torch.empty_like(V_t),
+               dK_d=[torch.empty_like(K_t) for _ in range(m)], dV_d=[torch.empty_like(K_t) for _ in range(m)],
+               workspace=ws)
+    arr = lambda ts: (ctypes.c_void_p * max(m, 1))(*[x.data_ptr() for x in ts])
+    sc = float(scale) if scale is not None else 1.0 / (D ** 0.5)
+    _ok(lib.hass_hca_attention_bwd(_p(Q), _p(K_t), _p(V_t), arr(K_d), arr(V_d), m, B, T, H, Hkv, D, ctypes.c_float(sc),
+                                   _p(O), _p(lse), _p(dO), _p(out["dQ"]), _p(out["dK_t"]), _p(out["dV_t"]),
+                                   arr(out["dK_d"]), arr(out["dV_d"]), _p(ws), ws.numel(), _stream(stream)),
+        "hass_hca_attention_bwd")
+    return out
+
+
 def check(workspace: torch.Tensor, stream=None) -> None:
     """Synchronises the stream and raises HassError if a kernel recorded a device-side problem."""
     _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")
 
 
 PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional",
-                 "hca_attention")
+                 "hca_attention", "hca_attention_bwd")
 
 
 def profile_enable(on: bool) -> None:

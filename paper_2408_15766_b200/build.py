@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 SRC_DIR = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhass_b200.so")
 SOURCES = ["hass_api.cu"]
-HEADERS = ["kernels.cuh", "hca_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "hass.h")]
+HEADERS = ["kernels.cuh", "hca_kernels.cuh", "hca_bwd_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "hass.h")]
 
 
 def _stale() -> bool:

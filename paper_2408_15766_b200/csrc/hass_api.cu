@@ -11,6 +11,7 @@
 #include "../../include/hass.h"
 #include "kernels.cuh"
 #include "hca_kernels.cuh"
+#include "hca_bwd_kernels.cuh"
 
 namespace hass {
 
@@ -19,7 +20,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, NUM_KINDS = 7 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_BWD = 7, NUM_KINDS = 8 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -76,6 +77,8 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
             // two CTAs of this kernel share an SM: ask for the largest shared-memory carve-out
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::DQ_SMEM_BYTES);
+            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::KV_SMEM_BYTES);
             if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
                 cudaGetLastError();
                 return HASS_ERR_CUDA;
@@ -1237,6 +1240,139 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
         hca::hca_attention_kernel<<<grid, hca::NUM_THREADS, hca::SMEM_BYTES, st>>>(p);
     }
     g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+    return HASS_OK;
+}
+
+// workspace of the HCA backward: status word, D [B, H, T], and the weights and dS of the substituted entries
+struct HcaBwdLayout {
+    size_t D, Pd, dSd, total;
+};
+static HcaBwdLayout hca_bwd_layout(int64_t B, int64_t T, int64_t H, int32_t m) {
+    HcaBwdLayout L;
+    auto up = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
+    const size_t rows = static_cast<size_t>(B) * H * T;
+    L.D = 256;
+    L.Pd = up(L.D + rows * 4);
+    L.dSd = up(L.Pd + rows * 4 * (m > 0 ? m : 1));
+    L.total = up(L.dSd + rows * 4 * (m > 0 ? m : 1));
+    return L;
+}
+
+int hass_hca_attention_bwd_workspace_bytes(int64_t B, int64_t T, int64_t H, int32_t m, size_t* bytes) {
+    if (!bytes || B < 1 || T < 1 || H < 1 || m < 0 || m > HASS_HCA_MAX_DRAFTS) return HASS_ERR_INVALID_ARG;
+    *bytes = hca_bwd_layout(B, T, H, m).total;
+    return HASS_OK;
+}
+
+int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,
+                           const void* const* V_d, int32_t m, int64_t B, int64_t T, int64_t H, int64_t Hkv, int64_t D,
+                           float scale, const void* O, const float* lse, const void* dO, void* dQ, void* dK_t,
+                           void* dV_t, void* const* dK_d, void* const* dV_d, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream) {
+    if (!Q || !K_t || !V_t || !O || !lse || !dO || !dQ || !dK_t || !dV_t) return HASS_ERR_INVALID_ARG;
+    if (m < 0 || m > HASS_HCA_MAX_DRAFTS || (m > 0 && (!K_d || !V_d || !dK_d || !dV_d))) return HASS_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || H < 1 || Hkv < 1 || H % Hkv != 0 || !(scale > 0.f) || !(scale < INFINITY))
+        return HASS_ERR_INVALID_ARG;
+    if (D != hca::HD) return HASS_ERR_UNSUPPORTED;
+    if (B > 65535 || T > (1 << 22) || H > 4096 || B * H * ((T + hca::QT - 1) / hca::QT) > INT_MAX / 2)
+        return HASS_ERR_UNSUPPORTED;
+    auto mis = [](const void* q, uintptr_t a) { return (reinterpret_cast<uintptr_t>(q) & (a - 1)) != 0; };
+    if (mis(Q, 16) || mis(K_t, 16) || mis(V_t, 16) || mis(O, 16) || mis(dO, 16) || mis(lse, 4) || mis(dQ, 32) ||
+        mis(dK_t, 32) || mis(dV_t, 32))
+        return HASS_ERR_INVALID_ARG;
+    for (int i = 0; i < m; ++i)
+        if (!K_d[i] || !V_d[i] || !dK_d[i] || !dV_d[i] || mis(K_d[i], 16) || mis(V_d[i], 16) || mis(dK_d[i], 16) ||
+            mis(dV_d[i], 16))
+            return HASS_ERR_INVALID_ARG;
+    const HcaBwdLayout L = hca_bwd_layout(B, T, H, m);
+    if (!workspace || workspace_bytes < L.total || mis(workspace, 256)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    float* Dv = reinterpret_cast<float*>(ws + L.D);
+    float* Pd = reinterpret_cast<float*>(ws + L.Pd);
+    float* dSd = reinterpret_cast<float*>(ws + L.dSd);
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    const int iB = static_cast<int>(B), iT = static_cast<int>(T), iH = static_cast<int>(H), iHkv = static_cast<int>(Hkv);
+    const float c2 = scale * 1.4426950408889634f;
+
+    hca_bwd::DqParams q;
+    std::memset(&q, 0, sizeof(q));
+    rc = make_tmap_seq(&q.tmQ, Q, B, T, H * hca::HD, 128);
+    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmdO, dO, B, T, H * hca::HD, 128);
+    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmK, K_t, B, T, Hkv * hca::HD, 64);
+    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmV, V_t, B, T, Hkv * hca::HD, 64);
+    for (int i = 0; i < m && rc == HASS_OK; ++i) {
+        rc = make_tmap_seq(&q.tmKd[i], K_d[i], B, T, Hkv * hca::HD, 64);
+        if (rc == HASS_OK) rc = make_tmap_seq(&q.tmVd[i], V_d[i], B, T, Hkv * hca::HD, 64);
+    }
+    hca_bwd::DkvParams k;
+    std::memset(&k, 0, sizeof(k));
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmK, K_t, B, T, Hkv * hca::HD, 128);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmV, V_t, B, T, Hkv * hca::HD, 128);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmQ, Q, B, T, H * hca::HD, 64);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmdO, dO, B, T, H * hca::HD, 64);
+    if (rc != HASS_OK) return rc;
+
+    {   // D = rowsum(dO * O)
+        KernelTimer kt(KIND_HCA_BWD, st);
+        const long long rows = static_cast<long long>(B) * T * H;
+        hca_bwd::hca_bwd_prep_kernel<<<static_cast<unsigned>((rows * 32 + 255) / 256), 256, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Dv, iB, iT, iH);
+    }
+    g_launches.fetch_add(1);
+
+    q.dQ = static_cast<__nv_bfloat16*>(dQ);
+    q.lse = lse;
+    q.D = Dv;
+    q.Pd = Pd;
+    q.dSd = dSd;
+    q.B = iB; q.T = iT; q.H = iH; q.Hkv = iHkv; q.m = m;
+    q.q_tiles = static_cast<int>((T + 127) / 128);
+    q.k_tiles = static_cast<int>((T + 63) / 64);
+    q.items = iB * iH * q.q_tiles;
+    q.c2 = c2;
+    q.scale = scale;
+    q.status = static_cast<unsigned int*>(workspace);
+    {
+        KernelTimer kt(KIND_HCA_BWD, st);
+        hca_bwd::hca_dq_kernel<<<q.items < di.sms ? q.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::DQ_SMEM_BYTES, st>>>(q);
+    }
+    g_launches.fetch_add(1);
+
+    k.dK = static_cast<__nv_bfloat16*>(dK_t);
+    k.dV = static_cast<__nv_bfloat16*>(dV_t);
+    k.lse = lse;
+    k.D = Dv;
+    k.B = iB; k.T = iT; k.H = iH; k.Hkv = iHkv; k.m = m;
+    k.kt_tiles = static_cast<int>((T + 127) / 128);
+    k.q_tiles64 = static_cast<int>((T + 63) / 64);
+    k.items = iB * iHkv * k.kt_tiles;
+    k.c2 = c2;
+    k.scale = scale;
+    k.status = static_cast<unsigned int*>(workspace);
+    {
+        KernelTimer kt(KIND_HCA_BWD, st);
+        hca_bwd::hca_dkv_kernel<<<k.items < di.sms ? k.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::KV_SMEM_BYTES, st>>>(k);
+    }
+    g_launches.fetch_add(1);
+
+    for (int i = 0; i < m; ++i) {
+        KernelTimer kt(KIND_HCA_BWD, st);
+        const long long warps = static_cast<long long>(B) * T * Hkv;
+        hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd,
+            static_cast<__nv_bfloat16*>(dK_d[i]), static_cast<__nv_bfloat16*>(dV_d[i]), i, m, iB, iT, iH, iHkv);
+        g_launches.fetch_add(1);
+    }
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     return HASS_OK;
 }

@@ -1,0 +1,772 @@
+// Backward of the HCA attention (Section 3.2) for sm_100a. With P = softmax weights (recomputed from the
+// forward's row normaliser), D[t] = <dO[t], O[t]> and dS = P * (dP - D) * scale, dP[t,s] = <dO[t], v(t,s)>:
+//   dQ[t]    = sum_s dS[t,s] k(t,s)                                  hca_dq_kernel (query tiles stationary)
+//   dK_t[s]  = sum_{t: t-s >= m} dS[t,s] Q[t],  dV_t[s] = sum_{t: t-s >= m} P[t,s] dO[t]
+//                                                                    hca_dkv_kernel (key tiles stationary)
+//   dK_d[i][s] = dS[s+i,s] Q[s+i],  dV_d[i][s] = P[s+i,s] dO[s+i]    hca_draft_grad_kernel (one term per
+//                                                                    query head of the group: row scalings)
+// hca_dq_kernel also leaves P and dS of the substituted entries (t, t-i) in the workspace for the last one.
+//
+// Both tensor-core kernels follow the forward kernel's organisation (warp 0 TMA producer, warp 1 MMA issuer
+// and TMEM owner, warps 2-5 one tile row per thread) and its bounded waits.
+#pragma once
+#include "hca_kernels.cuh"
+
+namespace hass {
+namespace hca_bwd {
+
+using hca::ex2;
+using hca::pack_bf16;
+using hca::st_shared_v4;
+using hca::tma_load_3d;
+
+constexpr int QT = 128;
+constexpr int KT = 64;
+constexpr int HD = 128;
+constexpr int MAX_DRAFTS = hca::MAX_DRAFTS;
+constexpr int NUM_THREADS = 192;
+constexpr int Q_BYTES = QT * HD * 2;
+constexpr int Q_HALF = Q_BYTES / 2;
+constexpr int KV_BYTES = KT * HD * 2;
+constexpr int KV_HALF = KV_BYTES / 2;
+constexpr int DS_BYTES = QT * KT * 2;
+
+// D[b, h, t] = <dO[b, t, h, :], O[b, t, h, :]>, one warp per row of 128.
+__global__ void hca_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
+                                    float* __restrict__ D, int B, int T, int H) {
+    const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, t, h)
+    const int lane = threadIdx.x & 31;
+    if (row >= static_cast<long long>(B) * T * H) return;
+    const uint2 a = __ldg(reinterpret_cast<const uint2*>(O + row * HD) + lane);
+    const uint2 c = __ldg(reinterpret_cast<const uint2*>(dO + row * HD) + lane);
+    auto lo = [](uint32_t w) { return __uint_as_float(w << 16); };
+    auto hi = [](uint32_t w) { return __uint_as_float(w & 0xffff0000u); };
+    float acc = lo(a.x) * lo(c.x) + hi(a.x) * hi(c.x) + lo(a.y) * lo(c.y) + hi(a.y) * hi(c.y);
+#pragma unroll
+    for (int sft = 16; sft >= 1; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+    if (lane == 0) {
+        const int h = static_cast<int>(row % H);
+        const long long bt = row / H;
+        const int t = static_cast<int>(bt % T);
+        const int b = static_cast<int>(bt / T);
+        D[(static_cast<long long>(b) * H + h) * T + t] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// dQ: a work item is (sequence, query head, tile of 128 query positions). Every element of its sweep - a key
+// tile of 64 keys, or half h of draft pass i fetched i rows early (the substituted entries sit on its
+// diagonal) - takes the same route: K and V stage by TMA; S = Q K^T and dP = dO V^T into TMEM; the row's
+// thread forms dS (full row, or its diagonal element only) as bf16 in shared memory; dQ += dS K with the
+// same K stage read MN-major.
+constexpr int DQ_SMEM_Q = 0;
+constexpr int DQ_SMEM_DO = DQ_SMEM_Q + Q_BYTES;
+constexpr int DQ_SMEM_K = DQ_SMEM_DO + Q_BYTES;        // 2 stages
+constexpr int DQ_SMEM_V = DQ_SMEM_K + 2 * KV_BYTES;    // 2 stages
+constexpr int DQ_SMEM_DS = DQ_SMEM_V + 2 * KV_BYTES;   // 2 buffers
+constexpr int DQ_SMEM_BAR = DQ_SMEM_DS + 2 * DS_BYTES;
+constexpr int DQ_NUM_BARS = 16;
+constexpr int DQ_SMEM_BYTES = DQ_SMEM_BAR + 256 + 1024 /*alignment slack*/;
+constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb, dP at 128 sb + 64; dQ at 256
+
+struct DqParams {
+    CUtensorMap tmQ, tmdO;         // [B, T, H * 128], box {64, 128, 1}
+    CUtensorMap tmK, tmV;          // [B, T, Hkv * 128], box {64, 64, 1}
+    CUtensorMap tmKd[MAX_DRAFTS];
+    CUtensorMap tmVd[MAX_DRAFTS];
+    __nv_bfloat16* dQ;             // [B, T, H, 128]
+    const float* lse;              // [B, H, T] natural-log normaliser from the forward
+    const float* D;                // [B, H, T]
+    float* Pd;                     // [B, H, T, m] weight of the substituted entry (t, t - i)
+    float* dSd;                    // [B, H, T, m] its dS
+    int B, T, H, Hkv, m;
+    int q_tiles, k_tiles, items;
+    float c2;                      // scale * log2(e)
+    float scale;
+    unsigned int* status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_constant__ DqParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar0 = base + DQ_SMEM_BAR;
+    const uint32_t qdo_full = bar0, qdo_empty = bar0 + 8;
+    auto kv_full = [&](int s) { return bar0 + 8u * (2 + s); };
+    auto kv_empty = [&](int s) { return bar0 + 8u * (4 + s); };
+    auto sdp_full = [&](int s) { return bar0 + 8u * (6 + s); };
+    auto sdp_empty = [&](int s) { return bar0 + 8u * (8 + s); };
+    auto ds_full = [&](int s) { return bar0 + 8u * (10 + s); };
+    auto ds_empty = [&](int s) { return bar0 + 8u * (12 + s); };
+    const uint32_t dq_done = bar0 + 8u * 14, dq_free = bar0 + 8u * 15;
+    uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + DQ_SMEM_BAR + 8 * DQ_NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(qdo_full, 1);
+        mbar_init(qdo_empty, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(kv_full(s), 1);
+            mbar_init(kv_empty(s), 1);
+            mbar_init(sdp_full(s), 1);
+            mbar_init(sdp_empty(s), 4);
+            mbar_init(ds_full(s), 4);
+            mbar_init(ds_empty(s), 1);
+        }
+        mbar_init(dq_done, 1);
+        mbar_init(dq_free, 4);
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&p.tmQ);
+        prefetch_tensormap(&p.tmdO);
+        prefetch_tensormap(&p.tmK);
+        prefetch_tensormap(&p.tmV);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_ptr_smem), DQ_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    const int BH = p.B * p.H;
+    const int rep = p.H / p.Hkv;
+    const int m = p.m;
+    auto decode = [&](int item, int& qt, int& b, int& h) {
+        qt = p.q_tiles - 1 - item / BH;
+        const int bh = item - (item / BH) * BH;
+        b = bh / p.H;
+        h = bh - b * p.H;
+    };
+    auto key_tiles = [&](int qt) { return min(2 * qt + 2, p.k_tiles); };
+    // elements of an item: key tiles 0 .. n-1, then draft pass i, half h (element n + 2i + h)
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t g = 0, it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+                int qt, b, h;
+                decode(item, qt, b, h);
+                const int col = (h / rep) * HD;
+                const int n = key_tiles(qt);
+                if (!wait_barrier(qdo_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1)) break;
+                mbar_arrive_expect_tx(qdo_full, 2 * Q_BYTES);
+                tma_load_3d(base + DQ_SMEM_Q, &p.tmQ, qdo_full, h * HD, qt * QT, b);
+                tma_load_3d(base + DQ_SMEM_Q + Q_HALF, &p.tmQ, qdo_full, h * HD + 64, qt * QT, b);
+                tma_load_3d(base + DQ_SMEM_DO, &p.tmdO, qdo_full, h * HD, qt * QT, b);
+                tma_load_3d(base + DQ_SMEM_DO + Q_HALF, &p.tmdO, qdo_full, h * HD + 64, qt * QT, b);
+                for (int e = 0; e < n + 2 * m && ok; ++e, ++g) {
+                    const int s = g & 1u;
+                    if (!wait_barrier(kv_empty(s), ((g >> 1) & 1u) ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
+                    const int d = e - n;
+                    const CUtensorMap* tk = e < n ? &p.tmK : &p.tmKd[d >> 1];
+                    const CUtensorMap* tv = e < n ? &p.tmV : &p.tmVd[d >> 1];
+                    const int row = e < n ? e * KT : qt * QT + 64 * (d & 1) - (d >> 1);
+                    mbar_arrive_expect_tx(kv_full(s), 2 * KV_BYTES);
+                    tma_load_3d(base + DQ_SMEM_K + s * KV_BYTES, tk, kv_full(s), col, row, b);
+                    tma_load_3d(base + DQ_SMEM_K + s * KV_BYTES + KV_HALF, tk, kv_full(s), col + 64, row, b);
+                    tma_load_3d(base + DQ_SMEM_V + s * KV_BYTES, tv, kv_full(s), col, row, b);
+                    tma_load_3d(base + DQ_SMEM_V + s * KV_BYTES + KV_HALF, tv, kv_full(s), col + 64, row, b);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
+            constexpr uint32_t idesc_q = make_idesc_bf16(QT, HD, 0, 1);
+            uint32_t gs = 0, gq = 0, it = 0;      // elements whose S/dP, resp. dQ product has been issued
+            bool ok = true;
+            auto issue_sdp = [&]() -> bool {
+                const int s = gs & 1u;
+                const uint32_t ph = (gs >> 1) & 1u;
+                if (!wait_barrier(kv_full(s), ph, abort_flag, p.status, 4)) return false;
+                if (!wait_barrier(sdp_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k) {
+                    const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
+                    umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + DQ_SMEM_Q + qo, 0, 1024),
+                              make_smem_desc_sw128(base + DQ_SMEM_K + s * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k) {
+                    const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
+                    umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + DQ_SMEM_DO + qo, 0, 1024),
+                              make_smem_desc_sw128(base + DQ_SMEM_V + s * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                }
+                umma_commit(sdp_full(s));
+                ++gs;
+                return true;
+            };
+            auto issue_dq = [&](bool first, bool last) -> bool {
+                const int s = gq & 1u;
+                if (!wait_barrier(ds_full(s), (gq >> 1) & 1u, abort_flag, p.status, 7)) return false;
+                if (first && !wait_barrier(dq_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < KT / 16; ++k)
+                    umma_bf16(tmem_base + 256, make_smem_desc_sw128(base + DQ_SMEM_DS + s * DS_BYTES + k * 32, 0, 1024),
+                              make_smem_desc_sw128(base + DQ_SMEM_K + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_q,
+                              (!first || k != 0) ? 1u : 0u);
+                umma_commit(kv_empty(s));
+                umma_commit(ds_empty(s));
+                if (last) umma_commit(dq_done);
+                ++gq;
+                return true;
+            };
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+                int qt, b, h;
+                decode(item, qt, b, h);
+                const int n_e = key_tiles(qt) + 2 * m;
+                if (!wait_barrier(qdo_full, it & 1u, abort_flag, p.status, 6)) break;
+                if (!issue_sdp()) break;
+                if (n_e == 1) umma_commit(qdo_empty);
+                for (int a = 0; a < n_e && ok; ++a) {
+                    if (a + 1 < n_e) {
+                        ok = issue_sdp();
+                        if (ok && a + 2 == n_e) umma_commit(qdo_empty);
+                    }
+                    if (ok) ok = issue_dq(a == 0, a + 1 == n_e);
+                }
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+        uint32_t g = 0, it = 0;
+        bool ok = true;
+        auto ds_addr = [&](int s, int chunk) {
+            return base + DQ_SMEM_DS + s * DS_BYTES + r * 128 + (((chunk ^ (r & 7)) & 7) << 4);
+        };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            int qt, b, h;
+            decode(item, qt, b, h);
+            const int n = key_tiles(qt);
+            const int t = qt * QT + r;
+            const bool valid = t < p.T;
+            const size_t row_idx = (static_cast<size_t>(b) * p.H + h) * p.T + (valid ? t : 0);
+            // P = 2^(S c2 - lse2); a row outside the sequence gets P = 0 through lse2 = +inf
+            const float nlse2 = valid ? -p.lse[row_idx] * 1.4426950408889634f : -INFINITY;
+            const float Dt = valid ? p.D[row_idx] : 0.f;
+            for (int e = 0; e < n + 2 * m; ++e, ++g) {
+                const int s = g & 1u;
+                const uint32_t ph = (g >> 1) & 1u;
+                if (!wait_barrier(sdp_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr;
+                if (e < n) {
+                    // ---- key tile: dS for the whole row ----
+                    const bool band = e * KT + KT - 1 > qt * QT - m;
+                    const int lim = t - m - e * KT;
+                    uint32_t sr[2][32], dr[2][32];
+                    tmem_ld32(tmem_s, sr[0]);
+                    tmem_ld32(tmem_s + 32, sr[1]);
+                    tmem_ld32(tmem_s + 64, dr[0]);
+                    tmem_ld32(tmem_s + 96, dr[1]);
+                    tmem_ld_wait(sr[0]);
+                    tmem_ld_wait(sr[1]);
+                    tmem_ld_wait(dr[0]);
+                    tmem_ld_wait(dr[1]);
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sdp_empty(s));
+                    float ds[2][32];
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            float pw = ex2(fmaf(__uint_as_float(sr[k][c]), p.c2, nlse2));
+                            if (band && 32 * k + c > lim) pw = 0.f;
+                            ds[k][c] = pw * (__uint_as_float(dr[k][c]) - Dt) * p.scale;
+                        }
+                    }
+                    if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            st_shared_v4(ds_addr(s, 4 * k + q4), pack_bf16(ds[k][8 * q4], ds[k][8 * q4 + 1]),
+                                         pack_bf16(ds[k][8 * q4 + 2], ds[k][8 * q4 + 3]),
+                                         pack_bf16(ds[k][8 * q4 + 4], ds[k][8 * q4 + 5]),
+                                         pack_bf16(ds[k][8 * q4 + 6], ds[k][8 * q4 + 7]));
+                    }
+                } else {
+                    // ---- draft pass i, half hf: only the diagonal element of the rows of that half ----
+                    const int i = (e - n) >> 1, hf = (e - n) & 1;
+                    float sv = 0.f, dv = 0.f;
+                    if ((quad >> 1) == hf) {
+                        uint32_t sr[32], dr[32];
+                        tmem_ld32(tmem_s + 32 * (quad & 1), sr);
+                        tmem_ld32(tmem_s + 64 + 32 * (quad & 1), dr);
+                        tmem_ld_wait(sr);
+                        tmem_ld_wait(dr);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            if (c == lane) {
+                                sv = __uint_as_float(sr[c]);
+                                dv = __uint_as_float(dr[c]);
+                            }
+                        }
+                    }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sdp_empty(s));
+                    const bool mine = (r >> 6) == hf && t - i >= 0 && valid;
+                    const float pw = mine ? ex2(fmaf(sv, p.c2, nlse2)) : 0.f;
+                    const float dsv = pw * (dv - Dt) * p.scale;
+                    if ((r >> 6) == hf && valid) {
+                        p.Pd[row_idx * m + i] = pw;
+                        p.dSd[row_idx * m + i] = dsv;
+                    }
+                    const uint32_t bits = pack_bf16(dsv, 0.f) << ((r & 1) * 16);
+                    if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
+#pragma unroll
+                    for (int chunk = 0; chunk < 8; ++chunk) {
+                        const bool here = chunk == ((r & 63) >> 3);
+                        const int w = (r & 7) >> 1;
+                        st_shared_v4(ds_addr(s, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
+                                     here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ds_full(s));
+            }
+            if (!ok) break;
+            // ---- epilogue: dQ as bf16, each thread stores its own 256-byte row ----
+            if (!wait_barrier(dq_done, it & 1u, abort_flag, p.status, 13)) break;
+            tc_fence_after_sync();
+            __nv_bfloat16* orow = p.dQ + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t raw[2][32];
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * hf, raw[0]);
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * hf + 32, raw[1]);
+                tmem_ld_wait(raw[0]);
+                tmem_ld_wait(raw[1]);
+                if (hf == 1) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(dq_free);
+                }
+                if (valid) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int q8 = 0; q8 < 2; ++q8) {
+                            const uint32_t* x = &raw[k][16 * q8];
+                            st_global_v8(orow + 64 * hf + 32 * k + 16 * q8,
+                                         pack_bf16(__uint_as_float(x[0]), __uint_as_float(x[1])),
+                                         pack_bf16(__uint_as_float(x[2]), __uint_as_float(x[3])),
+                                         pack_bf16(__uint_as_float(x[4]), __uint_as_float(x[5])),
+                                         pack_bf16(__uint_as_float(x[6]), __uint_as_float(x[7])),
+                                         pack_bf16(__uint_as_float(x[8]), __uint_as_float(x[9])),
+                                         pack_bf16(__uint_as_float(x[10]), __uint_as_float(x[11])),
+                                         pack_bf16(__uint_as_float(x[12]), __uint_as_float(x[13])),
+                                         pack_bf16(__uint_as_float(x[14]), __uint_as_float(x[15])));
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, DQ_TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// dK_t, dV_t: a work item is (sequence, key/value head, tile of 128 key positions), kept in shared memory; it
+// sweeps the query heads of its group and, per head, the tiles of 64 queries at or after it. Per element:
+//   S^T = K Q^T and dP^T = V dO^T      tcgen05.mma, 128 x 64 x 128, into TMEM (rows = keys, one per thread)
+//   threads                             P^T = 2^(S^T c2 - lse2[t]) on the entries the target's keys really met
+//                                       (t - s >= m), dS^T = P^T (dP^T - D[t]) scale; both as bf16 in shared memory
+//   dV += P^T dO, dK += dS^T Q          the Q / dO stage read MN-major
+// The per-query vectors -lse2[t] and D[t] of an element travel with its Q / dO stage: the producer warp's
+// lanes copy them into shared memory next to the TMA loads.
+constexpr int KV_SMEM_K = 0;                               // 128 keys x 128: two halves of 16 KB
+constexpr int KV_SMEM_V = KV_SMEM_K + Q_BYTES;
+constexpr int KV_SMEM_Q = KV_SMEM_V + Q_BYTES;             // 2 stages of 64 queries
+constexpr int KV_SMEM_DO = KV_SMEM_Q + 2 * KV_BYTES;       // 2 stages
+constexpr int KV_SMEM_PT = KV_SMEM_DO + 2 * KV_BYTES;      // P^T, 128 x 64 bf16
+constexpr int KV_SMEM_DST = KV_SMEM_PT + DS_BYTES;         // dS^T
+constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // 2 stages x (64 x -lse2, 64 x D) floats
+constexpr int KV_SMEM_BAR = KV_SMEM_VEC + 2 * 512;
+constexpr int KV_NUM_BARS = 14;
+constexpr int KV_SMEM_BYTES = KV_SMEM_BAR + 256 + 1024 /*alignment slack*/;
+constexpr int KV_TMEM_COLS = 512;   // buffer sb: S^T at 128 sb, dP^T at 128 sb + 64; dV at 256, dK at 384
+
+struct DkvParams {
+    CUtensorMap tmK, tmV;          // [B, T, Hkv * 128], box {64, 128, 1}
+    CUtensorMap tmQ, tmdO;         // [B, T, H * 128], box {64, 64, 1}
+    __nv_bfloat16* dK;             // [B, T, Hkv, 128]
+    __nv_bfloat16* dV;
+    const float* lse;              // [B, H, T]
+    const float* D;                // [B, H, T]
+    int B, T, H, Hkv, m;
+    int kt_tiles;                  // ceil(T / 128) key tiles
+    int q_tiles64;                 // ceil(T / 64) query tiles
+    int items;                     // B * Hkv * kt_tiles
+    float c2, scale;
+    unsigned int* status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_constant__ DkvParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar0 = base + KV_SMEM_BAR;
+    const uint32_t kv_full = bar0, kv_empty = bar0 + 8;
+    auto qd_full = [&](int s) { return bar0 + 8u * (2 + s); };
+    auto qd_empty = [&](int s) { return bar0 + 8u * (4 + s); };
+    auto st_full = [&](int s) { return bar0 + 8u * (6 + s); };
+    auto st_empty = [&](int s) { return bar0 + 8u * (8 + s); };
+    const uint32_t pds_full = bar0 + 8u * 10, pds_empty = bar0 + 8u * 11;
+    const uint32_t acc_done = bar0 + 8u * 12, acc_free = bar0 + 8u * 13;
+    uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + KV_SMEM_BAR + 8 * KV_NUM_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
+    float* vec = reinterpret_cast<float*>(smem_gen + KV_SMEM_VEC);     // [stage][0..63 -lse2 | 64..127 D]
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_full, 1);
+        mbar_init(kv_empty, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(qd_full(s), 2);      // the TMA transaction's arrival and the producer warp's vectors
+            mbar_init(qd_empty(s), 1);
+            mbar_init(st_full(s), 1);
+            mbar_init(st_empty(s), 4);
+        }
+        mbar_init(pds_full, 4);
+        mbar_init(pds_empty, 1);
+        mbar_init(acc_done, 1);
+        mbar_init(acc_free, 4);
+        *abort_flag = 0;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        prefetch_tensormap(&p.tmK);
+        prefetch_tensormap(&p.tmV);
+        prefetch_tensormap(&p.tmQ);
+        prefetch_tensormap(&p.tmdO);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_ptr_smem), KV_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    const int BG = p.B * p.Hkv;
+    const int rep = p.H / p.Hkv;
+    const int m = p.m;
+    // item -> (key tile, sequence, key/value head): the first key tiles meet the most queries and come first
+    auto decode = [&](int item, int& kt, int& b, int& g) {
+        kt = item / BG;
+        const int bg = item - kt * BG;
+        b = bg / p.Hkv;
+        g = bg - b * p.Hkv;
+    };
+    // elements of an item: for each head of the group, the 64-query tiles 2 kt .. q_tiles64 - 1
+    auto q_count = [&](int kt) { return p.q_tiles64 - 2 * kt; };
+
+    if (warp == 0) {
+        // ===================== producer: TMA by lane 0, the per-query vectors by all lanes =====================
+        uint32_t gq = 0, it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            int kt, b, g;
+            decode(item, kt, b, g);
+            const int nq = q_count(kt);
+            if (lane == 0) {
+                ok = wait_barrier(kv_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1);
+                if (ok) {
+                    mbar_arrive_expect_tx(kv_full, 2 * Q_BYTES);
+                    tma_load_3d(base + KV_SMEM_K, &p.tmK, kv_full, g * HD, kt * QT, b);
+                    tma_load_3d(base + KV_SMEM_K + Q_HALF, &p.tmK, kv_full, g * HD + 64, kt * QT, b);
+                    tma_load_3d(base + KV_SMEM_V, &p.tmV, kv_full, g * HD, kt * QT, b);
+                    tma_load_3d(base + KV_SMEM_V + Q_HALF, &p.tmV, kv_full, g * HD + 64, kt * QT, b);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            for (int e = 0; e < rep * nq && ok; ++e, ++gq) {
+                const int h = g * rep + e / nq;
+                const int jq = 2 * kt + e % nq;
+                const int s = gq & 1u;
+                if (lane == 0) ok = wait_barrier(qd_empty(s), ((gq >> 1) & 1u) ^ 1u, abort_flag, p.status, 2);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(qd_full(s), 2 * KV_BYTES);
+                    tma_load_3d(base + KV_SMEM_Q + s * KV_BYTES, &p.tmQ, qd_full(s), h * HD, jq * KT, b);
+                    tma_load_3d(base + KV_SMEM_Q + s * KV_BYTES + KV_HALF, &p.tmQ, qd_full(s), h * HD + 64, jq * KT, b);
+                    tma_load_3d(base + KV_SMEM_DO + s * KV_BYTES, &p.tmdO, qd_full(s), h * HD, jq * KT, b);
+                    tma_load_3d(base + KV_SMEM_DO + s * KV_BYTES + KV_HALF, &p.tmdO, qd_full(s), h * HD + 64, jq * KT, b);
+                }
+                // -lse2[t] (or -inf past the sequence, which zeroes the weight) and D[t] for the 64 queries
+                const size_t rowbase = (static_cast<size_t>(b) * p.H + h) * p.T;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int c = lane + 32 * u;
+                    const int t = jq * KT + c;
+                    vec[s * 128 + c] = t < p.T ? -p.lse[rowbase + t] * 1.4426950408889634f : -INFINITY;
+                    vec[s * 128 + 64 + c] = t < p.T ? p.D[rowbase + t] : 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(qd_full(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
+            constexpr uint32_t idesc_a = make_idesc_bf16(QT, HD, 0, 1);
+            uint32_t gs = 0, ga = 0, it = 0;
+            bool ok = true;
+            auto issue_st = [&]() -> bool {
+                const int s = gs & 1u;
+                const uint32_t ph = (gs >> 1) & 1u;
+                if (!wait_barrier(qd_full(s), ph, abort_flag, p.status, 4)) return false;
+                if (!wait_barrier(st_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k) {
+                    const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
+                    umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + KV_SMEM_K + ao, 0, 1024),
+                              make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                }
+#pragma unroll
+                for (int k = 0; k < HD / 16; ++k) {
+                    const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
+                    umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + KV_SMEM_V + ao, 0, 1024),
+                              make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                }
+                umma_commit(st_full(s));
+                ++gs;
+                return true;
+            };
+            auto issue_acc = [&](bool first, bool last) -> bool {
+                const int s = ga & 1u;
+                if (!wait_barrier(pds_full, ga & 1u, abort_flag, p.status, 7)) return false;
+                if (first && !wait_barrier(acc_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < KT / 16; ++k)
+                    umma_bf16(tmem_base + 256, make_smem_desc_sw128(base + KV_SMEM_PT + k * 32, 0, 1024),
+                              make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
+                              (!first || k != 0) ? 1u : 0u);
+#pragma unroll
+                for (int k = 0; k < KT / 16; ++k)
+                    umma_bf16(tmem_base + 384, make_smem_desc_sw128(base + KV_SMEM_DST + k * 32, 0, 1024),
+                              make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
+                              (!first || k != 0) ? 1u : 0u);
+                umma_commit(qd_empty(s));
+                umma_commit(pds_empty);
+                if (last) umma_commit(acc_done);
+                ++ga;
+                return true;
+            };
+            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+                int kt, b, g;
+                decode(item, kt, b, g);
+                const int n_e = rep * q_count(kt);
+                if (!wait_barrier(kv_full, it & 1u, abort_flag, p.status, 6)) break;
+                if (!issue_st()) break;
+                if (n_e == 1) umma_commit(kv_empty);
+                for (int a = 0; a < n_e && ok; ++a) {
+                    if (a + 1 < n_e) {
+                        ok = issue_st();
+                        if (ok && a + 2 == n_e) umma_commit(kv_empty);     // K and V are free once the last S^T / dP^T has read them
+                    }
+                    if (ok) ok = issue_acc(a == 0, a + 1 == n_e);
+                }
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                 // key row of the tile
+        const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+        uint32_t gq = 0, it = 0;
+        bool ok = true;
+        auto row_addr = [&](int buf_off, int chunk) { return base + buf_off + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
+        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            int kt, b, g;
+            decode(item, kt, b, g);
+            const int nq = q_count(kt);
+            const int spos = kt * QT + r;               // key position
+            for (int e = 0; e < rep * nq; ++e, ++gq) {
+                const int jq = 2 * kt + e % nq;
+                const int s = gq & 1u;
+                const uint32_t ph = (gq >> 1) & 1u;
+                if (!wait_barrier(st_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
+                if (!wait_barrier(qd_full(s), ph, abort_flag, p.status, 15)) { ok = false; break; }   // the element's vectors
+                tc_fence_after_sync();
+                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr;
+                // the target's key at spos met query t only if t - spos >= m: columns below lo are empty
+                const int lo = spos + m - jq * KT;
+                const bool band = lo > 0;
+                uint32_t sr[2][32], dr[2][32];
+                tmem_ld32(tmem_s, sr[0]);
+                tmem_ld32(tmem_s + 32, sr[1]);
+                tmem_ld32(tmem_s + 64, dr[0]);
+                tmem_ld32(tmem_s + 96, dr[1]);
+                tmem_ld_wait(sr[0]);
+                tmem_ld_wait(sr[1]);
+                tmem_ld_wait(dr[0]);
+                tmem_ld_wait(dr[1]);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(st_empty(s));
+                const float4* nl = reinterpret_cast<const float4*>(vec + s * 128);
+                const float4* dd = reinterpret_cast<const float4*>(vec + s * 128 + 64);
+                float pw[2][32], ds[2][32];
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4) {
+                        const float4 a = nl[8 * k + c4], d = dd[8 * k + c4];
+                        const float av[4] = {a.x, a.y, a.z, a.w}, dv[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int c = 4 * c4 + u;
+                            float w = ex2(fmaf(__uint_as_float(sr[k][c]), p.c2, av[u]));
+                            if (band && 32 * k + c < lo) w = 0.f;
+                            pw[k][c] = w;
+                            ds[k][c] = w * (__uint_as_float(dr[k][c]) - dv[u]) * p.scale;
+                        }
+                    }
+                }
+                if (!wait_barrier(pds_empty, (gq & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        st_shared_v4(row_addr(KV_SMEM_PT, 4 * k + q4), pack_bf16(pw[k][8 * q4], pw[k][8 * q4 + 1]),
+                                     pack_bf16(pw[k][8 * q4 + 2], pw[k][8 * q4 + 3]),
+                                     pack_bf16(pw[k][8 * q4 + 4], pw[k][8 * q4 + 5]),
+                                     pack_bf16(pw[k][8 * q4 + 6], pw[k][8 * q4 + 7]));
+                        st_shared_v4(row_addr(KV_SMEM_DST, 4 * k + q4), pack_bf16(ds[k][8 * q4], ds[k][8 * q4 + 1]),
+                                     pack_bf16(ds[k][8 * q4 + 2], ds[k][8 * q4 + 3]),
+                                     pack_bf16(ds[k][8 * q4 + 4], ds[k][8 * q4 + 5]),
+                                     pack_bf16(ds[k][8 * q4 + 6], ds[k][8 * q4 + 7]));
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pds_full);
+            }
+            if (!ok) break;
+            // ---- epilogue: this key row of dV and dK as bf16 ----
+            if (!wait_barrier(acc_done, it & 1u, abort_flag, p.status, 13)) break;
+            tc_fence_after_sync();
+            const bool valid = spos < p.T;
+            const size_t orow = ((static_cast<size_t>(b) * p.T + (valid ? spos : 0)) * p.Hkv + g) * HD;
+#pragma unroll
+            for (int part = 0; part < 4; ++part) {      // dV columns 0..63, 64..127, then dK likewise
+                __nv_bfloat16* dst = (part < 2 ? p.dV : p.dK) + orow + 64 * (part & 1);
+                uint32_t raw[2][32];
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * part, raw[0]);
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * part + 32, raw[1]);
+                tmem_ld_wait(raw[0]);
+                tmem_ld_wait(raw[1]);
+                if (part == 3) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_free);
+                }
+                if (valid) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int q8 = 0; q8 < 2; ++q8) {
+                            const uint32_t* x = &raw[k][16 * q8];
+                            st_global_v8(dst + 32 * k + 16 * q8, pack_bf16(__uint_as_float(x[0]), __uint_as_float(x[1])),
+                                         pack_bf16(__uint_as_float(x[2]), __uint_as_float(x[3])),
+                                         pack_bf16(__uint_as_float(x[4]), __uint_as_float(x[5])),
+                                         pack_bf16(__uint_as_float(x[6]), __uint_as_float(x[7])),
+                                         pack_bf16(__uint_as_float(x[8]), __uint_as_float(x[9])),
+                                         pack_bf16(__uint_as_float(x[10]), __uint_as_float(x[11])),
+                                         pack_bf16(__uint_as_float(x[12]), __uint_as_float(x[13])),
+                                         pack_bf16(__uint_as_float(x[14]), __uint_as_float(x[15])));
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, KV_TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Gradients of the draft passes' keys and values: position s of pass i meets exactly one query per head,
+// t = s + i, so dK_d[i][s] = sum over the group's query heads of dS[t, s] Q[t] and likewise for the values.
+// One warp per (sequence, position s, key/value head, pass i); lane = 4 of the 128 columns.
+__global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
+                                      const float* __restrict__ Pd, const float* __restrict__ dSd,
+                                      __nv_bfloat16* dKd, __nv_bfloat16* dVd, int i, int m, int B, int T, int H,
+                                      int Hkv) {
+    const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, s, g)
+    const int lane = threadIdx.x & 31;
+    if (w >= static_cast<long long>(B) * T * Hkv) return;
+    const int g = static_cast<int>(w % Hkv);
+    const long long bs = w / Hkv;
+    const int s = static_cast<int>(bs % T);
+    const int b = static_cast<int>(bs / T);
+    const int t = s + i;
+    const int rep = H / Hkv;
+    auto lo = [](uint32_t x) { return __uint_as_float(x << 16); };
+    auto hi = [](uint32_t x) { return __uint_as_float(x & 0xffff0000u); };
+    float k0 = 0.f, k1 = 0.f, k2 = 0.f, k3 = 0.f, v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+    if (t < T) {
+        for (int hh = 0; hh < rep; ++hh) {
+            const int h = g * rep + hh;
+            const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m + i;
+            const float pw = Pd[ri], ds = dSd[ri];
+            const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
+            const uint2 q = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
+            const uint2 d = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
+            k0 = fmaf(ds, lo(q.x), k0);
+            k1 = fmaf(ds, hi(q.x), k1);
+            k2 = fmaf(ds, lo(q.y), k2);
+            k3 = fmaf(ds, hi(q.y), k3);
+            v0 = fmaf(pw, lo(d.x), v0);
+            v1 = fmaf(pw, hi(d.x), v1);
+            v2 = fmaf(pw, lo(d.y), v2);
+            v3 = fmaf(pw, hi(d.y), v3);
+        }
+    }
+    const size_t orow = ((static_cast<size_t>(b) * T + s) * Hkv + g) * HD;
+    *(reinterpret_cast<uint2*>(dKd + orow) + lane) = make_uint2(pack_bf16(k0, k1), pack_bf16(k2, k3));
+    *(reinterpret_cast<uint2*>(dVd + orow) + lane) = make_uint2(pack_bf16(v0, v1), pack_bf16(v2, v3));
+}
+
+}  // namespace hca_bwd
+}  // namespace hass
