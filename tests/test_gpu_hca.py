@@ -121,3 +121,69 @@ def test_full_size_sampled_heads(name):
     O, lse = _run(inp)
     pairs = [(0, 0), (wl.B - 1, wl.H - 1), (1, 5), (2, wl.H // 2 + 1)]
     print(_compare(inp, O, lse, pairs=pairs))
+
+
+# ---- backward ---------------------------------------------------------------------------------------
+# Tolerance: every gradient within 1.5e-2 of its tensor's largest entry (the weights and dS pass through
+# bf16 before their products, outputs are bf16; observed <= 7e-3), with a floor for gradients that are
+# zero by construction (a single position has softmax weight 1 and dS = 0).
+G_TOL = 1.5e-2
+
+
+def _run_bwd(inp, scale=None, pairs=None):
+    hass = _hass()
+    dev = torch.device("cuda:0")
+    wl = inp.wl
+    g = torch.Generator().manual_seed(wl.seed + 77)
+    dO = torch.randn(inp.Q.shape, generator=g).to(torch.bfloat16)
+    d = lambda x: x.to(dev)
+    Kd, Vd = [d(x) for x in inp.K_d], [d(x) for x in inp.V_d]
+    fw = hass.hca_attention_fwd(d(inp.Q), d(inp.K_t), d(inp.V_t), Kd, Vd, scale=scale)
+    bw = hass.hca_attention_bwd(d(inp.Q), d(inp.K_t), d(inp.V_t), Kd, Vd, fw["O"], fw["lse"], d(dO), scale=scale)
+    hass.check(bw["workspace"])
+    got = dict(dQ=bw["dQ"].cpu(), dK_t=bw["dK_t"].cpu(), dV_t=bw["dV_t"].cpu(),
+               dK_d=[x.cpu() for x in bw["dK_d"]], dV_d=[x.cpu() for x in bw["dV_d"]])
+    # oracle per sequence and key/value group (a group's heads share their keys' gradients)
+    rep = wl.H // wl.Hkv
+    if pairs is None:
+        pairs = [(b, g_) for b in range(wl.B) for g_ in range(wl.Hkv)]
+    worst = 0.0
+    for b, gk in pairs:
+        hs = slice(gk * rep, (gk + 1) * rep)
+        sq = lambda x: _f64(x[b:b + 1, :, hs, :])
+        sk = lambda x: _f64(x[b:b + 1, :, gk:gk + 1, :])
+        ref = ho.hca_attention_grad(sq(inp.Q), sk(inp.K_t), sk(inp.V_t), [sk(x) for x in inp.K_d],
+                                    [sk(x) for x in inp.V_d], sq(dO), scale=scale)
+        cmp = [(sq(got["dQ"]), ref[0]), (sk(got["dK_t"]), ref[1]), (sk(got["dV_t"]), ref[2])]
+        cmp += [(sk(got["dK_d"][i]), ref[3][i]) for i in range(wl.m)]
+        cmp += [(sk(got["dV_d"][i]), ref[4][i]) for i in range(wl.m)]
+        for mine, want in cmp:
+            err = np.abs(mine - want).max() / max(np.abs(want).max(), 1e-2)
+            worst = max(worst, err)
+    assert worst <= G_TOL, f"gradient error {worst:.3e} of the tensor's maximum"
+    return worst
+
+
+@pytest.mark.parametrize("name", ["hca-tiny", "hca-mid"])
+def test_backward_small_workloads(name):
+    print(_run_bwd(hi.make_hca_inputs(hi.HCA_WORKLOADS[name])))
+
+
+@pytest.mark.parametrize("B,T,H,Hkv,m", [
+    (1, 1, 1, 1, 1), (1, 128, 2, 2, 8), (1, 129, 2, 1, 8), (2, 256, 3, 3, 0), (1, 515, 4, 2, 5),
+    (2, 700, 16, 4, 2), (3, 64, 5, 5, 4), (1, 70, 1, 1, 8),
+])
+def test_backward_awkward_shapes(B, T, H, Hkv, m):
+    inp = hi.make_hca_inputs(hi.HcaWorkload("custom", B=B, T=T, H=H, Hkv=Hkv, m=m, seed=T + m))
+    pairs = None if B * Hkv <= 6 else [(0, 0), (B - 1, Hkv - 1), (B - 1, 1)]
+    print(_run_bwd(inp, pairs=pairs))
+
+
+def test_backward_steep_scores():
+    inp = hi.make_hca_inputs(hi.HcaWorkload("steep", B=1, T=640, H=2, Hkv=1, m=2, seed=3))
+    print(_run_bwd(inp, scale=0.5))
+
+
+def test_backward_full_size_sampled_groups():
+    wl = hi.HCA_WORKLOADS["hca-l3-8b"]
+    print(_run_bwd(hi.make_hca_inputs(wl), pairs=[(0, 0), (wl.B - 1, wl.Hkv - 1)]))
