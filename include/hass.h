@@ -346,10 +346,11 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
  * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
  * launches of the exact route behind a fused call (they return at once unless it is needed),
- * 6 HCA attention forward, 7 HCA attention backward (all its kernels).
+ * 6 HCA attention forward, 7 / 8 / 9 HCA attention backward: dQ kernel, dK_t/dV_t kernel, row kernels
+ * (row sums and the draft passes' gradients).
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */
-#define HASS_PROFILE_KINDS 8
+#define HASS_PROFILE_KINDS 10
 int hass_profile_enable(int on);
 int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
 

@@ -392,7 +392,7 @@ def check(workspace: torch.Tensor, stream=None) -> None:
 
 
 PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional",
-                 "hca_attention", "hca_attention_bwd")
+                 "hca_attention", "hca_bwd_dq", "hca_bwd_dkv", "hca_bwd_rows")
 
 
 def profile_enable(on: bool) -> None:

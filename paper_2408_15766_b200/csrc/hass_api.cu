@@ -20,7 +20,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_BWD = 7, NUM_KINDS = 8 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_DQ = 7, KIND_HCA_DKV = 8, KIND_HCA_BWD_ROWS = 9, NUM_KINDS = 10 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -1323,7 +1323,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     if (rc != HASS_OK) return rc;
 
     {   // D = rowsum(dO * O)
-        KernelTimer kt(KIND_HCA_BWD, st);
+        KernelTimer kt(KIND_HCA_BWD_ROWS, st);
         const long long rows = static_cast<long long>(B) * T * H;
         hca_bwd::hca_bwd_prep_kernel<<<static_cast<unsigned>((rows * 32 + 255) / 256), 256, 0, st>>>(
             static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Dv, iB, iT, iH);
@@ -1343,7 +1343,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     q.scale = scale;
     q.status = static_cast<unsigned int*>(workspace);
     {
-        KernelTimer kt(KIND_HCA_BWD, st);
+        KernelTimer kt(KIND_HCA_DQ, st);
         hca_bwd::hca_dq_kernel<<<q.items < di.sms ? q.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::DQ_SMEM_BYTES, st>>>(q);
     }
     g_launches.fetch_add(1);
@@ -1360,13 +1360,13 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     k.scale = scale;
     k.status = static_cast<unsigned int*>(workspace);
     {
-        KernelTimer kt(KIND_HCA_BWD, st);
+        KernelTimer kt(KIND_HCA_DKV, st);
         hca_bwd::hca_dkv_kernel<<<k.items < di.sms ? k.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::KV_SMEM_BYTES, st>>>(k);
     }
     g_launches.fetch_add(1);
 
     for (int i = 0; i < m; ++i) {
-        KernelTimer kt(KIND_HCA_BWD, st);
+        KernelTimer kt(KIND_HCA_BWD_ROWS, st);
         const long long warps = static_cast<long long>(B) * T * Hkv;
         hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, st>>>(
             static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd,

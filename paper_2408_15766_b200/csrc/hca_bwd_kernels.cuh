@@ -134,6 +134,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    // items are sorted longest first; round k deals items k*G .. k*G + G-1 to the G CTAs in alternating direction
+    auto round_item = [&](uint32_t k) {
+        const int G = gridDim.x, c = blockIdx.x;
+        return static_cast<int>(k) * G + ((k & 1u) ? G - 1 - c : c);
+    };
 
     const int BH = p.B * p.H;
     const int rep = p.H / p.Hkv;
@@ -151,7 +156,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
         if (lane == 0) {
             uint32_t g = 0, it = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int col = (h / rep) * HD;
@@ -221,7 +226,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 ++gq;
                 return true;
             };
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int n_e = key_tiles(qt) + 2 * m;
@@ -246,7 +251,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
         auto ds_addr = [&](int s, int chunk) {
             return base + DQ_SMEM_DS + s * DS_BYTES + r * 128 + (((chunk ^ (r & 7)) & 7) << 4);
         };
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int qt, b, h;
             decode(item, qt, b, h);
             const int n = key_tiles(qt);
@@ -475,6 +480,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    // items are sorted longest first; round k deals items k*G .. k*G + G-1 to the G CTAs in alternating direction
+    auto round_item = [&](uint32_t k) {
+        const int G = gridDim.x, c = blockIdx.x;
+        return static_cast<int>(k) * G + ((k & 1u) ? G - 1 - c : c);
+    };
 
     const int BG = p.B * p.Hkv;
     const int rep = p.H / p.Hkv;
@@ -493,7 +503,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
         // ===================== producer: TMA by lane 0, the per-query vectors by all lanes =====================
         uint32_t gq = 0, it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int kt, b, g;
             decode(item, kt, b, g);
             const int nq = q_count(kt);
@@ -584,7 +594,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                 ++ga;
                 return true;
             };
-            for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+            for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
                 int kt, b, g;
                 decode(item, kt, b, g);
                 const int n_e = rep * q_count(kt);
@@ -607,7 +617,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
         uint32_t gq = 0, it = 0;
         bool ok = true;
         auto row_addr = [&](int buf_off, int chunk) { return base + buf_off + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
-        for (int item = blockIdx.x; item < p.items && ok; item += gridDim.x, ++it) {
+        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int kt, b, g;
             decode(item, kt, b, g);
             const int nq = q_count(kt);
