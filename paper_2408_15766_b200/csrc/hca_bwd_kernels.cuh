@@ -261,6 +261,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             // P = 2^(S c2 - lse2); a row outside the sequence gets P = 0 through lse2 = +inf
             const float nlse2 = valid ? -p.lse[row_idx] * 1.4426950408889634f : -INFINITY;
             const float Dt = valid ? p.D[row_idx] : 0.f;
+            const float nDs = -Dt * p.scale;
             for (int e = 0; e < n + 2 * m; ++e, ++g) {
                 const int s = g & 1u;
                 const uint32_t ph = (g >> 1) & 1u;
@@ -283,14 +284,24 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(sdp_empty(s));
+                    if (band) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (32 * k + c > lim) sr[k][c] = 0xff800000u;       // -inf: weight 0
+                        }
+                    }
+                    // dS = P (dP - D) scale = 2^(S c2 - lse2) (dP scale - D scale), two columns per instruction
                     float ds[2][32];
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            float pw = ex2(fmaf(__uint_as_float(sr[k][c]), p.c2, nlse2));
-                            if (band && 32 * k + c > lim) pw = 0.f;
-                            ds[k][c] = pw * (__uint_as_float(dr[k][c]) - Dt) * p.scale;
+                        for (int c = 0; c < 32; c += 2) {
+                            float x0, x1, y0, y1;
+                            ffma2(x0, x1, __uint_as_float(sr[k][c]), __uint_as_float(sr[k][c + 1]), p.c2, p.c2, nlse2, nlse2);
+                            ffma2(y0, y1, __uint_as_float(dr[k][c]), __uint_as_float(dr[k][c + 1]), p.scale, p.scale, nDs, nDs);
+                            fmul2(ds[k][c], ds[k][c + 1], ex2(x0), ex2(x1), y0, y1);
                         }
                     }
                     if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
@@ -403,7 +414,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
 //   threads                             P^T = 2^(S^T c2 - lse2[t]) on the entries the target's keys really met
 //                                       (t - s >= m), dS^T = P^T (dP^T - D[t]) scale; both as bf16 in shared memory
 //   dV += P^T dO, dK += dS^T Q          the Q / dO stage read MN-major
-// The per-query vectors -lse2[t] and D[t] of an element travel with its Q / dO stage: the producer warp's
+// The per-query vectors -lse2[t] and -D[t] scale of an element travel with its Q / dO stage: the producer warp's
 // lanes copy them into shared memory next to the TMA loads.
 constexpr int KV_SMEM_K = 0;                               // 128 keys x 128: two halves of 16 KB
 constexpr int KV_SMEM_V = KV_SMEM_K + Q_BYTES;
@@ -411,7 +422,7 @@ constexpr int KV_SMEM_Q = KV_SMEM_V + Q_BYTES;             // 2 stages of 64 que
 constexpr int KV_SMEM_DO = KV_SMEM_Q + 2 * KV_BYTES;       // 2 stages
 constexpr int KV_SMEM_PT = KV_SMEM_DO + 2 * KV_BYTES;      // P^T, 128 x 64 bf16
 constexpr int KV_SMEM_DST = KV_SMEM_PT + DS_BYTES;         // dS^T
-constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // 2 stages x (64 x -lse2, 64 x D) floats
+constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // 2 stages x (64 x -lse2, 64 x -D scale) floats
 constexpr int KV_SMEM_BAR = KV_SMEM_VEC + 2 * 512;
 constexpr int KV_NUM_BARS = 14;
 constexpr int KV_SMEM_BYTES = KV_SMEM_BAR + 256 + 1024 /*alignment slack*/;
@@ -532,14 +543,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                     tma_load_3d(base + KV_SMEM_DO + s * KV_BYTES, &p.tmdO, qd_full(s), h * HD, jq * KT, b);
                     tma_load_3d(base + KV_SMEM_DO + s * KV_BYTES + KV_HALF, &p.tmdO, qd_full(s), h * HD + 64, jq * KT, b);
                 }
-                // -lse2[t] (or -inf past the sequence, which zeroes the weight) and D[t] for the 64 queries
+                // -lse2[t] (or -inf past the sequence, which zeroes the weight) and -D[t] scale for the 64 queries
                 const size_t rowbase = (static_cast<size_t>(b) * p.H + h) * p.T;
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     const int c = lane + 32 * u;
                     const int t = jq * KT + c;
                     vec[s * 128 + c] = t < p.T ? -p.lse[rowbase + t] * 1.4426950408889634f : -INFINITY;
-                    vec[s * 128 + 64 + c] = t < p.T ? p.D[rowbase + t] : 0.f;
+                    vec[s * 128 + 64 + c] = t < p.T ? -p.D[rowbase + t] * p.scale : 0.f;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(qd_full(s));
@@ -647,21 +658,33 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                 if (lane == 0) mbar_arrive(st_empty(s));
                 const float4* nl = reinterpret_cast<const float4*>(vec + s * 128);
                 const float4* dd = reinterpret_cast<const float4*>(vec + s * 128 + 64);
+                if (band) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (32 * k + c < lo) sr[k][c] = 0xff800000u;       // -inf: weight 0
+                    }
+                }
+                // P^T = 2^(S^T c2 - lse2[t]), dS^T = P^T (dP^T scale - D[t] scale), two columns per instruction
                 float pw[2][32], ds[2][32];
 #pragma unroll
                 for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int c4 = 0; c4 < 8; ++c4) {
                         const float4 a = nl[8 * k + c4], d = dd[8 * k + c4];
-                        const float av[4] = {a.x, a.y, a.z, a.w}, dv[4] = {d.x, d.y, d.z, d.w};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int c = 4 * c4 + u;
-                            float w = ex2(fmaf(__uint_as_float(sr[k][c]), p.c2, av[u]));
-                            if (band && 32 * k + c < lo) w = 0.f;
-                            pw[k][c] = w;
-                            ds[k][c] = w * (__uint_as_float(dr[k][c]) - dv[u]) * p.scale;
-                        }
+                        const int c = 4 * c4;
+                        float x0, x1, y0, y1;
+                        ffma2(x0, x1, __uint_as_float(sr[k][c]), __uint_as_float(sr[k][c + 1]), p.c2, p.c2, a.x, a.y);
+                        ffma2(y0, y1, __uint_as_float(dr[k][c]), __uint_as_float(dr[k][c + 1]), p.scale, p.scale, d.x, d.y);
+                        pw[k][c] = ex2(x0);
+                        pw[k][c + 1] = ex2(x1);
+                        fmul2(ds[k][c], ds[k][c + 1], pw[k][c], pw[k][c + 1], y0, y1);
+                        ffma2(x0, x1, __uint_as_float(sr[k][c + 2]), __uint_as_float(sr[k][c + 3]), p.c2, p.c2, a.z, a.w);
+                        ffma2(y0, y1, __uint_as_float(dr[k][c + 2]), __uint_as_float(dr[k][c + 3]), p.scale, p.scale, d.z, d.w);
+                        pw[k][c + 2] = ex2(x0);
+                        pw[k][c + 3] = ex2(x1);
+                        fmul2(ds[k][c + 2], ds[k][c + 3], pw[k][c + 2], pw[k][c + 3], y0, y1);
                     }
                 }
                 if (!wait_barrier(pds_empty, (gq & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
