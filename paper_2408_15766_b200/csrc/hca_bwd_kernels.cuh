@@ -8,7 +8,8 @@
 // hca_dq_kernel also leaves P and dS of the substituted entries (t, t-i) in the workspace for the last one.
 //
 // Both tensor-core kernels follow the forward kernel's organisation (warp 0 TMA producer, warp 1 MMA issuer
-// and TMEM owner, warps 2-5 one tile row per thread) and its bounded waits.
+// and TMEM owner, then row-owning warps - here two groups of four, each taking half of a tile's columns,
+// which needs no exchange because the backward has no running row statistics) and its bounded waits.
 #pragma once
 #include "hca_kernels.cuh"
 
@@ -24,7 +25,7 @@ constexpr int QT = 128;
 constexpr int KT = 64;
 constexpr int HD = 128;
 constexpr int MAX_DRAFTS = hca::MAX_DRAFTS;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;        // producer, MMA issuer, two groups of four row-owning warps
 constexpr int Q_BYTES = QT * HD * 2;
 constexpr int Q_HALF = Q_BYTES / 2;
 constexpr int KV_BYTES = KT * HD * 2;
@@ -112,12 +113,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             mbar_init(kv_full(s), 1);
             mbar_init(kv_empty(s), 1);
             mbar_init(sdp_full(s), 1);
-            mbar_init(sdp_empty(s), 4);
-            mbar_init(ds_full(s), 4);
+            mbar_init(sdp_empty(s), 8);
+            mbar_init(ds_full(s), 8);
             mbar_init(ds_empty(s), 1);
         }
         mbar_init(dq_done, 1);
-        mbar_init(dq_free, 4);
+        mbar_init(dq_free, 8);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -243,6 +244,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             }
         }
     } else {
+        // two groups of four warps share every row: group grp takes columns 32 grp .. 32 grp + 31 of each
+        // 64-column tile (nothing crosses columns here), and half of the dQ row in the epilogue
+        const int grp = (warp - 2) >> 2;
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
@@ -267,61 +271,49 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 const uint32_t ph = (g >> 1) & 1u;
                 if (!wait_barrier(sdp_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr;
+                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr + 32 * grp;
                 if (e < n) {
-                    // ---- key tile: dS for the whole row ----
+                    // ---- key tile: dS for this group's 32 columns of the row ----
                     const bool band = e * KT + KT - 1 > qt * QT - m;
-                    const int lim = t - m - e * KT;
-                    uint32_t sr[2][32], dr[2][32];
-                    tmem_ld32(tmem_s, sr[0]);
-                    tmem_ld32(tmem_s + 32, sr[1]);
-                    tmem_ld32(tmem_s + 64, dr[0]);
-                    tmem_ld32(tmem_s + 96, dr[1]);
-                    tmem_ld_wait(sr[0]);
-                    tmem_ld_wait(sr[1]);
-                    tmem_ld_wait(dr[0]);
-                    tmem_ld_wait(dr[1]);
+                    const int lim = t - m - e * KT - 32 * grp;
+                    uint32_t sr[32], dr[32];
+                    tmem_ld32(tmem_s, sr);
+                    tmem_ld32(tmem_s + 64, dr);
+                    tmem_ld_wait(sr);
+                    tmem_ld_wait(dr);
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(sdp_empty(s));
                     if (band) {
 #pragma unroll
-                        for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (32 * k + c > lim) sr[k][c] = 0xff800000u;       // -inf: weight 0
-                        }
+                        for (int c = 0; c < 32; ++c)
+                            if (c > lim) sr[c] = 0xff800000u;       // -inf: weight 0
                     }
                     // dS = P (dP - D) scale = 2^(S c2 - lse2) (dP scale - D scale), two columns per instruction
-                    float ds[2][32];
+                    float ds[32];
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            float x0, x1, y0, y1;
-                            ffma2(x0, x1, __uint_as_float(sr[k][c]), __uint_as_float(sr[k][c + 1]), p.c2, p.c2, nlse2, nlse2);
-                            ffma2(y0, y1, __uint_as_float(dr[k][c]), __uint_as_float(dr[k][c + 1]), p.scale, p.scale, nDs, nDs);
-                            fmul2(ds[k][c], ds[k][c + 1], ex2(x0), ex2(x1), y0, y1);
-                        }
+                    for (int c = 0; c < 32; c += 2) {
+                        float x0, x1, y0, y1;
+                        ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), p.c2, p.c2, nlse2, nlse2);
+                        ffma2(y0, y1, __uint_as_float(dr[c]), __uint_as_float(dr[c + 1]), p.scale, p.scale, nDs, nDs);
+                        fmul2(ds[c], ds[c + 1], ex2(x0), ex2(x1), y0, y1);
                     }
                     if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4)
-                            st_shared_v4(ds_addr(s, 4 * k + q4), pack_bf16(ds[k][8 * q4], ds[k][8 * q4 + 1]),
-                                         pack_bf16(ds[k][8 * q4 + 2], ds[k][8 * q4 + 3]),
-                                         pack_bf16(ds[k][8 * q4 + 4], ds[k][8 * q4 + 5]),
-                                         pack_bf16(ds[k][8 * q4 + 6], ds[k][8 * q4 + 7]));
-                    }
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        st_shared_v4(ds_addr(s, 4 * grp + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
+                                     pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
+                                     pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
                 } else {
-                    // ---- draft pass i, half hf: only the diagonal element of the rows of that half ----
+                    // ---- draft pass i, half hf: only the diagonal element of the rows of that half; it lies in
+                    //      this group's columns when (r & 63) / 32 == grp ----
                     const int i = (e - n) >> 1, hf = (e - n) & 1;
+                    const bool holder = (r >> 6) == hf && (quad & 1) == grp;
                     float sv = 0.f, dv = 0.f;
-                    if ((quad >> 1) == hf) {
+                    if (holder) {               // warp-uniform
                         uint32_t sr[32], dr[32];
-                        tmem_ld32(tmem_s + 32 * (quad & 1), sr);
-                        tmem_ld32(tmem_s + 64 + 32 * (quad & 1), dr);
+                        tmem_ld32(tmem_s, sr);
+                        tmem_ld32(tmem_s + 64, dr);
                         tmem_ld_wait(sr);
                         tmem_ld_wait(dr);
 #pragma unroll
@@ -335,17 +327,18 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(sdp_empty(s));
-                    const bool mine = (r >> 6) == hf && t - i >= 0 && valid;
+                    const bool mine = holder && t - i >= 0 && valid;
                     const float pw = mine ? ex2(fmaf(sv, p.c2, nlse2)) : 0.f;
-                    const float dsv = pw * (dv - Dt) * p.scale;
-                    if ((r >> 6) == hf && valid) {
+                    const float dsv = pw * fmaf(dv, p.scale, nDs);
+                    if (holder && valid) {
                         p.Pd[row_idx * m + i] = pw;
-                        p.dSd[row_idx * m + i] = dsv;
+                        p.dSd[row_idx * m + i] = mine ? dsv : 0.f;
                     }
-                    const uint32_t bits = pack_bf16(dsv, 0.f) << ((r & 1) * 16);
+                    const uint32_t bits = mine ? pack_bf16(dsv, 0.f) << ((r & 1) * 16) : 0u;
                     if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
 #pragma unroll
-                    for (int chunk = 0; chunk < 8; ++chunk) {
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const int chunk = 4 * grp + q4;
                         const bool here = chunk == ((r & 63) >> 3);
                         const int w = (r & 7) >> 1;
                         st_shared_v4(ds_addr(s, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
@@ -357,29 +350,26 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 if (lane == 0) mbar_arrive(ds_full(s));
             }
             if (!ok) break;
-            // ---- epilogue: dQ as bf16, each thread stores its own 256-byte row ----
+            // ---- epilogue: this group's half of the dQ row as bf16 ----
             if (!wait_barrier(dq_done, it & 1u, abort_flag, p.status, 13)) break;
             tc_fence_after_sync();
-            __nv_bfloat16* orow = p.dQ + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
+            __nv_bfloat16* orow = p.dQ + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD + 64 * grp;
+            {
                 uint32_t raw[2][32];
-                tmem_ld32(tmem_base + 256 + lane_addr + 64 * hf, raw[0]);
-                tmem_ld32(tmem_base + 256 + lane_addr + 64 * hf + 32, raw[1]);
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * grp, raw[0]);
+                tmem_ld32(tmem_base + 256 + lane_addr + 64 * grp + 32, raw[1]);
                 tmem_ld_wait(raw[0]);
                 tmem_ld_wait(raw[1]);
-                if (hf == 1) {
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(dq_free);
-                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(dq_free);
                 if (valid) {
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
 #pragma unroll
                         for (int q8 = 0; q8 < 2; ++q8) {
                             const uint32_t* x = &raw[k][16 * q8];
-                            st_global_v8(orow + 64 * hf + 32 * k + 16 * q8,
+                            st_global_v8(orow + 32 * k + 16 * q8,
                                          pack_bf16(__uint_as_float(x[0]), __uint_as_float(x[1])),
                                          pack_bf16(__uint_as_float(x[2]), __uint_as_float(x[3])),
                                          pack_bf16(__uint_as_float(x[4]), __uint_as_float(x[5])),
@@ -469,12 +459,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             mbar_init(qd_full(s), 2);      // the TMA transaction's arrival and the producer warp's vectors
             mbar_init(qd_empty(s), 1);
             mbar_init(st_full(s), 1);
-            mbar_init(st_empty(s), 4);
+            mbar_init(st_empty(s), 8);
         }
-        mbar_init(pds_full, 4);
+        mbar_init(pds_full, 8);
         mbar_init(pds_empty, 1);
         mbar_init(acc_done, 1);
-        mbar_init(acc_free, 4);
+        mbar_init(acc_free, 8);
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -622,6 +612,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             }
         }
     } else {
+        // two groups of four warps share every key row: group grp takes the query columns 32 grp .. 32 grp + 31
+        // of each element, and in the epilogue dV (group 0) or dK (group 1)
+        const int grp = (warp - 2) >> 2;
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                 // key row of the tile
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
@@ -640,87 +633,72 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                 if (!wait_barrier(st_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
                 if (!wait_barrier(qd_full(s), ph, abort_flag, p.status, 15)) { ok = false; break; }   // the element's vectors
                 tc_fence_after_sync();
-                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr;
+                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr + 32 * grp;
                 // the target's key at spos met query t only if t - spos >= m: columns below lo are empty
-                const int lo = spos + m - jq * KT;
-                const bool band = lo > 0;
-                uint32_t sr[2][32], dr[2][32];
-                tmem_ld32(tmem_s, sr[0]);
-                tmem_ld32(tmem_s + 32, sr[1]);
-                tmem_ld32(tmem_s + 64, dr[0]);
-                tmem_ld32(tmem_s + 96, dr[1]);
-                tmem_ld_wait(sr[0]);
-                tmem_ld_wait(sr[1]);
-                tmem_ld_wait(dr[0]);
-                tmem_ld_wait(dr[1]);
+                const int lo = spos + m - jq * KT - 32 * grp;
+                const bool band = spos + m - jq * KT > 0;
+                uint32_t sr[32], dr[32];
+                tmem_ld32(tmem_s, sr);
+                tmem_ld32(tmem_s + 64, dr);
+                tmem_ld_wait(sr);
+                tmem_ld_wait(dr);
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(st_empty(s));
-                const float4* nl = reinterpret_cast<const float4*>(vec + s * 128);
-                const float4* dd = reinterpret_cast<const float4*>(vec + s * 128 + 64);
                 if (band) {
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (32 * k + c < lo) sr[k][c] = 0xff800000u;       // -inf: weight 0
-                    }
+                    for (int c = 0; c < 32; ++c)
+                        if (c < lo) sr[c] = 0xff800000u;       // -inf: weight 0
                 }
                 // P^T = 2^(S^T c2 - lse2[t]), dS^T = P^T (dP^T scale - D[t] scale), two columns per instruction
-                float pw[2][32], ds[2][32];
+                const float4* nl = reinterpret_cast<const float4*>(vec + s * 128 + 32 * grp);
+                const float4* dd = reinterpret_cast<const float4*>(vec + s * 128 + 64 + 32 * grp);
+                float pw[32], ds[32];
 #pragma unroll
-                for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4) {
-                        const float4 a = nl[8 * k + c4], d = dd[8 * k + c4];
-                        const int c = 4 * c4;
-                        float x0, x1, y0, y1;
-                        ffma2(x0, x1, __uint_as_float(sr[k][c]), __uint_as_float(sr[k][c + 1]), p.c2, p.c2, a.x, a.y);
-                        ffma2(y0, y1, __uint_as_float(dr[k][c]), __uint_as_float(dr[k][c + 1]), p.scale, p.scale, d.x, d.y);
-                        pw[k][c] = ex2(x0);
-                        pw[k][c + 1] = ex2(x1);
-                        fmul2(ds[k][c], ds[k][c + 1], pw[k][c], pw[k][c + 1], y0, y1);
-                        ffma2(x0, x1, __uint_as_float(sr[k][c + 2]), __uint_as_float(sr[k][c + 3]), p.c2, p.c2, a.z, a.w);
-                        ffma2(y0, y1, __uint_as_float(dr[k][c + 2]), __uint_as_float(dr[k][c + 3]), p.scale, p.scale, d.z, d.w);
-                        pw[k][c + 2] = ex2(x0);
-                        pw[k][c + 3] = ex2(x1);
-                        fmul2(ds[k][c + 2], ds[k][c + 3], pw[k][c + 2], pw[k][c + 3], y0, y1);
-                    }
+                for (int c4 = 0; c4 < 8; ++c4) {
+                    const float4 a = nl[c4], d = dd[c4];
+                    const int c = 4 * c4;
+                    float x0, x1, y0, y1;
+                    ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), p.c2, p.c2, a.x, a.y);
+                    ffma2(y0, y1, __uint_as_float(dr[c]), __uint_as_float(dr[c + 1]), p.scale, p.scale, d.x, d.y);
+                    pw[c] = ex2(x0);
+                    pw[c + 1] = ex2(x1);
+                    fmul2(ds[c], ds[c + 1], pw[c], pw[c + 1], y0, y1);
+                    ffma2(x0, x1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]), p.c2, p.c2, a.z, a.w);
+                    ffma2(y0, y1, __uint_as_float(dr[c + 2]), __uint_as_float(dr[c + 3]), p.scale, p.scale, d.z, d.w);
+                    pw[c + 2] = ex2(x0);
+                    pw[c + 3] = ex2(x1);
+                    fmul2(ds[c + 2], ds[c + 3], pw[c + 2], pw[c + 3], y0, y1);
                 }
                 if (!wait_barrier(pds_empty, (gq & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
 #pragma unroll
-                for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        st_shared_v4(row_addr(KV_SMEM_PT, 4 * k + q4), pack_bf16(pw[k][8 * q4], pw[k][8 * q4 + 1]),
-                                     pack_bf16(pw[k][8 * q4 + 2], pw[k][8 * q4 + 3]),
-                                     pack_bf16(pw[k][8 * q4 + 4], pw[k][8 * q4 + 5]),
-                                     pack_bf16(pw[k][8 * q4 + 6], pw[k][8 * q4 + 7]));
-                        st_shared_v4(row_addr(KV_SMEM_DST, 4 * k + q4), pack_bf16(ds[k][8 * q4], ds[k][8 * q4 + 1]),
-                                     pack_bf16(ds[k][8 * q4 + 2], ds[k][8 * q4 + 3]),
-                                     pack_bf16(ds[k][8 * q4 + 4], ds[k][8 * q4 + 5]),
-                                     pack_bf16(ds[k][8 * q4 + 6], ds[k][8 * q4 + 7]));
-                    }
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    st_shared_v4(row_addr(KV_SMEM_PT, 4 * grp + q4), pack_bf16(pw[8 * q4], pw[8 * q4 + 1]),
+                                 pack_bf16(pw[8 * q4 + 2], pw[8 * q4 + 3]), pack_bf16(pw[8 * q4 + 4], pw[8 * q4 + 5]),
+                                 pack_bf16(pw[8 * q4 + 6], pw[8 * q4 + 7]));
+                    st_shared_v4(row_addr(KV_SMEM_DST, 4 * grp + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
+                                 pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
+                                 pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pds_full);
             }
             if (!ok) break;
-            // ---- epilogue: this key row of dV and dK as bf16 ----
+            // ---- epilogue: this key row of dV (group 0) or dK (group 1) as bf16 ----
             if (!wait_barrier(acc_done, it & 1u, abort_flag, p.status, 13)) break;
             tc_fence_after_sync();
             const bool valid = spos < p.T;
             const size_t orow = ((static_cast<size_t>(b) * p.T + (valid ? spos : 0)) * p.Hkv + g) * HD;
 #pragma unroll
-            for (int part = 0; part < 4; ++part) {      // dV columns 0..63, 64..127, then dK likewise
-                __nv_bfloat16* dst = (part < 2 ? p.dV : p.dK) + orow + 64 * (part & 1);
+            for (int part = 0; part < 2; ++part) {      // columns 0..63, 64..127
+                __nv_bfloat16* dst = (grp == 0 ? p.dV : p.dK) + orow + 64 * part;
                 uint32_t raw[2][32];
-                tmem_ld32(tmem_base + 256 + lane_addr + 64 * part, raw[0]);
-                tmem_ld32(tmem_base + 256 + lane_addr + 64 * part + 32, raw[1]);
+                tmem_ld32(tmem_base + 256 + 128 * grp + lane_addr + 64 * part, raw[0]);
+                tmem_ld32(tmem_base + 256 + 128 * grp + lane_addr + 64 * part + 32, raw[1]);
                 tmem_ld_wait(raw[0]);
                 tmem_ld_wait(raw[1]);
-                if (part == 3) {
+                if (part == 1) {
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acc_free);
