@@ -62,11 +62,12 @@ __global__ void hca_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const _
 // same K stage read MN-major.
 constexpr int DQ_SMEM_Q = 0;
 constexpr int DQ_SMEM_DO = DQ_SMEM_Q + Q_BYTES;
-constexpr int DQ_SMEM_K = DQ_SMEM_DO + Q_BYTES;        // 2 stages
-constexpr int DQ_SMEM_V = DQ_SMEM_K + 2 * KV_BYTES;    // 2 stages
-constexpr int DQ_SMEM_DS = DQ_SMEM_V + 2 * KV_BYTES;   // 2 buffers
+constexpr int DQ_STAGES = 4;        // a K/V stage is held until its dQ product is done, long after the next S/dP products need theirs
+constexpr int DQ_SMEM_K = DQ_SMEM_DO + Q_BYTES;
+constexpr int DQ_SMEM_V = DQ_SMEM_K + DQ_STAGES * KV_BYTES;
+constexpr int DQ_SMEM_DS = DQ_SMEM_V + DQ_STAGES * KV_BYTES;   // 2 buffers
 constexpr int DQ_SMEM_BAR = DQ_SMEM_DS + 2 * DS_BYTES;
-constexpr int DQ_NUM_BARS = 16;
+constexpr int DQ_NUM_BARS = 2 * DQ_STAGES + 12;
 constexpr int DQ_SMEM_BYTES = DQ_SMEM_BAR + 256 + 1024 /*alignment slack*/;
 constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb, dP at 128 sb + 64; dQ at 256
 
@@ -94,12 +95,12 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
     const uint32_t bar0 = base + DQ_SMEM_BAR;
     const uint32_t qdo_full = bar0, qdo_empty = bar0 + 8;
     auto kv_full = [&](int s) { return bar0 + 8u * (2 + s); };
-    auto kv_empty = [&](int s) { return bar0 + 8u * (4 + s); };
-    auto sdp_full = [&](int s) { return bar0 + 8u * (6 + s); };
-    auto sdp_empty = [&](int s) { return bar0 + 8u * (8 + s); };
-    auto ds_full = [&](int s) { return bar0 + 8u * (10 + s); };
-    auto ds_empty = [&](int s) { return bar0 + 8u * (12 + s); };
-    const uint32_t dq_done = bar0 + 8u * 14, dq_free = bar0 + 8u * 15;
+    auto kv_empty = [&](int s) { return bar0 + 8u * (2 + DQ_STAGES + s); };
+    auto sdp_full = [&](int s) { return bar0 + 8u * (2 + 2 * DQ_STAGES + s); };
+    auto sdp_empty = [&](int s) { return bar0 + 8u * (4 + 2 * DQ_STAGES + s); };
+    auto ds_full = [&](int s) { return bar0 + 8u * (6 + 2 * DQ_STAGES + s); };
+    auto ds_empty = [&](int s) { return bar0 + 8u * (8 + 2 * DQ_STAGES + s); };
+    const uint32_t dq_done = bar0 + 8u * (10 + 2 * DQ_STAGES), dq_free = bar0 + 8u * (11 + 2 * DQ_STAGES);
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + DQ_SMEM_BAR + 8 * DQ_NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
@@ -109,9 +110,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
     if (threadIdx.x == 0) {
         mbar_init(qdo_full, 1);
         mbar_init(qdo_empty, 1);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < DQ_STAGES; ++s) {
             mbar_init(kv_full(s), 1);
             mbar_init(kv_empty(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(sdp_full(s), 1);
             mbar_init(sdp_empty(s), 8);
             mbar_init(ds_full(s), 8);
@@ -169,8 +172,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 tma_load_3d(base + DQ_SMEM_DO, &p.tmdO, qdo_full, h * HD, qt * QT, b);
                 tma_load_3d(base + DQ_SMEM_DO + Q_HALF, &p.tmdO, qdo_full, h * HD + 64, qt * QT, b);
                 for (int e = 0; e < n + 2 * m && ok; ++e, ++g) {
-                    const int s = g & 1u;
-                    if (!wait_barrier(kv_empty(s), ((g >> 1) & 1u) ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
+                    const int s = g % DQ_STAGES;
+                    if (!wait_barrier(kv_empty(s), ((g / DQ_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
                     const int d = e - n;
                     const CUtensorMap* tk = e < n ? &p.tmK : &p.tmKd[d >> 1];
                     const CUtensorMap* tv = e < n ? &p.tmV : &p.tmVd[d >> 1];
@@ -190,38 +193,40 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             uint32_t gs = 0, gq = 0, it = 0;      // elements whose S/dP, resp. dQ product has been issued
             bool ok = true;
             auto issue_sdp = [&]() -> bool {
-                const int s = gs & 1u;
+                const int s = gs & 1u;                  // S / dP buffer
+                const int ks = gs % DQ_STAGES;          // K / V stage
                 const uint32_t ph = (gs >> 1) & 1u;
-                if (!wait_barrier(kv_full(s), ph, abort_flag, p.status, 4)) return false;
+                if (!wait_barrier(kv_full(ks), (gs / DQ_STAGES) & 1u, abort_flag, p.status, 4)) return false;
                 if (!wait_barrier(sdp_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
                     umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + DQ_SMEM_Q + qo, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_K + s * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                              make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
                 }
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
                     umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + DQ_SMEM_DO + qo, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_V + s * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                              make_smem_desc_sw128(base + DQ_SMEM_V + ks * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
                 }
                 umma_commit(sdp_full(s));
                 ++gs;
                 return true;
             };
             auto issue_dq = [&](bool first, bool last) -> bool {
-                const int s = gq & 1u;
+                const int s = gq & 1u;                  // dS buffer
+                const int ks = gq % DQ_STAGES;          // K stage
                 if (!wait_barrier(ds_full(s), (gq >> 1) & 1u, abort_flag, p.status, 7)) return false;
                 if (first && !wait_barrier(dq_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k)
                     umma_bf16(tmem_base + 256, make_smem_desc_sw128(base + DQ_SMEM_DS + s * DS_BYTES + k * 32, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_K + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_q,
+                              make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_q,
                               (!first || k != 0) ? 1u : 0u);
-                umma_commit(kv_empty(s));
+                umma_commit(kv_empty(ks));
                 umma_commit(ds_empty(s));
                 if (last) umma_commit(dq_done);
                 ++gq;
@@ -408,13 +413,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
 // lanes copy them into shared memory next to the TMA loads.
 constexpr int KV_SMEM_K = 0;                               // 128 keys x 128: two halves of 16 KB
 constexpr int KV_SMEM_V = KV_SMEM_K + Q_BYTES;
-constexpr int KV_SMEM_Q = KV_SMEM_V + Q_BYTES;             // 2 stages of 64 queries
-constexpr int KV_SMEM_DO = KV_SMEM_Q + 2 * KV_BYTES;       // 2 stages
-constexpr int KV_SMEM_PT = KV_SMEM_DO + 2 * KV_BYTES;      // P^T, 128 x 64 bf16
+constexpr int KV_STAGES = 3;        // a Q/dO stage is held until its dV/dK products are done
+constexpr int KV_SMEM_Q = KV_SMEM_V + Q_BYTES;             // stages of 64 queries
+constexpr int KV_SMEM_DO = KV_SMEM_Q + KV_STAGES * KV_BYTES;
+constexpr int KV_SMEM_PT = KV_SMEM_DO + KV_STAGES * KV_BYTES;      // P^T, 128 x 64 bf16
 constexpr int KV_SMEM_DST = KV_SMEM_PT + DS_BYTES;         // dS^T
-constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // 2 stages x (64 x -lse2, 64 x -D scale) floats
-constexpr int KV_SMEM_BAR = KV_SMEM_VEC + 2 * 512;
-constexpr int KV_NUM_BARS = 14;
+constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // per stage: 64 x -lse2, 64 x -D scale (floats)
+constexpr int KV_SMEM_BAR = KV_SMEM_VEC + KV_STAGES * 512;
+constexpr int KV_NUM_BARS = 2 * KV_STAGES + 10;
 constexpr int KV_SMEM_BYTES = KV_SMEM_BAR + 256 + 1024 /*alignment slack*/;
 constexpr int KV_TMEM_COLS = 512;   // buffer sb: S^T at 128 sb, dP^T at 128 sb + 64; dV at 256, dK at 384
 
@@ -440,11 +446,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
     const uint32_t bar0 = base + KV_SMEM_BAR;
     const uint32_t kv_full = bar0, kv_empty = bar0 + 8;
     auto qd_full = [&](int s) { return bar0 + 8u * (2 + s); };
-    auto qd_empty = [&](int s) { return bar0 + 8u * (4 + s); };
-    auto st_full = [&](int s) { return bar0 + 8u * (6 + s); };
-    auto st_empty = [&](int s) { return bar0 + 8u * (8 + s); };
-    const uint32_t pds_full = bar0 + 8u * 10, pds_empty = bar0 + 8u * 11;
-    const uint32_t acc_done = bar0 + 8u * 12, acc_free = bar0 + 8u * 13;
+    auto qd_empty = [&](int s) { return bar0 + 8u * (2 + KV_STAGES + s); };
+    auto st_full = [&](int s) { return bar0 + 8u * (2 + 2 * KV_STAGES + s); };
+    auto st_empty = [&](int s) { return bar0 + 8u * (4 + 2 * KV_STAGES + s); };
+    const uint32_t pds_full = bar0 + 8u * (6 + 2 * KV_STAGES), pds_empty = bar0 + 8u * (7 + 2 * KV_STAGES);
+    const uint32_t acc_done = bar0 + 8u * (8 + 2 * KV_STAGES), acc_free = bar0 + 8u * (9 + 2 * KV_STAGES);
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + KV_SMEM_BAR + 8 * KV_NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
     float* vec = reinterpret_cast<float*>(smem_gen + KV_SMEM_VEC);     // [stage][0..63 -lse2 | 64..127 D]
@@ -455,9 +461,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
         mbar_init(kv_empty, 1);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < KV_STAGES; ++s) {
             mbar_init(qd_full(s), 2);      // the TMA transaction's arrival and the producer warp's vectors
             mbar_init(qd_empty(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(st_full(s), 1);
             mbar_init(st_empty(s), 8);
         }
@@ -522,8 +530,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             for (int e = 0; e < rep * nq && ok; ++e, ++gq) {
                 const int h = g * rep + e / nq;
                 const int jq = 2 * kt + e % nq;
-                const int s = gq & 1u;
-                if (lane == 0) ok = wait_barrier(qd_empty(s), ((gq >> 1) & 1u) ^ 1u, abort_flag, p.status, 2);
+                const int s = gq % KV_STAGES;
+                if (lane == 0) ok = wait_barrier(qd_empty(s), ((gq / KV_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2);
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
                 if (lane == 0) {
@@ -553,29 +561,30 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             uint32_t gs = 0, ga = 0, it = 0;
             bool ok = true;
             auto issue_st = [&]() -> bool {
-                const int s = gs & 1u;
+                const int s = gs & 1u;                  // S^T / dP^T buffer
+                const int qs = gs % KV_STAGES;          // Q / dO stage
                 const uint32_t ph = (gs >> 1) & 1u;
-                if (!wait_barrier(qd_full(s), ph, abort_flag, p.status, 4)) return false;
+                if (!wait_barrier(qd_full(qs), (gs / KV_STAGES) & 1u, abort_flag, p.status, 4)) return false;
                 if (!wait_barrier(st_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
                     umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + KV_SMEM_K + ao, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                              make_smem_desc_sw128(base + KV_SMEM_Q + qs * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
                 }
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
                     umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + KV_SMEM_V + ao, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                              make_smem_desc_sw128(base + KV_SMEM_DO + qs * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
                 }
                 umma_commit(st_full(s));
                 ++gs;
                 return true;
             };
             auto issue_acc = [&](bool first, bool last) -> bool {
-                const int s = ga & 1u;
+                const int s = ga % KV_STAGES;           // Q / dO stage
                 if (!wait_barrier(pds_full, ga & 1u, abort_flag, p.status, 7)) return false;
                 if (first && !wait_barrier(acc_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
                 tc_fence_after_sync();
@@ -628,10 +637,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             const int spos = kt * QT + r;               // key position
             for (int e = 0; e < rep * nq; ++e, ++gq) {
                 const int jq = 2 * kt + e % nq;
-                const int s = gq & 1u;
+                const int s = gq & 1u;                  // S^T / dP^T buffer
+                const int qs = gq % KV_STAGES;          // the element's Q / dO stage, for its vectors
                 const uint32_t ph = (gq >> 1) & 1u;
                 if (!wait_barrier(st_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
-                if (!wait_barrier(qd_full(s), ph, abort_flag, p.status, 15)) { ok = false; break; }   // the element's vectors
+                if (!wait_barrier(qd_full(qs), (gq / KV_STAGES) & 1u, abort_flag, p.status, 15)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t tmem_s = tmem_base + s * 128 + lane_addr + 32 * grp;
                 // the target's key at spos met query t only if t - spos >= m: columns below lo are empty
@@ -651,8 +661,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                         if (c < lo) sr[c] = 0xff800000u;       // -inf: weight 0
                 }
                 // P^T = 2^(S^T c2 - lse2[t]), dS^T = P^T (dP^T scale - D[t] scale), two columns per instruction
-                const float4* nl = reinterpret_cast<const float4*>(vec + s * 128 + 32 * grp);
-                const float4* dd = reinterpret_cast<const float4*>(vec + s * 128 + 64 + 32 * grp);
+                const float4* nl = reinterpret_cast<const float4*>(vec + qs * 128 + 32 * grp);
+                const float4* dd = reinterpret_cast<const float4*>(vec + qs * 128 + 64 + 32 * grp);
                 float pw[32], ds[32];
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4) {
