@@ -285,8 +285,8 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
  *   dQ [B, T, H, D], dK_t, dV_t [B, T, Hkv, D] bf16      out (32-byte aligned)
  *   dK_d, dV_d   HOST arrays of m DEVICE pointers, each [B, T, Hkv, D] bf16, out
  *   workspace    hass_hca_attention_bwd_workspace_bytes(B, T, H, m) bytes, 256-byte aligned
- * Four kinds of kernels are enqueued on cuda_stream (row sums, dQ, dK_t/dV_t, one row-scaling kernel per
- * draft pass). Errors as for the forward.
+ * Four kernels are enqueued on cuda_stream (row sums, dQ, dK_t/dV_t, and for m > 0 a row-scaling kernel for
+ * the draft passes). Errors as for the forward.
  */
 int hass_hca_attention_bwd_workspace_bytes(int64_t B, int64_t T, int64_t H, int32_t m, size_t* bytes);
 int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,

@@ -1365,12 +1365,17 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     }
     g_launches.fetch_add(1);
 
-    for (int i = 0; i < m; ++i) {
+    if (m > 0) {
+        hca_bwd::DraftGradParams dg;
+        std::memset(&dg, 0, sizeof(dg));
+        for (int i = 0; i < m; ++i) {
+            dg.dKd[i] = static_cast<__nv_bfloat16*>(dK_d[i]);
+            dg.dVd[i] = static_cast<__nv_bfloat16*>(dV_d[i]);
+        }
         KernelTimer kt(KIND_HCA_BWD_ROWS, st);
         const long long warps = static_cast<long long>(B) * T * Hkv;
         hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd,
-            static_cast<__nv_bfloat16*>(dK_d[i]), static_cast<__nv_bfloat16*>(dV_d[i]), i, m, iB, iT, iH, iHkv);
+            static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd, dg, m, iB, iT, iH, iHkv);
         g_launches.fetch_add(1);
     }
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;

@@ -749,44 +749,68 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------------
 // Gradients of the draft passes' keys and values: position s of pass i meets exactly one query per head,
 // t = s + i, so dK_d[i][s] = sum over the group's query heads of dS[t, s] Q[t] and likewise for the values.
-// One warp per (sequence, position s, key/value head, pass i); lane = 4 of the 128 columns.
+// One warp per (sequence, query position t, key/value head): it reads the group's Q[t] and dO[t] rows once
+// and writes row t - i of every pass i; the last i rows of pass i have no query and are zeroed by the warp
+// of the same index. Lane = 4 of the 128 columns.
+struct DraftGradParams {
+    __nv_bfloat16* dKd[MAX_DRAFTS];
+    __nv_bfloat16* dVd[MAX_DRAFTS];
+};
+
 __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
                                       const float* __restrict__ Pd, const float* __restrict__ dSd,
-                                      __nv_bfloat16* dKd, __nv_bfloat16* dVd, int i, int m, int B, int T, int H,
-                                      int Hkv) {
-    const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, s, g)
+                                      const __grid_constant__ DraftGradParams out, int m, int B, int T, int H, int Hkv) {
+    const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, t, g)
     const int lane = threadIdx.x & 31;
     if (w >= static_cast<long long>(B) * T * Hkv) return;
     const int g = static_cast<int>(w % Hkv);
-    const long long bs = w / Hkv;
-    const int s = static_cast<int>(bs % T);
-    const int b = static_cast<int>(bs / T);
-    const int t = s + i;
+    const long long bt = w / Hkv;
+    const int t = static_cast<int>(bt % T);
+    const int b = static_cast<int>(bt / T);
     const int rep = H / Hkv;
     auto lo = [](uint32_t x) { return __uint_as_float(x << 16); };
     auto hi = [](uint32_t x) { return __uint_as_float(x & 0xffff0000u); };
-    float k0 = 0.f, k1 = 0.f, k2 = 0.f, k3 = 0.f, v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
-    if (t < T) {
-        for (int hh = 0; hh < rep; ++hh) {
-            const int h = g * rep + hh;
-            const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m + i;
-            const float pw = Pd[ri], ds = dSd[ri];
-            const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
-            const uint2 q = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
-            const uint2 d = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
-            k0 = fmaf(ds, lo(q.x), k0);
-            k1 = fmaf(ds, hi(q.x), k1);
-            k2 = fmaf(ds, lo(q.y), k2);
-            k3 = fmaf(ds, hi(q.y), k3);
-            v0 = fmaf(pw, lo(d.x), v0);
-            v1 = fmaf(pw, hi(d.x), v1);
-            v2 = fmaf(pw, lo(d.y), v2);
-            v3 = fmaf(pw, hi(d.y), v3);
+    float kacc[MAX_DRAFTS][4], vacc[MAX_DRAFTS][4];
+#pragma unroll
+    for (int i = 0; i < MAX_DRAFTS; ++i)
+#pragma unroll
+        for (int u = 0; u < 4; ++u) kacc[i][u] = vacc[i][u] = 0.f;
+    for (int hh = 0; hh < rep; ++hh) {
+        const int h = g * rep + hh;
+        const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
+        const uint2 d = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
+        const float qf[4] = {lo(q.x), hi(q.x), lo(q.y), hi(q.y)}, df[4] = {lo(d.x), hi(d.x), lo(d.y), hi(d.y)};
+        const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m;
+#pragma unroll
+        for (int i = 0; i < MAX_DRAFTS; ++i) {
+            if (i < m) {
+                const float pw = Pd[ri + i], ds = dSd[ri + i];     // zero where t - i < 0
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    kacc[i][u] = fmaf(ds, qf[u], kacc[i][u]);
+                    vacc[i][u] = fmaf(pw, df[u], vacc[i][u]);
+                }
+            }
         }
     }
-    const size_t orow = ((static_cast<size_t>(b) * T + s) * Hkv + g) * HD;
-    *(reinterpret_cast<uint2*>(dKd + orow) + lane) = make_uint2(pack_bf16(k0, k1), pack_bf16(k2, k3));
-    *(reinterpret_cast<uint2*>(dVd + orow) + lane) = make_uint2(pack_bf16(v0, v1), pack_bf16(v2, v3));
+#pragma unroll
+    for (int i = 0; i < MAX_DRAFTS; ++i) {
+        if (i < m) {
+            if (t - i >= 0) {
+                const size_t orow = ((static_cast<size_t>(b) * T + (t - i)) * Hkv + g) * HD;
+                *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) =
+                    make_uint2(pack_bf16(kacc[i][0], kacc[i][1]), pack_bf16(kacc[i][2], kacc[i][3]));
+                *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) =
+                    make_uint2(pack_bf16(vacc[i][0], vacc[i][1]), pack_bf16(vacc[i][2], vacc[i][3]));
+            }
+            if (t + i >= T) {       // position t of pass i would meet query t + i, past the sequence
+                const size_t orow = ((static_cast<size_t>(b) * T + t) * Hkv + g) * HD;
+                *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) = make_uint2(0u, 0u);
+                *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) = make_uint2(0u, 0u);
+            }
+        }
+    }
 }
 
 }  // namespace hca_bwd
