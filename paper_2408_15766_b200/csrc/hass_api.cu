@@ -1325,7 +1325,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     {   // D = rowsum(dO * O)
         KernelTimer kt(KIND_HCA_BWD_ROWS, st);
         const long long rows = static_cast<long long>(B) * T * H;
-        hca_bwd::hca_bwd_prep_kernel<<<static_cast<unsigned>((rows * 32 + 255) / 256), 256, 0, st>>>(
+        hca_bwd::hca_bwd_prep_kernel<<<static_cast<unsigned>((rows * 16 + 255) / 256), 256, 0, st>>>(
             static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Dv, iB, iT, iH);
     }
     g_launches.fetch_add(1);

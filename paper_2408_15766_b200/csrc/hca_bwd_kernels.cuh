@@ -32,20 +32,24 @@ constexpr int KV_BYTES = KT * HD * 2;
 constexpr int KV_HALF = KV_BYTES / 2;
 constexpr int DS_BYTES = QT * KT * 2;
 
-// D[b, h, t] = <dO[b, t, h, :], O[b, t, h, :]>, one warp per row of 128.
+// D[b, h, t] = <dO[b, t, h, :], O[b, t, h, :]>, half a warp per row of 128 (16 bytes per lane and tensor).
 __global__ void hca_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                     float* __restrict__ D, int B, int T, int H) {
-    const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, t, h)
-    const int lane = threadIdx.x & 31;
-    if (row >= static_cast<long long>(B) * T * H) return;
-    const uint2 a = __ldg(reinterpret_cast<const uint2*>(O + row * HD) + lane);
-    const uint2 c = __ldg(reinterpret_cast<const uint2*>(dO + row * HD) + lane);
+    const long long row = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;   // (b, t, h)
+    const int sub = threadIdx.x & 15;
+    const bool live = row < static_cast<long long>(B) * T * H;
     auto lo = [](uint32_t w) { return __uint_as_float(w << 16); };
     auto hi = [](uint32_t w) { return __uint_as_float(w & 0xffff0000u); };
-    float acc = lo(a.x) * lo(c.x) + hi(a.x) * hi(c.x) + lo(a.y) * lo(c.y) + hi(a.y) * hi(c.y);
+    float acc = 0.f;
+    if (live) {
+        const uint4 a = __ldg(reinterpret_cast<const uint4*>(O + row * HD) + sub);
+        const uint4 c = __ldg(reinterpret_cast<const uint4*>(dO + row * HD) + sub);
+        acc = lo(a.x) * lo(c.x) + hi(a.x) * hi(c.x) + lo(a.y) * lo(c.y) + hi(a.y) * hi(c.y) + lo(a.z) * lo(c.z) +
+              hi(a.z) * hi(c.z) + lo(a.w) * lo(c.w) + hi(a.w) * hi(c.w);
+    }
 #pragma unroll
-    for (int sft = 16; sft >= 1; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
-    if (lane == 0) {
+    for (int sft = 8; sft >= 1; sft >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sft);
+    if (live && sub == 0) {
         const int h = static_cast<int>(row % H);
         const long long bt = row / H;
         const int t = static_cast<int>(bt % T);
@@ -775,6 +779,7 @@ __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const
     for (int i = 0; i < MAX_DRAFTS; ++i)
 #pragma unroll
         for (int u = 0; u < 4; ++u) kacc[i][u] = vacc[i][u] = 0.f;
+#pragma unroll 4
     for (int hh = 0; hh < rep; ++hh) {
         const int h = g * rep + hh;
         const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
