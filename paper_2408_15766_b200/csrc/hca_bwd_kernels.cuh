@@ -774,45 +774,62 @@ __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const
     const int rep = H / Hkv;
     auto lo = [](uint32_t x) { return __uint_as_float(x << 16); };
     auto hi = [](uint32_t x) { return __uint_as_float(x & 0xffff0000u); };
-    float kacc[MAX_DRAFTS][4], vacc[MAX_DRAFTS][4];
+    // two passes at a time (the group's rows are re-read from cache for further pairs): few registers, many warps in flight
+    for (int i0 = 0; i0 < m; i0 += 2) {
+        float kacc[2][4], vacc[2][4];
 #pragma unroll
-    for (int i = 0; i < MAX_DRAFTS; ++i)
+        for (int j = 0; j < 2; ++j)
 #pragma unroll
-        for (int u = 0; u < 4; ++u) kacc[i][u] = vacc[i][u] = 0.f;
-#pragma unroll 4
-    for (int hh = 0; hh < rep; ++hh) {
-        const int h = g * rep + hh;
-        const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
-        const uint2 q = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
-        const uint2 d = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
-        const float qf[4] = {lo(q.x), hi(q.x), lo(q.y), hi(q.y)}, df[4] = {lo(d.x), hi(d.x), lo(d.y), hi(d.y)};
-        const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m;
+            for (int c = 0; c < 4; ++c) kacc[j][c] = vacc[j][c] = 0.f;
+        // four heads of the group at a time, all their loads issued before any is used
+        for (int h0 = 0; h0 < rep; h0 += 4) {
+            uint2 q[4], d[4];
+            float pw[4][2], ds[4][2];
 #pragma unroll
-        for (int i = 0; i < MAX_DRAFTS; ++i) {
-            if (i < m) {
-                const float pw = Pd[ri + i], ds = dSd[ri + i];     // zero where t - i < 0
+            for (int u = 0; u < 4; ++u) {
+                const bool on = h0 + u < rep;
+                const int h = g * rep + (on ? h0 + u : 0);
+                const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
+                q[u] = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
+                d[u] = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
+                const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    kacc[i][u] = fmaf(ds, qf[u], kacc[i][u]);
-                    vacc[i][u] = fmaf(pw, df[u], vacc[i][u]);
+                for (int j = 0; j < 2; ++j) {
+                    const bool use = on && i0 + j < m;
+                    pw[u][j] = use ? __ldg(Pd + ri + i0 + j) : 0.f;      // zero where t - i < 0
+                    ds[u][j] = use ? __ldg(dSd + ri + i0 + j) : 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float qf[4] = {lo(q[u].x), hi(q[u].x), lo(q[u].y), hi(q[u].y)};
+                const float df[4] = {lo(d[u].x), hi(d[u].x), lo(d[u].y), hi(d[u].y)};
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        kacc[j][c] = fmaf(ds[u][j], qf[c], kacc[j][c]);
+                        vacc[j][c] = fmaf(pw[u][j], df[c], vacc[j][c]);
+                    }
                 }
             }
         }
-    }
 #pragma unroll
-    for (int i = 0; i < MAX_DRAFTS; ++i) {
-        if (i < m) {
-            if (t - i >= 0) {
-                const size_t orow = ((static_cast<size_t>(b) * T + (t - i)) * Hkv + g) * HD;
-                *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) =
-                    make_uint2(pack_bf16(kacc[i][0], kacc[i][1]), pack_bf16(kacc[i][2], kacc[i][3]));
-                *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) =
-                    make_uint2(pack_bf16(vacc[i][0], vacc[i][1]), pack_bf16(vacc[i][2], vacc[i][3]));
-            }
-            if (t + i >= T) {       // position t of pass i would meet query t + i, past the sequence
-                const size_t orow = ((static_cast<size_t>(b) * T + t) * Hkv + g) * HD;
-                *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) = make_uint2(0u, 0u);
-                *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) = make_uint2(0u, 0u);
+        for (int j = 0; j < 2; ++j) {
+            const int i = i0 + j;
+            if (i < m) {
+                if (t - i >= 0) {
+                    const size_t orow = ((static_cast<size_t>(b) * T + (t - i)) * Hkv + g) * HD;
+                    *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) =
+                        make_uint2(pack_bf16(kacc[j][0], kacc[j][1]), pack_bf16(kacc[j][2], kacc[j][3]));
+                    *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) =
+                        make_uint2(pack_bf16(vacc[j][0], vacc[j][1]), pack_bf16(vacc[j][2], vacc[j][3]));
+                }
+                if (t + i >= T) {       // position t of pass i would meet query t + i, past the sequence
+                    const size_t orow = ((static_cast<size_t>(b) * T + t) * Hkv + g) * HD;
+                    *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) = make_uint2(0u, 0u);
+                    *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) = make_uint2(0u, 0u);
+                }
             }
         }
     }
