@@ -183,11 +183,12 @@ def run_reference(args, rank: int, world: int):
 
 # ---- HCA attention of the draft layer (Section 3.2) ---------------------------------------------------
 HCA_METRIC = "tokens/sec HCA attention fwd"
+HCA_METRIC_BWD = "tokens/sec HCA attention fwd+bwd"
 
 
-def time_hca_oracle(inp, pairs):
+def time_hca_oracle(inp, pairs, backward=False):
     """fp64 oracle on whole (sequence, head) pairs; returns token-equivalents per second (a pair is
-    T / H of a sequence's attention work)."""
+    T / H of a sequence's attention work). With backward, the gradients for dO = Q are computed too."""
     from oracle import hca_oracle as ho
     wl = inp.wl
     rep = wl.H // wl.Hkv
@@ -195,8 +196,11 @@ def time_hca_oracle(inp, pairs):
     t0 = time.perf_counter()
     for b, h in pairs:
         g = h // rep
-        ho.hca_attention(f(inp.Q, b, h), f(inp.K_t, b, g), f(inp.V_t, b, g), [f(x, b, g) for x in inp.K_d],
-                         [f(x, b, g) for x in inp.V_d])
+        a = (f(inp.Q, b, h), f(inp.K_t, b, g), f(inp.V_t, b, g), [f(x, b, g) for x in inp.K_d],
+             [f(x, b, g) for x in inp.V_d])
+        ho.hca_attention(*a)
+        if backward:
+            ho.hca_attention_grad(*a, a[0])
     dt = time.perf_counter() - t0
     return len(pairs) * wl.T / wl.H / dt, dt
 
@@ -209,8 +213,11 @@ def hca_pairs(wl, n, seed=0):
 def main_hca(args):
     wl = hi.HCA_WORKLOADS[args.workload]
     tokens = wl.B * wl.T
+    bwd = args.hca_pass == "fwd_bwd"
+    metric = HCA_METRIC_BWD if bwd else HCA_METRIC
     config = {"workload": wl.name, "B": wl.B, "T": wl.T, "heads": wl.H, "kv_heads": wl.Hkv, "head_dim": wl.D,
-              "draft_passes_m": wl.m, "aligning_step": wl.m + 1, "path": "hass_hca_attention_fwd"}
+              "draft_passes_m": wl.m, "aligning_step": wl.m + 1,
+              "path": "hass_hca_attention_fwd + hass_hca_attention_bwd" if bwd else "hass_hca_attention_fwd"}
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
             return
@@ -218,12 +225,12 @@ def main_hca(args):
         n_pairs = args.oracle_rows or 4
         vals = []
         for i in range(args.warmup + args.steps):
-            v = time_hca_oracle(inp, hca_pairs(wl, n_pairs, seed=i))
+            v = time_hca_oracle(inp, hca_pairs(wl, n_pairs, seed=i), backward=bwd)
             if i >= args.warmup:
                 vals.append(v)
         tps = float(np.mean([v[0] for v in vals]))
         sample = f"{n_pairs} of {wl.B * wl.H} (sequence, head) pairs per step, all {wl.T} positions"
-        print(json.dumps({"impl": "reference", "metric": HCA_METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+        print(json.dumps({"impl": "reference", "metric": metric, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
                           "steps": args.steps, "warmup": args.warmup,
                           "ms_per_step": float(np.mean([v[1] for v in vals]) * 1e3), "higher_is_better": True,
                           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -244,15 +251,23 @@ def main_hca(args):
     Q, K_t, V_t = (x.to(dev) for x in host[:3])
     K_d, V_d = [x.to(dev) for x in inp.K_d], [x.to(dev) for x in inp.V_d]
     ws = torch.zeros(hass.hca_attention_workspace_bytes(), dtype=torch.uint8, device=dev)
+    ws_b = torch.zeros(hass.hca_attention_bwd_workspace_bytes(wl.B, wl.T, wl.H, wl.m), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
     in_bytes = sum(x.numel() * 2 for x in host)
+    g = torch.Generator().manual_seed(wl.seed + 77)
+    dO_host = torch.randn(inp.Q.shape, generator=g).to(torch.bfloat16)     # upstream gradient of the attention output
+    dO = dO_host.to(dev)
 
     def step():
-        return hass.hca_attention_fwd(Q, K_t, V_t, K_d, V_d, workspace=ws, stream=stream)
+        out = hass.hca_attention_fwd(Q, K_t, V_t, K_d, V_d, workspace=ws, stream=stream)
+        if bwd:
+            hass.hca_attention_bwd(Q, K_t, V_t, K_d, V_d, out["O"], out["lse"], dO, workspace=ws_b, stream=stream)
+        return out
 
     for _ in range(args.warmup):
         step()
     hass.check(ws)
+    hass.check(ws_b)
     barrier(world)
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
@@ -272,6 +287,7 @@ def main_hca(args):
     hass.profile_enable(False)
     clocks = sampler.stop()
     hass.check(ws)
+    hass.check(ws_b)
     ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
 
     # end to end: projected features from pinned host memory, O back to host, through the public call
@@ -279,12 +295,19 @@ def main_hca(args):
     if not args.no_e2e:
         pinned = [x.pin_memory() for x in host]
         O_h = torch.empty_like(inp.Q).pin_memory()
+        dO_pin = dO_host.pin_memory()
+        grads_h = [torch.empty_like(x).pin_memory() for x in host] if bwd else []
 
         def step_e2e():
             d_ = [x.to(dev, non_blocking=True) for x in pinned]
             out = hass.hca_attention_fwd(d_[0], d_[1], d_[2], d_[3:3 + wl.m], d_[3 + wl.m:], workspace=ws,
-                                         want_lse=False, stream=stream)
+                                         want_lse=bwd, stream=stream)
             O_h.copy_(out["O"], non_blocking=True)
+            if bwd:
+                gr = hass.hca_attention_bwd(d_[0], d_[1], d_[2], d_[3:3 + wl.m], d_[3 + wl.m:], out["O"], out["lse"],
+                                            dO_pin.to(dev, non_blocking=True), workspace=ws_b, stream=stream)
+                for dst, src in zip(grads_h, [gr["dQ"], gr["dK_t"], gr["dV_t"], *gr["dK_d"], *gr["dV_d"]]):
+                    dst.copy_(src, non_blocking=True)
 
         for _ in range(3):
             step_e2e()
@@ -299,21 +322,31 @@ def main_hca(args):
         barrier(world)
         ms_e2e = max_over_ranks(e0.elapsed_time(e1) / n_e2e, world, dev)
         e2e = {"value": aggregate(tokens, world, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
-               "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": inp.Q.numel() * 2,
-               "note": "Q, K_t, V_t and the draft passes' K/V from pinned host memory, O back to host"}
+               "h2d_bytes_per_step": in_bytes + (inp.Q.numel() * 2 if bwd else 0),
+               "d2h_bytes_per_step": inp.Q.numel() * 2 + (in_bytes if bwd else 0),
+               "note": "Q, K_t, V_t and the draft passes' K/V (and dO) from pinned host memory, O (and all "
+                       "gradients) back to host"}
     if rank != 0:
         return
-    # causal attention: two products of 2 * D flops per (query, key) pair with key <= query
-    flops = 4.0 * wl.D * wl.B * wl.H * wl.T * (wl.T + 1) / 2
-    ms_k, cnt = prof["hca_attention"]
+    # causal attention: one product = 2 * D flops per (query, key) pair with key <= query; the forward runs 2,
+    # the dQ kernel 3 (S, dP, dQ), the dK/dV kernel 4 (S^T, dP^T, dV, dK): 7 executed for 5 algorithmic
+    prod = 2.0 * wl.D * wl.B * wl.H * wl.T * (wl.T + 1) / 2
+    products = {"hca_attention": 2, "hca_bwd_dq": 3, "hca_bwd_dkv": 4}
+    kernel_rows = {k: {"ms_per_step": ms / args.steps, "launches_per_step": c / args.steps,
+                       **({"tflops": products[k] * prod / (ms / c * 1e-3) / 1e12} if k in products else {})}
+                   for k, (ms, c) in prof.items() if c}
+    dom = max(products, key=lambda k: prof[k][0])
+    ms_k, cnt = prof[dom]
+    flops = products[dom] * prod
     achieved = flops / (ms_k / cnt * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
-    line = {"metric": HCA_METRIC, "value": aggregate(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
+    line = {"metric": metric, "value": aggregate(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": dict(config, l2="inputs and output (%.0f MB) larger than L2" % ((in_bytes + inp.Q.numel() * 2) / 1e6)),
             "clocks": clocks, "gpu_launches": launches,
-            "roofline": {"bound": "tensor", "kernel": "hca_attention", "achieved": achieved, "peak": peak,
+            "kernels": kernel_rows,
+            "roofline": {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
                          "peak_kind": f"bf16_tflops (burst), of {peak_kind} (a sub-millisecond kernel timed alone)",
                          "flops_per_launch": flops, "avg_launch_ms": ms_k / cnt}}
@@ -321,7 +354,9 @@ def main_hca(args):
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
         n_pairs = args.oracle_rows or min(wl.B * wl.H, 192)      # about 10 s of CPU work at T = 2048
-        tps, dt = time_hca_oracle(inp, hca_pairs(wl, n_pairs))
+        if bwd and not args.oracle_rows:
+            n_pairs = max(8, n_pairs // 4)
+        tps, dt = time_hca_oracle(inp, hca_pairs(wl, n_pairs), backward=bwd)
         line["cpu_baseline"] = {"value": tps, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                 "sample": f"{n_pairs} (sequence, head) pairs drawn with replacement from {wl.B * wl.H}, all {wl.T} positions, {dt:.1f} s"}
     print(json.dumps(line), flush=True)
@@ -342,6 +377,8 @@ def main():
                          "+ w * Top-K in one call (8 N d V tensor FLOPs); top_p (P = 0.5, at most K tokens) and "
                          "normed (Normed Top-K: only the target product, 2 N d V) and bidir (Bi-directional "
                          "Top-K) are the loss variants of Section 4.3")
+    ap.add_argument("--hca-pass", default="fwd", choices=["fwd", "fwd_bwd"],
+                    help="hca-* workloads: time the forward alone, or forward + backward (all input gradients)")
     ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
