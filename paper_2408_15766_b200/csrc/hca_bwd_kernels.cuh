@@ -120,8 +120,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(sdp_full(s), 1);
-            mbar_init(sdp_empty(s), 8);
-            mbar_init(ds_full(s), 8);
+            mbar_init(sdp_empty(s), 4);
+            mbar_init(ds_full(s), 4);
             mbar_init(ds_empty(s), 1);
         }
         mbar_init(dq_done, 1);
@@ -253,8 +253,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             }
         }
     } else {
-        // two groups of four warps share every row: group grp takes columns 32 grp .. 32 grp + 31 of each
-        // 64-column tile (nothing crosses columns here), and half of the dQ row in the epilogue
+        // two groups of four warps: group grp takes the elements with (running index & 1) == grp, i.e. always the
+        // S / dP buffer and the dS buffer of its own index, so each group has two element slots of time for its
+        // chain TMEM load -> row math -> dS store (nothing is carried from one element to the next); in the
+        // epilogue each group stores half of the dQ row
         const int grp = (warp - 2) >> 2;
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
@@ -276,53 +278,60 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             const float Dt = valid ? p.D[row_idx] : 0.f;
             const float nDs = -Dt * p.scale;
             for (int e = 0; e < n + 2 * m; ++e, ++g) {
-                const int s = g & 1u;
+                if ((g & 1u) != static_cast<uint32_t>(grp)) continue;
+                const int s = grp;
                 const uint32_t ph = (g >> 1) & 1u;
                 if (!wait_barrier(sdp_full(s), ph, abort_flag, p.status, 10)) { ok = false; break; }
                 tc_fence_after_sync();
-                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr + 32 * grp;
+                const uint32_t tmem_s = tmem_base + s * 128 + lane_addr;
                 if (e < n) {
-                    // ---- key tile: dS for this group's 32 columns of the row ----
+                    // ---- key tile: dS for the row, 32 columns at a time ----
                     const bool band = e * KT + KT - 1 > qt * QT - m;
-                    const int lim = t - m - e * KT - 32 * grp;
-                    uint32_t sr[32], dr[32];
-                    tmem_ld32(tmem_s, sr);
-                    tmem_ld32(tmem_s + 64, dr);
-                    tmem_ld_wait(sr);
-                    tmem_ld_wait(dr);
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(sdp_empty(s));
-                    if (band) {
+                    bool stop = false;
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (c > lim) sr[c] = 0xff800000u;       // -inf: weight 0
-                    }
-                    // dS = P (dP - D) scale = 2^(S c2 - lse2) (dP scale - D scale), two columns per instruction
-                    float ds[32];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float x0, x1, y0, y1;
-                        ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), p.c2, p.c2, nlse2, nlse2);
-                        ffma2(y0, y1, __uint_as_float(dr[c]), __uint_as_float(dr[c + 1]), p.scale, p.scale, nDs, nDs);
-                        fmul2(ds[c], ds[c + 1], ex2(x0), ex2(x1), y0, y1);
-                    }
-                    if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        st_shared_v4(ds_addr(s, 4 * grp + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
-                                     pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
-                                     pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
-                } else {
-                    // ---- draft pass i, half hf: only the diagonal element of the rows of that half; it lies in
-                    //      this group's columns when (r & 63) / 32 == grp ----
-                    const int i = (e - n) >> 1, hf = (e - n) & 1;
-                    const bool holder = (r >> 6) == hf && (quad & 1) == grp;
-                    float sv = 0.f, dv = 0.f;
-                    if (holder) {               // warp-uniform
+                    for (int hc = 0; hc < 2; ++hc) {
+                        const int lim = t - m - e * KT - 32 * hc;
                         uint32_t sr[32], dr[32];
-                        tmem_ld32(tmem_s, sr);
-                        tmem_ld32(tmem_s + 64, dr);
+                        tmem_ld32(tmem_s + 32 * hc, sr);
+                        tmem_ld32(tmem_s + 64 + 32 * hc, dr);
+                        tmem_ld_wait(sr);
+                        tmem_ld_wait(dr);
+                        if (hc == 1) {
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(sdp_empty(s));
+                        }
+                        if (band) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c > lim) sr[c] = 0xff800000u;       // -inf: weight 0
+                        }
+                        // dS = P (dP - D) scale = 2^(S c2 - lse2) (dP scale - D scale), two columns per instruction
+                        float ds[32];
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            float x0, x1, y0, y1;
+                            ffma2(x0, x1, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]), p.c2, p.c2, nlse2, nlse2);
+                            ffma2(y0, y1, __uint_as_float(dr[c]), __uint_as_float(dr[c + 1]), p.scale, p.scale, nDs, nDs);
+                            fmul2(ds[c], ds[c + 1], ex2(x0), ex2(x1), y0, y1);
+                        }
+                        if (hc == 0 && !wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { stop = true; break; }
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            st_shared_v4(ds_addr(s, 4 * hc + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
+                                         pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
+                                         pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
+                    }
+                    if (stop) { ok = false; break; }
+                } else {
+                    // ---- draft pass i, half hf: only the diagonal element of the rows of that half ----
+                    const int i = (e - n) >> 1, hf = (e - n) & 1;
+                    const bool holder = (r >> 6) == hf;        // warp-uniform
+                    float sv = 0.f, dv = 0.f;
+                    if (holder) {
+                        uint32_t sr[32], dr[32];
+                        tmem_ld32(tmem_s + 32 * (quad & 1), sr);
+                        tmem_ld32(tmem_s + 64 + 32 * (quad & 1), dr);
                         tmem_ld_wait(sr);
                         tmem_ld_wait(dr);
 #pragma unroll
@@ -338,17 +347,16 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                     if (lane == 0) mbar_arrive(sdp_empty(s));
                     const bool mine = holder && t - i >= 0 && valid;
                     const float pw = mine ? ex2(fmaf(sv, p.c2, nlse2)) : 0.f;
-                    const float dsv = pw * fmaf(dv, p.scale, nDs);
+                    const float dsv = mine ? pw * fmaf(dv, p.scale, nDs) : 0.f;
                     if (holder && valid) {
                         p.Pd[row_idx * m + i] = pw;
-                        p.dSd[row_idx * m + i] = mine ? dsv : 0.f;
+                        p.dSd[row_idx * m + i] = dsv;
                     }
-                    const uint32_t bits = mine ? pack_bf16(dsv, 0.f) << ((r & 1) * 16) : 0u;
+                    const uint32_t bits = pack_bf16(dsv, 0.f) << ((r & 1) * 16);
                     if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const int chunk = 4 * grp + q4;
-                        const bool here = chunk == ((r & 63) >> 3);
+                    for (int chunk = 0; chunk < 8; ++chunk) {
+                        const bool here = holder && chunk == ((r & 63) >> 3);
                         const int w = (r & 7) >> 1;
                         st_shared_v4(ds_addr(s, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
                                      here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
