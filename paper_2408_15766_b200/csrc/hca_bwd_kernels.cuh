@@ -191,48 +191,60 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        // The whole warp runs this loop so that addresses and descriptors stay warp-uniform; one elected lane
+        // issues the tensor-core instructions.
+        {
             constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
             constexpr uint32_t idesc_q = make_idesc_bf16(QT, HD, 0, 1);
             uint32_t gs = 0, gq = 0, it = 0;      // elements whose S/dP, resp. dQ product has been issued
             bool ok = true;
+            auto wait_all = [&](uint32_t bar, uint32_t parity, unsigned code) {
+                return __all_sync(0xffffffffu, wait_barrier(bar, parity, abort_flag, p.status, code)) != 0;
+            };
             auto issue_sdp = [&]() -> bool {
                 const int s = gs & 1u;                  // S / dP buffer
                 const int ks = gs % DQ_STAGES;          // K / V stage
                 const uint32_t ph = (gs >> 1) & 1u;
-                if (!wait_barrier(kv_full(ks), (gs / DQ_STAGES) & 1u, abort_flag, p.status, 4)) return false;
-                if (!wait_barrier(sdp_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
+                if (!wait_all(kv_full(ks), (gs / DQ_STAGES) & 1u, 4)) return false;
+                if (!wait_all(sdp_empty(s), ph ^ 1u, 5)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
-                    umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + DQ_SMEM_Q + qo, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                    const uint64_t dq_ = make_smem_desc_sw128(base + DQ_SMEM_Q + qo, 0, 1024);
+                    const uint64_t dk_ = make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + ko, 0, 1024);
+                    const uint64_t do_ = make_smem_desc_sw128(base + DQ_SMEM_DO + qo, 0, 1024);
+                    const uint64_t dv_ = make_smem_desc_sw128(base + DQ_SMEM_V + ks * KV_BYTES + ko, 0, 1024);
+                    if (leader) {
+                        umma_bf16(tmem_base + s * 128, dq_, dk_, idesc_s, k != 0 ? 1u : 0u);
+                        umma_bf16(tmem_base + s * 128 + 64, do_, dv_, idesc_s, k != 0 ? 1u : 0u);
+                    }
                 }
-#pragma unroll
-                for (int k = 0; k < HD / 16; ++k) {
-                    const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
-                    umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + DQ_SMEM_DO + qo, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_V + ks * KV_BYTES + ko, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
-                }
-                umma_commit(sdp_full(s));
+                if (leader) umma_commit(sdp_full(s));
+                __syncwarp();
                 ++gs;
                 return true;
             };
             auto issue_dq = [&](bool first, bool last) -> bool {
                 const int s = gq & 1u;                  // dS buffer
                 const int ks = gq % DQ_STAGES;          // K stage
-                if (!wait_barrier(ds_full(s), (gq >> 1) & 1u, abort_flag, p.status, 7)) return false;
-                if (first && !wait_barrier(dq_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                if (!wait_all(ds_full(s), (gq >> 1) & 1u, 7)) return false;
+                if (first && !wait_all(dq_free, (it & 1u) ^ 1u, 9)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
-                for (int k = 0; k < KT / 16; ++k)
-                    umma_bf16(tmem_base + 256, make_smem_desc_sw128(base + DQ_SMEM_DS + s * DS_BYTES + k * 32, 0, 1024),
-                              make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_q,
-                              (!first || k != 0) ? 1u : 0u);
-                umma_commit(kv_empty(ks));
-                umma_commit(ds_empty(s));
-                if (last) umma_commit(dq_done);
+                for (int k = 0; k < KT / 16; ++k) {
+                    const uint64_t da_ = make_smem_desc_sw128(base + DQ_SMEM_DS + s * DS_BYTES + k * 32, 0, 1024);
+                    const uint64_t db_ = make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
+                    if (leader) umma_bf16(tmem_base + 256, da_, db_, idesc_q, (!first || k != 0) ? 1u : 0u);
+                }
+                if (leader) {
+                    umma_commit(kv_empty(ks));
+                    umma_commit(ds_empty(s));
+                    if (last) umma_commit(dq_done);
+                }
+                __syncwarp();
                 ++gq;
                 return true;
             };
@@ -240,13 +252,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int n_e = key_tiles(qt) + 2 * m;
-                if (!wait_barrier(qdo_full, it & 1u, abort_flag, p.status, 6)) break;
+                if (!wait_all(qdo_full, it & 1u, 6)) break;
                 if (!issue_sdp()) break;
-                if (n_e == 1) umma_commit(qdo_empty);
+                if (n_e == 1 && elect_one()) umma_commit(qdo_empty);
                 for (int a = 0; a < n_e && ok; ++a) {
                     if (a + 1 < n_e) {
                         ok = issue_sdp();
-                        if (ok && a + 2 == n_e) umma_commit(qdo_empty);
+                        if (ok && a + 2 == n_e && elect_one()) umma_commit(qdo_empty);
                     }
                     if (ok) ok = issue_dq(a == 0, a + 1 == n_e);
                 }
