@@ -71,9 +71,10 @@ constexpr int DQ_SMEM_K = DQ_SMEM_DO + Q_BYTES;
 constexpr int DQ_SMEM_V = DQ_SMEM_K + DQ_STAGES * KV_BYTES;
 constexpr int DQ_SMEM_DS = DQ_SMEM_V + DQ_STAGES * KV_BYTES;   // 2 buffers
 constexpr int DQ_SMEM_BAR = DQ_SMEM_DS + 2 * DS_BYTES;
-constexpr int DQ_NUM_BARS = 2 * DQ_STAGES + 12;
+constexpr int DQ_NUM_BARS = 2 * DQ_STAGES + 14;
 constexpr int DQ_SMEM_BYTES = DQ_SMEM_BAR + 256 + 1024 /*alignment slack*/;
-constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb, dP at 128 sb + 64; dQ at 256
+constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb, dP at 128 sb + 64; dQ at 256; Q at 384 and dO at 448 as bf16 pairs
+constexpr int DQ_TMEM_Q = 384, DQ_TMEM_DO = 448;
 
 struct DqParams {
     CUtensorMap tmQ, tmdO;         // [B, T, H * 128], box {64, 128, 1}
@@ -105,6 +106,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
     auto ds_full = [&](int s) { return bar0 + 8u * (6 + 2 * DQ_STAGES + s); };
     auto ds_empty = [&](int s) { return bar0 + 8u * (8 + 2 * DQ_STAGES + s); };
     const uint32_t dq_done = bar0 + 8u * (10 + 2 * DQ_STAGES), dq_free = bar0 + 8u * (11 + 2 * DQ_STAGES);
+    const uint32_t qt_ready = bar0 + 8u * (12 + 2 * DQ_STAGES);    // Q and dO of the item copied into tensor memory
+    const uint32_t qt_free = bar0 + 8u * (13 + 2 * DQ_STAGES);     // ... and read by the item's last S / dP product
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_gen + DQ_SMEM_BAR + 8 * DQ_NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
@@ -113,7 +116,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
 
     if (threadIdx.x == 0) {
         mbar_init(qdo_full, 1);
-        mbar_init(qdo_empty, 1);
+        mbar_init(qdo_empty, 8);
+        mbar_init(qt_ready, 8);
+        mbar_init(qt_free, 1);
         for (int s = 0; s < DQ_STAGES; ++s) {
             mbar_init(kv_full(s), 1);
             mbar_init(kv_empty(s), 1);
@@ -211,14 +216,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
-                    const uint32_t qo = (k >> 2) * Q_HALF + (k & 3) * 32, ko = (k >> 2) * KV_HALF + (k & 3) * 32;
-                    const uint64_t dq_ = make_smem_desc_sw128(base + DQ_SMEM_Q + qo, 0, 1024);
+                    const uint32_t ko = (k >> 2) * KV_HALF + (k & 3) * 32;
+                    // A (Q, dO) comes from tensor memory, 8 columns per K step: only B is read from shared memory
                     const uint64_t dk_ = make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + ko, 0, 1024);
-                    const uint64_t do_ = make_smem_desc_sw128(base + DQ_SMEM_DO + qo, 0, 1024);
                     const uint64_t dv_ = make_smem_desc_sw128(base + DQ_SMEM_V + ks * KV_BYTES + ko, 0, 1024);
                     if (leader) {
-                        umma_bf16(tmem_base + s * 128, dq_, dk_, idesc_s, k != 0 ? 1u : 0u);
-                        umma_bf16(tmem_base + s * 128 + 64, do_, dv_, idesc_s, k != 0 ? 1u : 0u);
+                        umma_bf16_ta(tmem_base + s * 128, tmem_base + DQ_TMEM_Q + 8 * k, dk_, idesc_s, k != 0 ? 1u : 0u);
+                        umma_bf16_ta(tmem_base + s * 128 + 64, tmem_base + DQ_TMEM_DO + 8 * k, dv_, idesc_s, k != 0 ? 1u : 0u);
                     }
                 }
                 if (leader) umma_commit(sdp_full(s));
@@ -252,13 +256,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int n_e = key_tiles(qt) + 2 * m;
-                if (!wait_all(qdo_full, it & 1u, 6)) break;
+                if (!wait_all(qt_ready, it & 1u, 6)) break;
                 if (!issue_sdp()) break;
-                if (n_e == 1 && elect_one()) umma_commit(qdo_empty);
+                if (n_e == 1 && elect_one()) umma_commit(qt_free);
                 for (int a = 0; a < n_e && ok; ++a) {
                     if (a + 1 < n_e) {
                         ok = issue_sdp();
-                        if (ok && a + 2 == n_e && elect_one()) umma_commit(qdo_empty);
+                        if (ok && a + 2 == n_e && elect_one()) umma_commit(qt_free);
                     }
                     if (ok) ok = issue_dq(a == 0, a + 1 == n_e);
                 }
@@ -289,6 +293,32 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             const float nlse2 = valid ? -p.lse[row_idx] * 1.4426950408889634f : -INFINITY;
             const float Dt = valid ? p.D[row_idx] : 0.f;
             const float nDs = -Dt * p.scale;
+            // ---- this row of Q (group 0) or dO (group 1) from shared memory into tensor memory, where the S and dP
+            //      products read it as their A operand ----
+            if (!wait_barrier(qdo_full, it & 1u, abort_flag, p.status, 16)) { ok = false; break; }
+            if (!wait_barrier(qt_free, (it & 1u) ^ 1u, abort_flag, p.status, 17)) { ok = false; break; }
+            tc_fence_after_sync();
+            {
+                const uint32_t src = base + (grp == 0 ? DQ_SMEM_Q : DQ_SMEM_DO) + r * 128;
+                const uint32_t dst = tmem_base + lane_addr + (grp == 0 ? DQ_TMEM_Q : DQ_TMEM_DO);
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(w[4 * j]), "=r"(w[4 * j + 1]), "=r"(w[4 * j + 2]), "=r"(w[4 * j + 3])
+                                     : "r"(src + hf * Q_HALF + (((j ^ (r & 7)) & 7) << 4)));
+                    hca::tmem_st32(dst + 32 * hf, w);
+                }
+                hca::tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(qt_ready);
+                    mbar_arrive(qdo_empty);     // the shared-memory copies may be refilled for the next item
+                }
+            }
             for (int e = 0; e < n + 2 * m; ++e, ++g) {
                 if ((g & 1u) != static_cast<uint32_t>(grp)) continue;
                 const int s = grp;
