@@ -5,9 +5,10 @@
 //   S = Q K_t^T            tcgen05.mma, 128 x 64 x 128, fp32 in TMEM (two S buffers)
 //   softmax warps          read S (one query row per thread), hide the columns past t - m (the causal
 //                          part and the m substituted entries), update the row's running reference
-//                          and sum, write P = 2^(x - ref) as bf16 into shared memory in the swizzled
-//                          layout the tensor core reads
-//   O += P V_t             tcgen05.mma with V_t as an MN-major operand, fp32 in TMEM
+//                          and sum, write P = 2^(x - ref) as bf16 pairs back into tensor memory, over
+//                          the scores they were made from
+//   O += P V_t             tcgen05.mma with P read from tensor memory and V_t as an MN-major operand
+//                          from shared memory, fp32 in TMEM
 // The substituted entries (t, t - i), i < m, ride the same pipeline as extra half-height tiles:
 //   before the key tiles   S_ih = Q K_d[i]^T for the two 64-key halves h of the K_d[i] tile fetched
 //                          i rows early, so that the wanted scores <Q[t], K_d[i][t - i]> sit on the
@@ -19,7 +20,7 @@
 // by more than 2^8 (the O accumulator in TMEM is then rescaled in place by the softmax warps), so P
 // stays within bf16 range and most tiles skip the rescale.
 //
-// Two CTAs share an SM (112 KB of shared memory and 256 TMEM columns each): while one CTA's softmax
+// Two CTAs share an SM (96 KB of shared memory and 256 TMEM columns each): while one CTA's softmax
 // warps wait for the tensor core, TMEM or a barrier, the other's keep the exp2 unit busy.
 // Warps: 0 = TMA producer (Q once per item, K and V tiles through two-stage rings),
 //        1 = MMA issuer and TMEM owner, 2-5 = softmax + epilogue (TMEM lane quadrant = warp % 4).
@@ -41,15 +42,13 @@ constexpr int Q_BYTES = QT * HD * 2;                 // two halves (64 columns o
 constexpr int Q_HALF = Q_BYTES / 2;
 constexpr int KV_BYTES = KT * HD * 2;                // two halves of 64 rows x 128 B
 constexpr int KV_HALF = KV_BYTES / 2;
-constexpr int P_BYTES = QT * KT * 2;                 // 128 rows x 128 B
 constexpr int SMEM_Q = 0;
 constexpr int SMEM_K = SMEM_Q + Q_BYTES;             // 2 stages
 constexpr int SMEM_V = SMEM_K + 2 * KV_BYTES;        // 2 stages
-constexpr int SMEM_P = SMEM_V + 2 * KV_BYTES;        // 1 buffer
-constexpr int SMEM_BAR = SMEM_P + P_BYTES;
-constexpr int NUM_BARS = 17;
-constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 114944: two CTAs fit the SM's 228 KB
-constexpr int TMEM_COLS = 256;     // S0 at 0, S1 at 64, O at 128
+constexpr int SMEM_BAR = SMEM_V + 2 * KV_BYTES;
+constexpr int NUM_BARS = 18;
+constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 98560: two CTAs fit the SM's 228 KB
+constexpr int TMEM_COLS = 256;     // S0 at 0, S1 at 64 (P as bf16 pairs overwrites the first 32 columns of its S), O at 128
 constexpr float RESCALE_LOG2 = 8.f;
 
 struct Params {
@@ -119,8 +118,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
     auto s_full = [&](int b) { return bar0 + 8u * (10 + b); };
     auto s_empty = [&](int b) { return bar0 + 8u * (12 + b); };
     const uint32_t p_full = bar0 + 8u * 14;
-    const uint32_t pv_done = bar0 + 8u * 15;
-    const uint32_t o_free = bar0 + 8u * 16;
+    auto pv_done = [&](int b) { return bar0 + 8u * (15 + b); };     // PV product that read P from S buffer b
+    const uint32_t o_free = bar0 + 8u * 17;
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_raw + SMEM_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
@@ -139,7 +138,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
             mbar_init(s_empty(b), 4);
         }
         mbar_init(p_full, 4);
-        mbar_init(pv_done, 1);
+        mbar_init(pv_done(0), 1);
+        mbar_init(pv_done(1), 1);
         mbar_init(o_free, 4);
         *abort_flag = 0;
         fence_barrier_init();
@@ -256,15 +256,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k) {
-                    // A = P: K-major, 64 keys = one 128-byte row. B = V: 64-column groups KV_HALF apart, 16 keys
-                    // further = 16 rows of 128 bytes.
-                    const uint64_t a_desc = make_smem_desc_sw128(base + SMEM_P + k * 32, 0, 1024);
+                    // A = P from tensor memory (8 columns of bf16 pairs per 16 keys, in the S buffer the scores came
+                    // from). B = V: 64-column groups KV_HALF apart, 16 keys further = 16 rows of 128 bytes.
                     const uint64_t b_desc =
                         make_smem_desc_sw128(base + SMEM_V + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
-                    umma_bf16(tmem_o, a_desc, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
+                    umma_bf16_ta(tmem_o, tmem_base + s * KT + 8 * k, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
                 }
                 umma_commit(v_empty(s));
-                umma_commit(pv_done);
+                umma_commit(pv_done(s));
                 ++gv;
                 return true;
             };
@@ -293,8 +292,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
         const uint32_t tmem_o = tmem_base + 2 * KT + lane_addr;
         uint32_t gk = 0, gv = 0;
         bool ok = true;
-        // 16-byte unit `chunk` (0..7) of this thread's 128-byte row of the P buffer, as the tensor core sees it
-        auto p_addr = [&](int chunk) { return base + SMEM_P + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
+        // The weights of value-sequence element gv go, as bf16 pairs, into the first 32 columns of S buffer gv & 1:
+        // for a key tile that is the buffer its scores came from (both sequences advance by the same even count
+        // per item), already copied to registers; the tensor core takes products in issue order, so the next
+        // score product into that buffer runs after the PV product that reads these weights.
+        // PV(x) complete <=> pv_done(x & 1) has finished phase x >> 1.
+        auto pv_wait = [&](uint32_t x, unsigned code) {
+            return wait_barrier(pv_done(x & 1u), (x >> 1) & 1u, abort_flag, p.status, code);
+        };
         for (int item = first_item(0), it = 0; item < p.items && ok; item = first_item(++it)) {
             int qt, b, h;
             decode(item, qt, b, h);
@@ -385,7 +390,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                             mref = cand;
                             l *= f;
                         }
-                        if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
+                        if (!pv_wait(gv - 1, 11)) { ok = false; break; }
                         tc_fence_after_sync();
 #pragma unroll 1
                         for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -421,16 +426,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                     for (int i = 0; i < MAX_DRAFTS; ++i)
                         if (i < m && t - i >= 0) l += ex2(fmaf(sd[i], p.c2, nref));
                 }
-                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }   // P has been read
+                if (gv >= 2 && !pv_wait(gv - 2, 12)) { ok = false; break; }     // the last weights in this buffer have been read
+                {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int k = 0; k < 2; ++k) {
+                    for (int k = 0; k < 2; ++k)
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4)
-                        st_shared_v4(p_addr(4 * k + q4), pack_bf16(v[k][8 * q4], v[k][8 * q4 + 1]),
-                                     pack_bf16(v[k][8 * q4 + 2], v[k][8 * q4 + 3]), pack_bf16(v[k][8 * q4 + 4], v[k][8 * q4 + 5]),
-                                     pack_bf16(v[k][8 * q4 + 6], v[k][8 * q4 + 7]));
+                        for (int c = 0; c < 32; c += 2) pk[16 * k + (c >> 1)] = pack_bf16(v[k][c], v[k][c + 1]);
+                    tmem_st32(tmem_s, pk);
+                    tmem_st_wait();
                 }
-                fence_proxy_async_smem();      // P visible to the tensor core's reads
+                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(p_full);
             }
@@ -447,23 +453,23 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                     if (ii == i) sdi = sd[ii];
                 const bool mine = (r >> 6) == (e & 1) && t - i >= 0;
                 const float pi = mine ? ex2(fmaf(sdi, p.c2, nref_f)) : 0.f;
-                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // column r & 63 sits in word (r & 7) / 2
-                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
+                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // key r & 63 sits in word (r & 63) / 2
+                if (gv >= 2 && !pv_wait(gv - 2, 14)) { ok = false; break; }
+                {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int chunk = 0; chunk < 8; ++chunk) {
-                    const bool here = chunk == ((r & 63) >> 3);
-                    const int w = (r & 7) >> 1;
-                    st_shared_v4(p_addr(chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
-                                 here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
+                    for (int w = 0; w < 32; ++w) pk[w] = (w == ((r & 63) >> 1)) ? bits : 0u;
+                    tmem_st32(tmem_base + (gv & 1u) * KT + lane_addr, pk);
+                    tmem_st_wait();
                 }
-                fence_proxy_async_smem();
+                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(p_full);
             }
             if (!ok) break;
             // ---- epilogue: O / l as bf16, each thread stores its own 256-byte row ----
             {
-                if (!wait_barrier(pv_done, (gv & 1u) ^ 1u, abort_flag, p.status, 13)) break;
+                if (!pv_wait(gv - 1, 13)) break;
                 tc_fence_after_sync();
                 const float inv = 1.f / l;
                 if (valid && p.lse != nullptr)
