@@ -46,7 +46,7 @@ constexpr int SMEM_Q = 0;
 constexpr int SMEM_K = SMEM_Q + Q_BYTES;             // 2 stages
 constexpr int SMEM_V = SMEM_K + 2 * KV_BYTES;        // 2 stages
 constexpr int SMEM_BAR = SMEM_V + 2 * KV_BYTES;
-constexpr int NUM_BARS = 18;
+constexpr int NUM_BARS = 19;
 constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 98560: two CTAs fit the SM's 228 KB
 constexpr int TMEM_COLS = 256;     // S0 at 0, S1 at 64 (P as bf16 pairs overwrites the first 32 columns of its S), O at 128
 constexpr float RESCALE_LOG2 = 8.f;
@@ -117,9 +117,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
     auto v_empty = [&](int b) { return bar0 + 8u * (8 + b); };
     auto s_full = [&](int b) { return bar0 + 8u * (10 + b); };
     auto s_empty = [&](int b) { return bar0 + 8u * (12 + b); };
-    const uint32_t p_full = bar0 + 8u * 14;
-    auto pv_done = [&](int b) { return bar0 + 8u * (15 + b); };     // PV product that read P from S buffer b
-    const uint32_t o_free = bar0 + 8u * 17;
+    // one per S buffer: with a single barrier a warp one element ahead could arrive twice in one phase
+    auto p_full = [&](int b) { return bar0 + 8u * (14 + b); };
+    auto pv_done = [&](int b) { return bar0 + 8u * (16 + b); };     // PV product that read P from S buffer b
+    const uint32_t o_free = bar0 + 8u * 18;
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_raw + SMEM_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
@@ -137,7 +138,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
             mbar_init(s_full(b), 1);
             mbar_init(s_empty(b), 4);
         }
-        mbar_init(p_full, 4);
+        mbar_init(p_full(0), 4);
+        mbar_init(p_full(1), 4);
         mbar_init(pv_done(0), 1);
         mbar_init(pv_done(1), 1);
         mbar_init(o_free, 4);
@@ -250,7 +252,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
             // next element of the value sequence: O (+)= P V
             auto issue_pv = [&](bool first) -> bool {
                 const int s = gv & 1u;
-                if (!wait_barrier(p_full, gv & 1u, abort_flag, p.status, 7)) return false;
+                if (!wait_barrier(p_full(s), (gv >> 1) & 1u, abort_flag, p.status, 7)) return false;
                 if (!wait_barrier(v_full(s), (gv >> 1) & 1u, abort_flag, p.status, 8)) return false;
                 if (first && !wait_barrier(o_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
                 tc_fence_after_sync();
@@ -438,7 +440,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 }
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full);
+                if (lane == 0) mbar_arrive(p_full(gv & 1u));
             }
             if (!ok) break;
             // ---- draft passes of the value sequence: P holds only the weights 2^(sd c2 - ref) of the rows of one
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 }
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(p_full);
+                if (lane == 0) mbar_arrive(p_full(gv & 1u));
             }
             if (!ok) break;
             // ---- epilogue: O / l as bf16, each thread stores its own 256-byte row ----
