@@ -62,18 +62,19 @@ __global__ void hca_bwd_prep_kernel(const __nv_bfloat16* __restrict__ O, const _
 // dQ: a work item is (sequence, query head, tile of 128 query positions). Every element of its sweep - a key
 // tile of 64 keys, or half h of draft pass i fetched i rows early (the substituted entries sit on its
 // diagonal) - takes the same route: K and V stage by TMA; S = Q K^T and dP = dO V^T into TMEM; the row's
-// thread forms dS (full row, or its diagonal element only) as bf16 in shared memory; dQ += dS K with the
-// same K stage read MN-major.
+// thread forms dS (full row, or its diagonal element only) as bf16 pairs in tensor memory, over the scores it
+// came from; dQ += dS K with dS read from tensor memory and the same K stage read MN-major. Q and dO are copied
+// into tensor memory once per item, so the S / dP products read only their B operands from shared memory.
 constexpr int DQ_SMEM_Q = 0;
 constexpr int DQ_SMEM_DO = DQ_SMEM_Q + Q_BYTES;
 constexpr int DQ_STAGES = 4;        // a K/V stage is held until its dQ product is done, long after the next S/dP products need theirs
 constexpr int DQ_SMEM_K = DQ_SMEM_DO + Q_BYTES;
 constexpr int DQ_SMEM_V = DQ_SMEM_K + DQ_STAGES * KV_BYTES;
-constexpr int DQ_SMEM_DS = DQ_SMEM_V + DQ_STAGES * KV_BYTES;   // 2 buffers
-constexpr int DQ_SMEM_BAR = DQ_SMEM_DS + 2 * DS_BYTES;
+constexpr int DQ_SMEM_BAR = DQ_SMEM_V + DQ_STAGES * KV_BYTES;
 constexpr int DQ_NUM_BARS = 2 * DQ_STAGES + 14;
 constexpr int DQ_SMEM_BYTES = DQ_SMEM_BAR + 256 + 1024 /*alignment slack*/;
-constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb, dP at 128 sb + 64; dQ at 256; Q at 384 and dO at 448 as bf16 pairs
+constexpr int DQ_TMEM_COLS = 512;   // buffer sb: S at 128 sb (dS as bf16 pairs later overwrites its first 32 columns), dP at
+                                    // 128 sb + 64; dQ at 256; Q at 384 and dO at 448 as bf16 pairs
 constexpr int DQ_TMEM_Q = 384, DQ_TMEM_DO = 448;
 
 struct DqParams {
@@ -239,9 +240,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k) {
-                    const uint64_t da_ = make_smem_desc_sw128(base + DQ_SMEM_DS + s * DS_BYTES + k * 32, 0, 1024);
+                    // A = dS from tensor memory, in the buffer its S came from (the next S / dP product into that
+                    // buffer is issued after this one and the tensor core keeps issue order)
                     const uint64_t db_ = make_smem_desc_sw128(base + DQ_SMEM_K + ks * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
-                    if (leader) umma_bf16(tmem_base + 256, da_, db_, idesc_q, (!first || k != 0) ? 1u : 0u);
+                    if (leader) umma_bf16_ta(tmem_base + 256, tmem_base + s * 128 + 8 * k, db_, idesc_q, (!first || k != 0) ? 1u : 0u);
                 }
                 if (leader) {
                     umma_commit(kv_empty(ks));
@@ -279,9 +281,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
         uint32_t g = 0, it = 0;
         bool ok = true;
-        auto ds_addr = [&](int s, int chunk) {
-            return base + DQ_SMEM_DS + s * DS_BYTES + r * 128 + (((chunk ^ (r & 7)) & 7) << 4);
-        };
         for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int qt, b, h;
             decode(item, qt, b, h);
@@ -358,11 +357,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                             fmul2(ds[c], ds[c + 1], ex2(x0), ex2(x1), y0, y1);
                         }
                         if (hc == 0 && !wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 12)) { stop = true; break; }
+                        // as bf16 pairs over the S columns already in registers (columns 16 hc .. 16 hc + 15)
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4)
-                            st_shared_v4(ds_addr(s, 4 * hc + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
-                                         pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
-                                         pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
+                        for (int c = 0; c < 32; c += 2) pk[c >> 1] = pack_bf16(ds[c], ds[c + 1]);
+                        hca::tmem_st16(tmem_s + 16 * hc, pk);
                     }
                     if (stop) { ok = false; break; }
                 } else {
@@ -396,15 +395,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                     }
                     const uint32_t bits = pack_bf16(dsv, 0.f) << ((r & 1) * 16);
                     if (!wait_barrier(ds_empty(s), ph ^ 1u, abort_flag, p.status, 14)) { ok = false; break; }
+                    uint32_t pk[32];
 #pragma unroll
-                    for (int chunk = 0; chunk < 8; ++chunk) {
-                        const bool here = holder && chunk == ((r & 63) >> 3);
-                        const int w = (r & 7) >> 1;
-                        st_shared_v4(ds_addr(s, chunk), here && w == 0 ? bits : 0u, here && w == 1 ? bits : 0u,
-                                     here && w == 2 ? bits : 0u, here && w == 3 ? bits : 0u);
-                    }
+                    for (int w = 0; w < 32; ++w) pk[w] = (holder && w == ((r & 63) >> 1)) ? bits : 0u;
+                    hca::tmem_st32(tmem_s, pk);
                 }
-                fence_proxy_async_smem();
+                hca::tmem_st_wait();
+                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ds_full(s));
             }
