@@ -458,22 +458,22 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
 // sweeps the query heads of its group and, per head, the tiles of 64 queries at or after it. Per element:
 //   S^T = K Q^T and dP^T = V dO^T      tcgen05.mma, 128 x 64 x 128, into TMEM (rows = keys, one per thread)
 //   threads                             P^T = 2^(S^T c2 - lse2[t]) on the entries the target's keys really met
-//                                       (t - s >= m), dS^T = P^T (dP^T - D[t]) scale; both as bf16 in shared memory
-//   dV += P^T dO, dK += dS^T Q          the Q / dO stage read MN-major
+//                                       (t - s >= m), dS^T = P^T (dP^T - D[t]) scale; both as bf16 pairs back into
+//                                       tensor memory, over the columns they were made from
+//   dV += P^T dO, dK += dS^T Q          A from tensor memory, the Q / dO stage read MN-major from shared memory
 // The per-query vectors -lse2[t] and -D[t] scale of an element travel with its Q / dO stage: the producer warp's
 // lanes copy them into shared memory next to the TMA loads.
 constexpr int KV_SMEM_K = 0;                               // 128 keys x 128: two halves of 16 KB
 constexpr int KV_SMEM_V = KV_SMEM_K + Q_BYTES;
-constexpr int KV_STAGES = 3;        // a Q/dO stage is held until its dV/dK products are done
+constexpr int KV_STAGES = 4;        // a Q/dO stage is held until its dV/dK products are done
 constexpr int KV_SMEM_Q = KV_SMEM_V + Q_BYTES;             // stages of 64 queries
 constexpr int KV_SMEM_DO = KV_SMEM_Q + KV_STAGES * KV_BYTES;
-constexpr int KV_SMEM_PT = KV_SMEM_DO + KV_STAGES * KV_BYTES;      // P^T, 128 x 64 bf16
-constexpr int KV_SMEM_DST = KV_SMEM_PT + DS_BYTES;         // dS^T
-constexpr int KV_SMEM_VEC = KV_SMEM_DST + DS_BYTES;        // per stage: 64 x -lse2, 64 x -D scale (floats)
+constexpr int KV_SMEM_VEC = KV_SMEM_DO + KV_STAGES * KV_BYTES;     // per stage: 64 x -lse2, 64 x -D scale (floats)
 constexpr int KV_SMEM_BAR = KV_SMEM_VEC + KV_STAGES * 512;
 constexpr int KV_NUM_BARS = 2 * KV_STAGES + 10;
 constexpr int KV_SMEM_BYTES = KV_SMEM_BAR + 256 + 1024 /*alignment slack*/;
-constexpr int KV_TMEM_COLS = 512;   // buffer sb: S^T at 128 sb, dP^T at 128 sb + 64; dV at 256, dK at 384
+constexpr int KV_TMEM_COLS = 512;   // buffer sb: S^T at 128 sb, dP^T at 128 sb + 64 (P^T and dS^T as bf16 pairs later overwrite
+                                    // columns 0..15 and 32..47 of each); dV at 256, dK at 384
 
 struct DkvParams {
     CUtensorMap tmK, tmV;          // [B, T, Hkv * 128], box {64, 128, 1}
@@ -640,15 +640,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                 if (first && !wait_barrier(acc_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
                 tc_fence_after_sync();
 #pragma unroll
-                for (int k = 0; k < KT / 16; ++k)
-                    umma_bf16(tmem_base + 256, make_smem_desc_sw128(base + KV_SMEM_PT + k * 32, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
-                              (!first || k != 0) ? 1u : 0u);
-#pragma unroll
-                for (int k = 0; k < KT / 16; ++k)
-                    umma_bf16(tmem_base + 384, make_smem_desc_sw128(base + KV_SMEM_DST + k * 32, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
-                              (!first || k != 0) ? 1u : 0u);
+                for (int k = 0; k < KT / 16; ++k) {
+                    // A from tensor memory: queries 16 k .. 16 k + 15 of P^T (dS^T) sit as 8 columns of bf16 pairs in
+                    // the part of the S^T (dP^T) buffer their own column group read: 0..15 for k < 2, 32..47 for k >= 2
+                    const uint32_t a_col = (ga & 1u) * 128 + (k < 2 ? 8 * k : 32 + 8 * (k - 2));
+                    umma_bf16_ta(tmem_base + 256, tmem_base + a_col,
+                                 make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
+                                 (!first || k != 0) ? 1u : 0u);
+                    umma_bf16_ta(tmem_base + 384, tmem_base + a_col + 64,
+                                 make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
+                                 (!first || k != 0) ? 1u : 0u);
+                }
                 umma_commit(qd_empty(s));
                 umma_commit(pds_empty);
                 if (last) umma_commit(acc_done);
@@ -680,7 +682,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
         uint32_t gq = 0, it = 0;
         bool ok = true;
-        auto row_addr = [&](int buf_off, int chunk) { return base + buf_off + r * 128 + (((chunk ^ (r & 7)) & 7) << 4); };
         for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int kt, b, g;
             decode(item, kt, b, g);
@@ -732,16 +733,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                     fmul2(ds[c + 2], ds[c + 3], pw[c + 2], pw[c + 3], y0, y1);
                 }
                 if (!wait_barrier(pds_empty, (gq & 1u) ^ 1u, abort_flag, p.status, 12)) { ok = false; break; }
+                {
+                    // bf16 pairs over the first 16 of the 32 columns this group read (S^T, resp. dP^T)
+                    uint32_t pk[16], dk[16];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    st_shared_v4(row_addr(KV_SMEM_PT, 4 * grp + q4), pack_bf16(pw[8 * q4], pw[8 * q4 + 1]),
-                                 pack_bf16(pw[8 * q4 + 2], pw[8 * q4 + 3]), pack_bf16(pw[8 * q4 + 4], pw[8 * q4 + 5]),
-                                 pack_bf16(pw[8 * q4 + 6], pw[8 * q4 + 7]));
-                    st_shared_v4(row_addr(KV_SMEM_DST, 4 * grp + q4), pack_bf16(ds[8 * q4], ds[8 * q4 + 1]),
-                                 pack_bf16(ds[8 * q4 + 2], ds[8 * q4 + 3]), pack_bf16(ds[8 * q4 + 4], ds[8 * q4 + 5]),
-                                 pack_bf16(ds[8 * q4 + 6], ds[8 * q4 + 7]));
+                    for (int c = 0; c < 32; c += 2) {
+                        pk[c >> 1] = pack_bf16(pw[c], pw[c + 1]);
+                        dk[c >> 1] = pack_bf16(ds[c], ds[c + 1]);
+                    }
+                    hca::tmem_st16(tmem_s, pk);
+                    hca::tmem_st16(tmem_s + 64, dk);
+                    hca::tmem_st_wait();
                 }
-                fence_proxy_async_smem();
+                tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pds_full);
             }
