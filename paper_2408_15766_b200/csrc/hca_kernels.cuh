@@ -232,48 +232,61 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
         }
     } else if (warp == 1) {
         // ===================== MMA issuer =====================
-        if (lane == 0) {
+        // The whole warp runs this loop so that addresses and descriptors stay warp-uniform; one elected lane
+        // issues the tensor-core instructions.
+        {
             constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
             constexpr uint32_t idesc_o = make_idesc_bf16(QT, HD, 0, 1);
             const uint32_t tmem_o = tmem_base + 2 * KT;
             uint32_t gk = 0, gv = 0, it = 0;
             bool ok = true;
+            auto wait_all = [&](uint32_t bar, uint32_t parity, unsigned code) {
+                return __all_sync(0xffffffffu, wait_barrier(bar, parity, abort_flag, p.status, code)) != 0;
+            };
             // next element of the score sequence: S = Q K^T into S buffer gk & 1
             auto issue_s = [&]() -> bool {
                 const int s = gk & 1u;
                 const uint32_t ph = (gk >> 1) & 1u;
-                if (!wait_barrier(k_full(s), ph, abort_flag, p.status, 4)) return false;
-                if (!wait_barrier(s_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
+                if (!wait_all(k_full(s), ph, 4)) return false;
+                if (!wait_all(s_empty(s), ph ^ 1u, 5)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint64_t a_desc = make_smem_desc_sw128(base + SMEM_Q + (k >> 2) * Q_HALF + (k & 3) * 32, 0, 1024);
                     const uint64_t b_desc =
                         make_smem_desc_sw128(base + SMEM_K + s * KV_BYTES + (k >> 2) * KV_HALF + (k & 3) * 32, 0, 1024);
-                    umma_bf16(tmem_base + s * KT, a_desc, b_desc, idesc_s, k != 0 ? 1u : 0u);
+                    if (leader) umma_bf16(tmem_base + s * KT, a_desc, b_desc, idesc_s, k != 0 ? 1u : 0u);
                 }
-                umma_commit(k_empty(s));
-                umma_commit(s_full(s));
+                if (leader) {
+                    umma_commit(k_empty(s));
+                    umma_commit(s_full(s));
+                }
+                __syncwarp();
                 ++gk;
                 return true;
             };
             // next element of the value sequence: O (+)= P V
             auto issue_pv = [&](bool first) -> bool {
                 const int s = gv & 1u;
-                if (!wait_barrier(p_full(s), (gv >> 1) & 1u, abort_flag, p.status, 7)) return false;
-                if (!wait_barrier(v_full(s), (gv >> 1) & 1u, abort_flag, p.status, 8)) return false;
-                if (first && !wait_barrier(o_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                if (!wait_all(p_full(s), (gv >> 1) & 1u, 7)) return false;
+                if (!wait_all(v_full(s), (gv >> 1) & 1u, 8)) return false;
+                if (first && !wait_all(o_free, (it & 1u) ^ 1u, 9)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k) {
                     // A = P from tensor memory (8 columns of bf16 pairs per 16 keys, in the S buffer the scores came
                     // from). B = V: 64-column groups KV_HALF apart, 16 keys further = 16 rows of 128 bytes.
                     const uint64_t b_desc =
                         make_smem_desc_sw128(base + SMEM_V + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
-                    umma_bf16_ta(tmem_o, tmem_base + s * KT + 8 * k, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
+                    if (leader) umma_bf16_ta(tmem_o, tmem_base + s * KT + 8 * k, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
                 }
-                umma_commit(v_empty(s));
-                umma_commit(pv_done(s));
+                if (leader) {
+                    umma_commit(v_empty(s));
+                    umma_commit(pv_done(s));
+                }
+                __syncwarp();
                 ++gv;
                 return true;
             };
@@ -281,13 +294,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 int qt, b, h;
                 decode(item, qt, b, h);
                 const int n_s = 2 * m + key_tiles(qt);
-                if (!wait_barrier(q_full, it & 1u, abort_flag, p.status, 6)) break;
+                if (!wait_all(q_full, it & 1u, 6)) break;
                 if (!issue_s()) break;
-                if (n_s == 1) umma_commit(q_empty);
+                if (n_s == 1 && elect_one()) umma_commit(q_empty);
                 for (int a = 0; a < n_s && ok; ++a) {
                     if (a + 1 < n_s) {
                         ok = issue_s();
-                        if (ok && a + 2 == n_s) umma_commit(q_empty);      // Q is free once the item's last S has read it
+                        if (ok && a + 2 == n_s && elect_one()) umma_commit(q_empty);      // Q is free once the item's last S has read it
                     }
                     if (ok && a >= 2 * m) ok = issue_pv(a == 2 * m);
                 }
