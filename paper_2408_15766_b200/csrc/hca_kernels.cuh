@@ -100,23 +100,6 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x for two finite arguments on the FMA and integer pipes instead of the exp2 unit: x = n + f with n the
-// nearest integer (magic-number rounding) and f in [-0.5, 0.5], 2^f by a cubic (relative error 1.0e-4, far
-// below the bf16 rounding the weights get), 2^n by adding n to the exponent field. x is clamped at -126.
-__device__ __forceinline__ void exp2_poly2(float& y0, float& y1, float x0, float x1) {
-    constexpr float MAGIC = 12582912.f;      // 1.5 * 2^23
-    x0 = fmaxf(x0, -126.f);
-    x1 = fmaxf(x1, -126.f);
-    float t0, t1, n0, n1, f0, f1, p0, p1;
-    fadd2(t0, t1, x0, x1, MAGIC, MAGIC);
-    fadd2(n0, n1, t0, t1, -MAGIC, -MAGIC);
-    ffma2(f0, f1, n0, n1, -1.f, -1.f, x0, x1);
-    ffma2(p0, p1, f0, f1, 0.05592203512787819f, 0.05592203512787819f, 0.24264007806777954f, 0.24264007806777954f);
-    ffma2(p0, p1, p0, p1, f0, f1, 0.6931210160255432f, 0.6931210160255432f);
-    ffma2(p0, p1, p0, p1, f0, f1, 0.9999244809150696f, 0.9999244809150696f);
-    y0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-    y1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -449,31 +432,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 2) hca_attention_kernel(const __g
                 // (a row whose columns were all hidden so far has ref = -inf; it gets P = 0, not 2^(-inf + inf))
                 const float nref = mref == -INFINITY ? 0.f : -mref;
                 float ls0 = 0.f, ls1 = 0.f;
-                if (band) {
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            float x0, x1;
-                            ffma2(x0, x1, v[k][c], v[k][c + 1], p.c2, p.c2, nref, nref);
-                            v[k][c] = ex2(x0);
-                            v[k][c + 1] = ex2(x1);
-                            fadd2(ls0, ls1, ls0, ls1, v[k][c], v[k][c + 1]);
-                        }
-                    }
-                } else {
-                    // no hidden columns, every argument finite: the exp2 unit is the scarce resource of this phase
-                    // (16 results per cycle and SM, shared by two CTAs), so half of the columns go through the FMA pipe
+                for (int k = 0; k < 2; ++k) {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        float x0, x1, z0, z1;
-                        ffma2(x0, x1, v[0][c], v[0][c + 1], p.c2, p.c2, nref, nref);
-                        ffma2(z0, z1, v[1][c], v[1][c + 1], p.c2, p.c2, nref, nref);
-                        v[0][c] = ex2(x0);
-                        v[0][c + 1] = ex2(x1);
-                        exp2_poly2(v[1][c], v[1][c + 1], z0, z1);
-                        fadd2(ls0, ls1, ls0, ls1, v[0][c], v[0][c + 1]);
-                        fadd2(ls0, ls1, ls0, ls1, v[1][c], v[1][c + 1]);
+                        float x0, x1;
+                        ffma2(x0, x1, v[k][c], v[k][c + 1], p.c2, p.c2, nref, nref);
+                        v[k][c] = ex2(x0);
+                        v[k][c + 1] = ex2(x1);
+                        fadd2(ls0, ls1, ls0, ls1, v[k][c], v[k][c + 1]);
                     }
                 }
                 l += ls0 + ls1;
