@@ -77,3 +77,32 @@ def test_no_device_is_an_error_not_a_fallback(hass):
     al = ctypes.c_void_p((ctypes.addressof(buf) + 255) & ~255)
     rc = hass.lib.hass_topk_distill_fwd(al, al, al, 4, 64, 64, 2, al, al, al, al, al, al, 1 << 15, None)
     assert rc in (-4, -6)
+
+
+def test_hca_attention_arguments_rejected_before_the_device(hass):
+    buf = ctypes.create_string_buffer(8192)
+    al = ctypes.c_void_p((ctypes.addressof(buf) + 255) & ~255)
+    mis = ctypes.c_void_p(al.value + 2)
+    arr = (ctypes.c_void_p * 9)(*([al.value] * 9))
+    f = hass.lib.hass_hca_attention_fwd
+    sc = ctypes.c_float(0.088)
+
+    def call(Q=al, m=1, H=2, Hkv=1, D=128, scale=sc, O=al, ws=al, wsz=256, kd=arr):
+        return f(Q, al, al, kd, arr, m, 1, 16, H, Hkv, D, scale, O, None, ws, wsz, None)
+
+    assert call(Q=None) == -1                     # null input
+    assert call(Q=mis) == -1                      # misaligned input
+    assert call(m=9) == -1                        # more draft passes than HASS_HCA_MAX_DRAFTS
+    assert call(m=1, kd=None) == -1               # passes announced, no pointers
+    assert call(H=3, Hkv=2) == -1                 # query heads not a multiple of key/value heads
+    assert call(scale=ctypes.c_float(0.0)) == -1
+    assert call(D=64) == -2                       # only head dimension 128
+    assert call(ws=None) == -3 and call(wsz=8) == -3
+    n = ctypes.c_size_t(0)
+    assert hass.lib.hass_hca_attention_workspace_bytes(ctypes.byref(n)) == 0 and n.value == 256
+    # backward: the workspace holds the status block, D and the two [B, H, T, m] arrays
+    assert hass.hca_attention_bwd_workspace_bytes(2, 100, 4, 3) >= 256 + 2 * 4 * 100 * 4 * (1 + 2 * 3)
+    assert hass.lib.hass_hca_attention_bwd_workspace_bytes(2, 100, 4, 9, ctypes.byref(n)) == -1
+    g = hass.lib.hass_hca_attention_bwd
+    assert g(al, al, al, arr, arr, 1, 1, 16, 2, 1, 128, sc, al, None, al, al, al, al, arr, arr, al, 1 << 20, None) == -1
+    assert g(al, al, al, arr, arr, 1, 1, 16, 2, 1, 128, sc, al, al, al, al, al, al, arr, arr, al, 16, None) == -3
