@@ -606,54 +606,64 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        // whole warp in the loop, one elected lane issues (see hca_dq_kernel)
+        {
             constexpr uint32_t idesc_s = make_idesc_bf16(QT, KT, 0, 0);
             constexpr uint32_t idesc_a = make_idesc_bf16(QT, HD, 0, 1);
             uint32_t gs = 0, ga = 0, it = 0;
             bool ok = true;
+            auto wait_all = [&](uint32_t bar, uint32_t parity, unsigned code) {
+                return __all_sync(0xffffffffu, wait_barrier(bar, parity, abort_flag, p.status, code)) != 0;
+            };
             auto issue_st = [&]() -> bool {
                 const int s = gs & 1u;                  // S^T / dP^T buffer
                 const int qs = gs % KV_STAGES;          // Q / dO stage
                 const uint32_t ph = (gs >> 1) & 1u;
-                if (!wait_barrier(qd_full(qs), (gs / KV_STAGES) & 1u, abort_flag, p.status, 4)) return false;
-                if (!wait_barrier(st_empty(s), ph ^ 1u, abort_flag, p.status, 5)) return false;
+                if (!wait_all(qd_full(qs), (gs / KV_STAGES) & 1u, 4)) return false;
+                if (!wait_all(st_empty(s), ph ^ 1u, 5)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < HD / 16; ++k) {
                     const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
-                    umma_bf16(tmem_base + s * 128, make_smem_desc_sw128(base + KV_SMEM_K + ao, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_Q + qs * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
+                    const uint64_t ak_ = make_smem_desc_sw128(base + KV_SMEM_K + ao, 0, 1024);
+                    const uint64_t bq_ = make_smem_desc_sw128(base + KV_SMEM_Q + qs * KV_BYTES + bo, 0, 1024);
+                    const uint64_t av_ = make_smem_desc_sw128(base + KV_SMEM_V + ao, 0, 1024);
+                    const uint64_t bd_ = make_smem_desc_sw128(base + KV_SMEM_DO + qs * KV_BYTES + bo, 0, 1024);
+                    if (leader) {
+                        umma_bf16(tmem_base + s * 128, ak_, bq_, idesc_s, k != 0 ? 1u : 0u);
+                        umma_bf16(tmem_base + s * 128 + 64, av_, bd_, idesc_s, k != 0 ? 1u : 0u);
+                    }
                 }
-#pragma unroll
-                for (int k = 0; k < HD / 16; ++k) {
-                    const uint32_t ao = (k >> 2) * Q_HALF + (k & 3) * 32, bo = (k >> 2) * KV_HALF + (k & 3) * 32;
-                    umma_bf16(tmem_base + s * 128 + 64, make_smem_desc_sw128(base + KV_SMEM_V + ao, 0, 1024),
-                              make_smem_desc_sw128(base + KV_SMEM_DO + qs * KV_BYTES + bo, 0, 1024), idesc_s, k != 0 ? 1u : 0u);
-                }
-                umma_commit(st_full(s));
+                if (leader) umma_commit(st_full(s));
+                __syncwarp();
                 ++gs;
                 return true;
             };
             auto issue_acc = [&](bool first, bool last) -> bool {
                 const int s = ga % KV_STAGES;           // Q / dO stage
-                if (!wait_barrier(pds_full, ga & 1u, abort_flag, p.status, 7)) return false;
-                if (first && !wait_barrier(acc_free, (it & 1u) ^ 1u, abort_flag, p.status, 9)) return false;
+                if (!wait_all(pds_full, ga & 1u, 7)) return false;
+                if (first && !wait_all(acc_free, (it & 1u) ^ 1u, 9)) return false;
                 tc_fence_after_sync();
+                const bool leader = elect_one();
 #pragma unroll
                 for (int k = 0; k < KT / 16; ++k) {
                     // A from tensor memory: queries 16 k .. 16 k + 15 of P^T (dS^T) sit as 8 columns of bf16 pairs in
                     // the part of the S^T (dP^T) buffer their own column group read: 0..15 for k < 2, 32..47 for k >= 2
                     const uint32_t a_col = (ga & 1u) * 128 + (k < 2 ? 8 * k : 32 + 8 * (k - 2));
-                    umma_bf16_ta(tmem_base + 256, tmem_base + a_col,
-                                 make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
-                                 (!first || k != 0) ? 1u : 0u);
-                    umma_bf16_ta(tmem_base + 384, tmem_base + a_col + 64,
-                                 make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024), idesc_a,
-                                 (!first || k != 0) ? 1u : 0u);
+                    const uint64_t bd_ = make_smem_desc_sw128(base + KV_SMEM_DO + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
+                    const uint64_t bq_ = make_smem_desc_sw128(base + KV_SMEM_Q + s * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
+                    if (leader) {
+                        umma_bf16_ta(tmem_base + 256, tmem_base + a_col, bd_, idesc_a, (!first || k != 0) ? 1u : 0u);
+                        umma_bf16_ta(tmem_base + 384, tmem_base + a_col + 64, bq_, idesc_a, (!first || k != 0) ? 1u : 0u);
+                    }
                 }
-                umma_commit(qd_empty(s));
-                umma_commit(pds_empty);
-                if (last) umma_commit(acc_done);
+                if (leader) {
+                    umma_commit(qd_empty(s));
+                    umma_commit(pds_empty);
+                    if (last) umma_commit(acc_done);
+                }
+                __syncwarp();
                 ++ga;
                 return true;
             };
@@ -661,13 +671,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
                 int kt, b, g;
                 decode(item, kt, b, g);
                 const int n_e = rep * q_count(kt);
-                if (!wait_barrier(kv_full, it & 1u, abort_flag, p.status, 6)) break;
+                if (!wait_all(kv_full, it & 1u, 6)) break;
                 if (!issue_st()) break;
-                if (n_e == 1) umma_commit(kv_empty);
+                if (n_e == 1 && elect_one()) umma_commit(kv_empty);
                 for (int a = 0; a < n_e && ok; ++a) {
                     if (a + 1 < n_e) {
                         ok = issue_st();
-                        if (ok && a + 2 == n_e) umma_commit(kv_empty);     // K and V are free once the last S^T / dP^T has read them
+                        if (ok && a + 2 == n_e && elect_one()) umma_commit(kv_empty);     // K and V are free once the last S^T / dP^T has read them
                     }
                     if (ok) ok = issue_acc(a == 0, a + 1 == n_e);
                 }
