@@ -281,6 +281,36 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
         uint32_t g = 0, it = 0;
         bool ok = true;
+        // This row of Q (group 0) or dO (group 1) of this CTA's item number `n_it`, from shared memory into tensor
+        // memory, where the S and dP products read it as their A operand. Done for the first item up front and
+        // for every later item as soon as the group has finished the previous item's elements, before its
+        // epilogue, so that the tensor core can start on the next item meanwhile.
+        auto copy_item = [&](uint32_t n_it) -> bool {
+            if (!wait_barrier(qdo_full, n_it & 1u, abort_flag, p.status, 16)) return false;
+            if (!wait_barrier(qt_free, (n_it & 1u) ^ 1u, abort_flag, p.status, 17)) return false;
+            tc_fence_after_sync();
+            const uint32_t src = base + (grp == 0 ? DQ_SMEM_Q : DQ_SMEM_DO) + r * 128;
+            const uint32_t dst = tmem_base + lane_addr + (grp == 0 ? DQ_TMEM_Q : DQ_TMEM_DO);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t w[32];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(w[4 * j]), "=r"(w[4 * j + 1]), "=r"(w[4 * j + 2]), "=r"(w[4 * j + 3])
+                                 : "r"(src + hf * Q_HALF + (((j ^ (r & 7)) & 7) << 4)));
+                hca::tmem_st32(dst + 32 * hf, w);
+            }
+            hca::tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(qt_ready);
+                mbar_arrive(qdo_empty);     // the shared-memory copies may be refilled for the item after
+            }
+            return true;
+        };
+        if (round_item(0) < p.items) ok = copy_item(0);
         for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
             int qt, b, h;
             decode(item, qt, b, h);
@@ -292,32 +322,6 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
             const float nlse2 = valid ? -p.lse[row_idx] * 1.4426950408889634f : -INFINITY;
             const float Dt = valid ? p.D[row_idx] : 0.f;
             const float nDs = -Dt * p.scale;
-            // ---- this row of Q (group 0) or dO (group 1) from shared memory into tensor memory, where the S and dP
-            //      products read it as their A operand ----
-            if (!wait_barrier(qdo_full, it & 1u, abort_flag, p.status, 16)) { ok = false; break; }
-            if (!wait_barrier(qt_free, (it & 1u) ^ 1u, abort_flag, p.status, 17)) { ok = false; break; }
-            tc_fence_after_sync();
-            {
-                const uint32_t src = base + (grp == 0 ? DQ_SMEM_Q : DQ_SMEM_DO) + r * 128;
-                const uint32_t dst = tmem_base + lane_addr + (grp == 0 ? DQ_TMEM_Q : DQ_TMEM_DO);
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t w[32];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(w[4 * j]), "=r"(w[4 * j + 1]), "=r"(w[4 * j + 2]), "=r"(w[4 * j + 3])
-                                     : "r"(src + hf * Q_HALF + (((j ^ (r & 7)) & 7) << 4)));
-                    hca::tmem_st32(dst + 32 * hf, w);
-                }
-                hca::tmem_st_wait();
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(qt_ready);
-                    mbar_arrive(qdo_empty);     // the shared-memory copies may be refilled for the next item
-                }
-            }
             for (int e = 0; e < n + 2 * m; ++e, ++g) {
                 if ((g & 1u) != static_cast<uint32_t>(grp)) continue;
                 const int s = grp;
@@ -406,6 +410,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dq_kernel(const __grid_con
                 if (lane == 0) mbar_arrive(ds_full(s));
             }
             if (!ok) break;
+            if (round_item(it + 1) < p.items && !copy_item(it + 1)) { ok = false; break; }
             // ---- epilogue: this group's half of the dQ row as bf16 ----
             if (!wait_barrier(dq_done, it & 1u, abort_flag, p.status, 13)) break;
             tc_fence_after_sync();
