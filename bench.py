@@ -34,8 +34,9 @@ METRIC = "tokens/sec fused top-K distill fwd+bwd"
 UNIT = "tokens/s"
 # dram__bytes_read + dram__bytes_write of the dominant kernel (the logits sweep) per launch, from the ncu
 # capture summarised in profiles/gemm_kernel_l2-7b_ncu_full.md (l2-7b shape, mean of the two chunk launches),
-# scaled to the bench shape by the vocabulary ratio; valid for the library version it was taken with.
-TRAFFIC_CAPTURE = {"version": 10100, "workload": "l3-8b", "bytes_per_launch": 0.965e9 * 128256 / 32000}
+# scaled to the bench shape by the vocabulary ratio; valid for the library version it was taken with (10200 added
+# the HCA attention entries and left the kernels of this path as captured).
+TRAFFIC_CAPTURE = {"version": 10200, "workload": "l3-8b", "bytes_per_launch": 0.965e9 * 128256 / 32000}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
