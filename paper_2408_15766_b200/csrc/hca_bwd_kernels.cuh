@@ -8,8 +8,9 @@
 // hca_dq_kernel also leaves P and dS of the substituted entries (t, t-i) in the workspace for the last one.
 //
 // Both tensor-core kernels follow the forward kernel's organisation (warp 0 TMA producer, warp 1 MMA issuer
-// and TMEM owner, then row-owning warps - here two groups of four, each taking half of a tile's columns,
-// which needs no exchange because the backward has no running row statistics) and its bounded waits.
+// and TMEM owner, then row-owning warps - here two groups of four, taking alternate elements (dQ) or half of
+// a tile's columns (dK/dV), which needs no exchange because the backward has no running row statistics) and
+// its bounded waits. The A operands of the products come from tensor memory wherever they fit.
 #pragma once
 #include "hca_kernels.cuh"
 
