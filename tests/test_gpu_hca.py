@@ -187,3 +187,19 @@ def test_backward_steep_scores():
 def test_backward_full_size_sampled_groups():
     wl = hi.HCA_WORKLOADS["hca-l3-8b"]
     print(_run_bwd(hi.make_hca_inputs(wl), pairs=[(0, 0), (wl.B - 1, wl.Hkv - 1)]))
+
+
+def test_draft_passes_equal_to_target_change_nothing_on_the_gpu():
+    # property that holds at any size: with K_d = K_t and V_d = V_t the substituted entries carry the same keys and
+    # values as the ones they replace, so the output must agree with plain causal attention (m = 0) up to the
+    # rounding of the two routes (tensor-core tile vs. diagonal tile)
+    hass = _hass()
+    dev = torch.device("cuda:0")
+    inp = hi.make_hca_inputs(hi.HcaWorkload("same", B=2, T=1000, H=8, Hkv=2, m=0, seed=5))
+    Q, K, V = inp.Q.to(dev), inp.K_t.to(dev), inp.V_t.to(dev)
+    base = hass.hca_attention_fwd(Q, K, V)
+    sub = hass.hca_attention_fwd(Q, K, V, [K] * 3, [V] * 3)
+    hass.check(sub["workspace"])
+    scale = base["O"].float().abs().max().item()
+    assert (base["O"].float() - sub["O"].float()).abs().max().item() <= 1e-2 * scale
+    assert (base["lse"] - sub["lse"]).abs().max().item() <= 1e-4
