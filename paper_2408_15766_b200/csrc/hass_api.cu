@@ -1374,7 +1374,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
         }
         KernelTimer kt(KIND_HCA_BWD_ROWS, st);
         const long long warps = static_cast<long long>(B) * T * Hkv;
-        hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, st>>>(
+        hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 16 + 255) / 256), 256, 0, st>>>(
             static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd, dg, m, iB, iT, iH, iHkv);
         g_launches.fetch_add(1);
     }

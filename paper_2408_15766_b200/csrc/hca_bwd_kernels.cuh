@@ -820,9 +820,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_dkv_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------------
 // Gradients of the draft passes' keys and values: position s of pass i meets exactly one query per head,
 // t = s + i, so dK_d[i][s] = sum over the group's query heads of dS[t, s] Q[t] and likewise for the values.
-// One warp per (sequence, query position t, key/value head): it reads the group's Q[t] and dO[t] rows once
-// and writes row t - i of every pass i; the last i rows of pass i have no query and are zeroed by the warp
-// of the same index. Lane = 4 of the 128 columns.
+// Half a warp per (sequence, query position t, key/value head): it reads the group's Q[t] and dO[t] rows once
+// and writes row t - i of every pass i; the last i rows of pass i have no query and are zeroed by the half-warp
+// of the same index. A thread covers 8 of the 128 columns (16-byte accesses).
 struct DraftGradParams {
     __nv_bfloat16* dKd[MAX_DRAFTS];
     __nv_bfloat16* dVd[MAX_DRAFTS];
@@ -831,8 +831,8 @@ struct DraftGradParams {
 __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ dO,
                                       const float* __restrict__ Pd, const float* __restrict__ dSd,
                                       const __grid_constant__ DraftGradParams out, int m, int B, int T, int H, int Hkv) {
-    const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;   // (b, t, g)
-    const int lane = threadIdx.x & 31;
+    const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;   // (b, t, g)
+    const int sub = threadIdx.x & 15;       // 8 of the 128 columns (16 bytes) per thread
     if (w >= static_cast<long long>(B) * T * Hkv) return;
     const int g = static_cast<int>(w % Hkv);
     const long long bt = w / Hkv;
@@ -841,24 +841,31 @@ __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const
     const int rep = H / Hkv;
     auto lo = [](uint32_t x) { return __uint_as_float(x << 16); };
     auto hi = [](uint32_t x) { return __uint_as_float(x & 0xffff0000u); };
-    // two passes at a time (the group's rows are re-read from cache for further pairs): few registers, many warps in flight
+    auto widen = [&](const uint4& v, float (&f)[8]) {
+        f[0] = lo(v.x); f[1] = hi(v.x); f[2] = lo(v.y); f[3] = hi(v.y);
+        f[4] = lo(v.z); f[5] = hi(v.z); f[6] = lo(v.w); f[7] = hi(v.w);
+    };
+    auto narrow = [&](const float (&f)[8]) {
+        return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+    };
+    // two passes at a time (the group's rows are re-read from cache for further pairs): few registers, many rows in flight
     for (int i0 = 0; i0 < m; i0 += 2) {
-        float kacc[2][4], vacc[2][4];
+        float kacc[2][8], vacc[2][8];
 #pragma unroll
         for (int j = 0; j < 2; ++j)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) kacc[j][c] = vacc[j][c] = 0.f;
-        // four heads of the group at a time, all their loads issued before any is used
-        for (int h0 = 0; h0 < rep; h0 += 4) {
-            uint2 q[4], d[4];
-            float pw[4][2], ds[4][2];
+            for (int c = 0; c < 8; ++c) kacc[j][c] = vacc[j][c] = 0.f;
+        // two heads of the group at a time, all their loads issued before any is used
+        for (int h0 = 0; h0 < rep; h0 += 2) {
+            uint4 q[2], d[2];
+            float pw[2][2], ds[2][2];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 2; ++u) {
                 const bool on = h0 + u < rep;
                 const int h = g * rep + (on ? h0 + u : 0);
                 const size_t row = ((static_cast<size_t>(b) * T + t) * H + h) * HD;
-                q[u] = __ldg(reinterpret_cast<const uint2*>(Q + row) + lane);
-                d[u] = __ldg(reinterpret_cast<const uint2*>(dO + row) + lane);
+                q[u] = __ldg(reinterpret_cast<const uint4*>(Q + row) + sub);
+                d[u] = __ldg(reinterpret_cast<const uint4*>(dO + row) + sub);
                 const size_t ri = ((static_cast<size_t>(b) * H + h) * T + t) * m;
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
@@ -868,13 +875,14 @@ __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float qf[4] = {lo(q[u].x), hi(q[u].x), lo(q[u].y), hi(q[u].y)};
-                const float df[4] = {lo(d[u].x), hi(d[u].x), lo(d[u].y), hi(d[u].y)};
+            for (int u = 0; u < 2; ++u) {
+                float qf[8], df[8];
+                widen(q[u], qf);
+                widen(d[u], df);
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 8; ++c) {
                         kacc[j][c] = fmaf(ds[u][j], qf[c], kacc[j][c]);
                         vacc[j][c] = fmaf(pw[u][j], df[c], vacc[j][c]);
                     }
@@ -887,15 +895,13 @@ __global__ void hca_draft_grad_kernel(const __nv_bfloat16* __restrict__ Q, const
             if (i < m) {
                 if (t - i >= 0) {
                     const size_t orow = ((static_cast<size_t>(b) * T + (t - i)) * Hkv + g) * HD;
-                    *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) =
-                        make_uint2(pack_bf16(kacc[j][0], kacc[j][1]), pack_bf16(kacc[j][2], kacc[j][3]));
-                    *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) =
-                        make_uint2(pack_bf16(vacc[j][0], vacc[j][1]), pack_bf16(vacc[j][2], vacc[j][3]));
+                    *(reinterpret_cast<uint4*>(out.dKd[i] + orow) + sub) = narrow(kacc[j]);
+                    *(reinterpret_cast<uint4*>(out.dVd[i] + orow) + sub) = narrow(vacc[j]);
                 }
                 if (t + i >= T) {       // position t of pass i would meet query t + i, past the sequence
                     const size_t orow = ((static_cast<size_t>(b) * T + t) * Hkv + g) * HD;
-                    *(reinterpret_cast<uint2*>(out.dKd[i] + orow) + lane) = make_uint2(0u, 0u);
-                    *(reinterpret_cast<uint2*>(out.dVd[i] + orow) + lane) = make_uint2(0u, 0u);
+                    *(reinterpret_cast<uint4*>(out.dKd[i] + orow) + sub) = make_uint4(0u, 0u, 0u, 0u);
+                    *(reinterpret_cast<uint4*>(out.dVd[i] + orow) + sub) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
         }
