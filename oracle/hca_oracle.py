@@ -60,6 +60,8 @@ def hca_attention(Q, K_t, V_t, K_d: Sequence = (), V_d: Sequence = (), scale: Op
             k_t, v_t = K_t[b, :, g, :], V_t[b, :, g, :]
             w = q @ k_t.T * scale + mask
             for i in range(len(K_d)):
+                if i >= T:
+                    continue        # sub-diagonal i of a T x T matrix is empty
                 ind_q, ind_k = idx[i:], idx[:T - i]
                 w_d = q @ K_d[i][b, :, g, :].T * scale
                 w[ind_q, ind_k] = w_d[ind_q, ind_k]
@@ -69,6 +71,8 @@ def hca_attention(Q, K_t, V_t, K_d: Sequence = (), V_d: Sequence = (), scale: Op
             wn = e / den
             out = wn @ v_t
             for i in range(len(V_d)):
+                if i >= T:
+                    continue        # sub-diagonal i of a T x T matrix is empty
                 ind_q, ind_k = idx[i:], idx[:T - i]
                 v_d = V_d[i][b, :, g, :]
                 out[ind_q] += wn[ind_q, ind_k][:, None] * (v_d[ind_k] - v_t[ind_k])
@@ -104,6 +108,8 @@ def hca_attention_grad(Q, K_t, V_t, K_d: Sequence, V_d: Sequence, dO, scale: Opt
             k_t, v_t = K_t[b, :, g, :], V_t[b, :, g, :]
             w = q @ k_t.T * scale + mask
             for i in range(m):
+                if i >= T:
+                    continue        # sub-diagonal i of a T x T matrix is empty
                 ind_q, ind_k = idx[i:], idx[:T - i]
                 w[ind_q, ind_k] = (q @ K_d[i][b, :, g, :].T * scale)[ind_q, ind_k]
             wn = np.exp(w - w.max(axis=1, keepdims=True))
@@ -111,6 +117,8 @@ def hca_attention_grad(Q, K_t, V_t, K_d: Sequence, V_d: Sequence, dO, scale: Opt
             # d(loss)/d(wn): against the value each pair actually uses
             dwn = do @ v_t.T
             for i in range(m):
+                if i >= T:
+                    continue        # sub-diagonal i of a T x T matrix is empty
                 ind_q, ind_k = idx[i:], idx[:T - i]
                 dwn[ind_q, ind_k] = np.einsum("td,td->t", do[ind_q], V_d[i][b, ind_k, g, :])
             ds = wn * (dwn - (wn * dwn).sum(axis=1, keepdims=True)) * scale
@@ -118,6 +126,8 @@ def hca_attention_grad(Q, K_t, V_t, K_d: Sequence, V_d: Sequence, dO, scale: Opt
             # and the sub-diagonals that meet draft keys/values
             wn_t, ds_t = wn.copy(), ds.copy()
             for i in range(m):
+                if i >= T:
+                    continue        # sub-diagonal i of a T x T matrix is empty
                 ind_q, ind_k = idx[i:], idx[:T - i]
                 wd, dsd = wn[ind_q, ind_k], ds[ind_q, ind_k]
                 wn_t[ind_q, ind_k] = 0.0

@@ -151,3 +151,14 @@ def test_first_step_gradients_against_autograd():
     o.backward(torch.from_numpy(dO).permute(0, 2, 1, 3))
     for mine, ref in ((dQ, q.grad), (dK, k.grad), (dV, v.grad)):
         np.testing.assert_allclose(mine, ref.permute(0, 2, 1, 3).numpy(), rtol=1e-11, atol=1e-12)
+
+
+def test_passes_beyond_the_sequence_length_are_inert():
+    # a sequence of T positions has sub-diagonals 0 .. T-1 only: further draft passes meet no (query, key) pair
+    Q, K_t, V_t, K_d, V_d = _case(B=1, T=3, H=1, Hkv=1, D=4, m=5, seed=17)
+    O5, l5 = ho.hca_attention(Q, K_t, V_t, K_d, V_d)
+    O3, l3 = ho.hca_attention(Q, K_t, V_t, K_d[:3], V_d[:3])
+    np.testing.assert_array_equal(O5, O3)
+    np.testing.assert_array_equal(l5, l3)
+    g = ho.hca_attention_grad(Q, K_t, V_t, K_d, V_d, np.ones_like(Q))
+    assert all(np.all(x == 0) for x in g[3][3:]) and all(np.all(x == 0) for x in g[4][3:])
