@@ -105,9 +105,46 @@ class ClockSampler:
 
 
 # ---- multi-rank plumbing ----------------------------------------------------------------------------
+def spawn_ranks(n: int, cmd=None, timeout=None) -> int:
+    """`bench.py --gpus N` started without a launcher: runs N copies of `cmd` (default: this script with its
+    own arguments), one process per GPU, with RANK / LOCAL_RANK / WORLD_SIZE / MASTER_ADDR / MASTER_PORT set the
+    way torch.distributed.run sets them. Rank 0's JSON line goes to this process's stdout. Returns 0 only if
+    every rank exits 0; when one fails, the others (these exact processes) are terminated."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, os.path.abspath(__file__)] + sys.argv[1:] if cmd is None else list(cmd)
+    env = dict(os.environ, WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    procs = [subprocess.Popen(cmd, env=dict(env, RANK=str(r), LOCAL_RANK=str(r))) for r in range(n)]
+    deadline = None if timeout is None else time.time() + timeout
+    rc = 0
+    while any(p.poll() is None for p in procs):
+        failed = [p for p in procs if p.poll() not in (None, 0)]
+        if failed or (deadline is not None and time.time() > deadline):
+            rc = failed[0].returncode if failed else 124
+            for p in procs:
+                if p.poll() is None:
+                    p.terminate()
+            break
+        time.sleep(0.05)
+    for p in procs:
+        try:
+            p.wait(timeout=10)
+        except subprocess.TimeoutExpired:
+            p.kill()
+        if rc == 0 and p.returncode != 0:
+            rc = p.returncode
+    return rc
+
+
 def dist_setup(n_gpus: int):
-    """Returns (rank, world, local_rank). One process per GPU when launched by torch.distributed.run."""
+    """Returns (rank, world, local_rank). One process per GPU, started by torch.distributed.run or by
+    spawn_ranks; `--gpus` must agree with the launcher's world size."""
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != n_gpus:
+        sys.exit(f"bench.py: --gpus {n_gpus} but WORLD_SIZE={world}; start with --gpus {world}, or unset WORLD_SIZE "
+                 f"and let bench.py spawn its own ranks")
     if world == 1:
         return 0, 1, 0
     import torch.distributed as dist
@@ -387,6 +424,13 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus < 1:
+        sys.exit("bench.py: --gpus must be at least 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: one process per GPU, started here
+        if args.impl == "ours" and torch.cuda.device_count() < args.gpus:
+            sys.exit(f"bench.py: --gpus {args.gpus} but {torch.cuda.device_count()} CUDA device(s) are visible")
+        sys.exit(spawn_ranks(args.gpus))
 
     if args.workload in hi.HCA_WORKLOADS:
         main_hca(args)

@@ -74,7 +74,8 @@ int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K
 /*
  * Forward: Eq. 1 of the paper, L_i = - sum_{x in Omega_hat_i} q_i(x) log p_i(x), per row.
  *
- * Steps (Section 3.1 and the training listing of Section 3.2: lm_head(hidden_states_target),
+ * Steps (Section 3.1 and the training listing of the appendix,
+ * "Implementation of Harmonized Context Alignment": lm_head(hidden_states_target),
  * lm_head(predict), logit loss): target logits z_t = H_t W^T and draft logits z_d = H_d W^T over
  * the whole vocabulary (computed tile by tile, never stored), their log-sum-exp, the K largest
  * target logits per row (= K most probable tokens under q), and the loss.
@@ -303,6 +304,20 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
 int hass_check(void* workspace, void* cuda_stream);
 
 /*
+ * Self-test of the library's failure detection (no counterpart in the paper). Every device-side wait of
+ * the kernels above is bounded: a wait that runs out records a code in the workspace's status word,
+ * raises a flag that ends the other waits of its CTA, and the kernel returns; hass_check then reports
+ * HASS_ERR_TIMEOUT. This call exercises exactly that path without making any real kernel wait: it enqueues
+ * one small kernel (one CTA of 128 threads, no copies, no tensor memory) whose threads wait on a barrier
+ * that nothing completes, the first thread for limit_ns nanoseconds (1000 .. 100000000), the others until
+ * the first one's give-up flag reaches them. Afterwards hass_check(workspace) must return
+ * HASS_ERR_TIMEOUT once and HASS_OK from then on.
+ *   workspace  at least 256 bytes, 256-byte aligned; word 0 is the status word; the kernel also writes
+ *              word 16 = number of threads whose wait gave up (128) and word 17 = nanoseconds waited.
+ */
+int hass_selftest_wait_expiry(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* cuda_stream);
+
+/*
  * Number of kernels of this library launched by the calling process so far (all entry points).
  * Lets a benchmark report how many of the library's own kernels ran in a timed region.
  */
@@ -318,9 +333,14 @@ int64_t hass_kernel_launch_count(void);
  * sweep live in an array built into the library's device image instead of a caller workspace.
  *
  *   - The array is HASS_STATIC_SCRATCH_MAX_BYTES (32 MiB) and every GPU that loads the library
- *     holds it until the process exits. A problem whose forward scratch does not fit (it grows
- *     with K and, slowly, with N; e.g. N = 8192, V = 128256 fits for K <= 16; larger K use much larger candidate buffers) is refused
- *     with HASS_ERR_UNSUPPORTED; use hass_topk_distill_fwd with a workspace then.
+ *     holds it until the process exits. The forward scratch of a problem is about
+ *     slots * 128 * (8 * cap(K) + 16) bytes: slots = the partial-result slots of its tile schedule
+ *     (the number of SMs for up to 128 rows, about three times that for thousands of rows) and
+ *     cap(K) = 16 for K <= 16, else K + max(K, 96) rounded up to a multiple of 32.
+ *     hass_topk_distill_fwd_static_scratch_bytes returns the exact figure. On a 148-SM device
+ *     N = 8192, V = 128256 needs 7.7 MiB for K <= 16 and 55.9 MiB for K = 17, so it is accepted up
+ *     to K = 16; N = 128 fits up to K = 96. A problem that does not fit is refused with
+ *     HASS_ERR_UNSUPPORTED before anything is launched; use hass_topk_distill_fwd with a workspace.
  *   - The call allocates and frees nothing, in this library or through any other.
  *   - The first call on each device looks up the array's device address (a CUDA runtime query,
  *     with that device current). Make that first call outside any stream capture.
@@ -333,6 +353,7 @@ int64_t hass_kernel_launch_count(void);
  *     it replaces hass_check, which needs a workspace pointer.
  */
 #define HASS_STATIC_SCRATCH_MAX_BYTES (32u << 20)
+int hass_topk_distill_fwd_static_scratch_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes);
 int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                                  int64_t V, int32_t K, float* loss, int32_t* topk_idx, float* topk_q,
                                  float* lse_t, float* lse_d, unsigned int* device_status,

@@ -60,7 +60,10 @@ def _load():
                                                 c_vp, c_vp, c_vp, c_vp]
         lib.hass_oracle_features_variant.restype = ctypes.c_int
         lib.hass_oracle_features_variant.argtypes = [c_vp, c_vp, c_vp, c_i64, c_i64, c_i64, c_i32, ctypes.c_int, c_dbl,
-                                                     c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
+                                                     c_vp, c_vp, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp]
+        lib.hass_oracle_row_on_set.restype = ctypes.c_int
+        lib.hass_oracle_row_on_set.argtypes = [c_vp, c_vp, c_i64, c_vp, c_i32, c_dbl, ctypes.c_int, c_vp, c_vp, c_vp,
+                                               c_vp, c_vp]
         lib.hass_oracle_logits_at.restype = ctypes.c_int
         lib.hass_oracle_logits_at.argtypes = [c_vp, c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_i64, c_vp]
         _lib = lib
@@ -118,8 +121,27 @@ def variant_from_logits(z_t, z_d, K: int, variant: int, param: float = 0.0, g: f
                 dz_d=dz)
 
 
-def variant_from_features(H_t, H_d, W, K: int, variant: int, param: float = 0.0, rows=None, grad_loss=None) -> dict:
-    """Feature-level loss variants on bf16 bit patterns; outputs indexed by position in ``rows``."""
+def on_set_from_logits(z_t, z_d, tokens, g: float = 1.0, normed: bool = False) -> dict:
+    """Eq. 1 (or, with ``normed``, the Normed Top-K loss) of ONE row of logits on a given set of token ids."""
+    z_t = np.ascontiguousarray(z_t, dtype=np.float64)
+    z_d = np.ascontiguousarray(z_d, dtype=np.float64)
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    V, n = z_t.shape[0], tok.shape[0]
+    loss, lse_t, lse_d = np.zeros(1), np.zeros(1), np.zeros(1)
+    q = np.zeros(n)
+    dz = np.zeros(V)
+    rc = _load().hass_oracle_row_on_set(_ptr(z_t), _ptr(z_d), V, _ptr(tok), n, float(g), int(bool(normed)),
+                                        _ptr(loss), _ptr(q), _ptr(lse_t), _ptr(lse_d), _ptr(dz))
+    if rc != 0:
+        raise ValueError("oracle: bad arguments")
+    return dict(loss=float(loss[0]), q_k=q, lse_t=float(lse_t[0]), lse_d=float(lse_d[0]), dz_d=dz)
+
+
+def variant_from_features(H_t, H_d, W, K: int, variant: int, param: float = 0.0, rows=None, grad_loss=None,
+                          forced_idx=None) -> dict:
+    """Feature-level loss variants on bf16 bit patterns; outputs indexed by position in ``rows``.
+    ``forced_idx`` [len(rows), K] (2K for the bi-directional variant): score each row on these token ids
+    (entries < 0 are padding) instead of on the oracle's own selection."""
     H_t, H_d, W = np.ascontiguousarray(H_t), np.ascontiguousarray(H_d), np.ascontiguousarray(W)
     assert H_t.dtype == H_d.dtype == W.dtype == np.uint16
     N, d = H_t.shape
@@ -133,9 +155,13 @@ def variant_from_features(H_t, H_d, W, K: int, variant: int, param: float = 0.0,
     q_k = np.zeros((n, kk))
     cnt = np.zeros(n, dtype=np.int32)
     dH = np.zeros((n, d))
+    f = None
+    if forced_idx is not None:
+        f = np.ascontiguousarray(forced_idx, dtype=np.int32)
+        assert f.shape == (n, kk)
     rc = _load().hass_oracle_features_variant(_ptr(H_t), _ptr(H_d), _ptr(W), N, d, V, K, int(variant), float(param),
-                                              _ptr(gl), _ptr(rows_a), n, _ptr(loss), _ptr(idx), _ptr(q_k), _ptr(cnt),
-                                              _ptr(lse_t), _ptr(lse_d), _ptr(dH))
+                                              _ptr(gl), _ptr(rows_a), n, _ptr(f), _ptr(loss), _ptr(idx), _ptr(q_k),
+                                              _ptr(cnt), _ptr(lse_t), _ptr(lse_d), _ptr(dH))
     if rc != 0:
         raise ValueError("oracle: bad arguments")
     return dict(loss=loss, idx=idx, q_k=q_k, n=cnt, lse_t=lse_t, lse_d=lse_d, dH_d=dH)

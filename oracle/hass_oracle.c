@@ -12,8 +12,9 @@
  * tokens with the highest target probability):
  *
  *   step 1  z_t[v] = sum_k H_t[i,k] W[v,k],  z_d[v] = sum_k H_d[i,k] W[v,k]
- *           (the shared LM head applied to target and draft features; training
- *            listing in Section 3.2: lm_head(hidden_states_target), lm_head(predict))
+ *           (the shared LM head applied to target and draft features; training listing of the
+ *            appendix "Implementation of Harmonized Context Alignment":
+ *            lm_head(hidden_states_target), lm_head(predict))
  *   step 2  q = softmax(z_t), p = softmax(z_d) over the whole vocabulary (Eq. 1: q and p
  *           are next-token probability distributions; they are NOT renormalised over
  *           Omega_hat - that is the separate "Normed Top-K" variant of Section 4.3)
@@ -306,11 +307,63 @@ int hass_oracle_row_variant(const double* z_t, const double* z_d, int64_t V, int
     return 0;
 }
 
-/* Feature-level loss variants for a set of rows (bf16 bit patterns); outputs as hass_oracle_features plus n. */
+/*
+ * Eq. 1 (normed = 0) or the Normed Top-K loss (normed = 1) of one row on a GIVEN token set: the sum of Eq. 1
+ * runs over `set` (n distinct token ids) instead of over a selection made here. Used to score a row on a set
+ * that a caller found by other means, when two selections are equally valid (a near-tie at the K-th place).
+ *   q_set  [n] out: q at the set's tokens, in the given order.
+ * Returns 0, or -1 on bad arguments (empty set, id out of range, repeated id).
+ */
+int hass_oracle_row_on_set(const double* z_t, const double* z_d, int64_t V, const int32_t* set, int32_t n, double g,
+                           int normed, double* loss, double* q_set, double* lse_t_out, double* lse_d_out,
+                           double* dz_d) {
+    if (V < 1 || n < 1 || n > V) return -1;
+    for (int32_t j = 0; j < n; ++j) {
+        if (set[j] < 0 || set[j] >= V) return -1;
+        for (int32_t i = 0; i < j; ++i)
+            if (set[i] == set[j]) return -1;
+    }
+    const double lse_t = log_sum_exp(z_t, V);
+    const double lse_d = log_sum_exp(z_d, V);
+    if (lse_t_out) *lse_t_out = lse_t;
+    if (lse_d_out) *lse_d_out = lse_d;
+    double S = 0.0;
+    for (int32_t j = 0; j < n; ++j) {
+        q_set[j] = exp(z_t[set[j]] - lse_t);
+        S += q_set[j];
+    }
+    double L = 0.0;
+    if (!normed) {
+        for (int32_t j = 0; j < n; ++j) L -= q_set[j] * (z_d[set[j]] - lse_d);
+        if (dz_d) {
+            for (int64_t v = 0; v < V; ++v) dz_d[v] = g * S * exp(z_d[v] - lse_d);
+            for (int32_t j = 0; j < n; ++j) dz_d[set[j]] -= g * q_set[j];
+        }
+    } else {
+        double m = z_d[set[0]];
+        for (int32_t j = 1; j < n; ++j)
+            if (z_d[set[j]] > m) m = z_d[set[j]];
+        double se = 0.0;
+        for (int32_t j = 0; j < n; ++j) se += exp(z_d[set[j]] - m);
+        const double lse_k = m + log(se);
+        for (int32_t j = 0; j < n; ++j) L -= (q_set[j] / S) * (z_d[set[j]] - lse_k);
+        if (dz_d) {
+            for (int64_t v = 0; v < V; ++v) dz_d[v] = 0.0;
+            for (int32_t j = 0; j < n; ++j) dz_d[set[j]] = g * (exp(z_d[set[j]] - lse_k) - q_set[j] / S);
+        }
+    }
+    *loss = L;
+    return 0;
+}
+
+/* Feature-level loss variants for a set of rows (bf16 bit patterns); outputs as hass_oracle_features plus n.
+ * forced_idx: NULL, or [n_rows, kk] (kk = 2K for variant 3, else K) token sets to score instead of the
+ * oracle's own selection: a row's entries >= 0 are its Omega_hat (hass_oracle_row_on_set); idx repeats them. */
 int hass_oracle_features_variant(const uint16_t* H_t, const uint16_t* H_d, const uint16_t* W, int64_t N, int64_t d,
                                  int64_t V, int32_t K, int variant, double param, const double* grad_loss,
-                                 const int64_t* rows, int64_t n_rows, double* loss, int32_t* idx, double* q_k,
-                                 int32_t* n_out, double* lse_t, double* lse_d, double* dH_d) {
+                                 const int64_t* rows, int64_t n_rows, const int32_t* forced_idx, double* loss,
+                                 int32_t* idx, double* q_k, int32_t* n_out, double* lse_t, double* lse_d,
+                                 double* dH_d) {
     if (N < 1 || d < 1 || V < 1 || K < 1 || K > V || n_rows < 0 || !rows) return -1;
     int status = 0;
 #pragma omp parallel
@@ -337,8 +390,23 @@ int hass_oracle_features_variant(const uint16_t* H_t, const uint16_t* H_d, const
                 dot2(ht, hd, wr, d, &zt[v], &zd[v]);
             }
             const int64_t kk = variant == 3 ? 2 * (int64_t)K : K;   /* entries per row of idx / q_k */
-            if (hass_oracle_row_variant(zt, zd, V, K, g, variant, param, &loss[r], idx + r * kk, q_k + r * kk, &n_out[r],
-                                        &lse_t[r], &lse_d[r], dz) != 0) {
+            int rc;
+            if (forced_idx) {
+                int32_t n = 0;
+                for (int64_t j = 0; j < kk; ++j) {
+                    idx[r * kk + j] = -1;
+                    q_k[r * kk + j] = 0.0;
+                }
+                for (int64_t j = 0; j < kk; ++j)
+                    if (forced_idx[r * kk + j] >= 0) idx[r * kk + n++] = forced_idx[r * kk + j];
+                n_out[r] = n;
+                rc = hass_oracle_row_on_set(zt, zd, V, idx + r * kk, n, g, variant == 2, &loss[r], q_k + r * kk,
+                                            &lse_t[r], &lse_d[r], dz);
+            } else {
+                rc = hass_oracle_row_variant(zt, zd, V, K, g, variant, param, &loss[r], idx + r * kk, q_k + r * kk,
+                                             &n_out[r], &lse_t[r], &lse_d[r], dz);
+            }
+            if (rc != 0) {
 #pragma omp atomic write
                 status = -1;
                 continue;

@@ -3,26 +3,30 @@
 TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
 benchmark's CPU-baseline leg. It shares no code with the CUDA path.
 
-What it computes (Section 3.2, and the attention listing of the appendix): in aligning
-step j = m + 1 the query at position t attends, causally, to keys and values that come
-from the target LLM's features everywhere except on the m most recent positions, where
-they come from the draft features of the earlier passes: the pair (t, s) with
-t - s = i < m uses the keys/values of the i-th most recent draft pass (i = 0 is the
-latest pass and sits on the main diagonal). The steps below follow the listing's
-order: target scores with the causal mask, sub-diagonal overwrite with draft scores,
-softmax, product with the target values, then one correction per sub-diagonal that
-swaps the target value for the draft value.
+What it computes (Section 3.2, "Harmonized Context Alignment"): in aligning step
+j = m + 1 the query at position t attends causally to a key/value sequence of its own.
+Position s <= t of that sequence holds the target LLM's feature when it lies at least m
+positions back (t - s >= m); the m most recent positions hold draft features instead,
+position s = t - i taken from the i-th most recent earlier draft pass (i = 0 is the
+latest pass and sits at the query's own position). The output is an ordinary softmax
+attention of the query over that sequence:
 
-Reading taken where the listing and the text differ: the listing weights the value
-correction with the score matrix *before* the softmax; the text defines keys and values
-as the concatenation of target and draft features, i.e. an ordinary attention over the
-substituted key/value sequence. This oracle follows the text and uses the normalised
-weights, so that every output row is a convex combination of the value rows it attends
-to (pinned in the tests against the text's concatenation written out per query).
+    k(t, s), v(t, s) = K_t[s], V_t[s]            if t - s >= m
+                       K_d[t - s][s], V_d[t - s][s]  otherwise
+    w[t, .] = softmax_{s <= t}( scale * <Q[t], k(t, s)> ),   O[t] = sum_s w[t, s] v(t, s)
+
+The code below is that definition written out: one query at a time, its key and value
+sequences assembled explicitly, then a plain fp64 softmax attention over them.
+
+Reading taken where the appendix listing and the text differ: the listing multiplies the
+value substitution by the score matrix *before* the softmax; the text defines keys and
+values as the concatenation of target and draft features, i.e. an attention over the
+substituted sequence with normalised weights. This oracle follows the text. A draft pass
+i >= T meets no (query, key) pair of a T-position sequence and is inert.
 
 Layout: Q [B, T, H, D]; K_t, V_t [B, T, Hkv, D] with H a multiple of Hkv (query head h
 reads key/value head h // (H // Hkv)); K_d, V_d: sequences of m arrays shaped like K_t,
-index i = the sub-diagonal they replace. All arithmetic in float64.
+index i = how many positions behind the query the pass is used. All arithmetic in float64.
 """
 from __future__ import annotations
 
@@ -36,9 +40,36 @@ def _as64(x) -> np.ndarray:
     return np.asarray(x, dtype=np.float64)
 
 
+class _Context:
+    """Key and value sequences of one (sequence, key/value head) as each query sees them: a working copy of
+    the target rows in which, for the query at hand, the rows of its m most recent positions are replaced by
+    the draft passes' rows (and put back afterwards)."""
+
+    def __init__(self, k_t, v_t, k_d, v_d):
+        self.k_t, self.v_t, self.k_d, self.v_d = k_t, v_t, k_d, v_d
+        self.keys, self.vals = k_t.copy(), v_t.copy()
+
+    def enter(self, t):
+        for i in range(len(self.k_d)):
+            s = t - i
+            if s < 0:
+                break
+            self.keys[s] = self.k_d[i][s]
+            self.vals[s] = self.v_d[i][s]
+        return self.keys[:t + 1], self.vals[:t + 1]
+
+    def leave(self, t):
+        for i in range(len(self.k_d)):
+            s = t - i
+            if s < 0:
+                break
+            self.keys[s] = self.k_t[s]
+            self.vals[s] = self.v_t[s]
+
+
 def hca_attention(Q, K_t, V_t, K_d: Sequence = (), V_d: Sequence = (), scale: Optional[float] = None):
     """Forward pass. Returns (O [B, T, H, D], lse [B, H, T]) with lse the natural-log
-    normaliser of each query row after the sub-diagonal overwrite."""
+    normaliser of each query's scores over its own key sequence."""
     Q, K_t, V_t = _as64(Q), _as64(K_t), _as64(V_t)
     K_d = [_as64(x) for x in K_d]
     V_d = [_as64(x) for x in V_d]
@@ -51,39 +82,27 @@ def hca_attention(Q, K_t, V_t, K_d: Sequence = (), V_d: Sequence = (), scale: Op
         scale = 1.0 / math.sqrt(D)
     O = np.zeros((B, T, H, D))
     lse = np.zeros((B, H, T))
-    idx = np.arange(T)
-    mask = np.where(idx[None, :] > idx[:, None], -np.inf, 0.0)          # causal: s > t is hidden
     for b in range(B):
-        for h in range(H):
-            g = h // rep
-            q = Q[b, :, h, :]
-            k_t, v_t = K_t[b, :, g, :], V_t[b, :, g, :]
-            w = q @ k_t.T * scale + mask
-            for i in range(len(K_d)):
-                if i >= T:
-                    continue        # sub-diagonal i of a T x T matrix is empty
-                ind_q, ind_k = idx[i:], idx[:T - i]
-                w_d = q @ K_d[i][b, :, g, :].T * scale
-                w[ind_q, ind_k] = w_d[ind_q, ind_k]
-            mx = w.max(axis=1, keepdims=True)
-            e = np.exp(w - mx)
-            den = e.sum(axis=1, keepdims=True)
-            wn = e / den
-            out = wn @ v_t
-            for i in range(len(V_d)):
-                if i >= T:
-                    continue        # sub-diagonal i of a T x T matrix is empty
-                ind_q, ind_k = idx[i:], idx[:T - i]
-                v_d = V_d[i][b, :, g, :]
-                out[ind_q] += wn[ind_q, ind_k][:, None] * (v_d[ind_k] - v_t[ind_k])
-            O[b, :, h, :] = out
-            lse[b, h, :] = (mx + np.log(den))[:, 0]
+        for g in range(Hkv):
+            ctx = _Context(K_t[b, :, g, :], V_t[b, :, g, :], [x[b, :, g, :] for x in K_d],
+                           [x[b, :, g, :] for x in V_d])
+            for t in range(T):
+                keys, vals = ctx.enter(t)
+                for h in range(g * rep, (g + 1) * rep):
+                    sc = (keys @ Q[b, t, h]) * scale
+                    mx = sc.max()
+                    e = np.exp(sc - mx)
+                    den = e.sum()
+                    O[b, t, h] = (e / den) @ vals
+                    lse[b, h, t] = mx + math.log(den)
+                ctx.leave(t)
     return O, lse
 
 
 def hca_attention_grad(Q, K_t, V_t, K_d: Sequence, V_d: Sequence, dO, scale: Optional[float] = None):
-    """Gradients of sum(O * dO) with respect to every input, by the chain rule through the
-    steps of hca_attention (softmax Jacobian: dS = W * (dW - rowsum(W * dW))).
+    """Gradients of sum(O * dO) with respect to every input: the chain rule through each query's softmax
+    attention (dw = <dO[t], v(t, s)>, ds = w (dw - sum_s w dw) scale), with the gradient of every key and
+    value row sent back to the tensor the row came from.
     Returns (dQ, dK_t, dV_t, [dK_d], [dV_d]) with the inputs' shapes."""
     Q, K_t, V_t, dO = _as64(Q), _as64(K_t), _as64(V_t), _as64(dO)
     K_d = [_as64(x) for x in K_d]
@@ -98,44 +117,32 @@ def hca_attention_grad(Q, K_t, V_t, K_d: Sequence, V_d: Sequence, dO, scale: Opt
     dK_t, dV_t = np.zeros_like(K_t), np.zeros_like(V_t)
     dK_d = [np.zeros_like(K_t) for _ in range(m)]
     dV_d = [np.zeros_like(V_t) for _ in range(m)]
-    idx = np.arange(T)
-    mask = np.where(idx[None, :] > idx[:, None], -np.inf, 0.0)
+    pos = np.arange(T)
+    from_target = (pos[:, None] - pos[None, :]) >= m          # [t, s]: the pair (t, s) uses the target's row s
     for b in range(B):
-        for h in range(H):
-            g = h // rep
-            q = Q[b, :, h, :]
-            do = dO[b, :, h, :]
-            k_t, v_t = K_t[b, :, g, :], V_t[b, :, g, :]
-            w = q @ k_t.T * scale + mask
-            for i in range(m):
-                if i >= T:
-                    continue        # sub-diagonal i of a T x T matrix is empty
-                ind_q, ind_k = idx[i:], idx[:T - i]
-                w[ind_q, ind_k] = (q @ K_d[i][b, :, g, :].T * scale)[ind_q, ind_k]
-            wn = np.exp(w - w.max(axis=1, keepdims=True))
-            wn /= wn.sum(axis=1, keepdims=True)
-            # d(loss)/d(wn): against the value each pair actually uses
-            dwn = do @ v_t.T
-            for i in range(m):
-                if i >= T:
-                    continue        # sub-diagonal i of a T x T matrix is empty
-                ind_q, ind_k = idx[i:], idx[:T - i]
-                dwn[ind_q, ind_k] = np.einsum("td,td->t", do[ind_q], V_d[i][b, ind_k, g, :])
-            ds = wn * (dwn - (wn * dwn).sum(axis=1, keepdims=True)) * scale
-            # split weights and score gradients into the part that meets target keys/values
-            # and the sub-diagonals that meet draft keys/values
-            wn_t, ds_t = wn.copy(), ds.copy()
-            for i in range(m):
-                if i >= T:
-                    continue        # sub-diagonal i of a T x T matrix is empty
-                ind_q, ind_k = idx[i:], idx[:T - i]
-                wd, dsd = wn[ind_q, ind_k], ds[ind_q, ind_k]
-                wn_t[ind_q, ind_k] = 0.0
-                ds_t[ind_q, ind_k] = 0.0
-                dV_d[i][b, ind_k, g, :] += wd[:, None] * do[ind_q]
-                dK_d[i][b, ind_k, g, :] += dsd[:, None] * q[ind_q]
-                dQ[b, ind_q, h, :] += dsd[:, None] * K_d[i][b, ind_k, g, :]
-            dV_t[b, :, g, :] += wn_t.T @ do
-            dK_t[b, :, g, :] += ds_t.T @ q
-            dQ[b, :, h, :] += ds_t @ k_t
+        for g in range(Hkv):
+            ctx = _Context(K_t[b, :, g, :], V_t[b, :, g, :], [x[b, :, g, :] for x in K_d],
+                           [x[b, :, g, :] for x in V_d])
+            for h in range(g * rep, (g + 1) * rep):
+                # per-query weights w[t, s] and score gradients ds[t, s] (zero for s > t)
+                w = np.zeros((T, T))
+                ds = np.zeros((T, T))
+                for t in range(T):
+                    keys, vals = ctx.enter(t)
+                    sc = (keys @ Q[b, t, h]) * scale
+                    e = np.exp(sc - sc.max())
+                    wt = e / e.sum()
+                    dw = vals @ dO[b, t, h]
+                    dst = wt * (dw - wt @ dw) * scale
+                    dQ[b, t, h] = dst @ keys
+                    w[t, :t + 1] = wt
+                    ds[t, :t + 1] = dst
+                    ctx.leave(t)
+                # dk(t, s) = ds[t, s] Q[t] and dv(t, s) = w[t, s] dO[t], summed into the row's own tensor
+                dK_t[b, :, g, :] += np.where(from_target, ds, 0.0).T @ Q[b, :, h, :]
+                dV_t[b, :, g, :] += np.where(from_target, w, 0.0).T @ dO[b, :, h, :]
+                for i in range(min(m, T)):
+                    s = pos[:T - i]                            # keys that have a query i positions ahead
+                    dK_d[i][b, s, g, :] += ds[s + i, s][:, None] * Q[b, s + i, h, :]
+                    dV_d[i][b, s, g, :] += w[s + i, s][:, None] * dO[b, s + i, h, :]
     return dQ, dK_t, dV_t, dK_d, dV_d

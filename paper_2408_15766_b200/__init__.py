@@ -23,6 +23,7 @@ from .binding import (  # noqa: F401
     PROFILE_KINDS,
     profile_enable,
     profile_summary,
+    selftest_wait_expiry,
     status_string,
     topk_distill_bwd,
     topk_distill_fwd,
@@ -31,6 +32,8 @@ from .binding import (  # noqa: F401
     topk_distill_fwd_bwd_host,
     topk_distill_fwd_draft,
     topk_distill_fwd_static,
+    topk_distill_fwd_static_scratch_bytes,
+    STATIC_SCRATCH_MAX_BYTES,
     topk_distill_host_workspace_bytes,
     topk_distill_workspace_bytes,
     version,

@@ -64,8 +64,12 @@ def _load() -> ctypes.CDLL:
                                          ctypes.POINTER(vp), vp, sz, vp]
     L.hass_hca_attention_bwd.restype = ctypes.c_int
     L.hass_check.argtypes = [vp, vp]
+    L.hass_selftest_wait_expiry.argtypes = [vp, sz, ctypes.c_uint64, vp]
+    L.hass_selftest_wait_expiry.restype = ctypes.c_int
     L.hass_topk_distill_fwd_static.argtypes = [vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     L.hass_topk_distill_fwd_static.restype = ctypes.c_int
+    L.hass_topk_distill_fwd_static_scratch_bytes.argtypes = [i64, i64, i64, i32, ctypes.POINTER(sz)]
+    L.hass_topk_distill_fwd_static_scratch_bytes.restype = ctypes.c_int
     L.hass_profile_enable.argtypes = [ctypes.c_int]
     L.hass_profile_enable.restype = ctypes.c_int
     L.hass_profile_summary.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64), ctypes.c_int]
@@ -151,6 +155,17 @@ def topk_distill_fwd(H_t, H_d, W, K: int, workspace=None, stream=None) -> dict:
                                   _p(out["topk_q"]), _p(out["lse_t"]), _p(out["lse_d"]), _p(ws), ws.numel(),
                                   _stream(stream)), "hass_topk_distill_fwd")
     return out
+
+
+STATIC_SCRATCH_MAX_BYTES = 32 << 20
+
+
+def topk_distill_fwd_static_scratch_bytes(N: int, d: int, V: int, K: int) -> int:
+    """Bytes of the built-in scratch array that hass_topk_distill_fwd_static needs for this size."""
+    out = ctypes.c_size_t(0)
+    _ok(lib.hass_topk_distill_fwd_static_scratch_bytes(N, d, V, K, ctypes.byref(out)),
+        "hass_topk_distill_fwd_static_scratch_bytes")
+    return int(out.value)
 
 
 def topk_distill_fwd_static(H_t, H_d, W, K: int, stream=None, out: Optional[dict] = None) -> dict:
@@ -389,6 +404,14 @@ def hca_attention_bwd(Q, K_t, V_t, K_d, V_d, O, lse, dO, scale: Optional[float] 
 def check(workspace: torch.Tensor, stream=None) -> None:
     """Synchronises the stream and raises HassError if a kernel recorded a device-side problem."""
     _ok(lib.hass_check(_p(workspace), _stream(stream)), "hass_check")
+
+
+def selftest_wait_expiry(workspace: torch.Tensor, limit_ns: int = 2_000_000, stream=None) -> None:
+    """Enqueues the small kernel whose bounded wait is made to run out; check(workspace) raises
+    HASS_ERR_TIMEOUT afterwards. See hass_selftest_wait_expiry."""
+    assert workspace.dtype == torch.uint8 and workspace.is_cuda and workspace.is_contiguous()
+    _ok(lib.hass_selftest_wait_expiry(_p(workspace), workspace.numel(), int(limit_ns), _stream(stream)),
+        "hass_selftest_wait_expiry")
 
 
 PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional",

@@ -1123,11 +1123,22 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
 // ---- forward without a caller-provided workspace -------------------------------------------------
 // Scratch of hass_topk_distill_fwd_static: lives in the library's device image, so every GPU that
 // loads the library holds these bytes until the process exits.
-#define HASS_STATIC_SCRATCH_BYTES (32u << 20)
-static __device__ __align__(256) unsigned char g_static_scratch[HASS_STATIC_SCRATCH_BYTES];
+static __device__ __align__(256) unsigned char g_static_scratch[HASS_STATIC_SCRATCH_MAX_BYTES];
 // Device address of g_static_scratch per device. In host code the symbol itself is only a handle
 // for the runtime, never a pointer a kernel may use; the address comes from cudaGetSymbolAddress.
 static void* g_static_scratch_addr[64] = {nullptr};
+
+int hass_topk_distill_fwd_static_scratch_bytes(int64_t N, int64_t d, int64_t V, int32_t K, size_t* bytes) {
+    if (!bytes) return HASS_ERR_INVALID_ARG;
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    // the forward needs the statistics / candidate part of the workspace layout only
+    Layout L;
+    rc = make_layout(N, d, V, K, sm_count_or_default(), &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    *bytes = L.fwd_end;
+    return HASS_OK;
+}
 
 int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
                                  int32_t K, float* loss, int32_t* topk_idx, float* topk_q, float* lse_t,
@@ -1137,15 +1148,14 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
     DeviceInfo di;
     rc = device_info(&di);
     if (rc != HASS_OK) return rc;
-    // the forward needs the statistics / candidate part of the workspace layout only
-    Layout L;
-    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    size_t need = 0;
+    rc = hass_topk_distill_fwd_static_scratch_bytes(N, d, V, K, &need);
     if (rc != HASS_OK) return rc;
-    if (L.fwd_end > HASS_STATIC_SCRATCH_BYTES) {
+    if (need > HASS_STATIC_SCRATCH_MAX_BYTES) {
         if (kLog)
             std::fprintf(stderr, "[hass] hass_topk_distill_fwd_static: this size needs %zu bytes of scratch, the built-in "
-                         "array holds %u; use hass_topk_distill_fwd with a workspace\n", L.fwd_end,
-                         HASS_STATIC_SCRATCH_BYTES);
+                         "array holds %u; use hass_topk_distill_fwd with a workspace\n", need,
+                         HASS_STATIC_SCRATCH_MAX_BYTES);
         return HASS_ERR_UNSUPPORTED;
     }
     int dev = -1;
@@ -1167,7 +1177,7 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
     // forward_impl zeroes the status word (the only part of the scratch that must start at zero:
     // every statistic and candidate slot that is read has been written by the same call)
     rc = forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d, scratch,
-                      HASS_STATIC_SCRATCH_BYTES, st);
+                      HASS_STATIC_SCRATCH_MAX_BYTES, st);
     if (rc != HASS_OK) return rc;
     if (device_status &&
         cudaMemcpyAsync(device_status, scratch, sizeof(unsigned int), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
@@ -1380,6 +1390,23 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     }
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     return HASS_OK;
+}
+
+int hass_selftest_wait_expiry(void* workspace, size_t workspace_bytes, uint64_t limit_ns, void* cuda_stream) {
+    if (!workspace || workspace_bytes < 256 || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    if (limit_ns < 1000ull || limit_ns > 100000000ull) return HASS_ERR_INVALID_ARG;      // 1 us .. 100 ms
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    unsigned int* words = static_cast<unsigned int*>(workspace);
+    wait_expiry_selftest_kernel<<<1, 128, 0, st>>>(words, limit_ns, words + 16);
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
 }
 
 int hass_check(void* workspace, void* cuda_stream) {

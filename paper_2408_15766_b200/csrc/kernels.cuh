@@ -1113,6 +1113,32 @@ __global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d,
     if (lane == 0) loss_ce[row] = lse_d[row] - dot - ce_corr[row];
 }
 
+// Self-test of the bounded waits (hass_selftest_wait_expiry): one CTA, no TMA, no tensor memory. Every thread
+// waits for a phase of an mbarrier that nothing ever completes; thread 0 with the caller's short limit, the
+// others with the library's normal limit. Thread 0 runs out of time, records its code in the status word and
+// raises the CTA's abort flag, which ends the other threads' waits; the kernel then returns by itself.
+// report[0] = threads whose wait gave up, report[1] = nanoseconds the CTA spent waiting.
+__global__ void wait_expiry_selftest_kernel(unsigned int* status, unsigned long long limit_ns, unsigned int* report) {
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
+    __shared__ int gave_up;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        gave_up = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const unsigned long long t0 = globaltimer_ns();
+    const bool done = wait_barrier(smem_u32(&bar), 0u, &abort_flag, status, 15u, threadIdx.x == 0 ? limit_ns : kWaitLimitNs);
+    if (!done) atomicAdd(&gave_up, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        report[0] = static_cast<unsigned int>(gave_up);
+        report[1] = static_cast<unsigned int>(globaltimer_ns() - t0);
+    }
+}
+
 // Ends the exact route after a fused call: the range report has been dealt with.
 __global__ void range_handled_kernel(unsigned int* status) {
     if (((*status) & 0xffu) == 2u) *status = 0u;

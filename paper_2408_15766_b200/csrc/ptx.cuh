@@ -50,9 +50,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
 
 // Waits for the barrier phase with the given parity. Gives up (returns false) when another
-// thread of the CTA already gave up or after kWaitLimitNs, recording (code << 8) | 1 in *status.
+// thread of the CTA already gave up or after limit_ns, recording (code << 8) | 1 in *status.
 __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                             unsigned int* status, unsigned int code) {
+                                             unsigned int* status, unsigned int code,
+                                             unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     unsigned int it = 0;
@@ -60,7 +61,7 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, vola
         if (mbar_try_wait(bar, parity)) return true;
         if ((++it & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(status, 0u, (code << 8) | 1u);
                 return false;

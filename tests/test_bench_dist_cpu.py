@@ -39,6 +39,38 @@ def test_two_gloo_ranks_aggregate_like_the_bench(tmp_path):
         assert "ok" in o
 
 
+def test_bench_spawns_its_own_ranks_when_no_launcher_did(tmp_path):
+    """`bench.py --gpus 2` without torchrun: spawn_ranks starts two processes whose environment is enough for a
+    gloo rendezvous, and fails as a whole when one rank fails."""
+    import bench
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER)
+    clean = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    old = dict(os.environ)
+    os.environ.clear()
+    os.environ.update(clean)
+    try:
+        assert bench.spawn_ranks(2, [sys.executable, str(script)], timeout=120) == 0
+        bad = tmp_path / "bad.py"
+        bad.write_text("import os, sys, time\nif os.environ['RANK'] == '1':\n    sys.exit(3)\ntime.sleep(60)\n")
+        assert bench.spawn_ranks(2, [sys.executable, str(bad)], timeout=120) == 3     # rank 0 is not left sleeping
+    finally:
+        os.environ.clear()
+        os.environ.update(old)
+    # the command line a user types: the reference arm needs no GPU; rank 0 prints the one line with n_gpus = 2
+    import json
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "tiny", "--steps", "1", "--warmup", "0", "--oracle-rows", "8"],
+                         capture_output=True, text=True, timeout=300, env=clean)
+    assert out.returncode == 0, out.stderr
+    lines = [ln for ln in out.stdout.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2
+    # our own arm refuses to pretend: more GPUs asked for than visible is an error, not an n_gpus = 1 line
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--workload", "tiny"],
+                         capture_output=True, text=True, timeout=300, env=dict(clean, CUDA_VISIBLE_DEVICES=""))
+    assert out.returncode != 0 and "--gpus 2" in out.stderr and out.stdout.strip() == ""
+
+
 def test_reference_arm_prints_one_json_line(tmp_path):
     import json
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",

@@ -2,7 +2,8 @@
 
 Tolerances (the kernel multiplies bf16 operands exactly, accumulates in fp32, rounds the softmax
 weights to bf16 before the value product and the output to bf16):
-  O    |error| <= 1e-2 * max|O|   (bf16 rounding of weights and output, 2^-9 relative each)
+  O    every row (one position of one head) within 1e-2 of that row's own largest entry, see
+       tests/hca_parity.py (bf16 rounding of weights and output, 2^-9 relative each)
   lse  |error| <= 2e-3            (fp32 sums, approximate exp2)
 """
 import numpy as np
@@ -10,6 +11,7 @@ import pytest
 import torch
 
 import hass_inputs as hi
+from hca_parity import rowwise_error, tilewise_error
 from oracle import hca_oracle as ho
 
 pytestmark = pytest.mark.gpu
@@ -50,10 +52,10 @@ def _compare(inp, O, lse, scale=None, m=None, pairs=None):
         sl = lambda x, hh: _f64(x[b:b + 1, :, hh:hh + 1, :])
         O_ref, lse_ref = ho.hca_attention(sl(inp.Q, h), sl(inp.K_t, g), sl(inp.V_t, g),
                                           [sl(x, g) for x in inp.K_d[:m]], [sl(x, g) for x in inp.V_d[:m]], scale=scale)
-        err = np.abs(_f64(O[b:b + 1, :, h:h + 1, :]) - O_ref).max() / np.abs(O_ref).max()
+        err = rowwise_error(_f64(O[b:b + 1, :, h:h + 1, :]), O_ref).max()
         lerr = np.abs(lse[b, h].to(torch.float64).numpy() - lse_ref[0, 0]).max()
         worst_o, worst_l = max(worst_o, err), max(worst_l, lerr)
-    assert worst_o <= O_TOL, f"O error {worst_o:.3e} of max|O|"
+    assert worst_o <= O_TOL, f"O error {worst_o:.3e} of the row's own scale"
     assert worst_l <= LSE_TOL, f"lse error {worst_l:.3e}"
     return worst_o, worst_l
 
@@ -125,13 +127,17 @@ def test_full_size_sampled_heads(name):
 
 
 # ---- backward ---------------------------------------------------------------------------------------
-# Tolerance: every gradient within 1.5e-2 of its tensor's largest entry (the weights and dS pass through
-# bf16 before their products, outputs are bf16; observed <= 7e-3), with a floor for gradients that are
-# zero by construction (a single position has softmax weight 1 and dS = 0).
+# Tolerance: every tile of 64 positions of every gradient within G_TOL of that tile's own largest entry
+# (tests/hca_parity.py explains why tiles and not single rows; the weights and dS pass through bf16 before their
+# products, D = <dO, O> is formed from the bf16 output, outputs are bf16; observed <= 5.3e-3), with the
+# comparator's floor for tiles that are zero by construction (a single position has softmax weight 1 and dS = 0).
+# `whole_tensor`: compare against the tensor's largest entry instead; only for the steep-score case, where nearly
+# every row attends to a single key, dS is a difference of two nearly equal numbers throughout, and the error of a
+# tile is set by the rounding of D, not by the tile's own (vanishing) gradient.
 G_TOL = 1.5e-2
 
 
-def _run_bwd(inp, scale=None, pairs=None):
+def _run_bwd(inp, scale=None, pairs=None, whole_tensor=False):
     hass = _hass()
     dev = torch.device("cuda:0")
     wl = inp.wl
@@ -158,10 +164,16 @@ def _run_bwd(inp, scale=None, pairs=None):
         cmp = [(sq(got["dQ"]), ref[0]), (sk(got["dK_t"]), ref[1]), (sk(got["dV_t"]), ref[2])]
         cmp += [(sk(got["dK_d"][i]), ref[3][i]) for i in range(wl.m)]
         cmp += [(sk(got["dV_d"][i]), ref[4][i]) for i in range(wl.m)]
-        for mine, want in cmp:
-            err = np.abs(mine - want).max() / max(np.abs(want).max(), 1e-2)
+        names = ["dQ", "dK_t", "dV_t"] + [f"dK_d[{i}]" for i in range(wl.m)] + [f"dV_d[{i}]" for i in range(wl.m)]
+        for name, (mine, want) in zip(names, cmp):
+            if np.abs(want).max() < 1e-2:                            # an all-zero gradient: absolute comparison
+                err = np.abs(mine - want).max() / 1e-2
+            elif whole_tensor:
+                err = np.abs(mine - want).max() / np.abs(want).max()
+            else:
+                err = tilewise_error(mine, want).max()
+            assert err <= G_TOL, f"{name} of (sequence {b}, group {gk}): error {err:.3e} of the tile's scale"
             worst = max(worst, err)
-    assert worst <= G_TOL, f"gradient error {worst:.3e} of the tensor's maximum"
     return worst
 
 
@@ -182,12 +194,13 @@ def test_backward_awkward_shapes(B, T, H, Hkv, m):
 
 def test_backward_steep_scores():
     inp = hi.make_hca_inputs(hi.HcaWorkload("steep", B=1, T=640, H=2, Hkv=1, m=2, seed=3))
-    print(_run_bwd(inp, scale=0.5))
+    print(_run_bwd(inp, scale=0.5, whole_tensor=True))
 
 
-def test_backward_full_size_sampled_groups():
-    wl = hi.HCA_WORKLOADS["hca-l3-8b"]
-    print(_run_bwd(hi.make_hca_inputs(wl), pairs=[(0, 0), (wl.B - 1, wl.Hkv - 1)]))
+@pytest.mark.parametrize("name", ["hca-l3-8b", "hca-l2-7b"])
+def test_backward_full_size_sampled_groups(name):
+    wl = hi.HCA_WORKLOADS[name]
+    print(_run_bwd(hi.make_hca_inputs(wl), pairs=[(0, 0), (wl.B - 1, wl.Hkv - 1), (1, wl.Hkv // 2)]))
 
 
 def test_draft_passes_equal_to_target_change_nothing_on_the_gpu():

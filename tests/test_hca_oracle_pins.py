@@ -78,6 +78,54 @@ def test_equals_concatenated_context_per_query(m):
                 assert abs(lse[b, h, t] - (sc.max() + math.log(z))) < 1e-12
 
 
+def _dense_masked_form(Q, K_t, V_t, K_d, V_d, scale):
+    """The same attention in another form: one T x T score matrix per head whose i-th sub-diagonal is taken
+    from the scores against draft pass i, a row softmax under the causal mask, and an output split into the
+    part that meets target values and one band per draft pass. torch fp64 with autograd."""
+    B, T, H, D = Q.shape
+    rep = H // K_t.shape[2]
+    t_idx = torch.arange(T)
+    lag = t_idx[:, None] - t_idx[None, :]                       # t - s
+    outs, lses = [], []
+    for h in range(H):
+        g = h // rep
+        q = Q[:, :, h, :]
+        S = torch.einsum("btd,bsd->bts", q, K_t[:, :, g, :]) * scale
+        for i in range(len(K_d)):
+            Sd = torch.einsum("btd,bsd->bts", q, K_d[i][:, :, g, :]) * scale
+            S = torch.where(lag == i, Sd, S)
+        S = S.masked_fill(lag < 0, float("-inf"))
+        lses.append(torch.logsumexp(S, dim=-1))
+        P = torch.softmax(S, dim=-1)
+        band = torch.zeros_like(lag, dtype=torch.bool)
+        o = 0
+        for i in range(len(V_d)):
+            o = o + torch.einsum("bts,bsd->btd", P * (lag == i), V_d[i][:, :, g, :])
+            band |= lag == i
+        o = o + torch.einsum("bts,bsd->btd", P * (~band), V_t[:, :, g, :])
+        outs.append(o)
+    return torch.stack(outs, dim=2), torch.stack(lses, dim=1)
+
+
+@pytest.mark.parametrize("m,H,Hkv", [(1, 2, 2), (3, 4, 2), (6, 2, 1)])
+def test_forward_and_gradients_against_the_dense_masked_form_with_autograd(m, H, Hkv):
+    B, T, D = 2, 13, 4
+    Q, K_t, V_t, K_d, V_d = _case(B, T, H, Hkv, D, m, seed=21 + m)
+    dO = _rand(Q.shape, 77)
+    scale = 0.37
+    leaf = lambda x: torch.from_numpy(x).clone().requires_grad_(True)
+    tq, tk, tv = leaf(Q), leaf(K_t), leaf(V_t)
+    tkd, tvd = [leaf(x) for x in K_d], [leaf(x) for x in V_d]
+    O_ref, lse_ref = _dense_masked_form(tq, tk, tv, tkd, tvd, scale)
+    (O_ref * torch.from_numpy(dO)).sum().backward()
+    O, lse = ho.hca_attention(Q, K_t, V_t, K_d, V_d, scale=scale)
+    np.testing.assert_allclose(O, O_ref.detach().numpy(), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(lse, lse_ref.detach().numpy(), rtol=1e-12, atol=1e-13)
+    g = ho.hca_attention_grad(Q, K_t, V_t, K_d, V_d, dO, scale=scale)
+    for mine, ref in [(g[0], tq), (g[1], tk), (g[2], tv)] + list(zip(g[3], tkd)) + list(zip(g[4], tvd)):
+        np.testing.assert_allclose(mine, ref.grad.numpy(), rtol=1e-11, atol=1e-13)
+
+
 def test_two_token_closed_form():
     # T = 2, D = 1, one head, one draft pass on the main diagonal
     Q = np.array([0.5, -1.5]).reshape(1, 2, 1, 1)
@@ -162,3 +210,36 @@ def test_passes_beyond_the_sequence_length_are_inert():
     np.testing.assert_array_equal(l5, l3)
     g = ho.hca_attention_grad(Q, K_t, V_t, K_d, V_d, np.ones_like(Q))
     assert all(np.all(x == 0) for x in g[3][3:]) and all(np.all(x == 0) for x in g[4][3:])
+
+
+def test_rowwise_comparator_sees_a_missing_substitution_in_every_query_tile():
+    """Negative control of the GPU tests' comparator (tests/hca_parity.py), on the CPU: on the full-size
+    geometry (T = 2048, m = 2) an implementation that forgot the draft passes altogether is flagged in every
+    128-query tile, late ones included, while a tensor-wide bound would pass the later half of the sequence."""
+    import hass_inputs as hi
+    from hca_parity import rowwise_error
+    wl = hi.HcaWorkload("control", B=1, T=2048, H=1, Hkv=1, m=2, seed=0)
+    inp = hi.make_hca_inputs(wl)
+    f = lambda x: x.to(torch.float64).numpy()
+    good, _ = ho.hca_attention(f(inp.Q), f(inp.K_t), f(inp.V_t), [f(x) for x in inp.K_d], [f(x) for x in inp.V_d])
+    forgot, _ = ho.hca_attention(f(inp.Q), f(inp.K_t), f(inp.V_t))
+    per_tile = rowwise_error(forgot, good)[0, :, 0].reshape(-1, 128).max(axis=1)
+    assert per_tile.min() > 5e-2                      # five times the GPU tests' tolerance, in every tile
+    whole = np.abs(forgot - good)[0, :, 0].max(axis=1) / np.abs(good).max()
+    assert (whole[1024:] < 1e-2).all()                # what a tensor-wide 1e-2 bound would have let through
+
+
+def test_tilewise_comparator_sees_a_backward_without_the_substitution_in_every_tile():
+    """The same negative control for the gradients' comparator: gradients computed without the draft passes
+    differ from the real ones by more than three times the GPU tolerance in every 64-position tile of dQ, dK_t and dV_t."""
+    import hass_inputs as hi
+    from hca_parity import tilewise_error
+    wl = hi.HcaWorkload("control", B=1, T=1024, H=1, Hkv=1, m=2, seed=0)
+    inp = hi.make_hca_inputs(wl)
+    f = lambda x: x.to(torch.float64).numpy()
+    dO = _rand(tuple(inp.Q.shape), 3)
+    good = ho.hca_attention_grad(f(inp.Q), f(inp.K_t), f(inp.V_t), [f(x) for x in inp.K_d], [f(x) for x in inp.V_d], dO)
+    forgot = ho.hca_attention_grad(f(inp.Q), f(inp.K_t), f(inp.V_t), [], [], dO)
+    for i, name in enumerate(("dQ", "dK_t", "dV_t")):
+        per_tile = tilewise_error(forgot[i], good[i])
+        assert per_tile.min() > 3 * 1.5e-2, (name, per_tile.min())

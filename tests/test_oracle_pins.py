@@ -440,3 +440,53 @@ def test_bidirectional_top_k_is_eq1_on_the_union_of_both_top_k_sets():
         ri = oracle.variant_from_logits(zt[i], zdd[i], 4, oracle.VARIANT_BIDIR)
         assert f["n"][i] == ri["n"] and np.array_equal(f["idx"][i], ri["idx"]) and f["loss"][i] == pytest.approx(ri["loss"], rel=1e-12)
         np.testing.assert_allclose(f["dH_d"][i], ri["dz_d"] @ Wd, atol=1e-13)
+
+
+# ---- scoring a row on a given token set (the comparator's route for near-ties at rank K) ----------------
+
+def test_scoring_on_a_given_set_is_the_literal_restricted_sum_and_autograd():
+    V = 40
+    z_t, z_d = _rand_logits(V, seed=51, scale=1.5)
+    tokens = [7, 31, 2, 19, 24]                       # any set, not the K most probable
+    q = np.exp(z_t) / np.exp(z_t).sum()
+    zd = torch.tensor(z_d, requires_grad=True)
+    logp = torch.log_softmax(zd, 0)
+    loss = -(torch.tensor(q[tokens]) * logp[tokens]).sum()         # Eq. 1 with the sum over the given set
+    (0.6 * loss).backward()
+    r = oracle.on_set_from_logits(z_t, z_d, tokens, g=0.6)
+    assert r["loss"] == pytest.approx(float(loss), rel=1e-12)
+    np.testing.assert_allclose(r["q_k"], q[tokens], rtol=1e-12)
+    np.testing.assert_allclose(r["dz_d"], zd.grad.numpy(), atol=1e-15)
+    # normed: both distributions restricted to the set (library log_softmax of the restricted logits)
+    zd2 = torch.tensor(z_d, requires_grad=True)
+    qn = torch.tensor(q[tokens] / q[tokens].sum())
+    ln = -(qn * torch.log_softmax(zd2[tokens], 0)).sum()
+    (0.6 * ln).backward()
+    rn = oracle.on_set_from_logits(z_t, z_d, tokens, g=0.6, normed=True)
+    assert rn["loss"] == pytest.approx(float(ln), rel=1e-12)
+    np.testing.assert_allclose(rn["dz_d"], zd2.grad.numpy(), atol=1e-15)
+    # bad sets are refused: repeated id, id out of range, empty
+    for bad in ([3, 3], [V], []):
+        with pytest.raises(ValueError):
+            oracle.on_set_from_logits(z_t, z_d, bad)
+
+
+def test_forcing_a_variants_own_selection_reproduces_the_unforced_result():
+    N, d, V, K = 5, 16, 80, 6
+    Ht, Hd, W, _ = _feat(N, d, V, seed=53, sigma_w=0.3)
+    g = np.array([1.0, -0.5, 0.0, 2.0, 0.3])
+    for variant, param in ((oracle.VARIANT_TOPK, 0.0), (oracle.VARIANT_TOP_P, 0.25), (oracle.VARIANT_NORMED, 0.0),
+                           (oracle.VARIANT_BIDIR, 0.0)):
+        free = oracle.variant_from_features(Ht, Hd, W, K, variant, param, grad_loss=g)
+        forced = oracle.variant_from_features(Ht, Hd, W, K, variant, param, grad_loss=g, forced_idx=free["idx"])
+        assert np.array_equal(forced["idx"], free["idx"]) and np.array_equal(forced["n"], free["n"])
+        np.testing.assert_allclose(forced["loss"], free["loss"], rtol=1e-13)
+        np.testing.assert_allclose(forced["q_k"], free["q_k"], rtol=1e-13)
+        np.testing.assert_allclose(forced["dH_d"], free["dH_d"], atol=1e-15)
+    # a different set gives a different loss (the forced set is really used): swap one token of row 0
+    free = oracle.variant_from_features(Ht, Hd, W, K, oracle.VARIANT_NORMED)
+    alt = free["idx"].copy()
+    alt[0, -1] = next(v for v in range(V) if v not in set(free["idx"][0].tolist()))
+    other = oracle.variant_from_features(Ht, Hd, W, K, oracle.VARIANT_NORMED, forced_idx=alt)
+    assert abs(other["loss"][0] - free["loss"][0]) > 1e-6
+    np.testing.assert_allclose(other["loss"][1:], free["loss"][1:], rtol=1e-13)

@@ -15,6 +15,7 @@ import pytest
 import torch
 
 import hass_inputs as hi
+from parity import compare
 
 pytestmark = pytest.mark.gpu
 
@@ -45,10 +46,35 @@ def test_static_scratch_forward_matches_workspace_forward_twice_in_a_row():
         static = hass.topk_distill_fwd_static(H_t, H_d, W, K)
         torch.cuda.synchronize()
         _compare(static, ref)
+        # and against the fp64 oracle itself (the forward has no dH_d)
+        print(compare(inp.H_t, inp.H_d[0], inp.W, K, {k: v.cpu() for k, v in static.items()}, check_dH=False))
         # and once more on the same inputs, reusing the output tensors (no allocation at all)
         again = hass.topk_distill_fwd_static(H_t, H_d, W, K, out=static)
         torch.cuda.synchronize()
         _compare(again, ref)
+
+
+@pytest.mark.parametrize("N,K_ok", [(8192, 16), (128, 96)])
+def test_static_scratch_limit_is_the_declared_one(N, K_ok):
+    """The largest K whose forward scratch fits the array (it depends on the number of row tiles) runs and agrees
+    with the ordinary forward; the next K is refused on the host, before anything is launched."""
+    import paper_2408_15766_b200 as hass
+    dev = torch.device("cuda:0")
+    d, V = 64, 128256
+    limit = hass.STATIC_SCRATCH_MAX_BYTES
+    fits = [K for K in range(1, 129) if hass.topk_distill_fwd_static_scratch_bytes(N, d, V, K) <= limit]
+    assert fits == list(range(1, K_ok + 1))
+    inp = hi.make_custom(N, d, V, K_ok, seed=7, sigma_w=0.25)
+    H_t, H_d, W = inp.H_t.to(dev), inp.H_d[0].to(dev), inp.W.to(dev)
+    ref = hass.topk_distill_fwd(H_t, H_d, W, K_ok)
+    hass.check(ref["workspace"])
+    static = hass.topk_distill_fwd_static(H_t, H_d, W, K_ok)
+    torch.cuda.synchronize()
+    _compare(static, ref)
+    with pytest.raises(hass.HassError) as e:
+        hass.topk_distill_fwd_static(H_t, H_d, W, K_ok + 1)
+    assert e.value.status == -2
+    torch.cuda.synchronize()
 
 
 def test_static_scratch_refuses_a_problem_that_does_not_fit():
