@@ -551,7 +551,11 @@ def main():
     normed = args.objective == "normed"
     flops_credit = (8.0 if combined else 2.0 if normed else 6.0) * N * d * V
     # executed tensor work per step, averaged over the timed steps (a draft-only step skips the target product)
-    kinds = {"stats_gemm": (2.0 * n_full if normed else 4.0 * n_full + 2.0 * n_draft) / args.steps * N * d * V,
+    # the Top-K and Top-P calls sweep the target rows and the draft rows in separate launches (timed as
+    # stats_gemm and stats_gemm_draft); the combined and Bi-directional calls sweep both in one launch
+    two_sweeps = args.objective in ("topk", "top_p")
+    kinds = {"stats_gemm": (2.0 * n_full if (normed or two_sweeps) else 4.0 * n_full) / args.steps * N * d * V,
+             "stats_gemm_draft": 2.0 * (n_full + n_draft) / args.steps * N * d * V if two_sweeps else 0.0,
              "dz_gemm": 2.0 * N * d * V,
              "dH_gemm": (4.0 if combined else 2.0) * N * d * V}
     total_ms = sum(v[0] for v in prof.values())

@@ -336,10 +336,10 @@ int64_t hass_kernel_launch_count(void);
  *     holds it until the process exits. The forward scratch of a problem is about
  *     slots * 128 * (8 * cap(K) + 16) bytes: slots = the partial-result slots of its tile schedule
  *     (the number of SMs for up to 128 rows, about three times that for thousands of rows) and
- *     cap(K) = 16 for K <= 16, else K + max(K, 96) rounded up to a multiple of 32.
+ *     cap(K) = 16 for K <= 16, else K + max(2 K, 96) + 32 rounded up to a multiple of 32.
  *     hass_topk_distill_fwd_static_scratch_bytes returns the exact figure. On a 148-SM device
- *     N = 8192, V = 128256 needs 7.7 MiB for K <= 16 and 55.9 MiB for K = 17, so it is accepted up
- *     to K = 16; N = 128 fits up to K = 96. A problem that does not fit is refused with
+ *     N = 8192, V = 128256 needs 7.7 MiB for K <= 16 and 69.6 MiB for K = 17, so it is accepted up
+ *     to K = 16; N = 128 fits up to K = 53. A problem that does not fit is refused with
  *     HASS_ERR_UNSUPPORTED before anything is launched; use hass_topk_distill_fwd with a workspace.
  *   - The call allocates and frees nothing, in this library or through any other.
  *   - The first call on each device looks up the array's device address (a CUDA runtime query,
@@ -368,10 +368,11 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
  * launches of the exact route behind a fused call (they return at once unless it is needed),
  * 6 HCA attention forward, 7 / 8 / 9 HCA attention backward: dQ kernel, dK_t/dV_t kernel, row kernels
- * (row sums and the draft passes' gradients).
+ * (row sums and the draft passes' gradients), 10 the sweep of the draft rows in hass_topk_distill_fwd_bwd, its
+ * _draft form and the Top-P variant (kind 0 is then the sweep of the target rows alone).
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */
-#define HASS_PROFILE_KINDS 10
+#define HASS_PROFILE_KINDS 11
 int hass_profile_enable(int on);
 int hass_profile_summary(double* ms_by_kind, int64_t* launches_by_kind, int n_kinds);
 

@@ -20,7 +20,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_DQ = 7, KIND_HCA_DKV = 8, KIND_HCA_BWD_ROWS = 9, NUM_KINDS = 10 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_DQ = 7, KIND_HCA_DKV = 8, KIND_HCA_BWD_ROWS = 9, KIND_STATS_DRAFT = 10, NUM_KINDS = 11 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -74,6 +74,7 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e1 = cudaFuncSetAttribute(gemm_kernel<MODE_PROBS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_NONE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
             // two CTAs of this kernel share an SM: ask for the largest shared-memory carve-out
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -201,7 +202,7 @@ static int topk_cap(int K) { return K <= K_REG ? K_REG : cand_cap(K); }
 static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 struct Layout {
-    size_t status, part_m, part_s, cand_v, cand_i, thr_share, fwd_end, sidx, sgq, coef, lse2, sparse, scratch, fixed_end;
+    size_t status, part_m, part_s, cand_v, cand_i, thr_share, fwd_end, sidx, sgq, coef, lse2, capz, sparse, scratch, fixed_end;
     size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
     long long p_pitch;
     int pref_chunk_tiles;
@@ -260,6 +261,8 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     off = align256(off + static_cast<size_t>(N) * 4);
     L->lse2 = off;
     off = align256(off + static_cast<size_t>(N) * 4);
+    L->capz = off;                          // fused path: draft logits at Omega_hat, captured by the draft sweep, [N, K]
+    off = align256(off + static_cast<size_t>(N) * K * 4);
     L->sparse = off;                        // fused path: Omega_hat term of one chunk of rows, fp32 [chunk rows, d]
     off = align256(off + static_cast<size_t>(pref) * BM * d * 4);
     L->scratch = off;
@@ -296,9 +299,11 @@ static void log_schedule(const char* what, const Schedule& s) {
 }
 
 template <int MODE>
-static int launch_gemm(const GemmParams& p, cudaStream_t st) {
-    KernelTimer timer(p.only_if_range ? KIND_CONDITIONAL : MODE, st);
-    if (MODE == MODE_STATS && p.K <= K_REG)
+static int launch_gemm(const GemmParams& p, cudaStream_t st, int kind = -1) {
+    KernelTimer timer(p.only_if_range ? KIND_CONDITIONAL : (kind >= 0 ? kind : MODE), st);
+    if (MODE == MODE_STATS && p.topk_row_tiles == 0 && p.cap_z != nullptr)
+        gemm_kernel<MODE_STATS, TOPK_NONE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
+    else if (MODE == MODE_STATS && p.K <= K_REG)
         gemm_kernel<MODE_STATS, TOPK_REG><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
     else
         gemm_kernel<MODE><<<p.sched.max_ctas, NUM_THREADS, SMEM_BYTES, st>>>(p);
@@ -745,6 +750,215 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     return HASS_OK;
 }
 
+// ---- fused forward + backward, Omega_hat known before the draft rows are swept -------------------------
+// The route of hass_topk_distill_fwd_bwd, its _draft form and the Top-P variant. Per chunk of row tiles:
+// (1) sweep of the chunk's TARGET rows: statistics and Top-K candidates; (2) select_kernel: lse_t, Omega_hat,
+// and the same set sorted by token id; (3) sweep of the chunk's DRAFT rows: statistics, the bf16 spill of
+// 2^(z_d log2e - ref2), and z_d at the row's Omega_hat copied out of the accumulator as the sweep passes those
+// columns; (4) loss_patch_kernel: lse_d, Eq. 1, the per-row scale, and the Omega_hat term of dz_d subtracted
+// from the K spilled entries it concerns; (5) the second GEMM with the row scale in its epilogue. No logit
+// is computed twice and no row of W is gathered, so the cost does not depend on K beyond the candidate
+// handling of (1). with_target = false: (1) is skipped and (2) only sorts the given Omega_hat.
+static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
+                       long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
+                       int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
+                       void* workspace, size_t workspace_bytes, cudaStream_t st, float top_p = 0.f,
+                       int* topk_n = nullptr) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
+        return HASS_ERR_INVALID_ARG;
+    if (with_target && (!H_t || !idx_out || !q_out || !lse_t || !aligned16(H_t))) return HASS_ERR_INVALID_ARG;
+    if (!with_target && (!idx_in || !q_in)) return HASS_ERR_INVALID_ARG;
+    if (dH_dtype != HASS_BF16 && dH_dtype != HASS_FP32) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.fixed_end + L.scratch_row_tile_bytes) return HASS_ERR_WORKSPACE;
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN), DT = ceil_div(d, BN);
+    long long fit = static_cast<long long>((workspace_bytes - L.fixed_end) / L.scratch_row_tile_bytes);
+    int chunk_tiles = L.pref_chunk_tiles;
+    if (fit < chunk_tiles) chunk_tiles = static_cast<int>(fit);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    int* sidx = reinterpret_cast<int*>(ws + L.sidx);
+    float* sq = reinterpret_cast<float*>(ws + L.sgq);
+    float* coef = reinterpret_cast<float*>(ws + L.coef);
+    float* capz = reinterpret_cast<float*>(ws + L.capz);
+    __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(ws + L.scratch);
+    unsigned int* status = reinterpret_cast<unsigned int*>(ws + L.status);
+    if (cudaMemsetAsync(status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    CUtensorMap tmHt, tmHd, tmWk, tmWn, tmP;
+    rc = make_tmap(&tmHd, H_d, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = with_target ? make_tmap(&tmHt, H_t, N, d, d, BK, BM) : make_tmap(&tmHt, H_d, N, d, d, BK, BM);
+    if (rc == HASS_OK) rc = make_tmap(&tmWk, W, V, d, d, BK, BN);
+    if (rc == HASS_OK) rc = make_tmap(&tmWn, W, V, d, d, 64, BK);
+    if (rc == HASS_OK) rc = make_tmap(&tmP, P, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
+    if (rc != HASS_OK) return rc;
+
+    for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
+        const int tiles = (RT - t0 < chunk_tiles) ? RT - t0 : chunk_tiles;
+        const int rows = static_cast<int>((N - static_cast<long long>(t0) * BM < static_cast<long long>(tiles) * BM)
+                                              ? N - static_cast<long long>(t0) * BM
+                                              : static_cast<long long>(tiles) * BM);
+        // both sweeps cover `tiles` row tiles and share one schedule
+        GemmParams p;
+        std::memset(&p, 0, sizeof(p));
+        rc = plan_schedule(tiles, CT, di.sms, &p.sched);
+        if (rc != HASS_OK) return rc;
+        if (p.sched.total_slots > L.slot_cap) return HASS_ERR_WORKSPACE;
+        log_schedule("fused sweep (target / draft)", p.sched);
+        p.tmB = tmWk;
+        p.row_tiles0 = tiles;
+        p.a_row_offset = t0 * BM;
+        p.row_global_offset = t0 * BM;
+        p.rows_valid = static_cast<int>(N);
+        p.n_cols = static_cast<int>(V);
+        p.col_tiles = CT;
+        p.k_blocks = ceil_div(d, BK);
+        p.K = K;
+        p.cap = topk_cap(K);
+        p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+        p.part_s = reinterpret_cast<float*>(ws + L.part_s);
+        p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
+        p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
+        p.p_pitch = L.p_pitch;
+        p.status = status;
+        if (with_target) {
+            // (1) target rows: statistics + candidates
+            GemmParams t = p;
+            t.tmA0 = tmHt;
+            t.tmA1 = tmHt;
+            t.topk_row_tiles = tiles;
+            t.spill_begin = INT_MAX;
+            t.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+            if (cudaMemsetAsync(t.thr_share, 0xff, static_cast<size_t>(t.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
+                cudaGetLastError();
+                return HASS_ERR_CUDA;
+            }
+            rc = launch_gemm<MODE_STATS>(t, st);
+            if (rc != HASS_OK) return rc;
+        }
+        // (2) Omega_hat of the chunk's rows
+        SelectParams sp;
+        std::memset(&sp, 0, sizeof(sp));
+        sp.sched = p.sched;
+        sp.K = K;
+        sp.cap = p.cap;
+        sp.row_begin = t0 * BM;
+        sp.rows = rows;
+        sp.from_sweep = with_target ? 1 : 0;
+        sp.part_m = p.part_m;
+        sp.part_s = p.part_s;
+        sp.cand = p.cand;
+        sp.cand_n = p.cand_n;
+        sp.idx_in = idx_in;
+        sp.q_in = q_in;
+        sp.idx_out = idx_out;
+        sp.q_out = q_out;
+        sp.lse_t = lse_t;
+        sp.n_out = topk_n;
+        sp.top_p = top_p;
+        sp.sidx = sidx;
+        sp.sq = sq;
+        {
+            KernelTimer timer(KIND_FINALIZE, st);
+            select_kernel<<<ceil_div(rows, SEL_WARPS), SEL_WARPS * 32, 0, st>>>(sp);
+        }
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+        // (3) draft rows: statistics, spill, z_d at Omega_hat
+        {
+            GemmParams q = p;
+            q.tmA0 = tmHd;
+            q.tmA1 = tmHd;
+            q.topk_row_tiles = 0;
+            q.spill_begin = 0;
+            q.sidx = sidx;
+            q.cap_z = capz;
+            q.P = P;
+            rc = launch_gemm<MODE_STATS>(q, st, KIND_STATS_DRAFT);
+            if (rc != HASS_OK) return rc;
+        }
+        // (4) lse_d, loss, row scale, Omega_hat term into the spill
+        LossPatchParams lp;
+        std::memset(&lp, 0, sizeof(lp));
+        lp.sched = p.sched;
+        lp.K = K;
+        lp.row_begin = t0 * BM;
+        lp.rows = rows;
+        lp.part_m = p.part_m;
+        lp.part_s = p.part_s;
+        lp.sidx = sidx;
+        lp.sq = sq;
+        lp.cap_z = capz;
+        lp.grad_loss = grad_loss;
+        lp.loss = loss;
+        lp.lse_d = lse_d;
+        lp.coef_out = coef;
+        lp.P = P;
+        lp.p_pitch = L.p_pitch;
+        {
+            KernelTimer timer(KIND_FINALIZE, st);
+            loss_patch_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(lp);
+        }
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+        // (5) dH_d rows of the chunk = row scale x (patched spill x W)
+        GemmParams o;
+        std::memset(&o, 0, sizeof(o));
+        rc = plan_schedule(tiles, DT, di.sms, &o.sched);
+        if (rc != HASS_OK) return rc;
+        log_schedule("fused dH_d", o.sched);
+        o.tmA0 = tmP;
+        o.tmA1 = tmP;
+        o.tmB = tmWn;
+        o.row_tiles0 = tiles;
+        o.spill_begin = INT_MAX;
+        o.a_row_offset = 0;
+        o.row_global_offset = t0 * BM;
+        o.rows_valid = static_cast<int>(N);
+        o.n_cols = static_cast<int>(d);
+        o.col_tiles = DT;
+        o.k_blocks = ceil_div(V, BK);
+        o.K = K;
+        o.coef = coef;
+        o.out = dH_d;
+        o.out_fp32 = dH_dtype == HASS_FP32 ? 1 : 0;
+        o.out_align32 = ((reinterpret_cast<uintptr_t>(dH_d) | static_cast<uintptr_t>(d * (dH_dtype == HASS_FP32 ? 4 : 2))) & 31u) == 0 ? 1 : 0;
+        o.out_pitch = d;
+        o.status = status;
+        rc = launch_gemm<MODE_OUT>(o, st);
+        if (rc != HASS_OK) return rc;
+    }
+    if (!(top_p > 0.f)) {
+        // Exact route, enqueued behind every plain fused call: if a sweep reported a row beyond its exponent
+        // range, the separate forward and the recomputing backward (which have no such limit) redo the call
+        // and the report is withdrawn; otherwise each of these launches returns at once.
+        rc = forward_impl(with_target, H_t, H_d, W, N, d, V, K, idx_in, q_in, loss, idx_out, q_out, lse_t, lse_d,
+                          workspace, workspace_bytes, st, status);
+        if (rc != HASS_OK) return rc;
+        rc = backward_impl(H_d, W, N, d, V, K, with_target ? idx_out : idx_in, with_target ? q_out : q_in, lse_d,
+                           grad_loss, dH_d, dH_dtype, workspace, workspace_bytes, st, false, status);
+        if (rc != HASS_OK) return rc;
+        {
+            KernelTimer timer(KIND_CONDITIONAL, st);
+            range_handled_kernel<<<1, 1, 0, st>>>(status);
+        }
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+    }
+    return HASS_OK;
+}
+
 // ---- Normed Top-K variant -----------------------------------------------------------------------------
 // Both distributions are renormalised over Omega_hat, so the loss and its gradient involve the draft
 // logits on Omega_hat only: one sweep over the TARGET rows (statistics + Top-K), then finalize computes the
@@ -935,16 +1149,16 @@ int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, i
                               int32_t K, const float* grad_loss, float* loss, int32_t* topk_idx, float* topk_q,
                               float* lse_t, float* lse_d, void* dH_d, int dH_dtype, void* workspace,
                               size_t workspace_bytes, void* cuda_stream) {
-    return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
-                      dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+    return fused2_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
+                       dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
                                     const int32_t* topk_idx, const float* topk_q, const float* grad_loss, float* loss,
                                     float* lse_d, void* dH_d, int dH_dtype, void* workspace, size_t workspace_bytes,
                                     void* cuda_stream) {
-    return fused_impl(false, nullptr, H_d, W, N, d, V, K, grad_loss, topk_idx, topk_q, loss, nullptr, nullptr, nullptr,
-                      lse_d, dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+    return fused2_impl(false, nullptr, H_d, W, N, d, V, K, grad_loss, topk_idx, topk_q, loss, nullptr, nullptr, nullptr,
+                       lse_d, dH_d, dH_dtype, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V,
@@ -955,12 +1169,12 @@ int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     switch (variant) {
         case HASS_LOSS_TOPK:
-            return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
-                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, 0.f, topk_n);
+            return fused2_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
+                               lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, 0.f, topk_n);
         case HASS_LOSS_TOP_P:
             if (!(param > 0.f)) return HASS_ERR_INVALID_ARG;
-            return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
-                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, param, topk_n);
+            return fused2_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
+                               lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, param, topk_n);
         case HASS_LOSS_BIDIR_TOPK:
             return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
                               lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, 0.f, topk_n, true);

@@ -79,6 +79,8 @@ struct GemmParams {
     const float* coef;     // [N] g * S_q
     const int* sidx;       // [N, K] Omega_hat sorted by token id
     const float* sgq;      // [N, K] g * q in the same order
+    float* cap_z;          // MODE_STATS, TOPK_NONE: [N, K] out, z_d at the tokens of sidx (same order); slots of
+                           // padding entries (token id INT_MAX) are left untouched
     __nv_bfloat16* P;      // [chunk rows, p_pitch]
     __nv_bfloat16* Pt;     // [chunk rows, p_pitch] spill of the target tiles, or nullptr
     long long p_pitch;
@@ -117,11 +119,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 // compacts it to the row's K best and raises the threshold to the K-th largest logit. Entries stay in
 // increasing token-id order, admission is strict (x > threshold), and among logits equal to the K-th the
 // lowest token ids are kept, so equal logits resolve to the lower token id.
-constexpr int CAND_CAP_MAX = 256;                 // largest buffer: K = 128
+constexpr int CAND_CAP_MAX = 416;                 // largest buffer: K = 128
 constexpr int CAND_REGS = CAND_CAP_MAX / 32;      // entries per lane during a compaction
+constexpr int CAND_SLACK = 32;                    // a compaction may leave up to K + CAND_SLACK entries
 
-// K + at least 96 spare entries (a compaction is triggered 32 entries before the end), multiple of 32
-__host__ __device__ constexpr int cand_cap(int K) { return ((K + (K > 96 ? K : 96)) + 31) / 32 * 32; }
+// K entries kept + room for max(2K, 96) new ones between compactions (each compaction then multiplies the
+// number of columns a threshold has seen by about three) + the 32 entries before the end at which a
+// compaction is triggered; a multiple of 32
+__host__ __device__ constexpr int cand_cap(int K) { return (K + (2 * K > 96 ? 2 * K : 96) + 32 + 31) / 32 * 32; }
 
 // order-preserving map from fp32 bit patterns to unsigned integers (and back); 0 is below every float
 __device__ __forceinline__ uint32_t ordered_key(uint32_t bits) {
@@ -131,9 +136,14 @@ __device__ __forceinline__ uint32_t key_bits(uint32_t key) {
     return (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
 }
 
-// Warp-collective: compacts the buffer `buf` holding n >= K entries to its K best, in place, keeping their
-// order. Returns the bit pattern of the K-th largest logit (the new admission threshold).
-__device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K, int cap, int lane) {
+// Warp-collective: compacts the buffer `buf` holding n >= K entries, in place, keeping their order, and
+// returns the bit pattern of the new admission threshold (only logits strictly above it can still belong to
+// the row's K best); n_out = entries left. The K-th largest key is searched bit by bit from the top. After
+// the upper 16 bits (bf16 resolution) the search stops if at most K + CAND_SLACK entries reach the prefix
+// found so far: all of them are kept and the threshold is the value just below the prefix. Otherwise the
+// search runs to the last bit, exactly K entries are kept (among logits equal to the K-th, the lowest token
+// ids) and the threshold is the K-th largest logit itself.
+__device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K, int cap, int lane, int& n_out) {
     uint32_t key[CAND_REGS];
     int id[CAND_REGS];
     const int groups = cap >> 5;
@@ -148,8 +158,10 @@ __device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K,
             id[t] = static_cast<int>(v.y);
         }
     }
-    // largest T with at least K keys >= T, bit by bit
+    // largest T with at least K keys >= T, bit by bit; cT = number of keys >= T
     uint32_t T = 0u;
+    int cT = n;
+    bool exact = true;
 #pragma unroll 1
     for (int bit = 31; bit >= 0; --bit) {
         const uint32_t cand = T | (1u << bit);
@@ -157,15 +169,37 @@ __device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K,
 #pragma unroll
         for (int t = 0; t < CAND_REGS; ++t) c += (key[t] >= cand) ? 1 : 0;
         c = __reduce_add_sync(0xffffffffu, c);
-        if (c >= K) T = cand;
+        if (c >= K) {
+            T = cand;
+            cT = c;
+        }
+        if (bit == 16 && cT <= K + CAND_SLACK) {
+            exact = false;
+            break;
+        }
+    }
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int out = 0;
+    if (!exact) {
+        // keep every entry that reaches the 16-bit prefix
+#pragma unroll
+        for (int t = 0; t < CAND_REGS; ++t) {
+            if (t < groups) {
+                const bool keep = key[t] >= T;
+                const uint32_t km = __ballot_sync(0xffffffffu, keep);
+                if (keep) buf[out + __popc(km & lt_mask)] = make_uint2(key_bits(key[t]), static_cast<uint32_t>(id[t]));
+                out += __popc(km);
+            }
+        }
+        n_out = out;
+        return key_bits(T - 1u);      // T >= 2^16 here: at least K keys reach it
     }
     int n_gt = 0;
 #pragma unroll
     for (int t = 0; t < CAND_REGS; ++t) n_gt += (key[t] > T) ? 1 : 0;
     n_gt = __reduce_add_sync(0xffffffffu, n_gt);
     const int need_eq = K - n_gt;             // >= 1: how many entries equal to the K-th are kept
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    int run_eq = 0, out = 0;
+    int run_eq = 0;
 #pragma unroll
     for (int t = 0; t < CAND_REGS; ++t) {
         if (t < groups) {
@@ -178,13 +212,16 @@ __device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K,
             out += __popc(km);
         }
     }
+    n_out = out;
     return key_bits(T);
 }
 
 // TOPK selects how MODE_STATS keeps a row's Top-K candidates: TOPK_REG (K <= K_REG) a sorted list in
 // registers, all lanes inserting in parallel - best while most rows still admit logits; TOPK_BUF (any K)
-// append buffers with warp-cooperative compaction - cost nearly independent of K.
-enum { TOPK_REG = 0, TOPK_BUF = 1 };
+// append buffers with warp-cooperative compaction - cost nearly independent of K; TOPK_NONE: a sweep of draft
+// rows whose Omega_hat is already known - no candidates are collected, instead each row's draft logits at its
+// Omega_hat tokens are copied out of the accumulator as the sweep passes them (GemmParams::cap_z).
+enum { TOPK_REG = 0, TOPK_BUF = 1, TOPK_NONE = 2 };
 constexpr int K_REG = 16;
 
 template <int MODE, int TOPK = TOPK_BUF>
@@ -342,6 +379,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         // K_REG-th largest: a list of exactly K entries with its K-th as threshold measured slower), and the
         // current chunk's admitted logits waiting in a small local-memory buffer
         constexpr bool USE_REG = MODE == MODE_STATS && TOPK == TOPK_REG;
+        constexpr bool HAS_TOPK = MODE == MODE_STATS && TOPK != TOPK_NONE;
+        constexpr bool CAPTURE = MODE == MODE_STATS && TOPK == TOPK_NONE;
         float tv[USE_REG ? K_REG : 1];
         int ti[USE_REG ? K_REG : 1];
         float pend_v[USE_REG ? 32 : 1];
@@ -363,8 +402,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             const float* sg = nullptr;
             int cur = 0, nxt = INT_MAX;
             if (MODE == MODE_STATS) {
-                want_topk = rt < p.topk_row_tiles;
-                cbuf = p.cand + (static_cast<long long>(slot) * BM + r_local) * p.cap;
+                want_topk = HAS_TOPK && rt < p.topk_row_tiles;
+                if (HAS_TOPK) cbuf = p.cand + (static_cast<long long>(slot) * BM + r_local) * p.cap;
                 cnt = 0;
                 if (USE_REG) {
 #pragma unroll
@@ -382,6 +421,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 nxt = si[0];
             }
             if (MODE == MODE_OUT && p.coef != nullptr && row_ok) coef = p.coef[g_row];
+            float* cz = nullptr;
+            if (CAPTURE && row_ok && p.cap_z != nullptr) {
+                // the row's Omega_hat in increasing token order; this lane meets its own column tiles in that order too
+                si = p.sidx + static_cast<long long>(g_row) * p.K;
+                cz = p.cap_z + static_cast<long long>(g_row) * p.K;
+                nxt = si[0];
+            }
             const int t0 = (spill && ln != 0) ? -1 : 0;
             const int nt = (p.col_tiles - ln + S - 1) / S;
             for (int t = t0; t < nt; ++t) {
@@ -412,35 +458,56 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     m = ref2 * (1.0f / LOG2E);
                     skip_tile = t < 0;
                 }
+                if (CAPTURE && !skip_tile) {
+                    while (nxt < col_base) {
+                        ++cur;
+                        nxt = cur < p.K ? si[cur] : INT_MAX;
+                    }
+                }
 #pragma unroll 1
                 for (int ch = 0; ch < BN / 32 && !skip_tile; ++ch) {
+                    if (MODE == MODE_STATS && !USE_REG && want_topk) {
+                        // make room for a whole chunk in every row's buffer (warp-uniform control flow), before the
+                        // chunk's logits occupy registers
+                        uint32_t full = __ballot_sync(0xffffffffu, cnt > p.cap - 32);
+                        while (full) {
+                            const int L = __ffs(full) - 1;
+                            full &= full - 1u;
+                            __syncwarp();
+                            const unsigned long long bp = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(cbuf), L);
+                            const int n = __shfl_sync(0xffffffffu, cnt, L);
+                            int left = 0;
+                            const uint32_t tb = compact_candidates(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane, left);
+                            __syncwarp();
+                            if (lane == L) {
+                                cnt = left;
+                                thr_own = __uint_as_float(tb);
+                                thr = fmaxf(thr_own, thr_sh);
+                            }
+                        }
+                    }
                     uint32_t r[32];
                     tmem_ld32(t_row + ch * 32, r);
                     tmem_ld_wait(r);
                     const int col0 = col_base + ch * 32;
                     if (MODE == MODE_STATS) {
-                        if (!USE_REG && want_topk) {
-                            // make room for a whole chunk in every row's buffer (warp-uniform control flow)
-                            uint32_t full = __ballot_sync(0xffffffffu, cnt > p.cap - 32);
-                            while (full) {
-                                const int L = __ffs(full) - 1;
-                                full &= full - 1u;
-                                __syncwarp();
-                                const unsigned long long bp = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(cbuf), L);
-                                const int n = __shfl_sync(0xffffffffu, cnt, L);
-                                const uint32_t tb = compact_candidates(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane);
-                                __syncwarp();
-                                if (lane == L) {
-                                    cnt = p.K;
-                                    thr_own = __uint_as_float(tb);
-                                    thr = fmaxf(thr_own, thr_sh);
-                                }
-                            }
-                        }
                         if (col0 + 32 > p.n_cols) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (col0 + j >= p.n_cols) r[j] = __float_as_uint(-INFINITY);
+                        }
+                        if (CAPTURE) {
+                            // draft logits at the row's Omega_hat, straight from the fp32 accumulator
+                            while (nxt < col0 + 32) {
+                                const int off = nxt - col0;
+                                uint32_t zb = 0u;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (j == off) zb = r[j];
+                                cz[cur] = __uint_as_float(zb);
+                                ++cur;
+                                nxt = cur < p.K ? si[cur] : INT_MAX;
+                            }
                         }
                         float cm = -INFINITY;     // the chunk's largest logit (not needed by a spill row without Top-K)
                         if (!spill || want_topk) {
@@ -1073,6 +1140,271 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
         p.loss[row] = loss;
         // dense part of dz_d: g S_q p (Top-K loss) or g (1 + w S_q) p (combined objective)
         if (p.coef_out) p.coef_out[row] = (combined ? g * (1.f + p.w_topk * S_q) : g * S_q) * expf(m_spill - lse_d);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// select_kernel: one warp per row, between the sweep of the target rows and the sweep of the draft rows of
+// the fused call. Merges the target's partial statistics into lse_t, picks Omega_hat from the sweep's
+// candidates (or takes it as an input), writes topk_idx / topk_q in descending q, and leaves the same set
+// sorted by token id (sidx, sq) for the draft sweep, which copies z_d at those tokens out of its accumulators.
+constexpr int SEL_WARPS = 4;          // warps (rows) per block
+constexpr int SEL_MAX = 1024;         // candidates of one row that fit its shared-memory window
+
+struct SelectParams {
+    Schedule sched;        // schedule of the target sweep; its row tile t = rows [128 t, 128 t + 128) of the chunk
+    int K, cap;
+    int row_begin, rows;   // global rows [row_begin, row_begin + rows)
+    int from_sweep;        // 1: Omega_hat from the sweep's candidates; 0: idx_in / q_in are given
+    const float* part_m;
+    const float* part_s;
+    const uint2* cand;
+    const int* cand_n;
+    const int* idx_in;     // [N, K]
+    const float* q_in;
+    int* idx_out;          // [N, K] (from_sweep)
+    float* q_out;
+    float* lse_t;
+    int* n_out;            // [N] |Omega_hat| (nullable)
+    float top_p;           // > 0: Omega_hat is cut to the shortest sorted prefix with cumulative q > top_p
+    int* sidx;             // [N, K] Omega_hat in increasing token id; unused entries INT_MAX
+    float* sq;             // [N, K] q in the same order; unused entries 0
+    const unsigned int* only_if_range;
+};
+
+// Warp-collective: the largest t such that at least `want` of the n keys satisfy key >= t (keys pass the
+// filter `use`); bit by bit from the top.
+template <typename KeyFn>
+__device__ __forceinline__ uint32_t kth_largest_key(int n, int want, int lane, KeyFn key_of) {
+    uint32_t T = 0u;
+#pragma unroll 1
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t c2 = T | (1u << bit);
+        int c = 0;
+        for (int e = lane; e < n; e += 32) {
+            uint32_t k;
+            if (key_of(e, k)) c += (k >= c2) ? 1 : 0;
+        }
+        c = __reduce_add_sync(0xffffffffu, c);
+        if (c >= want) T = c2;
+    }
+    return T;
+}
+
+__global__ void __launch_bounds__(SEL_WARPS * 32) select_kernel(const __grid_constant__ SelectParams p) {
+    if (p.only_if_range != nullptr && ((*p.only_if_range) & 0xffu) != 2u) return;
+    __shared__ uint32_t sh_key[SEL_WARPS][SEL_MAX];   // ordered keys of the row's candidates
+    __shared__ int sh_id[SEL_WARPS][SEL_MAX];
+    __shared__ int sel_tok[SEL_WARPS][K_CAP];         // Omega_hat in descending q
+    __shared__ float sel_q[SEL_WARPS][K_CAP];
+    const int lane = threadIdx.x & 31;
+    const int wib = threadIdx.x >> 5;
+    const int local = blockIdx.x * SEL_WARPS + wib;
+    if (local >= p.rows) return;
+    const int row = p.row_begin + local;
+    const int rt = local / BM, r = local % BM;
+    const int K = p.K;
+    const long long ro = static_cast<long long>(row) * K;
+
+    if (p.from_sweep) {
+        int slot0, S;
+        find_slots(p.sched, rt, slot0, S);
+        const float lse_t = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
+        if (lane == 0) p.lse_t[row] = lse_t;
+        // Pool of candidates in shared memory. The slots' lists are appended one after the other; whenever the
+        // next list might not fit, the pool is cut to its K best (logit descending, lower token id first among
+        // equal logits) and the K-th logit becomes a floor below which later candidates are not even copied.
+        uint32_t* kk = sh_key[wib];
+        int* ii = sh_id[wib];
+        int n = 0;
+        uint32_t floor_key = 0u;
+        const uint32_t lt_mask = (1u << lane) - 1u;
+        auto cut_to_k = [&]() {
+            // K-th largest logit, then (only if several candidates share it) the id bound among those
+            const uint32_t T = kth_largest_key(n, K, lane, [&](int e, uint32_t& k) { k = kk[e]; return true; });
+            int n_gt = 0, n_eq = 0;
+            for (int e = lane; e < n; e += 32) {
+                n_gt += kk[e] > T ? 1 : 0;
+                n_eq += kk[e] == T ? 1 : 0;
+            }
+            n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+            n_eq = __reduce_add_sync(0xffffffffu, n_eq);
+            const int need_eq = K - n_gt;
+            uint32_t T2 = 0u;      // among the candidates equal to T: those with ~id >= T2 (the lowest ids) are kept
+            if (n_eq > need_eq)
+                T2 = kth_largest_key(n, need_eq, lane, [&](int e, uint32_t& k) { k = ~static_cast<uint32_t>(ii[e]); return kk[e] == T; });
+            int np = 0;
+            for (int e0 = 0; e0 < n; e0 += 32) {
+                const int e = e0 + lane;
+                uint32_t ke = 0u;
+                int ie = 0;
+                if (e < n) {
+                    ke = kk[e];
+                    ie = ii[e];
+                }
+                const bool take = e < n && (ke > T || (ke == T && ~static_cast<uint32_t>(ie) >= T2));
+                const uint32_t bm = __ballot_sync(0xffffffffu, take);
+                __syncwarp();
+                if (take) {
+                    const int at = np + __popc(bm & lt_mask);      // at <= e: in place
+                    kk[at] = ke;
+                    ii[at] = ie;
+                }
+                np += __popc(bm);
+                __syncwarp();
+            }
+            n = np;
+            floor_key = T;
+        };
+        for (int sl = 0; sl < S; ++sl) {
+            const long long so = static_cast<long long>(slot0 + sl) * BM + r;
+            const int cn = p.cand_n[so];
+            if (n + cn > SEL_MAX && n > K) cut_to_k();
+            for (int e0 = 0; e0 < cn; e0 += 32) {
+                const int e = e0 + lane;
+                bool ok = false;
+                uint2 ce = make_uint2(0u, 0u);
+                uint32_t key = 0u;
+                if (e < cn) {
+                    ce = p.cand[so * p.cap + e];
+                    key = ordered_key(ce.x);
+                    // unused register-list entries carry id -1; anything below the floor cannot be among the K best
+                    ok = static_cast<int>(ce.y) >= 0 && key >= floor_key;
+                }
+                const uint32_t bm = __ballot_sync(0xffffffffu, ok);
+                if (ok) {
+                    const int at = n + __popc(bm & lt_mask);
+                    kk[at] = key;
+                    ii[at] = static_cast<int>(ce.y);
+                }
+                n += __popc(bm);
+            }
+            __syncwarp();
+        }
+        if (n > K) cut_to_k();
+        __syncwarp();
+        // order the K picks: logit descending, token id ascending
+        for (int j = lane; j < K; j += 32) {
+            const uint32_t kj = j < n ? kk[j] : 0u;
+            const int ij = j < n ? ii[j] : 0;
+            int rank = 0;
+            for (int i = 0; i < K; ++i) {
+                const uint32_t ki = i < n ? kk[i] : 0u;
+                const int i2 = i < n ? ii[i] : 0;
+                rank += (ki > kj || (ki == kj && (i2 < ij || (i2 == ij && i < j)))) ? 1 : 0;
+            }
+            sel_tok[wib][rank] = ij;
+            sel_q[wib][rank] = j < n ? expf(__uint_as_float(key_bits(kj)) - lse_t) : 0.f;
+        }
+        __syncwarp();
+        int n_sel = K;
+        if (p.top_p > 0.f) {
+            // Top-P: a token belongs to Omega_hat while the probability of those before it is <= P
+            int n = 0;
+            if (lane == 0) {
+                float cum = 0.f;
+                for (int j = 0; j < K; ++j) {
+                    if (cum > p.top_p) {
+                        sel_tok[wib][j] = -1;
+                        sel_q[wib][j] = 0.f;
+                    } else {
+                        ++n;
+                    }
+                    cum += sel_q[wib][j];
+                }
+            }
+            __syncwarp();
+            n_sel = __shfl_sync(0xffffffffu, n, 0);
+        }
+        for (int j = lane; j < K; j += 32) {
+            p.idx_out[ro + j] = sel_tok[wib][j];
+            p.q_out[ro + j] = sel_q[wib][j];
+        }
+        if (lane == 0 && p.n_out) p.n_out[row] = n_sel;
+    } else {
+        for (int j = lane; j < K; j += 32) {
+            sel_tok[wib][j] = p.idx_in[ro + j];
+            sel_q[wib][j] = p.q_in[ro + j];
+        }
+        if (lane == 0 && p.n_out) p.n_out[row] = K;
+    }
+    __syncwarp();
+    // the same set in increasing token id (entries cut by Top-P go to the end as INT_MAX / 0)
+    for (int j = lane; j < K; j += 32) {
+        const int tj = sel_tok[wib][j] < 0 ? INT_MAX : sel_tok[wib][j];
+        int rank = 0;
+        for (int i = 0; i < K; ++i) {
+            const int ti = sel_tok[wib][i] < 0 ? INT_MAX : sel_tok[wib][i];
+            rank += (ti < tj || (ti == tj && i < j)) ? 1 : 0;
+        }
+        p.sidx[ro + rank] = tj;
+        p.sq[ro + rank] = tj == INT_MAX ? 0.f : sel_q[wib][j];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// loss_patch_kernel: one warp per row, after the sweep of the draft rows of the fused call. Merges the draft's
+// partial statistics into lse_d, evaluates Eq. 1 from the captured draft logits, writes the per-row scale of the
+// spilled tiles, and puts the Omega_hat term of dz_d into the spill itself: with the spilled value
+// P~(v) = 2^(z_d(v) log2e - ref2), dz_d(v) = coef (P~(v) - [v in Omega_hat] q(v) / (S_q e^(m_spill - lse_d))),
+// so the K entries of the row at its Omega_hat tokens are lowered in place (bf16) and the second GEMM needs
+// nothing but the row scale in its epilogue.
+struct LossPatchParams {
+    Schedule sched;        // schedule of the draft sweep
+    int K;
+    int row_begin, rows;
+    const float* part_m;
+    const float* part_s;
+    const int* sidx;       // [N, K]
+    const float* sq;
+    const float* cap_z;    // [N, K] z_d at sidx
+    const float* grad_loss;
+    float* loss;
+    float* lse_d;
+    float* coef_out;       // [N] g S_q e^(m_spill - lse_d)
+    __nv_bfloat16* P;      // spill of the chunk [rows, p_pitch]
+    long long p_pitch;
+};
+
+__global__ void __launch_bounds__(256) loss_patch_kernel(const __grid_constant__ LossPatchParams p) {
+    const int lane = threadIdx.x & 31;
+    const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (local >= p.rows) return;
+    const int row = p.row_begin + local;
+    const int rt = local / BM, r = local % BM;
+    const int K = p.K;
+    int slot0, S;
+    find_slots(p.sched, rt, slot0, S);
+    const float lse_d = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
+    const float m_spill = p.part_m[static_cast<long long>(slot0) * BM + r];
+    const float g = p.grad_loss ? p.grad_loss[row] : 1.f;
+    const long long ro = static_cast<long long>(row) * K;
+    float S_q = 0.f, loss = 0.f;
+    for (int j = lane; j < K; j += 32) {
+        if (p.sidx[ro + j] != INT_MAX) {
+            const float qv = p.sq[ro + j];
+            S_q += qv;
+            loss += qv * (lse_d - p.cap_z[ro + j]);     // -q log p,  log p = z_d - lse_d
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        S_q += __shfl_xor_sync(0xffffffffu, S_q, o);
+        loss += __shfl_xor_sync(0xffffffffu, loss, o);
+    }
+    const float scale = S_q * expf(m_spill - lse_d);     // coef / g
+    if (lane == 0) {
+        p.loss[row] = loss;
+        p.lse_d[row] = lse_d;
+        p.coef_out[row] = g * scale;
+    }
+    if (g != 0.f && scale > 0.f && scale < INFINITY) {
+        const float inv = 1.f / scale;
+        __nv_bfloat16* prow = p.P + static_cast<long long>(local) * p.p_pitch;
+        for (int j = lane; j < K; j += 32) {
+            const int tok = p.sidx[ro + j];
+            if (tok != INT_MAX) prow[tok] = __float2bfloat16_rn(__bfloat162float(prow[tok]) - p.sq[ro + j] * inv);
+        }
     }
 }
 
