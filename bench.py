@@ -32,11 +32,13 @@ import hass_inputs as hi  # noqa: E402
 
 METRIC = "tokens/sec fused top-K distill fwd+bwd"
 UNIT = "tokens/s"
-# dram__bytes_read + dram__bytes_write of the dominant kernel (the logits sweep) per launch, from the ncu
-# capture summarised in profiles/gemm_kernel_l2-7b_ncu_full.md (l2-7b shape, mean of the two chunk launches),
-# scaled to the bench shape by the vocabulary ratio; valid for the library version it was taken with (10200 added
-# the HCA attention entries and left the kernels of this path as captured).
-TRAFFIC_CAPTURE = {"version": 10200, "workload": "l3-8b", "bytes_per_launch": 0.965e9 * 128256 / 32000}
+# dram__bytes_read + dram__bytes_write per launch of the three GEMM kernels of the fused call, from the ncu
+# captures summarised in profiles/gemm_kernels_l2-7b_ncu_full.md (l2-7b shape, K = 10; mean of the two row-chunk
+# launches of one step). Valid for the library version they were taken with; for the l3-8b shape the figures
+# are scaled by the vocabulary ratio (W, the spill and its re-reads all grow with V; the 2 x 39 MB of H rows
+# and the dH_d rows that do not are 6 % of the total).
+TRAFFIC_CAPTURE = {"version": 10300, "workload": "l2-7b", "V": 32000, "K": 10,
+                   "bytes_per_launch": {"stats_gemm": 494.0e6, "stats_gemm_draft": 755.4e6, "dH_gemm": 1211.9e6}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -378,16 +380,25 @@ def main_hca(args):
     flops = products[dom] * prod
     achieved = flops / (ms_k / cnt * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
+    # the attention itself needs 2 products forward and 5 backward; the two backward kernels execute 7
+    algorithmic = (7 if bwd else 2) * prod
+    executed = (9 if bwd else 2) * prod
     line = {"metric": metric, "value": aggregate(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": dict(config, l2="inputs and output (%.0f MB) larger than L2" % ((in_bytes + inp.Q.numel() * 2) / 1e6)),
             "clocks": clocks, "gpu_launches": launches,
+            "tensor": {"algorithmic_flops_per_step": algorithmic, "executed_flops_per_step": executed,
+                       "algorithmic_tflops": algorithmic / (ms_step * 1e-3) / 1e12,
+                       "executed_tflops": executed / (ms_step * 1e-3) / 1e12,
+                       "frac_of_burst_algorithmic": algorithmic / (ms_step * 1e-3) / 1e12 / peak,
+                       "frac_of_burst_executed": executed / (ms_step * 1e-3) / 1e12 / peak, "peaks": peak_kind},
             "kernels": kernel_rows,
             "roofline": {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
                          "peak_kind": f"bf16_tflops (burst), of {peak_kind} (a sub-millisecond kernel timed alone)",
-                         "flops_per_launch": flops, "avg_launch_ms": ms_k / cnt}}
+                         "flops_per_launch": flops, "avg_launch_ms": ms_k / cnt,
+                         "note": "achieved counts the products this kernel executes; see tensor.* for the step"}}
     if e2e:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
@@ -570,15 +581,29 @@ def main():
     dom_ms, dom_cnt = prof[dom]
     flops_per_launch = kinds[dom] * args.steps / dom_cnt
     achieved = flops_per_launch / (dom_ms / dom_cnt * 1e-3) / 1e12
-    peak = float(peaks["bf16_tflops_sustained"])
+    # a timed region under a second never settles at the power cap: compare it with the burst figure
+    timed_s = ms_step * args.steps * 1e-3
+    peak_key = "bf16_tflops_sustained" if timed_s >= 1.0 else "bf16_tflops"
+    peak = float(peaks[peak_key])
+    traffic, traffic_note = None, "no capture for this kernel, objective, shape or library version"
+    cap = TRAFFIC_CAPTURE
+    if (args.objective == "topk" and hass.version() == cap["version"] and dom in cap["bytes_per_launch"]
+            and wl.name in ("l2-7b", "l3-8b") and K <= 16):
+        traffic = cap["bytes_per_launch"][dom] * V / cap["V"]
+        traffic_note = ("ncu dram bytes of this kernel captured on %s (K = %d), mean of the step's two launches"
+                        % (cap["workload"], cap["K"]) + ("" if wl.name == cap["workload"] else
+                                                         ", scaled by the vocabulary ratio %d / %d" % (V, cap["V"])))
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak,
-                "traffic": (TRAFFIC_CAPTURE["bytes_per_launch"]
-                            if dom == "stats_gemm" and args.objective == "topk" and wl.name == TRAFFIC_CAPTURE["workload"]
-                            and hass.version() == TRAFFIC_CAPTURE["version"] else None),
-                "peak_kind": f"bf16_tflops_sustained, of {peak_kind} (kernel timed inside a long step)",
+                "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
+                "peak_kind": "%s, of %s (timed region %.2f s: %s)" % (
+                    peak_key, peak_kind, timed_s,
+                    "long enough to sit at the power cap" if timed_s >= 1.0 else "too short to reach the power cap"),
                 "frac_of_burst": achieved / float(peaks["bf16_tflops"]),
+                "frac_of_sustained": achieved / float(peaks["bf16_tflops_sustained"]),
                 "flops_per_launch": flops_per_launch, "avg_launch_ms": dom_ms / dom_cnt}
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    chunk_rows = min(max(sms // 4, 1) * 128, (N + 127) // 128 * 128)     # the library's chunk: #SM / 4 row tiles
+    V_pad = (V + 255) // 256 * 256
     step_tflops = flops_credit / (ms_step * 1e-3) / 1e12
     executed = sum(f for k, f in kinds.items() if prof[k][1] > 0)
 
@@ -588,6 +613,9 @@ def main():
             "config": {"workload": wl.name, "N": N, "d": d, "V": V, "K": K, "rows_per_gpu": N,
                        "l2": "inputs larger than L2 (W alone is %.0f MB)" % (V * d * 2 / 1e6),
                        "dH_dtype": "bf16", "aligning_steps": wl.steps, "objective": args.objective,
+                       "spill_scratch": "un-normalised bf16 draft probabilities of one chunk of %d rows x %d tokens "
+                                        "= %.0f MB live at a time (the N x V matrix would be %.0f MB)" % (
+                                            chunk_rows, V_pad, chunk_rows * V_pad * 2 / 1e6, N * V * 2 / 1e6),
                        "target_stats": ("recomputed every step" if wl.steps == 1 else
                                         "computed in aligning step 1, reused in steps 2..%d" % wl.steps),
                        "path": {"combined": "hass_combined_distill_fwd_bwd", "top_p": "hass_variant_distill_fwd_bwd (Top-P)",

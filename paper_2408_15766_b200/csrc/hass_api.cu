@@ -1070,7 +1070,7 @@ const char* hass_status_string(int status) {
     }
 }
 
-int hass_version(void) { return 10200; }
+int hass_version(void) { return 10300; }
 
 int64_t hass_kernel_launch_count(void) { return g_launches.load(); }
 
