@@ -457,7 +457,10 @@ def main():
     import paper_2408_15766_b200 as hass   # fails loudly if the CUDA library is missing
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
     wl = hi.WORKLOADS[args.workload]
-    K = args.K or wl.K
+    # Top-P: on these near-uniform synthetic rows (largest q about 2e-3) P = 0.01 gives prefixes of a handful of
+    # tokens, well inside the cap of K = 64 tokens, so the variant does not degenerate into plain Top-K
+    TOP_P = 0.01
+    K = args.K or (64 if args.objective == "top_p" else wl.K)
     dev = torch.device(f"cuda:{local}")
     torch.cuda.set_device(dev)
     peaks, peak_kind = load_peaks()
@@ -482,6 +485,7 @@ def main():
     stream = torch.cuda.current_stream()
 
     counts = {"full": 0, "draft": 0, "i": 0}
+    var_out = {}          # outputs of the latest variant call
 
     def step():
         # Aligning step j of harmonized context alignment: step 1 computes the target side too, steps >= 2
@@ -494,8 +498,8 @@ def main():
         elif args.objective in ("top_p", "normed", "bidir"):
             counts["full"] += 1
             variant = {"top_p": hass.LOSS_TOP_P, "normed": hass.LOSS_NORMED_TOPK, "bidir": hass.LOSS_BIDIR_TOPK}
-            hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, variant[args.objective], 0.5, workspace=ws,
-                                         stream=stream)
+            var_out.update(hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, variant[args.objective], TOP_P,
+                                                        workspace=ws, stream=stream))
         elif j == 0:
             counts["full"] += 1
             hass.topk_distill_fwd_bwd(H_t, H_d_steps[0], W, K, workspace=ws, out=out, stream=stream)
@@ -613,6 +617,8 @@ def main():
             "config": {"workload": wl.name, "N": N, "d": d, "V": V, "K": K, "rows_per_gpu": N,
                        "l2": "inputs larger than L2 (W alone is %.0f MB)" % (V * d * 2 / 1e6),
                        "dH_dtype": "bf16", "aligning_steps": wl.steps, "objective": args.objective,
+                       **({"top_p": TOP_P, "prefix_tokens_mean": float(var_out["topk_n"].abs().float().mean()),
+                           "rows_cut_by_the_cap": int((var_out["topk_n"] < 0).sum())} if args.objective == "top_p" else {}),
                        "spill_scratch": "un-normalised bf16 draft probabilities of one chunk of %d rows x %d tokens "
                                         "= %.0f MB live at a time (the N x V matrix would be %.0f MB)" % (
                                             chunk_rows, V_pad, chunk_rows * V_pad * 2 / 1e6, N * V * 2 / 1e6),

@@ -3,7 +3,11 @@
  *
  * The library computes, for N rows of target features H_t and draft features H_d and the
  * frozen LM head W that both share, the Top-K distillation loss of HASS and its gradient
- * with respect to H_d, without ever holding an N x V logit matrix in memory.
+ * with respect to H_d. No N x V logit matrix is ever held in memory: logits exist tile by tile in
+ * tensor memory. What does pass through the workspace, between the forward sweep and the
+ * back-projection of the fused call, is a bounded chunk of un-normalised bf16 draft probabilities
+ * (chunk rows x V, chunk rows = 128 x a quarter of the SM count, 4736 on a 148-SM device whatever
+ * N is: 1.2 GB for V = 128256); see hass_topk_distill_fwd_bwd.
  *
  * Notation follows the paper (Section 3.1): q = softmax(H_t W^T) is the target LLM's
  * next-token distribution, p = softmax(H_d W^T) the draft model's, Omega the vocabulary
@@ -129,19 +133,25 @@ int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, 
 /*
  * Forward and backward in one call (the whole hot path of one aligning step): the same results as
  * hass_topk_distill_fwd followed by hass_topk_distill_bwd, up to rounding, but no logit is
- * computed twice. Rows are processed in bounded chunks; while a chunk's draft logits are swept
- * for the forward statistics they are also written to the workspace as bf16 values
+ * computed twice and no row of W is gathered. Rows are processed in bounded chunks. Per chunk the
+ * target rows are swept first (statistics and Top-K candidates), Omega_hat is selected, then the
+ * draft rows are swept: their statistics, their logits at the row's Omega_hat (copied out of the
+ * fp32 accumulator for Eq. 1), and the tile itself, written to the workspace as bf16 values
  * 2^(z_d log2(e) - ref2), ref2 a per-row exponent fixed from the row's largest logit among the
- * first 256 tokens, and dH_d = coef (spill W) - sum_{x in Omega_hat} g q(x) W[x,:] is formed by
- * the second GEMM, whose epilogue applies the per-row scale coef = g S_q 2^ref2 / sum_v e^{z_d}
- * and the sparse term.
+ * first 256 tokens. With coef = g S_q 2^ref2 / sum_v e^{z_d},
+ *     dz_d(v) = coef ( spill(v) - [v in Omega_hat] g q(v) / coef ),
+ * so the K entries of a row at its Omega_hat tokens are lowered in place (in bf16) and
+ * dH_d = coef (spill W) is formed by the second GEMM, whose epilogue applies the row scale.
+ * Precision: every entry of dz_d, the Omega_hat entries included, reaches the tensor cores in bf16
+ * (2^-9 relative); the loss uses fp32 logits throughout.
  * Range condition: the fixed exponent holds as long as no draft logit of a row exceeds that
  * row's largest logit among tokens 0..255 by more than about 130 (natural-log units; a probability
  * ratio of e^130). The sweep detects a violation; the call therefore also enqueues the separate
  * forward and the recomputing backward as conditional launches that return at once unless a
  * violation was detected, in which case they redo the whole call exactly. The result is correct
- * either way; the conditional launches cost about 0.1 % when they have nothing to do.
- * (hass_combined_distill_fwd_bwd and the Top-P / Bi-directional variants have no such second route:
+ * either way; the conditional launches cost about 0.3 % when they have nothing to do. The _draft
+ * form and the Top-P variant work the same way.
+ * (hass_combined_distill_fwd_bwd and the Bi-directional variant have no such second route:
  * there hass_check reports HASS_ERR_RANGE and loss, lse_d and dH_d are invalid.)
  */
 int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
@@ -202,7 +212,9 @@ int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* 
  *                          topk_idx / topk_q must hold 2K entries per row: the target's K in descending q,
  *                          then the draft's tokens not among them in descending p, then -1 / 0. K <= 64.
  *
- * topk_n [N] (nullable) receives |Omega_hat| per row. The other arguments are those of
+ * topk_n [N] (nullable) receives |Omega_hat| per row; for HASS_LOSS_TOP_P the count is negated (-K) on a row
+ * whose K most probable tokens together still do not exceed P, i.e. whose prefix was cut by the cap of K
+ * tokens rather than by P (K may be as large as HASS_K_MAX). The other arguments are those of
  * hass_topk_distill_fwd_bwd. The Recall@k surrogate and BiLD losses of that section are not built (the
  * paper does not define them).
  */

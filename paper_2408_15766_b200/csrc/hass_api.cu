@@ -316,7 +316,8 @@ static int launch_gemm(const GemmParams& p, cudaStream_t st, int kind = -1) {
 static int forward_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
                         long long V, int K, const int* idx_in, const float* q_in, float* loss, int* idx_out,
                         float* q_out, float* lse_t, float* lse_d, void* workspace, size_t workspace_bytes,
-                        cudaStream_t st, const unsigned int* only_if_range = nullptr) {
+                        cudaStream_t st, const unsigned int* only_if_range = nullptr, float top_p = 0.f,
+                        int* topk_n = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !aligned16(H_d) || !aligned16(W)) return HASS_ERR_INVALID_ARG;
@@ -408,6 +409,8 @@ static int forward_impl(bool with_target, const void* H_t, const void* H_d, cons
     f.lse_t = lse_t;
     f.lse_d = lse_d;
     f.only_if_range = only_if_range;
+    f.top_p = top_p;
+    f.n_out = topk_n;
     const int warps_per_block = 8;
     {
         KernelTimer timer(only_if_range ? KIND_CONDITIONAL : KIND_FINALIZE, st);
@@ -939,12 +942,12 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
     }
-    if (!(top_p > 0.f)) {
-        // Exact route, enqueued behind every plain fused call: if a sweep reported a row beyond its exponent
+    {
+        // Exact route, enqueued behind every call of this route: if a sweep reported a row beyond its exponent
         // range, the separate forward and the recomputing backward (which have no such limit) redo the call
         // and the report is withdrawn; otherwise each of these launches returns at once.
         rc = forward_impl(with_target, H_t, H_d, W, N, d, V, K, idx_in, q_in, loss, idx_out, q_out, lse_t, lse_d,
-                          workspace, workspace_bytes, st, status);
+                          workspace, workspace_bytes, st, status, top_p, topk_n);
         if (rc != HASS_OK) return rc;
         rc = backward_impl(H_d, W, N, d, V, K, with_target ? idx_out : idx_in, with_target ? q_out : q_in, lse_d,
                            grad_loss, dH_d, dH_dtype, workspace, workspace_bytes, st, false, status);

@@ -1084,7 +1084,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
             }
         }
     }
-    if (lane == 0 && p.n_out) p.n_out[row] = n_sel;
+    if (lane == 0 && p.n_out) p.n_out[row] = (p.top_p > 0.f && !(cum_q > p.top_p)) ? -n_sel : n_sel;
     if (p.normed) {
         // Normed Top-K: qn = q / S_q, pn = softmax of the draft logits restricted to Omega_hat
         __syncwarp();
@@ -1312,6 +1312,7 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) select_kernel(const __grid_con
                     }
                     cum += sel_q[wib][j];
                 }
+                if (!(cum > p.top_p)) n = -n;      // all K tokens taken and P still not exceeded: the cap cut the prefix
             }
             __syncwarp();
             n_sel = __shfl_sync(0xffffffffu, n, 0);

@@ -102,6 +102,13 @@ def compare_variant(H_t, H_d, W, K, variant, param, gpu: dict, rows=None, grad_l
     ref = oracle.variant_from_features(Hb_t, Hb_d, Wb, K, variant, param, rows=rows, grad_loss=gl)
     g = {k: _np(v) for k, v in gpu.items() if v is not None and k != "workspace"}
     g_idx, g_n = g["topk_idx"][rows], g["topk_n"][rows]
+    if top_p:
+        # Top-P: a negative count marks a row whose prefix took all K tokens without exceeding P
+        cut = g_n < 0
+        g_n = np.abs(g_n)
+        tot = ref["q_k"].sum(1)
+        assert np.all(g_n[cut] == K) and np.all(tot[cut] <= param + 1e-5), "cap flag on a row that reached P"
+        assert np.all(tot[(~cut) & (g_n == K)] > param - 1e-5), "a row cut by the cap is not flagged"
     kk = g_idx.shape[1]
     assert kk == ref["idx"].shape[1]
     assert g_idx.max() < V and np.all((g_idx >= 0) == (np.arange(kk)[None, :] < g_n[:, None])), "padding / count mismatch"

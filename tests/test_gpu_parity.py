@@ -180,8 +180,14 @@ def test_rows_beyond_the_exponent_range_of_the_spill_are_redone_exactly():
                                          dH_dtype=hass.HASS_FP32, workspace=out["workspace"])
     hass.check(out["workspace"])
     assert torch.allclose(d2["loss"], out["loss"], rtol=1e-5) and torch.allclose(d2["dH_d"], out["dH_d"], atol=1e-6)
-    # the variants without a second route report it
-    v = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, hass.LOSS_TOP_P, 0.5)
+    # the Top-P variant has the same second route ...
+    import oracle
+    v = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, hass.LOSS_TOP_P, 0.004,
+                                     dH_dtype=hass.HASS_FP32)
+    hass.check(v["workspace"])
+    print("top-p, exact route", compare_variant(inp.H_t, H_d, W, K, oracle.VARIANT_TOP_P, 0.004, _to_cpu(v)))
+    # ... the Bi-directional variant has none and reports the range
+    v = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, hass.LOSS_BIDIR_TOPK, 0.0)
     with pytest.raises(hass.HassError) as e:
         hass.check(v["workspace"])
     assert e.value.status == -7 and hass.status_string(-7) == "HASS_ERR_RANGE"
@@ -417,9 +423,26 @@ def test_top_p_variant_matches_oracle(N, d, V, K, P):
     import oracle
     inp = hi.make_custom(N, d, V, K, seed=N + K + 2, sigma_w=2.0 / np.sqrt(d))
     cpu = _run_variant(inp, K, _hass().LOSS_TOP_P, P)
-    n_gpu = cpu["topk_n"].numpy()
+    n_gpu = np.abs(cpu["topk_n"].numpy())
     assert n_gpu.min() >= 1 and n_gpu.max() <= K and len(np.unique(n_gpu)) > 1
     print("top-p", compare_variant(inp.H_t, inp.H_d[0], inp.W, K, oracle.VARIANT_TOP_P, P, cpu))
+
+
+def test_top_p_reports_rows_whose_prefix_was_cut_by_the_cap():
+    """With K = 4 and P = 0.9 on near-uniform rows no prefix of 4 tokens reaches P: topk_n = -4 on those rows;
+    a peaked row (one dominant token) reaches P with its first token: topk_n = 1."""
+    import oracle
+    N, d, V, K, P = 96, 64, 900, 4, 0.9
+    inp = hi.make_custom(N, d, V, K, seed=11, sigma_w=0.05)
+    H_t = inp.H_t.clone()
+    u = torch.where(torch.rand(d, generator=torch.Generator().manual_seed(5)) < 0.5, -1.0, 1.0)
+    W = inp.W.clone()
+    W[123] = (0.25 * u).to(torch.bfloat16)
+    H_t[::3] = (2.0 * u).to(torch.bfloat16)            # z_t[123] = 64 * 0.25 * 2 = 32 on every third row: q(123) ~ 1
+    cpu = _run_variant(hi.Inputs(inp.wl, H_t, inp.H_d, W), K, _hass().LOSS_TOP_P, P)
+    n = cpu["topk_n"].numpy()
+    assert np.all(n[::3] == 1) and np.all(np.delete(n, np.arange(0, N, 3)) == -K)
+    print("top-p cap", compare_variant(H_t, inp.H_d[0], W, K, oracle.VARIANT_TOP_P, P, cpu))
 
 
 @pytest.mark.parametrize("N,d,V,K", [(64, 256, 1024, 10), (300, 128, 5000, 24), (4800, 64, 700, 6)])
