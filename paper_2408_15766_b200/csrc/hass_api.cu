@@ -11,6 +11,7 @@
 #include "../../include/hass.h"
 #include "kernels.cuh"
 #include "hca_kernels.cuh"
+#include "hca_pair_kernel.cuh"
 #include "hca_bwd_kernels.cuh"
 
 namespace hass {
@@ -78,6 +79,7 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
             // two CTAs of this kernel share an SM: ask for the largest shared-memory carve-out
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca2::hca_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca2::SMEM_BYTES);
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::DQ_SMEM_BYTES);
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::KV_SMEM_BYTES);
             if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
@@ -1435,6 +1437,47 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
     if (rc != HASS_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
+    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    static const bool old_kernel = [] {
+        const char* e = std::getenv("HASS_HCA_OLD");
+        return e && e[0] == '1';
+    }();
+    if (!old_kernel) {
+        hca2::Params p;
+        std::memset(&p, 0, sizeof(p));
+        rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca2::HD, hca2::QT);
+        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca2::HD, hca2::KT);
+        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca2::HD, hca2::KT);
+        for (int i = 0; i < m && rc == HASS_OK; ++i) {
+            rc = make_tmap_seq(&p.tmKd[i], K_d[i], B, T, Hkv * hca2::HD, hca2::KT);
+            if (rc == HASS_OK) rc = make_tmap_seq(&p.tmVd[i], V_d[i], B, T, Hkv * hca2::HD, hca2::KT);
+        }
+        if (rc != HASS_OK) return rc;
+        p.O = static_cast<__nv_bfloat16*>(O);
+        p.lse = lse;
+        p.B = static_cast<int>(B);
+        p.T = static_cast<int>(T);
+        p.H = static_cast<int>(H);
+        p.Hkv = static_cast<int>(Hkv);
+        p.m = m;
+        p.q_tiles = static_cast<int>((T + hca2::QT - 1) / hca2::QT);
+        // two query heads of one key/value group per CTA when the group size is even, else two query tiles of one head
+        p.head_pairing = ((H / Hkv) % 2 == 0) ? 1 : 0;
+        p.pairs = p.head_pairing ? static_cast<int>(B * (H / 2)) * p.q_tiles : static_cast<int>(B * H) * ((p.q_tiles + 1) / 2);
+        p.c2 = scale * 1.4426950408889634f;
+        p.status = static_cast<unsigned int*>(workspace);
+        const int grid = p.pairs < di.sms ? p.pairs : di.sms;
+        {
+            KernelTimer kt(KIND_HCA, st);
+            hca2::hca_attention_pair_kernel<<<grid, hca2::NUM_THREADS, hca2::SMEM_BYTES, st>>>(p);
+        }
+        g_launches.fetch_add(1);
+        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+        return HASS_OK;
+    }
     hca::Params p;
     std::memset(&p, 0, sizeof(p));
     rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca::HD, hca::QT);
@@ -1457,10 +1500,6 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
     p.items = static_cast<int>(B * H) * p.q_tiles;
     p.c2 = scale * 1.4426950408889634f;
     p.status = static_cast<unsigned int*>(workspace);
-    if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
-        cudaGetLastError();
-        return HASS_ERR_CUDA;
-    }
     const int grid = p.items < 2 * di.sms ? p.items : 2 * di.sms;      // two CTAs per SM
     {
         KernelTimer kt(KIND_HCA, st);
