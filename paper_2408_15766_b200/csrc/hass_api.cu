@@ -76,10 +76,7 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e2 = cudaFuncSetAttribute(gemm_kernel<MODE_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_NONE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-            cudaError_t e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca::SMEM_BYTES);
-            // two CTAs of this kernel share an SM: ask for the largest shared-memory carve-out
-            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca::hca_attention_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca2::hca_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca2::SMEM_BYTES);
+            cudaError_t e4 = cudaFuncSetAttribute(hca2::hca_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca2::SMEM_BYTES);
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::DQ_SMEM_BYTES);
             if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::KV_SMEM_BYTES);
             if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
@@ -1441,11 +1438,7 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
         cudaGetLastError();
         return HASS_ERR_CUDA;
     }
-    static const bool old_kernel = [] {
-        const char* e = std::getenv("HASS_HCA_OLD");
-        return e && e[0] == '1';
-    }();
-    if (!old_kernel) {
+    {
         hca2::Params p;
         std::memset(&p, 0, sizeof(p));
         rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca2::HD, hca2::QT);
@@ -1478,36 +1471,6 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
         if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
         return HASS_OK;
     }
-    hca::Params p;
-    std::memset(&p, 0, sizeof(p));
-    rc = make_tmap_seq(&p.tmQ, Q, B, T, H * hca::HD, hca::QT);
-    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmK, K_t, B, T, Hkv * hca::HD, hca::KT);
-    if (rc == HASS_OK) rc = make_tmap_seq(&p.tmV, V_t, B, T, Hkv * hca::HD, hca::KT);
-    for (int i = 0; i < m && rc == HASS_OK; ++i) {
-        rc = make_tmap_seq(&p.tmKd[i], K_d[i], B, T, Hkv * hca::HD, hca::KT);
-        if (rc == HASS_OK) rc = make_tmap_seq(&p.tmVd[i], V_d[i], B, T, Hkv * hca::HD, hca::KT);
-    }
-    if (rc != HASS_OK) return rc;
-    p.O = static_cast<__nv_bfloat16*>(O);
-    p.lse = lse;
-    p.B = static_cast<int>(B);
-    p.T = static_cast<int>(T);
-    p.H = static_cast<int>(H);
-    p.Hkv = static_cast<int>(Hkv);
-    p.m = m;
-    p.q_tiles = static_cast<int>((T + hca::QT - 1) / hca::QT);
-    p.k_tiles = static_cast<int>((T + hca::KT - 1) / hca::KT);
-    p.items = static_cast<int>(B * H) * p.q_tiles;
-    p.c2 = scale * 1.4426950408889634f;
-    p.status = static_cast<unsigned int*>(workspace);
-    const int grid = p.items < 2 * di.sms ? p.items : 2 * di.sms;      // two CTAs per SM
-    {
-        KernelTimer kt(KIND_HCA, st);
-        hca::hca_attention_kernel<<<grid, hca::NUM_THREADS, hca::SMEM_BYTES, st>>>(p);
-    }
-    g_launches.fetch_add(1);
-    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
-    return HASS_OK;
 }
 
 // workspace of the HCA backward: status word, D [B, H, T], and the weights and dS of the substituted entries

@@ -57,7 +57,8 @@ constexpr int SMEM_Q = 0;                            // 2 slots
 constexpr int SMEM_K = SMEM_Q + 2 * Q_BYTES;
 constexpr int SMEM_V = SMEM_K + KV_STAGES * KV_BYTES;
 constexpr int SMEM_BAR = SMEM_V + KV_STAGES * KV_BYTES;
-constexpr int NUM_BARS = 4 + 4 * KV_STAGES + 6;
+constexpr int SCHED_DEPTH = 4;       // pair indices published ahead by the producer
+constexpr int NUM_BARS = 4 + 4 * KV_STAGES + 6 + 2 * SCHED_DEPTH;
 constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 196864
 constexpr int TMEM_COLS = 512;     // S of slot s at 128 s (P overwrites its first 64 columns), O of slot s at 256 + 128 s
 constexpr float RESCALE_LOG2 = 8.f;
@@ -126,8 +127,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
     auto s_full = [&](int s) { return bar0 + 8u * (4 + 4 * KV_STAGES + s); };
     auto p_full = [&](int s) { return bar0 + 8u * (6 + 4 * KV_STAGES + s); };
     auto pv_done = [&](int s) { return bar0 + 8u * (8 + 4 * KV_STAGES + s); };
+    auto sched_full = [&](int e) { return bar0 + 8u * (10 + 4 * KV_STAGES + e); };
+    auto sched_empty = [&](int e) { return bar0 + 8u * (10 + 4 * KV_STAGES + SCHED_DEPTH + e); };
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_raw + SMEM_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
+    volatile int* sched_idx = reinterpret_cast<volatile int*>(tmem_ptr_smem + 2);      // [SCHED_DEPTH]
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -146,6 +150,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             mbar_init(v_full(st), 1);
             mbar_init(v_empty(st), 1);
         }
+        for (int e = 0; e < SCHED_DEPTH; ++e) {
+            mbar_init(sched_full(e), 1);
+            mbar_init(sched_empty(e), 9);      // the MMA warp and the eight softmax warps
+        }
         *abort_flag = 0;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -162,11 +170,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
 
-    // Pairs are sorted longest first; round k hands pairs k*G .. k*G + G-1 to the G CTAs, in alternating
-    // direction, so that a CTA that got a long pair in one round gets a short one in the next.
-    auto pair_of_round = [&](uint32_t k) {
-        const int G = gridDim.x, c = blockIdx.x;
-        return static_cast<int>(k) * G + ((k & 1u) ? G - 1 - c : c);
+    // Pairs are sorted longest first and handed out dynamically: the producer takes the next index from a counter in
+    // the workspace (word 1, zeroed by the host before the launch) and publishes it to the other roles through a
+    // small queue in shared memory, so a CTA that falls behind simply takes fewer pairs. An index >= pairs ends a role.
+    // next_pair(k): the k-th index this CTA works on (every consumer warp calls it once per k).
+    auto next_pair = [&](uint32_t k, unsigned code) -> int {
+        const int e = k % SCHED_DEPTH;
+        if (!wait_barrier(sched_full(e), (k / SCHED_DEPTH) & 1u, abort_flag, p.status, code)) return INT_MAX;
+        const int idx = sched_idx[e];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sched_empty(e));
+        return idx;
     };
 
     // Per item and slot the tensor core runs, in this order:
@@ -174,7 +188,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
     //                            scores <Q[t], K_d[i][t - i]> sit on the tile's diagonal; the row's thread keeps its own
     //   n key tiles              S = Q K_t^T -> softmax -> O += P V_t
     //   m draft value products   O += diag(p_i) V_d[i] (V_d[i] fetched i rows early; P holds the row's weight on
-    //                            the diagonal and zeros elsewhere)
+    //                            the diagonal and zeros elsewhere), two passes per arrival of the softmax warps
     // Every product of a slot but the first S follows an arrival of the slot's softmax warps on p_full.
     // The K ring carries the draft key tiles, then the key tiles; the V ring the value tiles, then the draft
     // value tiles. A tile both slots use (always, when the pair is two heads of one group; the key/value
@@ -204,7 +218,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
                 ++gv;
                 return true;
             };
-            for (int idx = pair_of_round(0); idx < p.pairs && ok; idx = pair_of_round(++it)) {
+            for (;; ++it) {
+                const int idx = static_cast<int>(atomicAdd(p.status + 1, 1u));
+                {
+                    const int e = it % SCHED_DEPTH;
+                    if (!wait_barrier(sched_empty(e), ((it / SCHED_DEPTH) & 1u) ^ 1u, abort_flag, p.status, 15)) break;
+                    sched_idx[e] = idx;
+                    mbar_arrive(sched_full(e));
+                }
+                if (idx >= p.pairs || !ok) break;
                 const Pair pr = decode_pair(p, idx);
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
@@ -259,17 +281,17 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             }
             __syncwarp();
         };
-        // O of slot s (+)= P V from V stage st
-        auto issue_pv = [&](int s, int st, bool first) {
+        // O of slot s (+)= P V: keys [16 k0, 16 k1) of V stage st, P read from the slot's S buffer starting at column
+        // a_col (8 columns of bf16 pairs per 16 keys). B = V: 64-column groups KV_HALF apart, 16 keys further = 16
+        // rows of 128 bytes. first: the item's first product into O; commit: signal pv_done afterwards.
+        auto issue_pv = [&](int s, int st, int a_col, int k0, int k1, bool first, bool commit) {
             tc_fence_after_sync();
 #pragma unroll
-            for (int k = 0; k < KT / 16; ++k) {
-                // A = P from tensor memory (8 columns of bf16 pairs per 16 keys). B = V: 64-column groups KV_HALF
-                // apart, 16 keys further = 16 rows of 128 bytes.
+            for (int k = k0; k < k1; ++k) {
                 const uint64_t b_desc = make_smem_desc_sw128(base + SMEM_V + st * KV_BYTES + k * 16 * 128, KV_HALF, 1024);
-                if (leader) umma_bf16_ta(tmem_base + 256 + s * HD, tmem_base + s * KT + 8 * k, b_desc, idesc_o, (!first || k != 0) ? 1u : 0u);
+                if (leader) umma_bf16_ta(tmem_base + 256 + s * HD, tmem_base + s * KT + a_col + 8 * (k - k0), b_desc, idesc_o, (!first || k != k0) ? 1u : 0u);
             }
-            if (leader) umma_commit(pv_done(s));
+            if (leader && commit) umma_commit(pv_done(s));
             __syncwarp();
         };
         auto k_acquire = [&](int& st) {
@@ -295,7 +317,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             ++gp[s];
             return r;
         };
-        for (int idx = pair_of_round(0); idx < p.pairs && ok; idx = pair_of_round(++it)) {
+
+        for (int idx = next_pair(0, 16); idx < p.pairs && ok; idx = next_pair(++it, 16)) {
             const Pair pr = decode_pair(p, idx);
             const int m = p.m;
             const int n1 = pr.qt[1] + 1;
@@ -362,7 +385,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
                 bool k_ready = false;
                 if (j < n0) {
                     if (!p_wait(0)) { ok = false; break; }
-                    issue_pv(0, vst, j == 0);
+                    issue_pv(0, vst, 0, 0, 8, j == 0, true);
                     if (j + 1 < n0) {
                         if (!k_acquire(st)) { ok = false; break; }
                         k_ready = true;
@@ -370,7 +393,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
                     }
                 }
                 if (!p_wait(1)) { ok = false; break; }
-                issue_pv(1, vst, j == 0);
+                issue_pv(1, vst, 0, 0, 8, j == 0, true);
                 v_release(vst);
                 if (j + 1 < n1) {
                     if (!k_ready && !k_acquire(st)) { ok = false; break; }
@@ -378,29 +401,38 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
                     k_release(st);
                 }
             }
-            // ---- draft value steps ----
-            for (int i = 0; i < m && ok; ++i) {
-                int vst;
-                if (shared) {
-                    if (!v_acquire(vst)) { ok = false; break; }
-                    if (a_on) {
-                        if (!p_wait(0)) { ok = false; break; }
-                        issue_pv(0, vst, false);
-                    }
-                    if (!p_wait(1)) { ok = false; break; }
-                    issue_pv(1, vst, false);
-                    v_release(vst);
-                } else {
-                    if (a_on) {
+            // ---- draft value rounds: two passes per arrival (their weights sit in the two halves of the S buffer) ----
+            for (int i0 = 0; i0 < m && ok; i0 += 2) {
+                const bool two = i0 + 1 < m;
+                bool waited0 = false, waited1 = false;
+                for (int e = 0; e < (two ? 2 : 1) && ok; ++e) {
+                    const bool fin = (e == 1) || !two;          // the slot's last product of the round
+                    int vst;
+                    if (shared) {
                         if (!v_acquire(vst)) { ok = false; break; }
-                        if (!p_wait(0)) { ok = false; break; }
-                        issue_pv(0, vst, false);
+                        if (a_on) {
+                            if (!waited0 && !p_wait(0)) { ok = false; break; }
+                            waited0 = true;
+                            issue_pv(0, vst, 64 * e, 0, 8, false, fin);
+                        }
+                        if (!waited1 && !p_wait(1)) { ok = false; break; }
+                        waited1 = true;
+                        issue_pv(1, vst, 64 * e, 0, 8, false, fin);
+                        v_release(vst);
+                    } else {
+                        if (a_on) {
+                            if (!v_acquire(vst)) { ok = false; break; }
+                            if (!waited0 && !p_wait(0)) { ok = false; break; }
+                            waited0 = true;
+                            issue_pv(0, vst, 64 * e, 0, 8, false, fin);
+                            v_release(vst);
+                        }
+                        if (!v_acquire(vst)) { ok = false; break; }
+                        if (!waited1 && !p_wait(1)) { ok = false; break; }
+                        waited1 = true;
+                        issue_pv(1, vst, 64 * e, 0, 8, false, fin);
                         v_release(vst);
                     }
-                    if (!v_acquire(vst)) { ok = false; break; }
-                    if (!p_wait(1)) { ok = false; break; }
-                    issue_pv(1, vst, false);
-                    v_release(vst);
                 }
             }
         }
@@ -417,7 +449,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
         const int m = p.m;
         uint32_t gs = 0, gpv = 0, it = 0;                     // S-type products seen, PV-type products requested
         bool ok = true;
-        for (int idx = pair_of_round(0); idx < p.pairs && ok; idx = pair_of_round(++it)) {
+        for (int idx = next_pair(0, 17); idx < p.pairs && ok; idx = next_pair(++it, 17)) {
             const Pair pr = decode_pair(p, idx);
             if (slot == 0 && !pr.act0) continue;
             const int qt = pr.qt[slot], h = pr.h[slot], b = pr.b;
@@ -539,25 +571,30 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
                 ++gpv;
             }
             if (!ok) break;
-            // ---- draft value steps: P holds only the weight 2^(sd c2 - ref) of each row, on the diagonal ----
+            // ---- draft value rounds: two passes at a time; P holds only the weight 2^(sd c2 - ref) of each row, on the
+            //      diagonal: pass i0 in the first 64 columns of the S buffer, pass i0 + 1 in the last 64 ----
             const float nref_f = mref == -INFINITY ? 0.f : -mref;
 #pragma unroll 1
-            for (int i = 0; i < m; ++i) {
-                float sdi = 0.f;
-#pragma unroll
-                for (int ii = 0; ii < MAX_DRAFTS; ++ii)
-                    if (ii == i) sdi = sd[ii];
-                const float pi = (t - i >= 0) ? ex2(fmaf(sdi, p.c2, nref_f)) : 0.f;
-                const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // key r sits in word r / 2
-                // the product that last read P must be complete before P is overwritten
+            for (int i0 = 0; i0 < m; i0 += 2) {
+                // the products that last read these columns must be complete before they are overwritten
                 if (!wait_barrier(pv_done(slot), (gpv - 1u) & 1u, abort_flag, p.status, 14)) { ok = false; break; }
                 tc_fence_after_sync();
+#pragma unroll 1
+                for (int e = 0; e < 2 && i0 + e < m; ++e) {
+                    const int i = i0 + e;
+                    float sdi = 0.f;
 #pragma unroll
-                for (int hw = 0; hw < 2; ++hw) {
-                    uint32_t pk[32];
+                    for (int ii = 0; ii < MAX_DRAFTS; ++ii)
+                        if (ii == i) sdi = sd[ii];
+                    const float pi = (t - i >= 0) ? ex2(fmaf(sdi, p.c2, nref_f)) : 0.f;
+                    const uint32_t bits = pack_bf16(pi, 0.f) << ((r & 1) * 16);        // key r sits in word r / 2
 #pragma unroll
-                    for (int w = 0; w < 32; ++w) pk[w] = (32 * hw + w == (r >> 1)) ? bits : 0u;
-                    tmem_st32(tmem_s + 32 * hw, pk);
+                    for (int hw = 0; hw < 2; ++hw) {
+                        uint32_t pk[32];
+#pragma unroll
+                        for (int w = 0; w < 32; ++w) pk[w] = (32 * hw + w == (r >> 1)) ? bits : 0u;
+                        tmem_st32(tmem_s + 64 * e + 32 * hw, pk);
+                    }
                 }
                 tmem_st_wait();
                 tc_fence_before_sync();
@@ -573,20 +610,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             if (valid && p.lse != nullptr)
                 p.lse[(static_cast<size_t>(b) * p.H + h) * p.T + t] = (mref + log2f(l)) * 0.6931471805599453f;
             __nv_bfloat16* orow = p.O + ((static_cast<size_t>(b) * p.T + (valid ? t : 0)) * p.H + h) * HD;
+            {
+                uint32_t raw[4][32];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t raw[2][32];
-                tmem_ld32(tmem_o + 64 * hf, raw[0]);
-                tmem_ld32(tmem_o + 64 * hf + 32, raw[1]);
-                tmem_ld_wait(raw[0]);
-                tmem_ld_wait(raw[1]);
+                for (int q = 0; q < 4; ++q) tmem_ld32(tmem_o + 32 * q, raw[q]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tmem_ld_wait(raw[q]);
                 if (valid) {
 #pragma unroll
-                    for (int k = 0; k < 2; ++k) {
+                    for (int q = 0; q < 4; ++q) {
 #pragma unroll
                         for (int q8 = 0; q8 < 2; ++q8) {
-                            const uint32_t* x = &raw[k][16 * q8];
-                            st_global_v8(orow + 64 * hf + 32 * k + 16 * q8,
+                            const uint32_t* x = &raw[q][16 * q8];
+                            st_global_v8(orow + 32 * q + 16 * q8,
                                          pack_bf16(__uint_as_float(x[0]) * inv, __uint_as_float(x[1]) * inv),
                                          pack_bf16(__uint_as_float(x[2]) * inv, __uint_as_float(x[3]) * inv),
                                          pack_bf16(__uint_as_float(x[4]) * inv, __uint_as_float(x[5]) * inv),

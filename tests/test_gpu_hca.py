@@ -78,6 +78,9 @@ def test_small_workloads_all_heads(name):
     (3, 64, 5, 5, 4),         # one key tile per item, five heads
     (1, 70, 1, 1, 8),         # the second key tile holds only hidden columns for most rows
     (2, 5, 2, 1, 8),          # more draft passes than positions
+    (1, 300, 3, 1, 2),        # an odd group size: a CTA pairs two query tiles of one head; three tiles leave one alone
+    (2, 640, 2, 2, 3),        # one query head per key/value head, five query tiles
+    (1, 384, 6, 3, 1),        # an even group size: a CTA pairs two heads of one group
 ])
 def test_awkward_shapes(B, T, H, Hkv, m):
     inp = hi.make_hca_inputs(hi.HcaWorkload("custom", B=B, T=T, H=H, Hkv=Hkv, m=m, seed=T + m))
