@@ -241,6 +241,11 @@ int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W
  * are then valid) and reports device-side errors like hass_check.
  * `workspace` must hold hass_topk_distill_host_workspace_bytes(...) bytes: the normal workspace
  * plus device staging for the inputs and outputs.
+ * The copies overlap the computation: the call works in row chunks, the rows of chunk c + 1 travel to the
+ * device while chunk c computes and the dH_d rows of chunk c travel back while chunk c + 1 computes. For this
+ * the library keeps, per device, two copy streams and a pool of events of its own (created by the first call
+ * on that device; no device memory); they are ordered after `cuda_stream` at the start of the call and
+ * `cuda_stream` is ordered after them at its end.
  */
 int hass_topk_distill_host_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K, int dH_dtype,
                                            size_t* bytes);

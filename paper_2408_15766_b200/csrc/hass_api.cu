@@ -761,11 +761,25 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
 // from the K spilled entries it concerns; (5) the second GEMM with the row scale in its epilogue. No logit
 // is computed twice and no row of W is gathered, so the cost does not depend on K beyond the candidate
 // handling of (1). with_target = false: (1) is skipped and (2) only sorts the given Omega_hat.
+// Hand-over between two copy streams and the compute stream, used by the host-buffer entry: the rows of a chunk
+// are copied to the device while the previous chunk computes, and a chunk's dH_d rows go back to the host while
+// the next chunk computes. H_t / H_d / dH_d of fused2_impl are then the device staging buffers.
+struct ChunkPipe {
+    cudaStream_t h2d, d2h;
+    const uint8_t* Ht_host;
+    const uint8_t* Hd_host;
+    uint8_t* dH_host;
+    size_t in_row_bytes, out_row_bytes;
+    cudaEvent_t* events;       // pool
+    int n_events, used;
+    cudaEvent_t next() { return used < n_events ? events[used++] : nullptr; }
+};
+
 static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
                        long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
                        int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
                        void* workspace, size_t workspace_bytes, cudaStream_t st, float top_p = 0.f,
-                       int* topk_n = nullptr) {
+                       int* topk_n = nullptr, ChunkPipe* pipe = nullptr) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
@@ -834,6 +848,25 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
         p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
         p.p_pitch = L.p_pitch;
         p.status = status;
+        cudaEvent_t ev_d = nullptr;
+        if (pipe) {
+            // this chunk's rows of H_t, then of H_d, on the inbound copy stream; the sweeps wait for them
+            const size_t off = static_cast<size_t>(t0) * BM * pipe->in_row_bytes, bytes = static_cast<size_t>(rows) * pipe->in_row_bytes;
+            cudaEvent_t ev_t = pipe->next();
+            ev_d = pipe->next();
+            if (!ev_t || !ev_d) return HASS_ERR_UNSUPPORTED;
+            bool ok = cudaMemcpyAsync(const_cast<uint8_t*>(static_cast<const uint8_t*>(H_t)) + off, pipe->Ht_host + off, bytes,
+                                      cudaMemcpyHostToDevice, pipe->h2d) == cudaSuccess;
+            ok = ok && cudaEventRecord(ev_t, pipe->h2d) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(const_cast<uint8_t*>(static_cast<const uint8_t*>(H_d)) + off, pipe->Hd_host + off, bytes,
+                                       cudaMemcpyHostToDevice, pipe->h2d) == cudaSuccess;
+            ok = ok && cudaEventRecord(ev_d, pipe->h2d) == cudaSuccess;
+            ok = ok && cudaStreamWaitEvent(st, ev_t, 0) == cudaSuccess;
+            if (!ok) {
+                cudaGetLastError();
+                return HASS_ERR_CUDA;
+            }
+        }
         if (with_target) {
             // (1) target rows: statistics + candidates
             GemmParams t = p;
@@ -878,6 +911,10 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
         g_launches.fetch_add(1);
         if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
         // (3) draft rows: statistics, spill, z_d at Omega_hat
+        if (pipe && cudaStreamWaitEvent(st, ev_d, 0) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
         {
             GemmParams q = p;
             q.tmA0 = tmHd;
@@ -940,6 +977,20 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
         o.status = status;
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
+        if (pipe) {
+            // the chunk's dH_d rows on the outbound copy stream
+            const size_t off = static_cast<size_t>(t0) * BM * pipe->out_row_bytes, bytes = static_cast<size_t>(rows) * pipe->out_row_bytes;
+            cudaEvent_t ev_o = pipe->next();
+            if (!ev_o) return HASS_ERR_UNSUPPORTED;
+            bool ok = cudaEventRecord(ev_o, st) == cudaSuccess;
+            ok = ok && cudaStreamWaitEvent(pipe->d2h, ev_o, 0) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(pipe->dH_host + off, static_cast<const uint8_t*>(dH_d) + off, bytes, cudaMemcpyDeviceToHost,
+                                       pipe->d2h) == cudaSuccess;
+            if (!ok) {
+                cudaGetLastError();
+                return HASS_ERR_CUDA;
+            }
+        }
     }
     {
         // Exact route, enqueued behind every call of this route: if a sweep reported a row beyond its exponent
@@ -1285,6 +1336,35 @@ int hass_topk_distill_host_workspace_bytes(int64_t N, int64_t d, int64_t V, int3
     return HASS_OK;
 }
 
+// Copy streams and events of the host-buffer entry, created on a device's first call (no device memory).
+struct HostPipeResources {
+    bool ready = false;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t events[256];
+};
+static HostPipeResources g_host_pipe[64];
+
+static int host_pipe_resources(HostPipeResources** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    HostPipeResources& r = g_host_pipe[dev];
+    if (!r.ready) {
+        bool ok = cudaStreamCreateWithFlags(&r.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&r.d2h, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; ok && i < 256; ++i) ok = cudaEventCreateWithFlags(&r.events[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        r.ready = true;
+    }
+    *out = &r;
+    return HASS_OK;
+}
+
 int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, const void* W, int64_t N, int64_t d,
                                    int64_t V, int32_t K, const float* grad_loss_host, float* loss_host,
                                    int32_t* topk_idx_host, float* topk_q_host, void* dH_d_host, int dH_dtype,
@@ -1302,12 +1382,9 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
     if (workspace_bytes < s.total) return HASS_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    const size_t hbytes = static_cast<size_t>(N) * d * 2;
-    if (cudaMemcpyAsync(ws + s.H_t, H_t_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(ws + s.H_d, H_d_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
-        cudaGetLastError();
-        return HASS_ERR_CUDA;
-    }
+    HostPipeResources* res = nullptr;
+    rc = host_pipe_resources(&res);
+    if (rc != HASS_OK) return rc;
     const float* grad_dev = nullptr;
     if (grad_loss_host) {
         if (cudaMemcpyAsync(ws + s.grad, grad_loss_host, static_cast<size_t>(N) * 4, cudaMemcpyHostToDevice, st) !=
@@ -1317,14 +1394,62 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
         }
         grad_dev = reinterpret_cast<const float*>(ws + s.grad);
     }
-    rc = hass_topk_distill_fwd_bwd(ws + s.H_t, ws + s.H_d, W, N, d, V, K, grad_dev, reinterpret_cast<float*>(ws + s.loss),
-                                   reinterpret_cast<int32_t*>(ws + s.idx), reinterpret_cast<float*>(ws + s.q),
-                                   reinterpret_cast<float*>(ws + s.lse_t), reinterpret_cast<float*>(ws + s.lse_d),
-                                   ws + s.dH, dH_dtype, workspace, base, st);
-    if (rc != HASS_OK) return rc;
+    // The copy streams start after whatever the caller's stream still does with the workspace. The rows of a chunk
+    // travel to the device while the previous chunk computes; a chunk's dH_d rows travel back while the next computes.
+    ChunkPipe pipe;
+    pipe.h2d = res->h2d;
+    pipe.d2h = res->d2h;
+    pipe.Ht_host = static_cast<const uint8_t*>(H_t_host);
+    pipe.Hd_host = static_cast<const uint8_t*>(H_d_host);
+    pipe.dH_host = static_cast<uint8_t*>(dH_d_host);
+    pipe.in_row_bytes = static_cast<size_t>(d) * 2;
+    pipe.out_row_bytes = static_cast<size_t>(d) * (dH_dtype == HASS_FP32 ? 4 : 2);
+    pipe.events = res->events;
+    pipe.n_events = 256;
+    pipe.used = 0;
+    cudaEvent_t ev_start = pipe.next();
+    if (cudaEventRecord(ev_start, st) != cudaSuccess || cudaStreamWaitEvent(pipe.h2d, ev_start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(pipe.d2h, ev_start, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    rc = fused2_impl(true, ws + s.H_t, ws + s.H_d, W, N, d, V, K, grad_dev, nullptr, nullptr,
+                     reinterpret_cast<float*>(ws + s.loss), reinterpret_cast<int32_t*>(ws + s.idx),
+                     reinterpret_cast<float*>(ws + s.q), reinterpret_cast<float*>(ws + s.lse_t),
+                     reinterpret_cast<float*>(ws + s.lse_d), ws + s.dH, dH_dtype, workspace, base, st, 0.f, nullptr, &pipe);
+    if (rc == HASS_ERR_UNSUPPORTED) {
+        // more row chunks than events (a very small workspace): one copy in, the call, one copy out
+        const size_t hbytes = static_cast<size_t>(N) * d * 2;
+        cudaStreamSynchronize(pipe.h2d);
+        cudaStreamSynchronize(pipe.d2h);
+        if (cudaMemcpyAsync(ws + s.H_t, H_t_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(ws + s.H_d, H_d_host, hbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        rc = fused2_impl(true, ws + s.H_t, ws + s.H_d, W, N, d, V, K, grad_dev, nullptr, nullptr,
+                         reinterpret_cast<float*>(ws + s.loss), reinterpret_cast<int32_t*>(ws + s.idx),
+                         reinterpret_cast<float*>(ws + s.q), reinterpret_cast<float*>(ws + s.lse_t),
+                         reinterpret_cast<float*>(ws + s.lse_d), ws + s.dH, dH_dtype, workspace, base, st);
+        if (rc == HASS_OK && cudaMemcpyAsync(dH_d_host, ws + s.dH, static_cast<size_t>(N) * pipe.out_row_bytes,
+                                             cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+    } else if (rc == HASS_OK) {
+        // the caller's stream ends after the last outbound copy
+        cudaEvent_t ev_out = pipe.next();
+        if (!ev_out || cudaEventRecord(ev_out, pipe.d2h) != cudaSuccess || cudaStreamWaitEvent(st, ev_out, 0) != cudaSuccess) {
+            cudaGetLastError();
+            cudaStreamSynchronize(pipe.d2h);
+        }
+    }
+    if (rc != HASS_OK) {
+        cudaStreamSynchronize(pipe.h2d);
+        cudaStreamSynchronize(pipe.d2h);
+        return rc;
+    }
     bool ok = cudaMemcpyAsync(loss_host, ws + s.loss, static_cast<size_t>(N) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(dH_d_host, ws + s.dH, static_cast<size_t>(N) * d * (dH_dtype == HASS_FP32 ? 4 : 2),
-                               cudaMemcpyDeviceToHost, st) == cudaSuccess;
     if (topk_idx_host)
         ok = ok && cudaMemcpyAsync(topk_idx_host, ws + s.idx, static_cast<size_t>(N) * K * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     if (topk_q_host)
@@ -1333,7 +1458,22 @@ int hass_topk_distill_fwd_bwd_host(const void* H_t_host, const void* H_d_host, c
         cudaGetLastError();
         return HASS_ERR_CUDA;
     }
-    return hass_check(workspace, cuda_stream);
+    // word 2 of the status block: the exact route ran after the chunks' dH_d rows had left; fetch them again
+    unsigned int redo = 0;
+    ok = cudaMemcpyAsync(&redo, ws + 8, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    rc = hass_check(workspace, cuda_stream);
+    cudaStreamSynchronize(pipe.d2h);
+    if (rc != HASS_OK) return rc;
+    if (!ok) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    if (redo != 0u &&
+        cudaMemcpy(dH_d_host, ws + s.dH, static_cast<size_t>(N) * pipe.out_row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    return HASS_OK;
 }
 
 // ---- forward without a caller-provided workspace -------------------------------------------------

@@ -1472,9 +1472,13 @@ __global__ void wait_expiry_selftest_kernel(unsigned int* status, unsigned long 
     }
 }
 
-// Ends the exact route after a fused call: the range report has been dealt with.
+// Ends the exact route after a fused call: the range report has been dealt with. Word 2 of the status block
+// records that the route ran (the host-buffer entry then copies dH_d to the host once more).
 __global__ void range_handled_kernel(unsigned int* status) {
-    if (((*status) & 0xffu) == 2u) *status = 0u;
+    if (((*status) & 0xffu) == 2u) {
+        *status = 0u;
+        status[2] = 1u;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -283,6 +283,39 @@ def test_host_buffer_entry_matches_device_entry():
     assert torch.equal(idx_h, ref["topk_idx"].cpu())
 
 
+def test_host_buffer_entry_with_several_row_chunks_and_the_exact_route():
+    """N = 4800 is two row chunks: the second chunk's rows travel to the device while the first computes and
+    the first chunk's dH_d rows travel back meanwhile; results equal the device entry's bit for bit. With a row
+    beyond the spill's exponent range the exact route redoes the call after the chunks' dH_d rows have left,
+    and the entry must fetch them again."""
+    hass = _hass()
+    N, d, V, K = 4800, 64, 700, 5
+    inp = hi.make_custom(N, d, V, K, seed=17, sigma_w=0.1)
+    dev = torch.device("cuda:0")
+    for hot in (False, True):
+        W, H_d = inp.W.clone(), inp.H_d[0].clone()
+        if hot:
+            u = torch.where(torch.rand(d, generator=torch.Generator().manual_seed(1)) < 0.5, -1.0, 1.0)
+            W[300] = (0.125 * u).to(torch.bfloat16)
+            H_d[[7, 4790]] = (37.5 * u).to(torch.bfloat16)        # z_d[300] = 300 on these rows
+        Wd = W.to(dev)
+        grad = torch.rand(N, generator=torch.Generator().manual_seed(2)) + 0.5
+        ref = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), Wd, K, grad_loss=grad.to(dev))
+        hass.check(ref["workspace"])
+        loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
+        dH_h = torch.full((N, d), float("nan"), dtype=torch.bfloat16).pin_memory()
+        q_h = torch.empty(N, K, dtype=torch.float32).pin_memory()
+        hass.topk_distill_fwd_bwd_host(inp.H_t.pin_memory(), H_d.pin_memory(), Wd, K, loss_h, dH_h,
+                                       grad_loss_host=grad.pin_memory(), topk_q_host=q_h)
+        assert torch.equal(loss_h, ref["loss"].cpu())
+        assert torch.equal(dH_h, ref["dH_d"].cpu())
+        assert torch.equal(q_h, ref["topk_q"].cpu())
+        if hot:
+            print(compare(inp.H_t, H_d, W, K, dict(loss=loss_h, topk_idx=ref["topk_idx"].cpu(), topk_q=q_h,
+                                                   lse_t=ref["lse_t"].cpu(), lse_d=ref["lse_d"].cpu(), dH_d=dH_h),
+                          rows=np.array([0, 7, 100, 4735, 4736, 4790, 4799]), grad_loss=grad.numpy().astype(np.float64)))
+
+
 def test_results_are_deterministic_run_to_run():
     hass = _hass()
     inp = hi.make_custom(500, 256, 9000, 10, seed=5, sigma_w=0.1)
