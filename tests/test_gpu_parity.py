@@ -105,6 +105,8 @@ def _guarded_fused(inp, K, grad, dH_fp32=True):
     (4800, 64, 700, 5),       # two row chunks, the second one ragged
     (260, 72, 20000, 17),     # smallest K on the buffered Top-K path, d not a multiple of 64
     (129, 4096, 128257, 10),  # a full-size hidden dimension, one row and one token past a tile boundary
+    (64, 64, 40000, 100),     # one row tile split over 148 lanes: the selection cuts its candidate pool many times
+    (100, 64, 33000, 128),    # the largest K, 129 lanes
 ])
 def test_awkward_shapes(N, d, V, K):
     inp = hi.make_custom(N, d, V, K, seed=N + V, sigma_w=0.5 / np.sqrt(d) * 4)
