@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 SRC_DIR = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhass_b200.so")
 SOURCES = ["hass_api.cu"]
-HEADERS = ["kernels.cuh", "hca_kernels.cuh", "hca_bwd_kernels.cuh", "ptx.cuh", os.path.join("..", "..", "include", "hass.h")]
+# every header under csrc/ and the public header: a change to any of them makes the library stale
+HEADERS = sorted(f for f in os.listdir(SRC_DIR) if f.endswith((".cuh", ".h"))) + [os.path.join("..", "..", "include", "hass.h")]
 
 
 def _stale() -> bool:
