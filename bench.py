@@ -428,6 +428,10 @@ def main():
                          "+ w * Top-K in one call (8 N d V tensor FLOPs); top_p (P = 0.5, at most K tokens) and "
                          "normed (Normed Top-K: only the target product, 2 N d V) and bidir (Bi-directional "
                          "Top-K) are the loss variants of Section 4.3")
+    ap.add_argument("--route", default="fused", choices=["fused", "split"],
+                    help="topk objective: fused = hass_topk_distill_fwd_bwd (6 N d V executed, the headline); split = "
+                         "hass_topk_distill_fwd followed by hass_topk_distill_bwd, which recomputes the draft logits "
+                         "(8 N d V executed for the same 6 N d V credited)")
     ap.add_argument("--hca-pass", default="fwd", choices=["fwd", "fwd_bwd"],
                     help="hca-* workloads: time the forward alone, or forward + backward (all input gradients)")
     ap.add_argument("--oracle-rows", type=int, default=None, help="rows of the CPU-baseline sample")
@@ -500,6 +504,11 @@ def main():
             variant = {"top_p": hass.LOSS_TOP_P, "normed": hass.LOSS_NORMED_TOPK, "bidir": hass.LOSS_BIDIR_TOPK}
             var_out.update(hass.variant_distill_fwd_bwd(H_t, H_d_steps[j], W, K, variant[args.objective], TOP_P,
                                                         workspace=ws, stream=stream))
+        elif args.route == "split":
+            counts["full"] += 1
+            f = hass.topk_distill_fwd(H_t, H_d_steps[j], W, K, workspace=ws, stream=stream)
+            hass.topk_distill_bwd(H_d_steps[j], W, f["topk_idx"], f["topk_q"], f["lse_d"], workspace=ws, stream=stream,
+                                  out=out["dH_d"])
         elif j == 0:
             counts["full"] += 1
             hass.topk_distill_fwd_bwd(H_t, H_d_steps[0], W, K, workspace=ws, out=out, stream=stream)
@@ -538,7 +547,7 @@ def main():
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region ----
     e2e = None
-    if not args.no_e2e and args.objective == "topk":
+    if not args.no_e2e and args.objective == "topk" and args.route == "fused":
         Ht_h, Hd_h = inp.H_t.pin_memory(), inp.H_d[0].pin_memory()
         loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
         dH_h = torch.empty(N, d, dtype=torch.bfloat16).pin_memory()
@@ -569,9 +578,10 @@ def main():
     # the Top-K and Top-P calls sweep the target rows and the draft rows in separate launches (timed as
     # stats_gemm and stats_gemm_draft); the combined and Bi-directional calls sweep both in one launch
     two_sweeps = args.objective in ("topk", "top_p")
+    split = args.objective == "topk" and args.route == "split"
     kinds = {"stats_gemm": (2.0 * n_full if (normed or two_sweeps) else 4.0 * n_full) / args.steps * N * d * V,
              "stats_gemm_draft": 2.0 * (n_full + n_draft) / args.steps * N * d * V if two_sweeps else 0.0,
-             "dz_gemm": 2.0 * N * d * V,
+             "dz_gemm": 2.0 * N * d * V if split else 0.0,
              "dH_gemm": (4.0 if combined else 2.0) * N * d * V}
     total_ms = sum(v[0] for v in prof.values())
     kernel_rows = {}
@@ -591,7 +601,7 @@ def main():
     peak = float(peaks[peak_key])
     traffic, traffic_note = None, "no capture for this kernel, objective, shape or library version"
     cap = TRAFFIC_CAPTURE
-    if (args.objective == "topk" and hass.version() == cap["version"] and dom in cap["bytes_per_launch"]
+    if (args.objective == "topk" and not split and hass.version() == cap["version"] and dom in cap["bytes_per_launch"]
             and wl.name in ("l2-7b", "l3-8b") and K <= 16):
         traffic = cap["bytes_per_launch"][dom] * V / cap["V"]
         traffic_note = ("ncu dram bytes of this kernel captured on %s (K = %d), mean of the step's two launches"
@@ -627,7 +637,8 @@ def main():
                        "path": {"combined": "hass_combined_distill_fwd_bwd", "top_p": "hass_variant_distill_fwd_bwd (Top-P)",
                                 "normed": "hass_variant_distill_fwd_bwd (Normed Top-K)",
                                 "bidir": "hass_variant_distill_fwd_bwd (Bi-directional Top-K)",
-                                "topk": "hass_topk_distill_fwd_bwd (no logit recompute)"}[args.objective]},
+                                "topk": ("hass_topk_distill_fwd + hass_topk_distill_bwd (draft logits recomputed)" if split else
+                                         "hass_topk_distill_fwd_bwd (no logit recompute)")}[args.objective]},
             "clocks": clocks, "gpu_launches": launches,
             "tensor": {"credited_tflops": step_tflops, "credited_flops_per_step": flops_credit,
                        "executed_tflops": executed / (ms_step * 1e-3) / 1e12, "executed_flops_per_step": executed,

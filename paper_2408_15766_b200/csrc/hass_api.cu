@@ -1012,6 +1012,134 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
     return HASS_OK;
 }
 
+// ---- forward alone, Omega_hat known before the draft rows are swept -----------------------------------
+// hass_topk_distill_fwd and hass_topk_distill_fwd_draft: the sweep of the target rows (statistics, candidates),
+// select_kernel, the sweep of the draft rows (statistics and z_d at the row's Omega_hat, copied out of the
+// accumulator) and loss_patch_kernel (lse_d, Eq. 1). Nothing is spilled and no row of W is gathered. Needs the
+// [N, K] lists of the workspace beyond the statistics; with a workspace that ends before them the older
+// single-sweep forward (forward_impl) runs instead.
+static int forward2_impl(bool with_target, const void* H_t, const void* H_d, const void* W, long long N, long long d,
+                         long long V, int K, const int* idx_in, const float* q_in, float* loss, int* idx_out,
+                         float* q_out, float* lse_t, float* lse_d, void* workspace, size_t workspace_bytes,
+                         cudaStream_t st) {
+    int rc = check_sizes(N, d, V, K);
+    if (rc != HASS_OK) return rc;
+    if (!H_d || !W || !loss || !lse_d || !aligned16(H_d) || !aligned16(W)) return HASS_ERR_INVALID_ARG;
+    if (with_target && (!H_t || !idx_out || !q_out || !lse_t || !aligned16(H_t))) return HASS_ERR_INVALID_ARG;
+    if (!with_target && (!idx_in || !q_in)) return HASS_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HASS_ERR_WORKSPACE;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc != HASS_OK) return rc;
+    rc = get_encode();
+    if (rc != HASS_OK) return rc;
+    Layout L;
+    rc = make_layout(N, d, V, K, di.sms, &L, nullptr);
+    if (rc != HASS_OK) return rc;
+    if (workspace_bytes < L.sparse)
+        return forward_impl(with_target, H_t, H_d, W, N, d, V, K, idx_in, q_in, loss, idx_out, q_out, lse_t, lse_d,
+                            workspace, workspace_bytes, st);
+    const int RT = ceil_div(N, BM), CT = ceil_div(V, BN);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws + L.status, 0, 256, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    rc = plan_schedule(RT, CT, di.sms, &p.sched);
+    if (rc != HASS_OK) return rc;
+    if (p.sched.total_slots > L.slot_cap) return HASS_ERR_WORKSPACE;
+    log_schedule("fwd sweep (target / draft)", p.sched);
+    rc = make_tmap(&p.tmB, W, V, d, d, BK, BN);
+    if (rc != HASS_OK) return rc;
+    p.row_tiles0 = RT;
+    p.spill_begin = INT_MAX;
+    p.rows_valid = static_cast<int>(N);
+    p.n_cols = static_cast<int>(V);
+    p.col_tiles = CT;
+    p.k_blocks = ceil_div(d, BK);
+    p.K = K;
+    p.cap = topk_cap(K);
+    p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+    p.part_s = reinterpret_cast<float*>(ws + L.part_s);
+    p.cand = reinterpret_cast<uint2*>(ws + L.cand_v);
+    p.cand_n = reinterpret_cast<int*>(ws + L.cand_i);
+    p.status = reinterpret_cast<unsigned int*>(ws + L.status);
+    int* sidx = reinterpret_cast<int*>(ws + L.sidx);
+    float* sq = reinterpret_cast<float*>(ws + L.sgq);
+    float* capz = reinterpret_cast<float*>(ws + L.capz);
+    if (with_target) {
+        GemmParams t = p;
+        rc = make_tmap(&t.tmA0, H_t, N, d, d, BK, BM);
+        if (rc != HASS_OK) return rc;
+        t.tmA1 = t.tmA0;
+        t.topk_row_tiles = RT;
+        t.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+        if (cudaMemsetAsync(t.thr_share, 0xff, static_cast<size_t>(t.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
+            cudaGetLastError();
+            return HASS_ERR_CUDA;
+        }
+        rc = launch_gemm<MODE_STATS>(t, st);
+        if (rc != HASS_OK) return rc;
+    }
+    SelectParams sp;
+    std::memset(&sp, 0, sizeof(sp));
+    sp.sched = p.sched;
+    sp.K = K;
+    sp.cap = p.cap;
+    sp.row_begin = 0;
+    sp.rows = static_cast<int>(N);
+    sp.from_sweep = with_target ? 1 : 0;
+    sp.part_m = p.part_m;
+    sp.part_s = p.part_s;
+    sp.cand = p.cand;
+    sp.cand_n = p.cand_n;
+    sp.idx_in = idx_in;
+    sp.q_in = q_in;
+    sp.idx_out = idx_out;
+    sp.q_out = q_out;
+    sp.lse_t = lse_t;
+    sp.sidx = sidx;
+    sp.sq = sq;
+    {
+        KernelTimer timer(KIND_FINALIZE, st);
+        select_kernel<<<ceil_div(N, SEL_WARPS), SEL_WARPS * 32, 0, st>>>(sp);
+    }
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
+    {
+        GemmParams q = p;
+        rc = make_tmap(&q.tmA0, H_d, N, d, d, BK, BM);
+        if (rc != HASS_OK) return rc;
+        q.tmA1 = q.tmA0;
+        q.topk_row_tiles = 0;
+        q.sidx = sidx;
+        q.cap_z = capz;
+        rc = launch_gemm<MODE_STATS>(q, st, KIND_STATS_DRAFT);
+        if (rc != HASS_OK) return rc;
+    }
+    LossPatchParams lp;
+    std::memset(&lp, 0, sizeof(lp));
+    lp.sched = p.sched;
+    lp.K = K;
+    lp.row_begin = 0;
+    lp.rows = static_cast<int>(N);
+    lp.part_m = p.part_m;
+    lp.part_s = p.part_s;
+    lp.sidx = sidx;
+    lp.sq = sq;
+    lp.cap_z = capz;
+    lp.loss = loss;
+    lp.lse_d = lse_d;
+    {
+        KernelTimer timer(KIND_FINALIZE, st);
+        loss_patch_kernel<<<ceil_div(N, 8), 256, 0, st>>>(lp);
+    }
+    g_launches.fetch_add(1);
+    return cudaGetLastError() == cudaSuccess ? HASS_OK : HASS_ERR_CUDA;
+}
+
 // ---- Normed Top-K variant -----------------------------------------------------------------------------
 // Both distributions are renormalised over Omega_hat, so the loss and its gradient involve the draft
 // logits on Omega_hat only: one sweep over the TARGET rows (statistics + Top-K), then finalize computes the
@@ -1180,15 +1308,15 @@ int hass_topk_distill_workspace_bytes(int64_t N, int64_t d, int64_t V, int32_t K
 int hass_topk_distill_fwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
                           float* loss, int32_t* topk_idx, float* topk_q, float* lse_t, float* lse_d, void* workspace,
                           size_t workspace_bytes, void* cuda_stream) {
-    return forward_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
-                        workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+    return forward2_impl(true, H_t, H_d, W, N, d, V, K, nullptr, nullptr, loss, topk_idx, topk_q, lse_t, lse_d,
+                         workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int hass_topk_distill_fwd_draft(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,
                                 const int32_t* topk_idx, const float* topk_q, float* loss, float* lse_d,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    return forward_impl(false, nullptr, H_d, W, N, d, V, K, topk_idx, topk_q, loss, nullptr, nullptr, nullptr, lse_d,
-                        workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+    return forward2_impl(false, nullptr, H_d, W, N, d, V, K, topk_idx, topk_q, loss, nullptr, nullptr, nullptr, lse_d,
+                         workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, int64_t V, int32_t K,

@@ -1397,9 +1397,9 @@ __global__ void __launch_bounds__(256) loss_patch_kernel(const __grid_constant__
     if (lane == 0) {
         p.loss[row] = loss;
         p.lse_d[row] = lse_d;
-        p.coef_out[row] = g * scale;
+        if (p.coef_out) p.coef_out[row] = g * scale;
     }
-    if (g != 0.f && scale > 0.f && scale < INFINITY) {
+    if (p.P != nullptr && g != 0.f && scale > 0.f && scale < INFINITY) {      // P == nullptr: forward only, nothing to patch
         const float inv = 1.f / scale;
         __nv_bfloat16* prow = p.P + static_cast<long long>(local) * p.p_pitch;
         for (int j = lane; j < K; j += 32) {
