@@ -42,7 +42,7 @@
 extern "C" {
 #endif
 
-#define HASS_K_MAX 128
+#define HASS_K_MAX 256
 
 typedef enum {
     HASS_OK = 0,
@@ -210,7 +210,7 @@ int hass_combined_distill_fwd_bwd(const void* H_t, const void* H_d, const void* 
  *   HASS_LOSS_BIDIR_TOPK   Omega_hat = the K most probable tokens under q united with the K most probable
  *                          under p (taken as a constant set); loss and gradient as Eq. 1 on the union.
  *                          topk_idx / topk_q must hold 2K entries per row: the target's K in descending q,
- *                          then the draft's tokens not among them in descending p, then -1 / 0. K <= 64.
+ *                          then the draft's tokens not among them in descending p, then -1 / 0. K <= HASS_K_MAX / 2.
  *
  * topk_n [N] (nullable) receives |Omega_hat| per row; for HASS_LOSS_TOP_P the count is negated (-K) on a row
  * whose K most probable tokens together still do not exceed P, i.e. whose prefix was cut by the cap of K

@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.environ.get("HASS_LIBRARY_PATH") or os.path.join(_HERE, "libhass_b200.so")
 
 HASS_BF16, HASS_FP32 = 0, 1
-K_MAX = 128
+K_MAX = 256
 
 
 class HassError(RuntimeError):

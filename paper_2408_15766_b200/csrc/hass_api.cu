@@ -457,7 +457,7 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
 
     {
         KernelTimer timer(only_if_range ? KIND_CONDITIONAL : KIND_PREP, st);
-        bwd_prep_kernel<<<ceil_div(N, 128), 128, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss,
+        bwd_prep_kernel<<<ceil_div(N, PREP_WARPS), PREP_WARPS * 32, 0, st>>>(static_cast<int>(N), K, topk_idx, topk_q, lse_d, grad_loss,
                                                            sidx, sgq, coef, lse2, only_if_range);
     }
     g_launches.fetch_add(1);
@@ -528,8 +528,9 @@ static int backward_impl(const void* H_d, const void* W, long long N, long long 
     return HASS_OK;
 }
 
-// ---- fused forward + backward -------------------------------------------------------------------
-// Per chunk of row tiles: (1) one sweep computes the logits of the chunk's target and draft rows,
+// ---- fused forward + backward with one sweep over target and draft rows ----------------------------
+// The route of the combined objective and of the Bi-directional variant (the plain Top-K call, its _draft form
+// and Top-P use fused2_impl below). Per chunk of row tiles: (1) one sweep computes the logits of the chunk's target and draft rows,
 // their statistics and Top-K candidates, and spills the draft tiles as 2^(z log2e - ref2) in bf16;
 // (2) finalize gives loss, Omega_hat, lse and the per-row scale of the spilled tiles; (3) the second
 // GEMM contracts the spilled tiles with W and applies scale and sparse term in its epilogue. No
@@ -547,7 +548,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
                       long long V, int K, const float* grad_loss, const int* idx_in, const float* q_in, float* loss,
                       int* idx_out, float* q_out, float* lse_t, float* lse_d, void* dH_d, int dH_dtype,
                       void* workspace, size_t workspace_bytes, cudaStream_t st, const Combined* cmb = nullptr,
-                      float top_p = 0.f, int* topk_n = nullptr, bool bidir = false) {
+                      int* topk_n = nullptr, bool bidir = false) {
     int rc = check_sizes(N, d, V, K);
     if (rc != HASS_OK) return rc;
     if (!H_d || !W || !loss || !lse_d || !dH_d || !aligned16(H_d) || !aligned16(W) || !aligned16(dH_d))
@@ -658,7 +659,6 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.coef_out = coef;
         f.gq_out = gq;
         f.sparse_out = sparse;
-        f.top_p = top_p;
         f.n_out = topk_n;
         f.bidir = bidir ? 1 : 0;
         f.H_t = static_cast<const __nv_bfloat16*>(H_t);
@@ -732,23 +732,7 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
     }
-    if (!cmb && !(top_p > 0.f) && !bidir) {
-        // Exact route, enqueued behind every plain fused call: if the sweep reported a row beyond its exponent
-        // range, the separate forward and the recomputing backward (which have no such limit) redo the call
-        // and the report is withdrawn; otherwise each of these launches returns at once.
-        rc = forward_impl(with_target, H_t, H_d, W, N, d, V, K, idx_in, q_in, loss, idx_out, q_out, lse_t, lse_d,
-                          workspace, workspace_bytes, st, status);
-        if (rc != HASS_OK) return rc;
-        rc = backward_impl(H_d, W, N, d, V, K, with_target ? idx_out : idx_in, with_target ? q_out : q_in, lse_d,
-                           grad_loss, dH_d, dH_dtype, workspace, workspace_bytes, st, false, status);
-        if (rc != HASS_OK) return rc;
-        {
-            KernelTimer timer(KIND_CONDITIONAL, st);
-            range_handled_kernel<<<1, 1, 0, st>>>(status);
-        }
-        g_launches.fetch_add(1);
-        if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
-    }
+    // no second route here: a row beyond the spill's exponent range is reported as HASS_ERR_RANGE by hass_check
     return HASS_OK;
 }
 
@@ -1358,7 +1342,7 @@ int hass_variant_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W
                                lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, param, topk_n);
         case HASS_LOSS_BIDIR_TOPK:
             return fused_impl(true, H_t, H_d, W, N, d, V, K, grad_loss, nullptr, nullptr, loss, topk_idx, topk_q, lse_t,
-                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, 0.f, topk_n, true);
+                              lse_d, dH_d, dH_dtype, workspace, workspace_bytes, st, nullptr, topk_n, true);
         case HASS_LOSS_NORMED_TOPK:
             return normed_impl(H_t, H_d, W, N, d, V, K, grad_loss, loss, topk_idx, topk_q, topk_n, lse_t, dH_d, dH_dtype,
                                workspace, workspace_bytes, st);

@@ -31,7 +31,7 @@ constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int NUM_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
 constexpr int MAX_PHASES = 48;
-constexpr int K_CAP = 128;         // == HASS_K_MAX
+constexpr int K_CAP = 256;         // == HASS_K_MAX
 constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float LOG2E = 1.4426950408889634f;
 
@@ -119,8 +119,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 // compacts it to the row's K best and raises the threshold to the K-th largest logit. Entries stay in
 // increasing token-id order, admission is strict (x > threshold), and among logits equal to the K-th the
 // lowest token ids are kept, so equal logits resolve to the lower token id.
-constexpr int CAND_CAP_MAX = 416;                 // largest buffer: K = 128
-constexpr int CAND_REGS = CAND_CAP_MAX / 32;      // entries per lane during a compaction
+constexpr int CAND_CAP_MAX = 800;                 // largest buffer: K = 256
+constexpr int CAND_REGS = CAND_CAP_MAX / 32;      // entries per lane during a compaction of the largest buffer
+constexpr int CAND_REGS_SMALL = 13;               // ... of a buffer of up to 416 entries (K <= 128)
 constexpr int CAND_SLACK = 32;                    // a compaction may leave up to K + CAND_SLACK entries
 
 // K entries kept + room for max(2K, 96) new ones between compactions (each compaction then multiplies the
@@ -143,7 +144,9 @@ __device__ __forceinline__ uint32_t key_bits(uint32_t key) {
 // found so far: all of them are kept and the threshold is the value just below the prefix. Otherwise the
 // search runs to the last bit, exactly K entries are kept (among logits equal to the K-th, the lowest token
 // ids) and the threshold is the K-th largest logit itself.
+template <int REGS>
 __device__ __forceinline__ uint32_t compact_candidates(uint2* buf, int n, int K, int cap, int lane, int& n_out) {
+    constexpr int CAND_REGS = REGS;
     uint32_t key[CAND_REGS];
     int id[CAND_REGS];
     const int groups = cap >> 5;
@@ -477,7 +480,9 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             const unsigned long long bp = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(cbuf), L);
                             const int n = __shfl_sync(0xffffffffu, cnt, L);
                             int left = 0;
-                            const uint32_t tb = compact_candidates(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane, left);
+                            const uint32_t tb = p.cap <= 32 * CAND_REGS_SMALL
+                                                    ? compact_candidates<CAND_REGS_SMALL>(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane, left)
+                                                    : compact_candidates<CAND_REGS>(reinterpret_cast<uint2*>(bp), n, p.K, p.cap, lane, left);
                             __syncwarp();
                             if (lane == L) {
                                 cnt = left;
@@ -1149,7 +1154,7 @@ __global__ void __launch_bounds__(256) finalize_kernel(const __grid_constant__ F
 // candidates (or takes it as an input), writes topk_idx / topk_q in descending q, and leaves the same set
 // sorted by token id (sidx, sq) for the draft sweep, which copies z_d at those tokens out of its accumulators.
 constexpr int SEL_WARPS = 4;          // warps (rows) per block
-constexpr int SEL_MAX = 1024;         // candidates of one row that fit its shared-memory window
+constexpr int SEL_MAX = 768;          // candidates of one row that fit its shared-memory window (> K_CAP + 32)
 
 struct SelectParams {
     Schedule sched;        // schedule of the target sweep; its row tile t = rows [128 t, 128 t + 128) of the chunk
@@ -1211,8 +1216,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) select_kernel(const __grid_con
         find_slots(p.sched, rt, slot0, S);
         const float lse_t = warp_lse(p.part_m, p.part_s, slot0, S, r, lane);
         if (lane == 0) p.lse_t[row] = lse_t;
-        // Pool of candidates in shared memory. The slots' lists are appended one after the other; whenever the
-        // next list might not fit, the pool is cut to its K best (logit descending, lower token id first among
+        // Pool of candidates in shared memory. The slots' lists are appended 32 entries at a time; whenever the
+        // next 32 might not fit, the pool is cut to its K best (logit descending, lower token id first among
         // equal logits) and the K-th logit becomes a floor below which later candidates are not even copied.
         uint32_t* kk = sh_key[wib];
         int* ii = sh_id[wib];
@@ -1259,8 +1264,8 @@ __global__ void __launch_bounds__(SEL_WARPS * 32) select_kernel(const __grid_con
         for (int sl = 0; sl < S; ++sl) {
             const long long so = static_cast<long long>(slot0 + sl) * BM + r;
             const int cn = p.cand_n[so];
-            if (n + cn > SEL_MAX && n > K) cut_to_k();
             for (int e0 = 0; e0 < cn; e0 += 32) {
+                if (n + 32 > SEL_MAX) cut_to_k();      // n > K here: the window holds more than K_CAP + 32 entries
                 const int e = e0 + lane;
                 bool ok = false;
                 uint2 ce = make_uint2(0u, 0u);
@@ -1482,38 +1487,46 @@ __global__ void range_handled_kernel(unsigned int* status) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// bwd_prep: one thread per row. Sorts Omega_hat by token id (the MODE_PROBS epilogue walks the
-// vocabulary in increasing order) and precomputes g * q, g * S_q and lse_d * log2(e).
-__global__ void bwd_prep_kernel(int N, int K, const int* __restrict__ idx, const float* __restrict__ q,
-                                const float* __restrict__ lse_d, const float* __restrict__ grad_loss,
-                                int* __restrict__ sidx, float* __restrict__ sgq, float* __restrict__ coef,
-                                float* __restrict__ lse2, const unsigned int* __restrict__ only_if_range) {
+// bwd_prep: one warp per row. Sorts Omega_hat by token id (the MODE_PROBS epilogue walks the vocabulary in
+// increasing order; entries cut by Top-P carry id -1 and come first) by ranking every entry against the
+// others, and precomputes g * q, g * S_q and lse_d * log2(e).
+constexpr int PREP_WARPS = 4;
+__global__ void __launch_bounds__(PREP_WARPS * 32) bwd_prep_kernel(int N, int K, const int* __restrict__ idx,
+                                                                    const float* __restrict__ q,
+                                                                    const float* __restrict__ lse_d,
+                                                                    const float* __restrict__ grad_loss,
+                                                                    int* __restrict__ sidx, float* __restrict__ sgq,
+                                                                    float* __restrict__ coef, float* __restrict__ lse2,
+                                                                    const unsigned int* __restrict__ only_if_range) {
     if (only_if_range != nullptr && ((*only_if_range) & 0xffu) != 2u) return;
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ int s_tok[PREP_WARPS][K_CAP];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int row = blockIdx.x * PREP_WARPS + wib;
     if (row >= N) return;
+    const long long ro = static_cast<long long>(row) * K;
     const float g = grad_loss ? grad_loss[row] : 1.f;
-    int li[K_CAP];
-    float lq[K_CAP];
     float S_q = 0.f;
-    for (int j = 0; j < K; ++j) {
-        const int x = idx[static_cast<long long>(row) * K + j];
-        const float qq = q[static_cast<long long>(row) * K + j];
-        S_q += qq;
-        int t = j;
-        while (t > 0 && li[t - 1] > x) {
-            li[t] = li[t - 1];
-            lq[t] = lq[t - 1];
-            --t;
+    for (int j = lane; j < K; j += 32) {
+        s_tok[wib][j] = idx[ro + j];
+        S_q += q[ro + j];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S_q += __shfl_xor_sync(0xffffffffu, S_q, o);
+    __syncwarp();
+    for (int j = lane; j < K; j += 32) {
+        const int tj = s_tok[wib][j];
+        int rank = 0;
+        for (int i = 0; i < K; ++i) {
+            const int ti = s_tok[wib][i];
+            rank += (ti < tj || (ti == tj && i < j)) ? 1 : 0;
         }
-        li[t] = x;
-        lq[t] = qq;
+        sidx[ro + rank] = tj;
+        sgq[ro + rank] = g * q[ro + j];
     }
-    for (int j = 0; j < K; ++j) {
-        sidx[static_cast<long long>(row) * K + j] = li[j];
-        sgq[static_cast<long long>(row) * K + j] = g * lq[j];
+    if (lane == 0) {
+        coef[row] = g * S_q;
+        lse2[row] = lse_d[row] * LOG2E;
     }
-    coef[row] = g * S_q;
-    lse2[row] = lse_d[row] * LOG2E;
 }
 
 }  // namespace hass

@@ -43,7 +43,7 @@ def test_workspace_bytes_is_bounded_in_N(hass):
 
 
 @pytest.mark.parametrize("N,d,V,K", [(0, 64, 64, 1), (4, 12, 64, 1), (4, 64, 64, 65), (4, 64, 64, 0),
-                                     (4, 64, 1000, 129), (4, 0, 64, 1)])
+                                     (4, 64, 1000, 257), (4, 0, 64, 1)])
 def test_bad_sizes_rejected_without_a_device(hass, N, d, V, K):
     out = ctypes.c_size_t(0)
     rc = hass.lib.hass_topk_distill_workspace_bytes(N, d, V, K, ctypes.byref(out))

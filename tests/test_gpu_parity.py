@@ -106,7 +106,8 @@ def _guarded_fused(inp, K, grad, dH_fp32=True):
     (260, 72, 20000, 17),     # smallest K on the buffered Top-K path, d not a multiple of 64
     (129, 4096, 128257, 10),  # a full-size hidden dimension, one row and one token past a tile boundary
     (64, 64, 40000, 100),     # one row tile split over 148 lanes: the selection cuts its candidate pool many times
-    (100, 64, 33000, 128),    # the largest K, 129 lanes
+    (100, 64, 33000, 256),    # the largest K, 129 lanes
+    (150, 64, 3000, 200),     # K above 128 with two row tiles and few lanes
 ])
 def test_awkward_shapes(N, d, V, K):
     inp = hi.make_custom(N, d, V, K, seed=N + V, sigma_w=0.5 / np.sqrt(d) * 4)
@@ -453,7 +454,8 @@ def test_normed_top_k_variant_matches_oracle(N, d, V, K):
     print("normed", compare_variant(inp.H_t, inp.H_d[0], inp.W, K, oracle.VARIANT_NORMED, 0.0, cpu, grad_loss=grad))
 
 
-@pytest.mark.parametrize("N,d,V,K,P", [(64, 256, 1024, 10, 0.2), (300, 128, 5000, 24, 0.3), (4800, 64, 700, 16, 0.5)])
+@pytest.mark.parametrize("N,d,V,K,P", [(64, 256, 1024, 10, 0.2), (300, 128, 5000, 24, 0.3), (4800, 64, 700, 16, 0.5),
+                                       (200, 128, 6000, 256, 0.6)])
 def test_top_p_variant_matches_oracle(N, d, V, K, P):
     import oracle
     inp = hi.make_custom(N, d, V, K, seed=N + K + 2, sigma_w=2.0 / np.sqrt(d))
