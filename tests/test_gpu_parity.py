@@ -319,6 +319,25 @@ def test_host_buffer_entry_with_several_row_chunks_and_the_exact_route():
                           rows=np.array([0, 7, 100, 4735, 4736, 4790, 4799]), grad_loss=grad.numpy().astype(np.float64)))
 
 
+def test_host_buffer_entry_with_more_row_chunks_than_it_has_events():
+    """409600 rows are 87 row chunks on a 148-SM device, more than the entry's event pool covers: it falls back to
+    one copy in, the call, one copy out, and the results still equal the device entry's."""
+    hass = _hass()
+    N, d, V, K = 3200 * 128, 8, 64, 2
+    inp = hi.make_custom(N, d, V, K, seed=5, sigma_w=0.3)
+    dev = torch.device("cuda:0")
+    W = inp.W.to(dev)
+    ref = hass.topk_distill_fwd_bwd(inp.H_t.to(dev), inp.H_d[0].to(dev), W, K)
+    hass.check(ref["workspace"])
+    loss_h = torch.empty(N, dtype=torch.float32).pin_memory()
+    dH_h = torch.empty(N, d, dtype=torch.bfloat16).pin_memory()
+    hass.topk_distill_fwd_bwd_host(inp.H_t.pin_memory(), inp.H_d[0].pin_memory(), W, K, loss_h, dH_h)
+    assert torch.equal(loss_h, ref["loss"].cpu())
+    assert torch.equal(dH_h, ref["dH_d"].cpu())
+    rows = hi.sample_rows(N, 300, seed=1)
+    print(compare(inp.H_t, inp.H_d[0], inp.W, K, _to_cpu(ref), rows=rows))
+
+
 def test_results_are_deterministic_run_to_run():
     hass = _hass()
     inp = hi.make_custom(500, 256, 9000, 10, seed=5, sigma_w=0.1)
