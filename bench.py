@@ -369,9 +369,9 @@ def main_hca(args):
     if rank != 0:
         return
     # causal attention: one product = 2 * D flops per (query, key) pair with key <= query; the forward runs 2,
-    # the dQ kernel 3 (S, dP, dQ), the dK/dV kernel 4 (S^T, dP^T, dV, dK): 7 executed for 5 algorithmic
+    # the backward kernel the 5 the chain rule needs (S^T, dP^T, dV, dK, dQ^T)
     prod = 2.0 * wl.D * wl.B * wl.H * wl.T * (wl.T + 1) / 2
-    products = {"hca_attention": 2, "hca_bwd_dq": 3, "hca_bwd_dkv": 4}
+    products = {"hca_attention": 2, "hca_bwd_fused": 5}
     kernel_rows = {k: {"ms_per_step": ms / args.steps, "launches_per_step": c / args.steps,
                        **({"tflops": products[k] * prod / (ms / c * 1e-3) / 1e12} if k in products else {})}
                    for k, (ms, c) in prof.items() if c}
@@ -380,9 +380,9 @@ def main_hca(args):
     flops = products[dom] * prod
     achieved = flops / (ms_k / cnt * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
-    # the attention itself needs 2 products forward and 5 backward; the two backward kernels execute 7
+    # the attention itself needs 2 products forward and 5 backward, and that is what the kernels execute
     algorithmic = (7 if bwd else 2) * prod
-    executed = (9 if bwd else 2) * prod
+    executed = (7 if bwd else 2) * prod
     line = {"metric": metric, "value": aggregate(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",

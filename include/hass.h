@@ -302,9 +302,12 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
  *   dO [B, T, H, D] bf16
  *   dQ [B, T, H, D], dK_t, dV_t [B, T, Hkv, D] bf16      out (32-byte aligned)
  *   dK_d, dV_d   HOST arrays of m DEVICE pointers, each [B, T, Hkv, D] bf16, out
- *   workspace    hass_hca_attention_bwd_workspace_bytes(B, T, H, m) bytes, 256-byte aligned
- * Four kernels are enqueued on cuda_stream (row sums, dQ, dK_t/dV_t, and for m > 0 a row-scaling kernel for
- * the draft passes). Errors as for the forward.
+ *   workspace    hass_hca_attention_bwd_workspace_bytes(B, T, H, m) bytes, 256-byte aligned: the status
+ *                word, Dt, and dQ in fp32 (4 B T H D bytes)
+ * Three kernels are enqueued on cuda_stream: a row kernel (Dt, the substituted entries with the draft passes'
+ * gradients and their share of dQ), one tensor-core kernel for dK_t, dV_t and the key tiles' shares of dQ, which
+ * it adds into the fp32 copy with atomic reductions (their order is not fixed, so dQ may differ between two
+ * runs in the last bits of that fp32 sum), and the conversion of dQ to bf16. Errors as for the forward.
  */
 int hass_hca_attention_bwd_workspace_bytes(int64_t B, int64_t T, int64_t H, int32_t m, size_t* bytes);
 int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, const void* const* K_d,
@@ -384,8 +387,8 @@ int hass_topk_distill_fwd_static(const void* H_t, const void* H_d, const void* W
  * entries, and clears the records. Kinds: 0 logits+statistics GEMM (forward), 1 dz_d GEMM
  * (backward, recompute), 2 dH_d GEMM (backward), 3 finalize, 4 backward preparation, 5 the conditional
  * launches of the exact route behind a fused call (they return at once unless it is needed),
- * 6 HCA attention forward, 7 / 8 / 9 HCA attention backward: dQ kernel, dK_t/dV_t kernel, row kernels
- * (row sums and the draft passes' gradients), 10 the sweep of the draft rows in hass_topk_distill_fwd_bwd, its
+ * 6 HCA attention forward, 7 / 8 / 9 HCA attention backward: conversion of dQ to bf16, the tensor-core kernel,
+ * the row kernel (row sums, substituted entries, the draft passes' gradients), 10 the sweep of the draft rows in hass_topk_distill_fwd_bwd, its
  * _draft form and the Top-P variant (kind 0 is then the sweep of the target rows alone).
  * At most 8192 launches are recorded between summaries. Not thread-safe.
  */

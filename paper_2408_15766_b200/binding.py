@@ -415,7 +415,7 @@ def selftest_wait_expiry(workspace: torch.Tensor, limit_ns: int = 2_000_000, str
 
 
 PROFILE_KINDS = ("stats_gemm", "dz_gemm", "dH_gemm", "finalize", "bwd_prep", "exact_route_conditional",
-                 "hca_attention", "hca_bwd_dq", "hca_bwd_dkv", "hca_bwd_rows", "stats_gemm_draft")
+                 "hca_attention", "hca_bwd_dq_convert", "hca_bwd_fused", "hca_bwd_rows", "stats_gemm_draft")
 
 
 def profile_enable(on: bool) -> None:

@@ -12,7 +12,7 @@
 #include "kernels.cuh"
 #include "hca_kernels.cuh"
 #include "hca_pair_kernel.cuh"
-#include "hca_bwd_kernels.cuh"
+#include "hca_bwd_fused_kernel.cuh"
 
 namespace hass {
 
@@ -21,7 +21,7 @@ static std::atomic<long long> g_launches{0};
 // ---- optional per-kernel timing (hass_profile_*) ------------------------------------------------
 // When enabled, every kernel launch is bracketed by a pair of CUDA events on its own stream; the
 // summary adds up the elapsed time per kernel kind. Off by default; not thread-safe.
-enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_DQ = 7, KIND_HCA_DKV = 8, KIND_HCA_BWD_ROWS = 9, KIND_STATS_DRAFT = 10, NUM_KINDS = 11 };
+enum { KIND_STATS = 0, KIND_PROBS = 1, KIND_OUT = 2, KIND_FINALIZE = 3, KIND_PREP = 4, KIND_CONDITIONAL = 5, KIND_HCA = 6, KIND_HCA_DQ_CONVERT = 7, KIND_HCA_BWD_FUSED = 8, KIND_HCA_BWD_ROWS = 9, KIND_STATS_DRAFT = 10, NUM_KINDS = 11 };
 constexpr int kMaxRecords = 8192;
 struct Profiler {
     bool on = false;
@@ -77,8 +77,7 @@ static int device_info(DeviceInfo* out) {
             cudaError_t e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_REG>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             if (e3 == cudaSuccess) e3 = cudaFuncSetAttribute(gemm_kernel<MODE_STATS, TOPK_NONE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             cudaError_t e4 = cudaFuncSetAttribute(hca2::hca_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca2::SMEM_BYTES);
-            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::DQ_SMEM_BYTES);
-            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::KV_SMEM_BYTES);
+            if (e4 == cudaSuccess) e4 = cudaFuncSetAttribute(hca_bwd::hca_bwd_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, hca_bwd::F_SMEM_BYTES);
             if (e0 != cudaSuccess || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) {
                 cudaGetLastError();
                 return HASS_ERR_CUDA;
@@ -1725,24 +1724,23 @@ int hass_hca_attention_fwd(const void* Q, const void* K_t, const void* V_t, cons
     }
 }
 
-// workspace of the HCA backward: status word, D [B, H, T], and the weights and dS of the substituted entries
+// workspace of the HCA backward: status word, D [B, H, T], and the fp32 dQ accumulator [B, T, H, 128]
 struct HcaBwdLayout {
-    size_t D, Pd, dSd, total;
+    size_t D, dQacc, total;
 };
-static HcaBwdLayout hca_bwd_layout(int64_t B, int64_t T, int64_t H, int32_t m) {
+static HcaBwdLayout hca_bwd_layout(int64_t B, int64_t T, int64_t H) {
     HcaBwdLayout L;
     auto up = [](size_t x) { return (x + 255) & ~static_cast<size_t>(255); };
     const size_t rows = static_cast<size_t>(B) * H * T;
     L.D = 256;
-    L.Pd = up(L.D + rows * 4);
-    L.dSd = up(L.Pd + rows * 4 * (m > 0 ? m : 1));
-    L.total = up(L.dSd + rows * 4 * (m > 0 ? m : 1));
+    L.dQacc = up(L.D + rows * 4);
+    L.total = up(L.dQacc + rows * hca::HD * 4);
     return L;
 }
 
 int hass_hca_attention_bwd_workspace_bytes(int64_t B, int64_t T, int64_t H, int32_t m, size_t* bytes) {
     if (!bytes || B < 1 || T < 1 || H < 1 || m < 0 || m > HASS_HCA_MAX_DRAFTS) return HASS_ERR_INVALID_ARG;
-    *bytes = hca_bwd_layout(B, T, H, m).total;
+    *bytes = hca_bwd_layout(B, T, H).total;
     return HASS_OK;
 }
 
@@ -1766,7 +1764,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
         if (!K_d[i] || !V_d[i] || !dK_d[i] || !dV_d[i] || mis(K_d[i], 16) || mis(V_d[i], 16) || mis(dK_d[i], 16) ||
             mis(dV_d[i], 16))
             return HASS_ERR_INVALID_ARG;
-    const HcaBwdLayout L = hca_bwd_layout(B, T, H, m);
+    const HcaBwdLayout L = hca_bwd_layout(B, T, H);
     if (!workspace || workspace_bytes < L.total || mis(workspace, 256)) return HASS_ERR_WORKSPACE;
     DeviceInfo di;
     int rc = device_info(&di);
@@ -1776,8 +1774,7 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     float* Dv = reinterpret_cast<float*>(ws + L.D);
-    float* Pd = reinterpret_cast<float*>(ws + L.Pd);
-    float* dSd = reinterpret_cast<float*>(ws + L.dSd);
+    float* dQacc = reinterpret_cast<float*>(ws + L.dQacc);
     if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) {
         cudaGetLastError();
         return HASS_ERR_CUDA;
@@ -1785,47 +1782,45 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     const int iB = static_cast<int>(B), iT = static_cast<int>(T), iH = static_cast<int>(H), iHkv = static_cast<int>(Hkv);
     const float c2 = scale * 1.4426950408889634f;
 
-    hca_bwd::DqParams q;
-    std::memset(&q, 0, sizeof(q));
-    rc = make_tmap_seq(&q.tmQ, Q, B, T, H * hca::HD, 128);
-    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmdO, dO, B, T, H * hca::HD, 128);
-    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmK, K_t, B, T, Hkv * hca::HD, 64);
-    if (rc == HASS_OK) rc = make_tmap_seq(&q.tmV, V_t, B, T, Hkv * hca::HD, 64);
-    for (int i = 0; i < m && rc == HASS_OK; ++i) {
-        rc = make_tmap_seq(&q.tmKd[i], K_d[i], B, T, Hkv * hca::HD, 64);
-        if (rc == HASS_OK) rc = make_tmap_seq(&q.tmVd[i], V_d[i], B, T, Hkv * hca::HD, 64);
-    }
-    hca_bwd::DkvParams k;
+    hca_bwd::FusedParams k;
     std::memset(&k, 0, sizeof(k));
-    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmK, K_t, B, T, Hkv * hca::HD, 128);
-    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmV, V_t, B, T, Hkv * hca::HD, 128);
-    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmQ, Q, B, T, H * hca::HD, 64);
-    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmdO, dO, B, T, H * hca::HD, 64);
+    rc = make_tmap_seq(&k.tmK, K_t, B, T, Hkv * hca::HD, hca_bwd::KEYS);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmV, V_t, B, T, Hkv * hca::HD, hca_bwd::KEYS);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmQ, Q, B, T, H * hca::HD, hca_bwd::QE);
+    if (rc == HASS_OK) rc = make_tmap_seq(&k.tmdO, dO, B, T, H * hca::HD, hca_bwd::QE);
+    if (rc == HASS_OK) {
+        // the fp32 accumulator [B, T, H * 128]: boxes of 32 positions x one head's 128 floats, rows as they lie in memory
+        cuuint64_t gdim[3] = {static_cast<cuuint64_t>(H * hca::HD), static_cast<cuuint64_t>(T), static_cast<cuuint64_t>(B)};
+        cuuint64_t gstride[2] = {gdim[0] * 4, gdim[0] * 4 * gdim[1]};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(hca::HD), 32, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (g_encode(&k.tmdQ, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dQacc, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            rc = HASS_ERR_CUDA;
+    }
     if (rc != HASS_OK) return rc;
 
-    {   // D = rowsum(dO * O)
+    {   // D, the substituted entries and everything that follows from them, the start value of the dQ accumulator
+        hca_bwd::RowsParams r;
+        std::memset(&r, 0, sizeof(r));
+        r.Q = static_cast<const __nv_bfloat16*>(Q);
+        r.O = static_cast<const __nv_bfloat16*>(O);
+        r.dO = static_cast<const __nv_bfloat16*>(dO);
+        for (int i = 0; i < m; ++i) {
+            r.Kd[i] = static_cast<const __nv_bfloat16*>(K_d[i]);
+            r.Vd[i] = static_cast<const __nv_bfloat16*>(V_d[i]);
+            r.dKd[i] = static_cast<__nv_bfloat16*>(dK_d[i]);
+            r.dVd[i] = static_cast<__nv_bfloat16*>(dV_d[i]);
+        }
+        r.lse = lse;
+        r.D = Dv;
+        r.dQacc = dQacc;
+        r.m = m; r.B = iB; r.T = iT; r.H = iH; r.Hkv = iHkv;
+        r.c2 = c2;
+        r.scale = scale;
         KernelTimer kt(KIND_HCA_BWD_ROWS, st);
-        const long long rows = static_cast<long long>(B) * T * H;
-        hca_bwd::hca_bwd_prep_kernel<<<static_cast<unsigned>((rows * 16 + 255) / 256), 256, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(O), static_cast<const __nv_bfloat16*>(dO), Dv, iB, iT, iH);
-    }
-    g_launches.fetch_add(1);
-
-    q.dQ = static_cast<__nv_bfloat16*>(dQ);
-    q.lse = lse;
-    q.D = Dv;
-    q.Pd = Pd;
-    q.dSd = dSd;
-    q.B = iB; q.T = iT; q.H = iH; q.Hkv = iHkv; q.m = m;
-    q.q_tiles = static_cast<int>((T + 127) / 128);
-    q.k_tiles = static_cast<int>((T + 63) / 64);
-    q.items = iB * iH * q.q_tiles;
-    q.c2 = c2;
-    q.scale = scale;
-    q.status = static_cast<unsigned int*>(workspace);
-    {
-        KernelTimer kt(KIND_HCA_DQ, st);
-        hca_bwd::hca_dq_kernel<<<q.items < di.sms ? q.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::DQ_SMEM_BYTES, st>>>(q);
+        const long long halves = static_cast<long long>(B) * T * Hkv;
+        hca_bwd::hca_bwd_rows_kernel<<<static_cast<unsigned>((halves * 16 + 255) / 256), 256, 0, st>>>(r);
     }
     g_launches.fetch_add(1);
 
@@ -1834,31 +1829,25 @@ int hass_hca_attention_bwd(const void* Q, const void* K_t, const void* V_t, cons
     k.lse = lse;
     k.D = Dv;
     k.B = iB; k.T = iT; k.H = iH; k.Hkv = iHkv; k.m = m;
-    k.kt_tiles = static_cast<int>((T + 127) / 128);
-    k.q_tiles64 = static_cast<int>((T + 63) / 64);
+    k.kt_tiles = static_cast<int>((T + hca_bwd::KEYS - 1) / hca_bwd::KEYS);
+    k.q_tiles64 = static_cast<int>((T + hca_bwd::QE - 1) / hca_bwd::QE);
     k.items = iB * iHkv * k.kt_tiles;
     k.c2 = c2;
     k.scale = scale;
     k.status = static_cast<unsigned int*>(workspace);
     {
-        KernelTimer kt(KIND_HCA_DKV, st);
-        hca_bwd::hca_dkv_kernel<<<k.items < di.sms ? k.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::KV_SMEM_BYTES, st>>>(k);
+        KernelTimer kt(KIND_HCA_BWD_FUSED, st);
+        hca_bwd::hca_bwd_fused_kernel<<<k.items < di.sms ? k.items : di.sms, hca_bwd::NUM_THREADS, hca_bwd::F_SMEM_BYTES, st>>>(k);
     }
     g_launches.fetch_add(1);
 
-    if (m > 0) {
-        hca_bwd::DraftGradParams dg;
-        std::memset(&dg, 0, sizeof(dg));
-        for (int i = 0; i < m; ++i) {
-            dg.dKd[i] = static_cast<__nv_bfloat16*>(dK_d[i]);
-            dg.dVd[i] = static_cast<__nv_bfloat16*>(dV_d[i]);
-        }
-        KernelTimer kt(KIND_HCA_BWD_ROWS, st);
-        const long long warps = static_cast<long long>(B) * T * Hkv;
-        hca_bwd::hca_draft_grad_kernel<<<static_cast<unsigned>((warps * 16 + 255) / 256), 256, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(dO), Pd, dSd, dg, m, iB, iT, iH, iHkv);
-        g_launches.fetch_add(1);
+    {
+        KernelTimer kt(KIND_HCA_DQ_CONVERT, st);
+        const long long n8 = static_cast<long long>(B) * T * H * (hca::HD / 8);
+        hca_bwd::hca_dq_convert_kernel<<<static_cast<unsigned>((n8 + 255) / 256), 256, 0, st>>>(
+            dQacc, static_cast<__nv_bfloat16*>(dQ), n8);
     }
+    g_launches.fetch_add(1);
     if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     return HASS_OK;
 }

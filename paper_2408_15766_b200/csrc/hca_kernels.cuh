@@ -1,4 +1,4 @@
-// Helpers shared by the HCA attention kernels (forward: hca_pair_kernel.cuh, backward: hca_bwd_kernels.cuh):
+// Helpers shared by the HCA attention kernels (forward: hca_pair_kernel.cuh, backward: hca_bwd_fused_kernel.cuh):
 // 3-D TMA loads, tensor-memory stores, exp2, bf16 packing.
 #pragma once
 #include <cuda_bf16.h>
