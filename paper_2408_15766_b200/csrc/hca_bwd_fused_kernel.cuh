@@ -75,14 +75,14 @@ __device__ __forceinline__ float sum16(float v) {
 
 // ------------------------------------------------------------------------------------------------------
 // Row work. Half a warp per (sequence, query position t, key/value head g); a lane covers 8 of the 128
-// columns (16-byte accesses). For every query head h of the group it reads Q[t], dO[t], O[t] once and forms
+// columns (16-byte accesses). For every query head h of the group Q[t], dO[t], O[t] are read once and give
 //   D[t] = <dO, O>;  for i < m:  s_i = <Q[t], K_d[i][t-i]>,  dp_i = <dO[t], V_d[i][t-i]>,
 //   P_i = 2^(s_i c2 - lse2[t]),  dS_i = P_i (dp_i - D) scale          (zero where t - i < 0)
 //   dQacc[t] = sum_i dS_i K_d[i][t-i]                                  (fp32; zero for m = 0)
 //   dK_d[i][t-i] = sum_h dS_i Q[t],  dV_d[i][t-i] = sum_h P_i dO[t]
 // Position s of pass i meets exactly one query per head (t = s + i), so each output row has one writer; the
 // last i rows of pass i meet none and are zeroed by the half-warp of the same index. Passes are taken two at
-// a time (few registers, many rows in flight).
+// a time; the rows of the next head are requested before the current head is worked on.
 struct RowsParams {
     const __nv_bfloat16* Q;        // [B, T, H, 128]
     const __nv_bfloat16* O;
@@ -98,11 +98,11 @@ struct RowsParams {
     float c2, scale;
 };
 
-__global__ void __launch_bounds__(256) hca_bwd_rows_kernel(const __grid_constant__ RowsParams p) {
+__global__ void __launch_bounds__(256, 2) hca_bwd_rows_kernel(const __grid_constant__ RowsParams p) {
     const long long w = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 4;   // (b, t, g)
     const int sub = threadIdx.x & 15;
-    // whole half-warps leave together; the shuffles below name all 32 lanes, so a warp whose upper half is past
-    // the end keeps that half running on clamped indices with its stores switched off
+    // no thread leaves early: the shuffles below name all 32 lanes, so a half-warp past the end runs on clamped
+    // indices with its stores switched off
     const long long total = static_cast<long long>(p.B) * p.T * p.Hkv;
     const bool live = w < total;
     const long long wc = live ? w : total - 1;
@@ -113,67 +113,83 @@ __global__ void __launch_bounds__(256) hca_bwd_rows_kernel(const __grid_constant
     const int rep = p.H / p.Hkv;
     const int m = p.m;
     const int passes = m > 0 ? m : 1;
+    const size_t row0 = ((static_cast<size_t>(b) * p.T + t) * p.H + g * rep) * HD;      // head g * rep; the group's heads follow
+    const size_t ri0 = (static_cast<size_t>(b) * p.H + g * rep) * p.T + t;              // ... at distance T here
     for (int i0 = 0; i0 < passes; i0 += 2) {
-        float kd[2][8], vd[2][8], kacc[2][8], vacc[2][8];
+        uint4 kraw[2], vraw[2];         // kept packed; widened where they are used
+        float kacc[2][8], vacc[2][8];
         bool use[2];
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int i = i0 + j;
             use[j] = i < m && t - i >= 0;
-            uint4 kraw = make_uint4(0u, 0u, 0u, 0u), vraw = kraw;
+            kraw[j] = vraw[j] = make_uint4(0u, 0u, 0u, 0u);
             if (use[j]) {
                 const size_t row = ((static_cast<size_t>(b) * p.T + (t - i)) * p.Hkv + g) * HD;
-                kraw = __ldg(reinterpret_cast<const uint4*>(p.Kd[i] + row) + sub);
-                vraw = __ldg(reinterpret_cast<const uint4*>(p.Vd[i] + row) + sub);
+                kraw[j] = __ldg(reinterpret_cast<const uint4*>(p.Kd[i] + row) + sub);
+                vraw[j] = __ldg(reinterpret_cast<const uint4*>(p.Vd[i] + row) + sub);
             }
-            widen8(kraw, kd[j]);
-            widen8(vraw, vd[j]);
 #pragma unroll
             for (int c = 0; c < 8; ++c) kacc[j][c] = vacc[j][c] = 0.f;
         }
+        uint4 qn = __ldg(reinterpret_cast<const uint4*>(p.Q + row0) + sub);
+        uint4 dn = __ldg(reinterpret_cast<const uint4*>(p.dO + row0) + sub);
+        uint4 on = i0 == 0 ? __ldg(reinterpret_cast<const uint4*>(p.O + row0) + sub) : make_uint4(0u, 0u, 0u, 0u);
+        float ln = __ldg(p.lse + ri0);
         for (int hh = 0; hh < rep; ++hh) {
-            const int h = g * rep + hh;
-            const size_t row = ((static_cast<size_t>(b) * p.T + t) * p.H + h) * HD;
-            const size_t ri = (static_cast<size_t>(b) * p.H + h) * p.T + t;
+            const size_t row = row0 + static_cast<size_t>(hh) * HD;
+            const size_t ri = ri0 + static_cast<size_t>(hh) * p.T;
             float qf[8], df[8];
-            widen8(__ldg(reinterpret_cast<const uint4*>(p.Q + row) + sub), qf);
-            widen8(__ldg(reinterpret_cast<const uint4*>(p.dO + row) + sub), df);
+            widen8(qn, qf);
+            widen8(dn, df);
+            const uint4 oc = on;
+            const float nlse2 = -ln * 1.4426950408889634f;
+            if (hh + 1 < rep) {
+                qn = __ldg(reinterpret_cast<const uint4*>(p.Q + row + HD) + sub);
+                dn = __ldg(reinterpret_cast<const uint4*>(p.dO + row + HD) + sub);
+                if (i0 == 0) on = __ldg(reinterpret_cast<const uint4*>(p.O + row + HD) + sub);
+                ln = __ldg(p.lse + ri + p.T);
+            }
             float Dt;
             if (i0 == 0) {
                 float of[8];
-                widen8(__ldg(reinterpret_cast<const uint4*>(p.O + row) + sub), of);
+                widen8(oc, of);
                 Dt = sum16(dot8(df, of));
                 if (live && sub == 0) p.D[ri] = Dt;
             } else {
-                Dt = p.D[ri];       // written by this half-warp's lane 0 in the first round
+                Dt = p.D[ri];           // written by this half-warp's first lane in the first round
                 Dt = __shfl_sync(0xffffffffu, Dt, threadIdx.x & 16);
             }
-            const float nlse2 = -__ldg(p.lse + ri) * 1.4426950408889634f;
             float dq[8];
 #pragma unroll
             for (int c = 0; c < 8; ++c) dq[c] = 0.f;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                const float sv = sum16(dot8(qf, kd[j]));
-                const float dv = sum16(dot8(df, vd[j]));
+                float kdf[8], vdf[8];
+                widen8(kraw[j], kdf);
+                widen8(vraw[j], vdf);
+                const float sv = sum16(dot8(qf, kdf));
+                const float dv = sum16(dot8(df, vdf));
                 const float pw = use[j] ? ex2(fmaf(sv, p.c2, nlse2)) : 0.f;
                 const float ds = pw * (dv - Dt) * p.scale;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    dq[c] = fmaf(ds, kd[j][c], dq[c]);
+                    dq[c] = fmaf(ds, kdf[c], dq[c]);
                     kacc[j][c] = fmaf(ds, qf[c], kacc[j][c]);
                     vacc[j][c] = fmaf(pw, df[c], vacc[j][c]);
                 }
             }
             if (live) {
-                float4* dst = reinterpret_cast<float4*>(p.dQacc + row) + 2 * sub;
+                float* dst = p.dQacc + row + 8 * sub;
                 if (i0 != 0) {
-                    const float4 a = dst[0], c4 = dst[1];
-                    dq[0] += a.x; dq[1] += a.y; dq[2] += a.z; dq[3] += a.w;
-                    dq[4] += c4.x; dq[5] += c4.y; dq[6] += c4.z; dq[7] += c4.w;
+                    float a[8];
+                    ld_global_v8(dst, a);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) dq[c] += a[c];
                 }
-                dst[0] = make_float4(dq[0], dq[1], dq[2], dq[3]);
-                dst[1] = make_float4(dq[4], dq[5], dq[6], dq[7]);
+                st_global_v8(dst, __float_as_uint(dq[0]), __float_as_uint(dq[1]), __float_as_uint(dq[2]),
+                             __float_as_uint(dq[3]), __float_as_uint(dq[4]), __float_as_uint(dq[5]),
+                             __float_as_uint(dq[6]), __float_as_uint(dq[7]));
             }
         }
 #pragma unroll
