@@ -30,7 +30,8 @@ constexpr int KEYS = 128;               // keys per item (stationary tile)
 constexpr int QE = 64;                  // queries per element of an item's sweep
 constexpr int HD = 128;
 constexpr int MAX_DRAFTS = hca::MAX_DRAFTS;
-constexpr int NUM_THREADS = 320;        // producer, MMA issuer, two groups of four row-owning warps
+constexpr int NUM_THREADS = 352;        // producer, MMA issuer, two groups of four row-owning warps, the vector warp
+constexpr int VEC_WARP = 10;
 constexpr int K_BYTES = KEYS * HD * 2;  // two halves (64 columns of the head dimension) of 128 rows x 128 B
 constexpr int K_HALF = K_BYTES / 2;
 constexpr int QE_BYTES = QE * HD * 2;
@@ -241,7 +242,8 @@ __global__ void __launch_bounds__(256) hca_dq_convert_kernel(const float* __rest
 //                                      threads the slowest stage.)
 // The tensor core completes products in issue order, so the issue order S^T(e+2) after the three products of
 // element e needs no barrier for the S^T columns; dP^T(e+2) waits until the threads have taken dQ^T(e) out.
-// The per-query vectors -lse2[t] and -D[t] scale of an element travel with its Q / dO stage.
+// The per-query vectors -lse2[t] and -D[t] scale of an element travel with its Q / dO stage (written by a warp
+// that does nothing else).
 constexpr int F_STAGES = 3;             // a Q / dO stage is held until the element's last product is done
 constexpr int F_SMEM_K = 0;
 constexpr int F_SMEM_V = F_SMEM_K + K_BYTES;
@@ -306,7 +308,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
         mbar_init(kv_full, 1);
         mbar_init(kv_empty, 1);
         for (int s = 0; s < F_STAGES; ++s) {
-            mbar_init(qd_full(s), 2);      // the TMA transaction's arrival and the producer warp's vectors
+            mbar_init(qd_full(s), 2);      // the TMA transaction's arrival and the vector warp's
             mbar_init(qd_empty(s), 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -356,46 +358,62 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
     auto q_count = [&](int kt) { return p.q_tiles64 - 2 * kt; };
 
     if (warp == 0) {
-        // ===================== producer: TMA by lane 0, the per-query vectors by all lanes =====================
-        uint32_t gq = 0, it = 0;
-        bool ok = true;
-        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
-            int kt, b, g;
-            decode(item, kt, b, g);
-            const int nq = q_count(kt);
-            if (lane == 0) {
-                ok = wait_barrier(kv_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1);
-                if (ok) {
-                    mbar_arrive_expect_tx(kv_full, 2 * K_BYTES);
-                    tma_load_3d(base + F_SMEM_K, &p.tmK, kv_full, g * HD, kt * KEYS, b);
-                    tma_load_3d(base + F_SMEM_K + K_HALF, &p.tmK, kv_full, g * HD + 64, kt * KEYS, b);
-                    tma_load_3d(base + F_SMEM_V, &p.tmV, kv_full, g * HD, kt * KEYS, b);
-                    tma_load_3d(base + F_SMEM_V + K_HALF, &p.tmV, kv_full, g * HD + 64, kt * KEYS, b);
-                }
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            for (int e = 0; e < rep * nq && ok; ++e, ++gq) {
-                const int h = g * rep + e / nq;
-                const int jq = 2 * kt + e % nq;
-                const int s = gq % F_STAGES;
-                if (lane == 0) ok = wait_barrier(qd_empty(s), ((gq / F_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2);
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) break;
-                if (lane == 0) {
+        // ===================== producer: TMA =====================
+        if (lane == 0) {
+            uint32_t gq = 0, it = 0;
+            bool ok = true;
+            for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+                int kt, b, g;
+                decode(item, kt, b, g);
+                const int nq = q_count(kt);
+                if (!wait_barrier(kv_empty, (it & 1u) ^ 1u, abort_flag, p.status, 1)) break;
+                mbar_arrive_expect_tx(kv_full, 2 * K_BYTES);
+                tma_load_3d(base + F_SMEM_K, &p.tmK, kv_full, g * HD, kt * KEYS, b);
+                tma_load_3d(base + F_SMEM_K + K_HALF, &p.tmK, kv_full, g * HD + 64, kt * KEYS, b);
+                tma_load_3d(base + F_SMEM_V, &p.tmV, kv_full, g * HD, kt * KEYS, b);
+                tma_load_3d(base + F_SMEM_V + K_HALF, &p.tmV, kv_full, g * HD + 64, kt * KEYS, b);
+                for (int e = 0; e < rep * nq; ++e, ++gq) {
+                    const int h = g * rep + e / nq;
+                    const int jq = 2 * kt + e % nq;
+                    const int s = gq % F_STAGES;
+                    if (!wait_barrier(qd_empty(s), ((gq / F_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2)) { ok = false; break; }
                     mbar_arrive_expect_tx(qd_full(s), 2 * QE_BYTES);
                     tma_load_3d(base + F_SMEM_Q + s * QE_BYTES, &p.tmQ, qd_full(s), h * HD, jq * QE, b);
                     tma_load_3d(base + F_SMEM_Q + s * QE_BYTES + QE_HALF, &p.tmQ, qd_full(s), h * HD + 64, jq * QE, b);
                     tma_load_3d(base + F_SMEM_DO + s * QE_BYTES, &p.tmdO, qd_full(s), h * HD, jq * QE, b);
                     tma_load_3d(base + F_SMEM_DO + s * QE_BYTES + QE_HALF, &p.tmdO, qd_full(s), h * HD + 64, jq * QE, b);
                 }
-                // -lse2[t] (or -inf past the sequence, which zeroes the weight) and -D[t] scale for the 64 queries
+            }
+        }
+    } else if (warp == VEC_WARP) {
+        // ===================== the per-query vectors of every element, next to its Q / dO stage =====================
+        // -lse2[t] (or -inf past the sequence, which zeroes the weight) and -D[t] scale for the 64 queries, two per
+        // lane. A warp of its own: the loads' latency then delays neither the TMA requests nor anything else.
+        uint32_t gq = 0, it = 0;
+        bool ok = true;
+        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+            int kt, b, g;
+            decode(item, kt, b, g);
+            const int nq = q_count(kt);
+            for (int e = 0; e < rep * nq && ok; ++e, ++gq) {
+                const int h = g * rep + e / nq;
+                const int jq = 2 * kt + e % nq;
+                const int s = gq % F_STAGES;
                 const size_t rowbase = (static_cast<size_t>(b) * p.H + h) * p.T;
+                float nl[2], nd[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const int c = lane + 32 * u;
-                    const int t = jq * QE + c;
-                    vec[s * 128 + c] = t < p.T ? -p.lse[rowbase + t] * 1.4426950408889634f : -INFINITY;
-                    vec[s * 128 + 64 + c] = t < p.T ? -p.D[rowbase + t] * p.scale : 0.f;
+                    const int t = jq * QE + lane + 32 * u;
+                    nl[u] = t < p.T ? -__ldg(p.lse + rowbase + t) * 1.4426950408889634f : -INFINITY;
+                    nd[u] = t < p.T ? -__ldg(p.D + rowbase + t) * p.scale : 0.f;
+                }
+                if (lane == 0) ok = wait_barrier(qd_empty(s), ((gq / F_STAGES) & 1u) ^ 1u, abort_flag, p.status, 3);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    vec[s * 128 + lane + 32 * u] = nl[u];
+                    vec[s * 128 + 64 + lane + 32 * u] = nd[u];
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(qd_full(s));
@@ -493,7 +511,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
                 if (ok && a + 2 < n_e) ok = issue_st();
             }
         }
-    } else {
+    } else if (warp < VEC_WARP) {
         // two groups of four warps share every key row: group grp takes the query columns 32 grp .. 32 grp + 31
         // of each element, and in the epilogue dV (group 0) or dK (group 1)
         const int grp = (warp - 2) >> 2;
