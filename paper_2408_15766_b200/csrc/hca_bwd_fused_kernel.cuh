@@ -343,6 +343,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
         const int G = gridDim.x, c = blockIdx.x;
         return static_cast<int>(k) * G + ((k & 1u) ? G - 1 - c : c);
     };
+    // Every CTA walks the rounds in rotated order, starting at round (its index mod rounds): its share of the work
+    // is the same, but at any moment different CTAs are in rounds of different item lengths, so that their item
+    // boundaries (pipeline drained, a burst of loads) do not coincide. next_item steps the round counter k to this
+    // CTA's next existing item and returns it, or -1.
+    const int n_rounds = (p.items + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    auto next_item = [&](int& k) {
+        while (k < n_rounds) {
+            const int item = round_item(static_cast<uint32_t>((k + static_cast<int>(blockIdx.x)) % n_rounds));
+            ++k;
+            if (item < p.items) return item;
+        }
+        return -1;
+    };
 
     const int BG = p.B * p.Hkv;
     const int rep = p.H / p.Hkv;
@@ -362,7 +375,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
         if (lane == 0) {
             uint32_t gq = 0, it = 0;
             bool ok = true;
-            for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+            for (int rk = 0, item = next_item(rk); item >= 0 && ok; item = next_item(rk), ++it) {
                 int kt, b, g;
                 decode(item, kt, b, g);
                 const int nq = q_count(kt);
@@ -391,7 +404,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
         // lane. A warp of its own: the loads' latency then delays neither the TMA requests nor anything else.
         uint32_t gq = 0, it = 0;
         bool ok = true;
-        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+        for (int rk = 0, item = next_item(rk); item >= 0 && ok; item = next_item(rk), ++it) {
             int kt, b, g;
             decode(item, kt, b, g);
             const int nq = q_count(kt);
@@ -499,7 +512,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
             ++ga;
             return true;
         };
-        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+        for (int rk = 0, item = next_item(rk); item >= 0 && ok; item = next_item(rk), ++it) {
             int kt, b, g;
             decode(item, kt, b, g);
             const int n_e = rep * q_count(kt);
@@ -558,7 +571,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
             ++nd;
             return true;
         };
-        for (int item = round_item(0); item < p.items && ok; item = round_item(++it)) {
+        for (int rk = 0, item = next_item(rk); item >= 0 && ok; item = next_item(rk), ++it) {
             int kt, b, g;
             decode(item, kt, b, g);
             const int nq = q_count(kt);
