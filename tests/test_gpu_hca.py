@@ -206,6 +206,34 @@ def test_backward_full_size_sampled_groups(name):
     print(_run_bwd(hi.make_hca_inputs(wl), pairs=[(0, 0), (wl.B - 1, wl.Hkv - 1), (1, wl.Hkv // 2)]))
 
 
+def test_backward_twice_gives_the_same_gradients():
+    # dK_t, dV_t and the draft passes' gradients have one writer per row and a fixed summation order: bit-identical
+    # between two calls. dQ is summed over the key tiles in fp32 by reductions whose order is not fixed: two calls
+    # may differ by the rounding of that sum, i.e. by one step of the bf16 result in rare entries and never more.
+    hass = _hass()
+    dev = torch.device("cuda:0")
+    inp = hi.make_hca_inputs(hi.HcaWorkload("twice", B=2, T=1500, H=8, Hkv=2, m=3, seed=11))
+    g = torch.Generator().manual_seed(5)
+    dO = torch.randn(inp.Q.shape, generator=g).to(torch.bfloat16).to(dev)
+    d = lambda x: x.to(dev)
+    Q, K, V = d(inp.Q), d(inp.K_t), d(inp.V_t)
+    Kd, Vd = [d(x) for x in inp.K_d], [d(x) for x in inp.V_d]
+    fw = hass.hca_attention_fwd(Q, K, V, Kd, Vd)
+    runs = []
+    for _ in range(2):
+        bw = hass.hca_attention_bwd(Q, K, V, Kd, Vd, fw["O"], fw["lse"], dO)
+        hass.check(bw["workspace"])
+        runs.append(bw)
+    a, b = runs
+    assert torch.equal(a["dK_t"], b["dK_t"]) and torch.equal(a["dV_t"], b["dV_t"])
+    for i in range(3):
+        assert torch.equal(a["dK_d"][i], b["dK_d"][i]) and torch.equal(a["dV_d"][i], b["dV_d"][i])
+    qa, qb = a["dQ"].float(), b["dQ"].float()
+    step = torch.maximum(qa.abs(), qb.abs()) * 2.0 ** -7        # one bf16 step is at most 2^-7 of the value
+    assert bool(((qa - qb).abs() <= step).all())
+    assert float((qa != qb).float().mean()) < 0.05
+
+
 def test_draft_passes_equal_to_target_change_nothing_on_the_gpu():
     # property that holds at any size: with K_d = K_t and V_d = V_t the substituted entries carry the same keys and
     # values as the ones they replace, so the output must agree with plain causal attention (m = 0) up to the
