@@ -801,6 +801,9 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
     if (rc == HASS_OK) rc = make_tmap(&tmWk, W, V, d, d, BK, BN);
     if (rc == HASS_OK) rc = make_tmap(&tmWn, W, V, d, d, 64, BK);
     if (rc == HASS_OK) rc = make_tmap(&tmP, P, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
+    // the same buffer as the draft sweep's TMA stores see it: boxes of 64 columns x 32 rows, every column up to the pitch
+    CUtensorMap tmPst;
+    if (rc == HASS_OK) rc = make_tmap(&tmPst, P, static_cast<long long>(chunk_tiles) * BM, L.p_pitch, L.p_pitch, 64, 32);
     if (rc != HASS_OK) return rc;
 
     for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
@@ -907,6 +910,7 @@ static int fused2_impl(bool with_target, const void* H_t, const void* H_d, const
             q.sidx = sidx;
             q.cap_z = capz;
             q.P = P;
+            q.tmSpill = tmPst;
             rc = launch_gemm<MODE_STATS>(q, st, KIND_STATS_DRAFT);
             if (rc != HASS_OK) return rc;
         }

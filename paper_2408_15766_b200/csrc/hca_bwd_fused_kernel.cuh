@@ -23,7 +23,6 @@ namespace hca_bwd {
 
 using hca::ex2;
 using hca::pack_bf16;
-using hca::st_shared_v4;
 using hca::tma_load_3d;
 
 constexpr int KEYS = 128;               // keys per item (stationary tile)
@@ -64,9 +63,6 @@ __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* tm, uint32_
                  "r"(smem_src), "r"(x), "r"(y), "r"(z)
                  : "memory");
 }
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // sum over the 16 lanes of a half-warp
 __device__ __forceinline__ float sum16(float v) {
 #pragma unroll
@@ -551,7 +547,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_bwd_fused_kernel(const __g
             __syncwarp();
             if (lane == 0) mbar_arrive(dp_free(s));
             if (issuer) {
-                bulk_wait_group_read0();            // the previous reduction has read the staging buffer
+                bulk_wait_group_read<0>();            // the previous reduction has read the staging buffer
                 mbar_arrive(stage_free(grp));
             }
             if (!wait_barrier(stage_free(grp), nd & 1u, abort_flag, p.status, 16)) return false;

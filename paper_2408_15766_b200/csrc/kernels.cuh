@@ -32,7 +32,10 @@ constexpr int NUM_THREADS = 192;   // warp 0: TMA, warp 1: MMA + TMEM owner, war
 constexpr int TMEM_COLS = 512;     // two accumulator buffers of BN fp32 columns
 constexpr int MAX_PHASES = 48;
 constexpr int K_CAP = 256;         // == HASS_K_MAX
-constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int SPILL_STAGE_BYTES = 32 * 128;   // 32 rows x 64 bf16 of a spilled tile on their way to global memory
+constexpr int SPILL_STAGES = 2;               // per epilogue warp
+constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * SPILL_STAGES * SPILL_STAGE_BYTES +
+                           1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr float LOG2E = 1.4426950408889634f;
 
 enum { MODE_STATS = 0, MODE_PROBS = 1, MODE_OUT = 2 };
@@ -54,6 +57,8 @@ struct Schedule {
 
 struct GemmParams {
     CUtensorMap tmA0, tmA1, tmB;
+    CUtensorMap tmSpill;   // MODE_STATS without Top-K lists (the draft sweep): the spill P as [chunk rows, p_pitch] bf16 with
+                           // boxes of 64 columns x 32 rows, 128-byte swizzle, for TMA stores
     Schedule sched;
     int row_tiles0;        // row tiles [0, row_tiles0) read A0, the others A1 (tile index - row_tiles0)
     int topk_row_tiles;    // leading row tiles whose rows collect Top-K candidates (MODE_STATS)
@@ -237,7 +242,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t smemA = smem_base;
     const uint32_t smemB = smem_base + STAGES * A_STAGE_BYTES;
-    const uint32_t bar_base = smemB + STAGES * B_STAGE_BYTES;
+    const uint32_t spill_stage = smemB + STAGES * B_STAGE_BYTES;      // [epilogue warp][SPILL_STAGES] x SPILL_STAGE_BYTES
+    const uint32_t bar_base = spill_stage + 4 * SPILL_STAGES * SPILL_STAGE_BYTES;
     // barriers: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then tmem pointer, abort flag
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
@@ -245,7 +251,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
     auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     uint32_t* tmem_ptr_smem =
-        reinterpret_cast<uint32_t*>(smem_gen + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 8 * (2 * STAGES + 4));
+        reinterpret_cast<uint32_t*>(smem_gen + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * SPILL_STAGES * SPILL_STAGE_BYTES +
+                                    8 * (2 * STAGES + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -378,6 +385,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         // Top-K candidates of this thread's row (MODE_STATS): buffer in the workspace, entries in use
         uint2* cbuf = nullptr;
         int cnt = 0;
+        uint32_t spill_boxes = 0;                  // chunks this warp has staged for TMA stores (two per box)
         // TOPK_REG: the K_REG largest logits so far sorted descending in tv[] (the admission threshold is the
         // K_REG-th largest: a list of exactly K entries with its K-th as threshold measured slower), and the
         // current chunk's admitted logits waiting in a small local-memory buffer
@@ -549,19 +557,46 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                                 fadd2(acc0, acc1, acc0, acc1, e[j], e[j + 1]);
                             }
                             s += acc0 + acc1;
-                            __nv_bfloat16* dst = (rt >= p.spill_begin
-                                                      ? p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch
-                                                      : p.Pt + static_cast<long long>(rt * BM + r_local) * p.p_pitch) + col0;
+                            if (TOPK == TOPK_NONE) {
+                                // The draft sweep hands its spill to the TMA unit: the row's 32 values go into the warp's
+                                // staging buffer (128-byte rows, swizzled), and after every second chunk one lane
+                                // requests the store of the 32 x 64 box. That is one request per 4 KB from this warp
+                                // instead of 64 store instructions that each touch 32 rows.
+                                const uint32_t buf = spill_stage + (quad * SPILL_STAGES + ((spill_boxes >> 1) & 1)) * SPILL_STAGE_BYTES;
+                                if ((ch & 1) == 0) {
+                                    // the store that read this buffer two boxes ago must have finished reading it
+                                    if (lane == 0) bulk_wait_group_read<SPILL_STAGES - 1>();
+                                    __syncwarp();
+                                }
 #pragma unroll
-                            for (int g16 = 0; g16 < 2; ++g16)
-                                st_global_v8(dst + 16 * g16, pack_bf16x2(e[16 * g16 + 0], e[16 * g16 + 1]),
-                                             pack_bf16x2(e[16 * g16 + 2], e[16 * g16 + 3]),
-                                             pack_bf16x2(e[16 * g16 + 4], e[16 * g16 + 5]),
-                                             pack_bf16x2(e[16 * g16 + 6], e[16 * g16 + 7]),
-                                             pack_bf16x2(e[16 * g16 + 8], e[16 * g16 + 9]),
-                                             pack_bf16x2(e[16 * g16 + 10], e[16 * g16 + 11]),
-                                             pack_bf16x2(e[16 * g16 + 12], e[16 * g16 + 13]),
-                                             pack_bf16x2(e[16 * g16 + 14], e[16 * g16 + 15]));
+                                for (int j = 0; j < 4; ++j)
+                                    st_shared_v4(buf + lane * 128 + ((((ch & 1) * 4 + j) ^ (lane & 7)) << 4),
+                                                 pack_bf16x2(e[8 * j + 0], e[8 * j + 1]), pack_bf16x2(e[8 * j + 2], e[8 * j + 3]),
+                                                 pack_bf16x2(e[8 * j + 4], e[8 * j + 5]), pack_bf16x2(e[8 * j + 6], e[8 * j + 7]));
+                                if (ch & 1) {
+                                    fence_proxy_async_smem();
+                                    __syncwarp();
+                                    if (lane == 0) {
+                                        tma_store_2d(&p.tmSpill, buf, col0 - 32, (rt - p.spill_begin) * BM + quad * 32);
+                                        bulk_commit_group();
+                                    }
+                                }
+                                ++spill_boxes;
+                            } else {
+                                __nv_bfloat16* dst = (rt >= p.spill_begin
+                                                          ? p.P + static_cast<long long>((rt - p.spill_begin) * BM + r_local) * p.p_pitch
+                                                          : p.Pt + static_cast<long long>(rt * BM + r_local) * p.p_pitch) + col0;
+#pragma unroll
+                                for (int g16 = 0; g16 < 2; ++g16)
+                                    st_global_v8(dst + 16 * g16, pack_bf16x2(e[16 * g16 + 0], e[16 * g16 + 1]),
+                                                 pack_bf16x2(e[16 * g16 + 2], e[16 * g16 + 3]),
+                                                 pack_bf16x2(e[16 * g16 + 4], e[16 * g16 + 5]),
+                                                 pack_bf16x2(e[16 * g16 + 6], e[16 * g16 + 7]),
+                                                 pack_bf16x2(e[16 * g16 + 8], e[16 * g16 + 9]),
+                                                 pack_bf16x2(e[16 * g16 + 10], e[16 * g16 + 11]),
+                                                 pack_bf16x2(e[16 * g16 + 12], e[16 * g16 + 13]),
+                                                 pack_bf16x2(e[16 * g16 + 14], e[16 * g16 + 15]));
+                            }
                         }
                         if (!USE_REG && want_topk && cm > thr) {
 #pragma unroll
@@ -759,6 +794,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             }
             return true;
         });
+        // shared memory must outlive the TMA stores that read it
+        if (MODE == MODE_STATS && TOPK == TOPK_NONE && lane == 0) bulk_wait_group0();
     }
 
     // ---- teardown ----

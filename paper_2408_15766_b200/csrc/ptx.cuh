@@ -184,6 +184,29 @@ __device__ __forceinline__ void ld_global_v8(const void* ptr, float (&v)[8]) {
     v[7] = __uint_as_float(h);
 }
 
+// ---- 128-bit shared-memory store (address 16-byte aligned) ----------------------------------------
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// ---- TMA stores (shared -> global), tracked by the issuing thread's bulk groups -------------------
+// 2-D tiled store of the map's box; x (innermost, elements) must make x * elem_size a multiple of 16 bytes and
+// neither coordinate may be negative; parts of the box outside the tensor are dropped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t smem_src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(tm)),
+                 "r"(smem_src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until all but the newest N groups of this thread have finished reading their shared-memory source
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+// waits until all of this thread's groups are complete
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ---- packed fp32 arithmetic (two lanes per instruction) and 3-input max ----------------------------
 __device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0,
                                       float c1) {
