@@ -52,9 +52,6 @@ __device__ __forceinline__ float dot8(const float (&a)[8], const float (&b)[8]) 
     for (int c = 1; c < 8; ++c) s = fmaf(a[c], b[c], s);
     return s;
 }
-__device__ __forceinline__ void st_shared_b32(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
 // Adds a [1, rows, cols] fp32 box from shared memory into global memory through the tensor map (element type and
 // box come from the map; parts outside the tensor are dropped). Completion is tracked by the thread's bulk groups.
 __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* tm, uint32_t smem_src, int x, int y, int z) {

@@ -394,8 +394,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
         constexpr bool CAPTURE = MODE == MODE_STATS && TOPK == TOPK_NONE;
         float tv[USE_REG ? K_REG : 1];
         int ti[USE_REG ? K_REG : 1];
-        float pend_v[USE_REG ? 32 : 1];
-        int pend_i[USE_REG ? 32 : 1];
+        // ... waiting in shared memory: entry q of thread T at word q * 128 + T of the values' array and of the
+        // tokens' array (16 KB each, the room the draft sweep uses for its spill boxes; this instantiation stores no
+        // boxes). With 200 KB of shared memory carved out little L1 is left, and a per-thread array in local memory
+        // cost about a thousand cycles per admitted logit here.
+        static_assert(4 * SPILL_STAGES * SPILL_STAGE_BYTES >= 2 * 32 * 128 * 4, "room for the pending logits");
+        const uint32_t pend_v = spill_stage + (threadIdx.x - 64) * 4;
+        const uint32_t pend_i = pend_v + 32 * 128 * 4;
         constexpr int lo = 0;
 
         for_each_item([&](int rt, int ln, int S, int slot) {
@@ -615,14 +620,14 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             for (int j = 0; j < 32; ++j) {
                                 const float x = __uint_as_float(r[j]);
                                 if (x > thr) {
-                                    pend_v[USE_REG ? np : 0] = x;
-                                    pend_i[USE_REG ? np : 0] = col0 + j;
+                                    st_shared_b32(pend_v + np * 512, __float_as_uint(x));
+                                    st_shared_b32(pend_i + np * 512, static_cast<uint32_t>(col0 + j));
                                     ++np;
                                 }
                             }
                             for (int q = 0; q < np; ++q) {
-                                const float x = pend_v[USE_REG ? q : 0];
-                                const int id = pend_i[USE_REG ? q : 0];
+                                const float x = __uint_as_float(ld_shared_b32(pend_v + q * 512));
+                                const int id = static_cast<int>(ld_shared_b32(pend_i + q * 512));
                                 if (!(x > thr)) continue;
                                 // sorted insertion; equal logits stay behind earlier (lower) token ids
 #pragma unroll
