@@ -474,6 +474,39 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     m = ref2 * (1.0f / LOG2E);
                     skip_tile = t < 0;
                 }
+                if (MODE == MODE_STATS && HAS_TOPK && !USE_REG && want_topk && t == 0 && p.n_cols - col_base >= BN) {
+                    // First tile of the sweep, buffer empty, no threshold yet: admitting all 256 logits would fill
+                    // the buffer and force a compaction of every row of the warp at once (32 warp-wide compactions
+                    // in a row, during which the tensor core runs out of free accumulators). Instead each thread
+                    // searches, bit by bit, the largest 12-bit prefix (sign, exponent, three mantissa bits) that at
+                    // least K of its row's 256 logits reach - comparisons against the tile in tensor memory, the same
+                    // instructions for every row - and starts from the threshold just below it: a valid lower bound
+                    // of the row's K-th largest logit that admits little more than K of the tile's logits.
+                    uint32_t T = 0u;
+#pragma unroll 1
+                    for (int bit = 31; bit >= 20; --bit) {
+                        const uint32_t cand = T | (1u << bit);
+                        const float fc = __uint_as_float(key_bits(cand));      // keys order like the floats they stand for
+                        int c = 0;
+#pragma unroll 1
+                        for (int ch = 0; ch < BN / 32; ++ch) {
+                            uint32_t r[32];
+                            tmem_ld32(t_row + ch * 32, r);
+                            tmem_ld_wait(r);
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) c += (__uint_as_float(r[j]) >= fc) ? 1 : 0;
+                        }
+                        if (c >= p.K) T = cand;
+                    }
+                    if (T >= (1u << 20)) {
+                        // the float just below the prefix; at the prefix of +0 that is -0, which compares equal to
+                        // the zeros that were counted, so step down to a float that is really smaller
+                        float below = __uint_as_float(key_bits(T - 1u));
+                        if (below == 0.f) below = -1.17549435e-38f;
+                        thr_own = below;
+                        thr = fmaxf(thr_own, thr_sh);
+                    }
+                }
                 if (CAPTURE && !skip_tile) {
                     while (nxt < col_base) {
                         ++cur;
