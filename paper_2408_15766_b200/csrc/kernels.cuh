@@ -637,12 +637,13 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             }
                         }
                         if (!USE_REG && want_topk && cm > thr) {
+                            // predicated stores, no branches: as 32 conditional blocks this section took about 5000
+                            // cycles whenever any row of the warp admitted a logit
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
-                                if (__uint_as_float(r[j]) > thr) {
-                                    cbuf[cnt] = make_uint2(r[j], static_cast<uint32_t>(col0 + j));
-                                    ++cnt;
-                                }
+                                const bool in = __uint_as_float(r[j]) > thr;
+                                st_global_v2_if(cbuf + cnt, r[j], static_cast<uint32_t>(col0 + j), in);
+                                cnt += in ? 1 : 0;
                             }
                         }
                         if (USE_REG && want_topk && cm > thr) {
@@ -652,11 +653,10 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
 #pragma unroll
                             for (int j = 0; j < 32; ++j) {
                                 const float x = __uint_as_float(r[j]);
-                                if (x > thr) {
-                                    st_shared_b32(pend_v + np * 512, __float_as_uint(x));
-                                    st_shared_b32(pend_i + np * 512, static_cast<uint32_t>(col0 + j));
-                                    ++np;
-                                }
+                                const bool in = x > thr;       // predicated stores, no branches
+                                st_shared_b32_if(pend_v + np * 512, __float_as_uint(x), in);
+                                st_shared_b32_if(pend_i + np * 512, static_cast<uint32_t>(col0 + j), in);
+                                np += in ? 1 : 0;
                             }
                             for (int q = 0; q < np; ++q) {
                                 const float x = __uint_as_float(ld_shared_b32(pend_v + q * 512));

@@ -192,6 +192,17 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 __device__ __forceinline__ void st_shared_b32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+// stores that happen only where `on` is true, as predicated instructions (no branch)
+__device__ __forceinline__ void st_shared_b32_if(uint32_t addr, uint32_t v, bool on) {
+    asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q st.shared.b32 [%0], %1;\n}" ::"r"(addr), "r"(v),
+                 "r"(static_cast<uint32_t>(on))
+                 : "memory");
+}
+__device__ __forceinline__ void st_global_v2_if(void* ptr, uint32_t a, uint32_t b, bool on) {
+    asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %3, 0;\n@q st.global.v2.b32 [%0], {%1, %2};\n}" ::"l"(ptr), "r"(a), "r"(b),
+                 "r"(static_cast<uint32_t>(on))
+                 : "memory");
+}
 __device__ __forceinline__ uint32_t ld_shared_b32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
