@@ -1238,7 +1238,7 @@ const char* hass_status_string(int status) {
     }
 }
 
-int hass_version(void) { return 10300; }
+int hass_version(void) { return 10400; }
 
 int64_t hass_kernel_launch_count(void) { return g_launches.load(); }
 
