@@ -362,6 +362,28 @@ def test_exact_ties_resolve_to_lower_token_id():
     print(compare(inp.H_t, inp.H_d[0], W, 4, _to_cpu(out) | {"dH_d": None}, check_dH=False))
 
 
+@pytest.mark.parametrize("K", [20, 64])
+def test_zero_rows_and_ties_with_buffered_candidates(K):
+    # K > 16 takes the candidate-buffer path, whose first threshold of a sweep is found by a search over the
+    # sweep's first tile. Rows of zeros make every logit +0 (the search ends at the prefix of zero, and the
+    # threshold must still admit the zeros); duplicated rows of W put ties everywhere, also at the K-th place.
+    hass = _hass()
+    inp = hi.make_custom(130, 64, 1500, K, seed=21, sigma_w=0.2)
+    W = inp.W.clone()
+    W[750:1500] = W[0:750]           # every logit appears twice: tokens v and v + 750
+    H_t, H_d = inp.H_t.clone(), inp.H_d[0].clone()
+    for r in (5, 77, 129):
+        H_t[r] = 0
+    H_d[5] = 0
+    dev = torch.device("cuda:0")
+    out = hass.topk_distill_fwd_bwd(H_t.to(dev), H_d.to(dev), W.to(dev), K)
+    hass.check(out["workspace"])
+    idx = out["topk_idx"].cpu().numpy()
+    for r in (5, 77, 129):
+        assert np.array_equal(np.sort(idx[r]), np.arange(K)), "all logits equal: the K lowest token ids"
+    print(compare(H_t, H_d, W, K, _to_cpu(out)))
+
+
 @pytest.mark.parametrize("name", ["l2-7b", "l3-8b"])
 def test_full_size_config_sampled_rows(name):
     wl = hi.WORKLOADS[name]
