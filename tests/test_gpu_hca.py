@@ -188,6 +188,7 @@ def test_backward_small_workloads(name):
 @pytest.mark.parametrize("B,T,H,Hkv,m", [
     (1, 1, 1, 1, 1), (1, 128, 2, 2, 8), (1, 129, 2, 1, 8), (2, 256, 3, 3, 0), (1, 515, 4, 2, 5),
     (2, 700, 16, 4, 2), (3, 64, 5, 5, 4), (1, 70, 1, 1, 8), (2, 5, 2, 1, 8), (1, 4096, 2, 1, 3),
+    (2, 300, 6, 2, 3), (1, 200, 10, 2, 1),
 ])
 def test_backward_awkward_shapes(B, T, H, Hkv, m):
     inp = hi.make_hca_inputs(hi.HcaWorkload("custom", B=B, T=T, H=H, Hkv=Hkv, m=m, seed=T + m))
