@@ -52,14 +52,16 @@ constexpr int Q_BYTES = QT * HD * 2;                 // two halves (64 columns o
 constexpr int Q_HALF = Q_BYTES / 2;
 constexpr int KV_BYTES = KT * HD * 2;
 constexpr int KV_HALF = KV_BYTES / 2;
-constexpr int KV_STAGES = 2;
+constexpr int KV_STAGES = 2;          // value tiles in flight
+constexpr int K_STAGES = 3;           // key tiles in flight: one more, the draft passes' key tiles occupy the ring at an item's start
 constexpr int SMEM_Q = 0;                            // 2 slots
 constexpr int SMEM_K = SMEM_Q + 2 * Q_BYTES;
-constexpr int SMEM_V = SMEM_K + KV_STAGES * KV_BYTES;
+constexpr int SMEM_V = SMEM_K + K_STAGES * KV_BYTES;
 constexpr int SMEM_BAR = SMEM_V + KV_STAGES * KV_BYTES;
 constexpr int SCHED_DEPTH = 4;       // pair indices published ahead by the producer
-constexpr int NUM_BARS = 4 + 4 * KV_STAGES + 6 + 2 * SCHED_DEPTH;
-constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 196864
+constexpr int NUM_BARS = 4 + 2 * K_STAGES + 2 * KV_STAGES + 6 + 2 * SCHED_DEPTH;
+constexpr int SMEM_BYTES = SMEM_BAR + 256;           // 229632
+static_assert(8 * NUM_BARS + 4 * (2 + SCHED_DEPTH) <= 256 && SMEM_BYTES <= 232448, "shared-memory window");
 constexpr int TMEM_COLS = 512;     // S of slot s at 128 s (P overwrites its first 64 columns), O of slot s at 256 + 128 s
 constexpr float RESCALE_LOG2 = 8.f;
 
@@ -121,14 +123,15 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
     auto q_full = [&](int s) { return bar0 + 8u * s; };
     auto q_empty = [&](int s) { return bar0 + 8u * (2 + s); };
     auto k_full = [&](int st) { return bar0 + 8u * (4 + st); };
-    auto k_empty = [&](int st) { return bar0 + 8u * (4 + KV_STAGES + st); };
-    auto v_full = [&](int st) { return bar0 + 8u * (4 + 2 * KV_STAGES + st); };
-    auto v_empty = [&](int st) { return bar0 + 8u * (4 + 3 * KV_STAGES + st); };
-    auto s_full = [&](int s) { return bar0 + 8u * (4 + 4 * KV_STAGES + s); };
-    auto p_full = [&](int s) { return bar0 + 8u * (6 + 4 * KV_STAGES + s); };
-    auto pv_done = [&](int s) { return bar0 + 8u * (8 + 4 * KV_STAGES + s); };
-    auto sched_full = [&](int e) { return bar0 + 8u * (10 + 4 * KV_STAGES + e); };
-    auto sched_empty = [&](int e) { return bar0 + 8u * (10 + 4 * KV_STAGES + SCHED_DEPTH + e); };
+    constexpr int KVB = 2 * K_STAGES + 2 * KV_STAGES;      // barriers of the two rings
+    auto k_empty = [&](int st) { return bar0 + 8u * (4 + K_STAGES + st); };
+    auto v_full = [&](int st) { return bar0 + 8u * (4 + 2 * K_STAGES + st); };
+    auto v_empty = [&](int st) { return bar0 + 8u * (4 + 2 * K_STAGES + KV_STAGES + st); };
+    auto s_full = [&](int s) { return bar0 + 8u * (4 + KVB + s); };
+    auto p_full = [&](int s) { return bar0 + 8u * (6 + KVB + s); };
+    auto pv_done = [&](int s) { return bar0 + 8u * (8 + KVB + s); };
+    auto sched_full = [&](int e) { return bar0 + 8u * (10 + KVB + e); };
+    auto sched_empty = [&](int e) { return bar0 + 8u * (10 + KVB + SCHED_DEPTH + e); };
     uint32_t* tmem_ptr_smem = reinterpret_cast<uint32_t*>(smem_raw + SMEM_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_ptr_smem + 1);
     volatile int* sched_idx = reinterpret_cast<volatile int*>(tmem_ptr_smem + 2);      // [SCHED_DEPTH]
@@ -144,9 +147,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             mbar_init(p_full(s), 4);
             mbar_init(pv_done(s), 1);
         }
-        for (int st = 0; st < KV_STAGES; ++st) {
+        for (int st = 0; st < K_STAGES; ++st) {
             mbar_init(k_full(st), 1);
             mbar_init(k_empty(st), 1);
+        }
+        for (int st = 0; st < KV_STAGES; ++st) {
             mbar_init(v_full(st), 1);
             mbar_init(v_empty(st), 1);
         }
@@ -201,8 +206,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             uint32_t gq[2] = {0u, 0u}, gk = 0, gv = 0, it = 0;
             bool ok = true;
             auto load_k = [&](const CUtensorMap* tm, int col, int row, int b) -> bool {
-                const int st = gk % KV_STAGES;
-                if (!wait_barrier(k_empty(st), ((gk / KV_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2)) return false;
+                const int st = gk % K_STAGES;
+                if (!wait_barrier(k_empty(st), ((gk / K_STAGES) & 1u) ^ 1u, abort_flag, p.status, 2)) return false;
                 mbar_arrive_expect_tx(k_full(st), KV_BYTES);
                 tma_load_3d(base + SMEM_K + st * KV_BYTES, tm, k_full(st), col, row, b);
                 tma_load_3d(base + SMEM_K + st * KV_BYTES + KV_HALF, tm, k_full(st), col + 64, row, b);
@@ -295,8 +300,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) hca_attention_pair_kernel(cons
             __syncwarp();
         };
         auto k_acquire = [&](int& st) {
-            st = gk % KV_STAGES;
-            return wait_all(k_full(st), (gk / KV_STAGES) & 1u, 4);
+            st = gk % K_STAGES;
+            return wait_all(k_full(st), (gk / K_STAGES) & 1u, 4);
         };
         auto k_release = [&](int st) {
             if (leader) umma_commit(k_empty(st));
