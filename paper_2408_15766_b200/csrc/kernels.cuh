@@ -9,9 +9,14 @@
 //               (the separate, recomputing backward)
 //   MODE_OUT    dH_d tile: coef * acc - Omega_hat row (fused), coef * acc (q W of the combined objective)
 //               or the accumulator as is (separate backward)
-// plus small kernels: finalize (merge partial statistics, pick Omega_hat, Eq. 1 and its variants, the
-// Omega_hat term of dH_d), ce_kernel (cross-entropy of the combined objective), bwd_prep (index-sorted
-// Top-K lists for MODE_PROBS) and range_handled_kernel.
+// plus small kernels: select (between the sweep of the target rows and the sweep of the draft rows: lse_t,
+// Omega_hat, the set sorted by token id), loss_patch (after the draft sweep: lse_d, Eq. 1, row scale, the
+// Omega_hat term into the spill), finalize (the single-sweep route: merge partial statistics, pick Omega_hat,
+// Eq. 1 and its variants, the Omega_hat term of dH_d), ce_kernel (cross-entropy of the combined objective),
+// bwd_prep (index-sorted Top-K lists for MODE_PROBS) and range_handled_kernel.
+// Beside the four operand stages the kernel's shared memory holds 32 KB that the epilogue warps use: staging
+// buffers for the TMA stores of the spill (draft sweep) or the logits waiting for admission to the register
+// Top-K lists (target sweep).
 #pragma once
 #include <cuda_bf16.h>
 #include <float.h>
