@@ -151,8 +151,12 @@ int hass_topk_distill_bwd(const void* H_d, const void* W, int64_t N, int64_t d, 
  * violation was detected, in which case they redo the whole call exactly. The result is correct
  * either way; the conditional launches cost about 0.3 % when they have nothing to do. The _draft
  * form and the Top-P variant work the same way.
- * (hass_combined_distill_fwd_bwd and the Bi-directional variant have no such second route:
- * there hass_check reports HASS_ERR_RANGE and loss, lse_d and dH_d are invalid.)
+ * hass_combined_distill_fwd_bwd and the Bi-directional variant handle a violation differently: their
+ * sweep records every row's largest logit, and the whole sequence is enqueued a second time as
+ * conditional launches that take each row's exponent from that record (no logit of the row can
+ * exceed it); a violation therefore costs one more pass and the result is correct either way.
+ * HASS_ERR_RANGE is what hass_check reports if a violation was detected and nothing redid the call
+ * (none of the entry points of this version leaves it at that).
  */
 int hass_topk_distill_fwd_bwd(const void* H_t, const void* H_d, const void* W, int64_t N, int64_t d,
                               int64_t V, int32_t K, const float* grad_loss, float* loss,
@@ -183,8 +187,9 @@ int hass_topk_distill_fwd_bwd_draft(const void* H_d, const void* W, int64_t N, i
  * i.e. the gradient of sum_i grad_loss[i] (loss_ce[i] + w loss_topk[i]) with respect to H_d. The
  * sweep spills the target tiles as well, a second GEMM forms q W per row, from which both the
  * cross-entropy, lse_d - <H_d[i], (q W)[i]>, and its gradient term follow; 8 N d V tensor FLOPs
- * are executed. Range condition and HASS_ERR_RANGE as for hass_topk_distill_fwd_bwd, for target
- * and draft logits alike. The other outputs are those of hass_topk_distill_fwd.
+ * are executed. Range condition as for hass_topk_distill_fwd_bwd, for target and draft logits
+ * alike; a violation is repaired by a second pass of the same sequence (see there). The other
+ * outputs are those of hass_topk_distill_fwd.
  * Workspace: hass_combined_distill_workspace_bytes (the normal workspace plus the target spill and
  * a q W buffer for one chunk of rows).
  */

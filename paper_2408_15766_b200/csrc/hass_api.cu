@@ -200,7 +200,7 @@ static int topk_cap(int K) { return K <= K_REG ? K_REG : cand_cap(K); }
 static inline size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 struct Layout {
-    size_t status, part_m, part_s, cand_v, cand_i, thr_share, fwd_end, sidx, sgq, coef, lse2, capz, sparse, scratch, fixed_end;
+    size_t status, part_m, part_s, cand_v, cand_i, thr_share, fwd_end, sidx, sgq, coef, lse2, capz, zmax, sparse, scratch, fixed_end;
     size_t scratch_row_tile_bytes;   // bytes of dz_d scratch per 128-row tile
     long long p_pitch;
     int pref_chunk_tiles;
@@ -261,6 +261,8 @@ static int make_layout(long long N, long long d, long long V, int K, int sms, La
     off = align256(off + static_cast<size_t>(N) * 4);
     L->capz = off;                          // fused path: draft logits at Omega_hat, captured by the draft sweep, [N, K]
     off = align256(off + static_cast<size_t>(N) * K * 4);
+    L->zmax = off;                          // single-sweep route: every spilling row's largest logit (target and draft rows)
+    off = align256(off + static_cast<size_t>(2 * RT) * BM * 4);
     L->sparse = off;                        // fused path: Omega_hat term of one chunk of rows, fp32 [chunk rows, d]
     off = align256(off + static_cast<size_t>(pref) * BM * d * 4);
     L->scratch = off;
@@ -590,6 +592,16 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
     if (rc == HASS_OK && cmb) rc = make_tmap(&tmPt, cmb->Pt, static_cast<long long>(chunk_tiles) * BM, V, L.p_pitch, BK, BM);
     if (rc != HASS_OK) return rc;
 
+    // Every spilling row records its largest logit. If the sweep reports a row beyond the exponent range of its spill
+    // (reference from column tile 0), the same sequence runs a second time as conditional launches with each row's
+    // reference taken from that record, which no logit of the row can exceed.
+    unsigned int* zmax = reinterpret_cast<unsigned int*>(ws + L.zmax);
+    if (cudaMemsetAsync(zmax, 0, static_cast<size_t>(2 * RT) * BM * 4, st) != cudaSuccess) {
+        cudaGetLastError();
+        return HASS_ERR_CUDA;
+    }
+    auto run = [&](bool retry) -> int {
+    const unsigned int* gate = retry ? status : nullptr;
     for (int t0 = 0; t0 < RT; t0 += chunk_tiles) {
         const int tiles = (RT - t0 < chunk_tiles) ? RT - t0 : chunk_tiles;
         const int rows = static_cast<int>((N - static_cast<long long>(t0) * BM < static_cast<long long>(tiles) * BM)
@@ -625,6 +637,9 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         p.p_pitch = L.p_pitch;
         p.status = status;
         p.thr_share = reinterpret_cast<float*>(ws + L.thr_share);
+        p.row_zmax = zmax + static_cast<size_t>(with_target ? 2 : 1) * t0 * BM;
+        p.use_row_zmax = retry ? 1 : 0;
+        p.only_if_range = gate;
     if (cudaMemsetAsync(p.thr_share, 0xff, static_cast<size_t>(p.sched.total_slots) * BM * 4, st) != cudaSuccess) {   // NaN
         cudaGetLastError();
         return HASS_ERR_CUDA;
@@ -666,8 +681,9 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         f.Pt = cmb ? cmb->Pt : nullptr;
         f.p_pitch = L.p_pitch;
         f.ce_corr_out = reinterpret_cast<float*>(ws + L.lse2);    // [N] floats, otherwise used by the split backward
+        f.only_if_range = gate;
         {
-            KernelTimer timer(KIND_FINALIZE, st);
+            KernelTimer timer(retry ? KIND_CONDITIONAL : KIND_FINALIZE, st);
             finalize_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(f);
         }
         g_launches.fetch_add(1);
@@ -698,13 +714,14 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
             t.out_align32 = 1;
             t.out_pitch = d;
             t.status = status;
+            t.only_if_range = gate;
             rc = launch_gemm<MODE_OUT>(t, st);
             if (rc != HASS_OK) return rc;
             {
-                KernelTimer timer(KIND_FINALIZE, st);
+                KernelTimer timer(retry ? KIND_CONDITIONAL : KIND_FINALIZE, st);
                 ce_kernel<<<ceil_div(rows, 8), 256, 0, st>>>(rows, t0 * BM, static_cast<int>(d),
                                                              static_cast<const __nv_bfloat16*>(H_d), cmb->T, lse_d, grad_loss,
-                                                             reinterpret_cast<const float*>(ws + L.lse2), cmb->loss_ce, sparse);
+                                                             reinterpret_cast<const float*>(ws + L.lse2), cmb->loss_ce, sparse, gate);
             }
             g_launches.fetch_add(1);
             if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
@@ -728,10 +745,22 @@ static int fused_impl(bool with_target, const void* H_t, const void* H_d, const 
         o.out_align32 = ((reinterpret_cast<uintptr_t>(dH_d) | static_cast<uintptr_t>(d * (dH_dtype == HASS_FP32 ? 4 : 2))) & 31u) == 0 ? 1 : 0;
         o.out_pitch = d;
         o.status = status;
+        o.only_if_range = gate;
         rc = launch_gemm<MODE_OUT>(o, st);
         if (rc != HASS_OK) return rc;
     }
-    // no second route here: a row beyond the spill's exponent range is reported as HASS_ERR_RANGE by hass_check
+    return HASS_OK;
+    };
+    rc = run(false);
+    if (rc != HASS_OK) return rc;
+    rc = run(true);
+    if (rc != HASS_OK) return rc;
+    {
+        KernelTimer timer(KIND_CONDITIONAL, st);
+        range_handled_kernel<<<1, 1, 0, st>>>(status);
+    }
+    g_launches.fetch_add(1);
+    if (cudaGetLastError() != cudaSuccess) return HASS_ERR_CUDA;
     return HASS_OK;
 }
 

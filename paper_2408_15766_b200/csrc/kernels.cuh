@@ -104,6 +104,12 @@ struct GemmParams {
     long long out_pitch;   // elements
     unsigned int* status;
     const unsigned int* only_if_range;   // nullptr, or: run only if this status word reports a range overflow
+    // The single-sweep route (spilling sweeps with Top-K lists): every spilling row leaves the ordered key of its
+    // largest logit in row_zmax[row tile * 128 + row] (atomicMax over the lanes of the row tile; zeroed by the
+    // host). A second sweep with use_row_zmax = 1 takes the row's fixed exponent from there instead of from
+    // column tile 0, so that no logit of the row can exceed it.
+    unsigned int* row_zmax;              // nullable
+    int use_row_zmax;
 };
 
 // MODE_STATS: does this row tile also write its tiles 2^(z log2e - ref2) as bf16? Draft tiles from spill_begin
@@ -417,6 +423,8 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
             float thr_sh = -INFINITY;                             // just below the best threshold published by the other lanes
             bool want_topk = false;
             const bool spill = MODE == MODE_STATS && spills(p, rt);
+            const bool track_zmax = MODE == MODE_STATS && TOPK != TOPK_NONE && spill && p.row_zmax != nullptr;
+            float zmax = -INFINITY;                               // the row's largest logit in this lane's column tiles
             float ref2 = 0.f;                                     // spill rows: exponent offset (log2 units)
             float lse2 = 0.f, coef = 0.f;                         // MODE_PROBS / fused MODE_OUT
             const int* si = nullptr;
@@ -464,14 +472,19 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                     // Reference exponent of this row: its largest logit in column tile 0. Every lane of
                     // the row tile computes tile 0 first and so derives the same value.
                     float mx = -INFINITY;
+                    if (TOPK != TOPK_NONE && p.use_row_zmax) {
+                        // second sweep after a range report: the row's largest logit is known
+                        mx = __uint_as_float(key_bits(p.row_zmax[rt * BM + r_local]));
+                    } else {
 #pragma unroll 1
-                    for (int ch = 0; ch < BN / 32; ++ch) {
-                        uint32_t r[32];
-                        tmem_ld32(t_row + ch * 32, r);
-                        tmem_ld_wait(r);
+                        for (int ch = 0; ch < BN / 32; ++ch) {
+                            uint32_t r[32];
+                            tmem_ld32(t_row + ch * 32, r);
+                            tmem_ld_wait(r);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (ch * 32 + j < p.n_cols) mx = fmaxf(mx, __uint_as_float(r[j]));
+                            for (int j = 0; j < 32; ++j)
+                                if (ch * 32 + j < p.n_cols) mx = fmaxf(mx, __uint_as_float(r[j]));
+                        }
                     }
                     // spilled values are 2^(z log2e - ref2) <= about 2^-64 for typical rows, which leaves
                     // 2^191 of headroom above the reference before bf16 / fp32 overflow
@@ -566,10 +579,11 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                             }
                         }
                         float cm = -INFINITY;     // the chunk's largest logit (not needed by a spill row without Top-K)
-                        if (!spill || want_topk) {
+                        if (!spill || want_topk || track_zmax) {
                             cm = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1]));
 #pragma unroll
                             for (int j = 2; j < 32; j += 2) cm = fmax3(cm, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+                            zmax = fmaxf(zmax, cm);
                         }
                         if (!spill) {
                             if (cm > m) {
@@ -826,6 +840,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1) gemm_kernel(const __grid_const
                 // a spilled value reached the top of the fp32 range: the row's logits spread too far
                 // above its reference for the fixed-exponent spill
                 if (spill && !(s < 1e38f)) atomicCAS(p.status, 0u, (5u << 8) | 2u);
+                if (track_zmax && !p.use_row_zmax) atomicMax(p.row_zmax + rt * BM + r_local, ordered_key(__float_as_uint(zmax)));
                 if (USE_REG && want_topk) {
                     // the register list goes out as a full buffer of K_REG entries (unused ones carry id -1)
 #pragma unroll
@@ -1501,7 +1516,9 @@ __global__ void __launch_bounds__(256) loss_patch_kernel(const __grid_constant__
 __global__ void __launch_bounds__(256) ce_kernel(int rows, int row_begin, int d, const __nv_bfloat16* __restrict__ H_d,
                                                  const float* __restrict__ T, const float* __restrict__ lse_d,
                                                  const float* __restrict__ grad_loss, const float* __restrict__ ce_corr,
-                                                 float* __restrict__ loss_ce, float* __restrict__ sparse) {
+                                                 float* __restrict__ loss_ce, float* __restrict__ sparse,
+                                                 const unsigned int* __restrict__ only_if_range) {
+    if (only_if_range != nullptr && ((*only_if_range) & 0xffu) != 2u) return;
     const int lane = threadIdx.x & 31;
     const int local = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (local >= rows) return;
