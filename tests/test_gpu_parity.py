@@ -237,6 +237,13 @@ def test_exact_route_with_two_row_chunks_when_only_some_rows_exceed_the_range():
     keep = np.setdiff1d(np.arange(N), hot)
     assert torch.equal(out["topk_idx"].cpu()[keep], ref["topk_idx"].cpu()[keep])
     assert torch.allclose(out["loss"].cpu()[keep], ref["loss"].cpu()[keep], rtol=1e-3, atol=1e-7)
+    # the Bi-directional variant on the same inputs: its second pass covers both chunks, every row keeps a valid result
+    import oracle
+    v = hass.variant_distill_fwd_bwd(inp.H_t.to(dev), H_d.to(dev), W.to(dev), K, hass.LOSS_BIDIR_TOPK, 0.0,
+                                     dH_dtype=hass.HASS_FP32)
+    hass.check(v["workspace"])
+    print("bidir, two chunks, second pass",
+          compare_variant(inp.H_t, H_d, W, K, oracle.VARIANT_BIDIR, 0.0, _to_cpu(v), rows=rows))
 
 
 def test_l3_8b_split_forward_and_recomputing_backward_sampled_rows():
