@@ -37,8 +37,8 @@ UNIT = "tokens/s"
 # launches of one step). Valid for the library version they were taken with; for the l3-8b shape the figures
 # are scaled by the vocabulary ratio (W, the spill and its re-reads all grow with V; the 2 x 39 MB of H rows
 # and the dH_d rows that do not are 6 % of the total).
-TRAFFIC_CAPTURE = {"version": 10400, "workload": "l2-7b", "V": 32000, "K": 10,
-                   "bytes_per_launch": {"stats_gemm": 497.1e6, "stats_gemm_draft": 753.4e6, "dH_gemm": 1211.7e6}}
+TRAFFIC_CAPTURE = {"version": 10410, "workload": "l2-7b", "V": 32000, "K": 10,
+                   "bytes_per_launch": {"stats_gemm": 495.0e6, "stats_gemm_draft": 759.1e6, "dH_gemm": 1212.1e6}}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -1267,7 +1267,7 @@ const char* hass_status_string(int status) {
     }
 }
 
-int hass_version(void) { return 10400; }
+int hass_version(void) { return 10410; }
 
 int64_t hass_kernel_launch_count(void) { return g_launches.load(); }
 
